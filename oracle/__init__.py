@@ -1,0 +1,211 @@
+"""ctypes front end of the CPU oracle (oracle/dynamo_oracle.c).
+
+TEST INFRASTRUCTURE ONLY: imported by tests/, the smoke check and the benchmark's CPU-baseline /
+reference arms, never by the CUDA package.  Builds the C file with gcc on first use (OpenMP, -O2).
+Array arguments are numpy arrays; fp32 tables and loads are promoted to fp64 inside the C code.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from types import SimpleNamespace
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "dynamo_oracle.c")
+_LIB = os.path.join(_HERE, "libdynamo_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle into oracle/libdynamo_oracle.so (rebuilds when the source is newer)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".{os.getpid()}.tmp"
+        subprocess.run(["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-Wall", "-Wextra",
+                        "-o", tmp, _SRC, "-lm"], check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+class _Profile(C.Structure):
+    _fields_ = [("C", C.c_int32), ("T", C.c_int32), ("R", C.c_int32), ("M", C.c_int32),
+                ("tp", C.c_void_p), ("f_grid", C.c_void_p), ("ttft", C.c_void_p), ("cap", C.c_void_p),
+                ("tbt", C.c_void_p), ("pw", C.c_void_p)]
+
+
+class _Space(C.Structure):
+    _fields_ = [("F", C.c_int32), ("Nmax", C.c_int32), ("f_cand", C.c_void_p),
+                ("slo_ttft", C.c_void_p), ("slo_tbt", C.c_void_p), ("gpu_budget", C.c_int32),
+                ("window_s", C.c_float)]
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.orc_num_threads.restype = C.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().orc_num_threads())
+
+
+def set_num_threads(n: int) -> None:
+    _load().orc_set_num_threads(C.c_int(int(n)))
+
+
+def _p(a):
+    return C.c_void_p(a.ctypes.data) if a is not None else C.c_void_p(0)
+
+
+def _arr(a, dt):
+    return np.ascontiguousarray(a, dtype=dt)
+
+
+def bin_trace(t_ms, in_tok, out_tok, window_ms, n_windows, in_edges, out_edges):
+    """Counts uint32 [W][C] and the number of requests past the last window."""
+    lib = _load()
+    t_ms, in_tok, out_tok = (_arr(x, np.uint32) for x in (t_ms, in_tok, out_tok))
+    ie, oe = _arr(in_edges, np.uint32), _arr(out_edges, np.uint32)
+    Cn = (len(ie) + 1) * (len(oe) + 1)
+    counts = np.empty((int(n_windows), Cn), dtype=np.uint32)
+    dropped = C.c_uint64(0)
+    rc = lib.orc_bin_trace(_p(t_ms), _p(in_tok), _p(out_tok), C.c_uint64(len(t_ms)),
+                           C.c_uint32(int(window_ms)), C.c_uint32(int(n_windows)),
+                           _p(ie), C.c_int32(len(ie)), _p(oe), C.c_int32(len(oe)),
+                           _p(counts), C.byref(dropped))
+    if rc != 0:
+        raise ValueError("orc_bin_trace: invalid argument")
+    return counts, int(dropped.value)
+
+
+def load_from_counts(counts, window_s):
+    counts = _arr(counts, np.uint32)
+    out = np.empty(counts.shape, dtype=np.float32)
+    _load().orc_load(_p(counts), C.c_uint64(counts.size), C.c_float(float(window_s)), _p(out))
+    return out
+
+
+def _structs(profile, space):
+    """Keep the numpy arrays alive next to the C structs that point into them."""
+    keep = SimpleNamespace(
+        tp=_arr(profile.tp, np.int32), fg=_arr(profile.f_grid_mhz, np.float32),
+        ttft=_arr(profile.ttft, np.float32), cap=_arr(profile.cap, np.float32),
+        tbt=_arr(profile.tbt, np.float32), pw=_arr(profile.pow, np.float32),
+        fc=_arr(space.f_cand_mhz, np.float32), sa=_arr(space.slo_ttft_s, np.float32),
+        sb=_arr(space.slo_tbt_s, np.float32))
+    Cn, T, R = keep.ttft.shape
+    M = keep.tbt.shape[3]
+    assert keep.tbt.shape == (Cn, T, R, M) and keep.pw.shape == (Cn, T, R, M) and keep.cap.shape == (Cn, T, R)
+    assert len(keep.tp) == T and len(keep.fg) == R and len(keep.sa) == Cn and len(keep.sb) == Cn
+    p = _Profile(Cn, T, R, M, keep.tp.ctypes.data, keep.fg.ctypes.data, keep.ttft.ctypes.data,
+                 keep.cap.ctypes.data, keep.tbt.ctypes.data, keep.pw.ctypes.data)
+    s = _Space(len(keep.fc), int(space.n_max), keep.fc.ctypes.data, keep.sa.ctypes.data,
+               keep.sb.ctypes.data, int(space.gpu_budget), float(space.window_s))
+    return p, s, keep
+
+
+def resolve(f_grid, f_cand):
+    fg, fc = _arr(f_grid, np.float32), _arr(f_cand, np.float32)
+    row = np.empty(len(fc), dtype=np.int32)
+    wt = np.empty(len(fc), dtype=np.float64)
+    rc = _load().orc_resolve(_p(fg), C.c_int32(len(fg)), _p(fc), C.c_int32(len(fc)), _p(row), _p(wt))
+    if rc != 0:
+        raise ValueError("orc_resolve: candidate frequency outside the table grid (or R < 2)")
+    return row, wt
+
+
+def eval_tile(profile, space, c, load, details=False):
+    """All J energies of one tile (fp64).  With details: also TBT, power, utilisation, margin."""
+    lib = _load()
+    p, s, keep = _structs(profile, space)
+    row, wt = resolve(keep.fg, keep.fc)
+    J = s.Nmax * p.T * s.F
+    E = np.empty(J)
+    if not details:
+        lib.orc_eval_tile(C.byref(p), C.byref(s), _p(row), _p(wt), C.c_int32(int(c)), C.c_double(float(load)),
+                          _p(E), None, None, None, None)
+        return E
+    tb, pw, u = np.empty(J), np.empty(J), np.empty(J)
+    mg = C.c_double(0.0)
+    lib.orc_eval_tile(C.byref(p), C.byref(s), _p(row), _p(wt), C.c_int32(int(c)), C.c_double(float(load)),
+                      _p(E), _p(tb), _p(pw), _p(u), C.byref(mg))
+    return E, tb, pw, u, float(mg.value)
+
+
+def eval_configs(profile, space, load):
+    """E fp64 [S][W][C][J] for loads float32 [S][W][C]."""
+    lib = _load()
+    p, s, keep = _structs(profile, space)
+    load = _arr(load, np.float32)
+    S, W, Cn = load.shape
+    assert Cn == p.C
+    J = s.Nmax * p.T * s.F
+    E = np.empty((S, W, Cn, J))
+    rc = lib.orc_eval_configs(C.byref(p), C.byref(s), _p(load), C.c_int64(S), C.c_int64(W), _p(E))
+    if rc != 0:
+        raise ValueError("orc_eval_configs: invalid argument")
+    return E
+
+
+def select_row(E):
+    E = _arr(E, np.float64)
+    idx, be, e2 = C.c_int32(0), C.c_double(0.0), C.c_double(0.0)
+    _load().orc_select_row(_p(E), C.c_int64(E.size), C.byref(idx), C.byref(be), C.byref(e2))
+    return int(idx.value), float(be.value), float(e2.value)
+
+
+def select(E):
+    """Per-tile argmin of E[..., J]: (best_idx int32, best_E, E2) shaped like E without its last axis."""
+    E = _arr(E, np.float64)
+    J = E.shape[-1]
+    tiles = E.size // J if J else 0
+    idx = np.empty(E.shape[:-1], dtype=np.int32)
+    be, e2 = np.empty(E.shape[:-1]), np.empty(E.shape[:-1])
+    _load().orc_select(_p(E), C.c_int64(tiles), C.c_int64(J), _p(idx), _p(be), _p(e2))
+    return idx, be, e2
+
+
+def eval_select(profile, space, load):
+    """Fused evaluate + select: dict(best_idx, best_E, E2, margin), each [S][W][C]."""
+    lib = _load()
+    p, s, keep = _structs(profile, space)
+    load = _arr(load, np.float32)
+    S, W, Cn = load.shape
+    assert Cn == p.C
+    idx = np.empty((S, W, Cn), dtype=np.int32)
+    be, e2, mg = np.empty((S, W, Cn)), np.empty((S, W, Cn)), np.empty((S, W, Cn))
+    rc = lib.orc_eval_select(C.byref(p), C.byref(s), _p(load), C.c_int64(S), C.c_int64(W),
+                             _p(idx), _p(be), _p(e2), _p(mg))
+    if rc != 0:
+        raise ValueError("orc_eval_select: invalid argument")
+    return dict(best_idx=idx, best_E=be, E2=e2, margin=mg)
+
+
+def config_tables(n_max, tp, F):
+    """n_of_j and tp_of_j for j = ((n-1)*T + t)*F + q."""
+    tp = np.asarray(tp, dtype=np.int32)
+    T = len(tp)
+    j = np.arange(int(n_max) * T * int(F))
+    return (j // (T * F) + 1).astype(np.int32), tp[(j // F) % T].astype(np.int32)
+
+
+def totals(best_idx, best_E, J, n_of_j=None, tp_of_j=None):
+    """dict(E_total[S], n_infeasible[S], E_window[S][W], hist[S][J], gpus[S][W] or None)."""
+    idx = _arr(best_idx, np.int32)
+    be = _arr(best_E, np.float64)
+    S, W, Cn = idx.shape
+    et = np.empty(S)
+    bad = np.empty(S, dtype=np.uint32)
+    ew = np.empty((S, W))
+    hist = np.empty((S, int(J)), dtype=np.uint32)
+    have = n_of_j is not None and tp_of_j is not None
+    gp = np.empty((S, W), dtype=np.uint32) if have else None
+    nj = _arr(n_of_j, np.int32) if have else None
+    tj = _arr(tp_of_j, np.int32) if have else None
+    _load().orc_totals(_p(idx), _p(be), C.c_int64(S), C.c_int64(W), C.c_int32(Cn), C.c_int64(int(J)),
+                       _p(nj), _p(tj), _p(et), _p(bad), _p(ew), _p(hist), _p(gp))
+    return dict(E_total=et, n_infeasible=bad, E_window=ew, hist=hist, gpus=gp)

@@ -1,0 +1,290 @@
+/*
+ * CPU oracle for the configuration-selection hot path of DynamoLLM (arXiv 2408.00741).
+ *
+ * TEST INFRASTRUCTURE ONLY.  Plain C, fp64, one loop per step of the definition, no blocking and
+ * no reordering.  It shares no code, header, table or constant with the CUDA library; only the
+ * tests, the smoke check and the benchmark's CPU-baseline / reference arms may call it.
+ *
+ * What it computes (paper passages in brackets):
+ *   orc_bin_trace     requests (timestamp, input tokens, output tokens) [Sec. 3, trace fields] are
+ *                     assigned a time window and one of KI*KO length classes [Sec. 3.1 and its
+ *                     thresholds table] and counted per (window, class) [Sec. 3.1 "Request loads",
+ *                     Sec. 3.2 load over time].
+ *   orc_load          count / window length = requests per second per (window, class).
+ *   orc_resolve       the profile function (load, class, TP, frequency) -> TTFT, TBT, power is a
+ *                     table over a few profiled frequencies and load levels with linear
+ *                     interpolation in between [Sec. 4.1 "Generating LLM profiles"; Sec. 5
+ *                     implementation: linear 1-D interpolation].
+ *   orc_eval_tile     for every candidate (N instances, TP, f): fair-share per-instance load,
+ *                     expected TBT and power, the constraints of Eq. 1 (GPU budget, load covered,
+ *                     performance within SLO) and the objective N x Energy^{TP,f}(L/N) [Sec. 4.1,
+ *                     Eq. 1]; infeasible candidates get +inf [Sec. 4.2 scale-up/down: filter out
+ *                     SLO-violating settings, then pick the minimum-energy one].
+ *   orc_select_row    minimum-energy feasible candidate, lowest index on ties [Sec. 4.2]; also the
+ *                     runner-up energy (for near-tie exemptions in parity tests).
+ *   orc_totals        cluster energy per scenario and per window, GPUs in use per window, histogram
+ *                     of chosen configurations [Sec. 6 cluster-level energy, GPUs per sharding].
+ *
+ * Readings of points the paper leaves open: class = number of edges <= value; window =
+ * t_ms / window_ms (unsigned integer division); utilisation u = (L/n)/cap with u > 1 infeasible; tables sampled at u_m = m/(M-1);
+ * config index j = ((n-1)*T + t)*F + q; no feasible candidate -> index -1, energy +inf, excluded
+ * from totals and counted in n_infeasible; energy in Wh per window.
+ *
+ * Parity pins (tests/ -m "not gpu"): closed forms of the synthetic profiles, Tables 1-3 of the
+ * paper as energy rows for orc_select_row, boundary values of the thresholds table, invariants and
+ * tiny-grid brute force.  Absolute energies versus the paper's Wh numbers: parity unpinned (the
+ * measured H100 profiles behind them are not available).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORC_OK 0
+#define ORC_EINVAL (-1)
+
+int orc_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+void orc_set_num_threads(int n) {
+#ifdef _OPENMP
+    if (n > 0) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
+/* ---- stage (a): classify, window, count -------------------------------------------------- */
+
+/* class of one length: how many ascending edges are <= the value */
+static int32_t edge_class(uint32_t v, const uint32_t *edges, int32_t n_edges) {
+    int32_t k = 0;
+    for (int32_t e = 0; e < n_edges; ++e)
+        if (edges[e] <= v) ++k;
+    return k;
+}
+
+int orc_bin_trace(const uint32_t *t_ms, const uint32_t *in_tok, const uint32_t *out_tok, uint64_t n_req,
+                  uint32_t window_ms, uint32_t n_windows,
+                  const uint32_t *in_edges, int32_t n_in_edges,
+                  const uint32_t *out_edges, int32_t n_out_edges,
+                  uint32_t *counts /* [W][C] */, uint64_t *dropped) {
+    if (window_ms == 0 || n_in_edges < 0 || n_out_edges < 0) return ORC_EINVAL;
+    const int32_t KO = n_out_edges + 1;
+    const int32_t C = (n_in_edges + 1) * KO;
+    memset(counts, 0, (size_t)n_windows * (size_t)C * sizeof(uint32_t));
+    uint64_t drop = 0;
+    for (uint64_t i = 0; i < n_req; ++i) {
+        uint32_t w = t_ms[i] / window_ms;
+        if (w >= n_windows) { ++drop; continue; }
+        int32_t ci = edge_class(in_tok[i], in_edges, n_in_edges);
+        int32_t co = edge_class(out_tok[i], out_edges, n_out_edges);
+        counts[(size_t)w * C + (size_t)(ci * KO + co)] += 1u;
+    }
+    *dropped = drop;
+    return ORC_OK;
+}
+
+/* load in requests/s, computed and rounded in fp32: this fp32 number is the input of stage (b) */
+void orc_load(const uint32_t *counts, uint64_t n_bins, float window_s, float *load) {
+    for (uint64_t i = 0; i < n_bins; ++i) load[i] = (float)counts[i] / window_s;
+}
+
+/* ---- stage (b): profile lookup, feasibility, energy -------------------------------------- */
+
+typedef struct {
+    int32_t C, T, R, M;
+    const int32_t *tp;         /* [T] */
+    const float *f_grid;       /* [R] ascending */
+    const float *ttft;         /* [C][T][R] */
+    const float *cap;          /* [C][T][R] */
+    const float *tbt;          /* [C][T][R][M] */
+    const float *pw;           /* [C][T][R][M] */
+} orc_profile;
+
+typedef struct {
+    int32_t F, Nmax;
+    const float *f_cand;       /* [F] */
+    const float *slo_ttft;     /* [C] */
+    const float *slo_tbt;      /* [C] */
+    int32_t gpu_budget;        /* <= 0: none */
+    float window_s;
+} orc_space;
+
+/* position of candidate frequency q in the table grid: row r and weight w in [0,1] */
+int orc_resolve(const float *f_grid, int32_t R, const float *f_cand, int32_t F,
+                int32_t *row, double *weight) {
+    if (R < 2) return ORC_EINVAL;
+    for (int32_t q = 0; q < F; ++q) {
+        double f = (double)f_cand[q];
+        if (f < (double)f_grid[0] || f > (double)f_grid[R - 1]) return ORC_EINVAL;
+        int32_t r = 0;
+        for (int32_t i = 0; i <= R - 2; ++i)
+            if ((double)f_grid[i] <= f) r = i;
+        row[q] = r;
+        weight[q] = (f - (double)f_grid[r]) / ((double)f_grid[r + 1] - (double)f_grid[r]);
+    }
+    return ORC_OK;
+}
+
+static double lerp(double a, double b, double w) { return (1.0 - w) * a + w * b; }
+
+/* value of a [R][M] table at (row r, weight om) x (knot m, weight nu): bilinear */
+static double table_at(const float *tab, int32_t M, int32_t r, double om, int32_t m, double nu) {
+    double lo = lerp((double)tab[(size_t)r * M + m], (double)tab[(size_t)r * M + m + 1], nu);
+    double hi = lerp((double)tab[(size_t)(r + 1) * M + m], (double)tab[(size_t)(r + 1) * M + m + 1], nu);
+    return lerp(lo, hi, om);
+}
+
+/*
+ * All J = Nmax*T*F candidates of one (window, class) tile with total load `load` (requests/s).
+ * E[j] in Wh (+inf if infeasible).  Optional outputs (NULL to skip): per-candidate TBT, power,
+ * utilisation; *margin = smallest relative distance of any deciding quantity to its bound
+ * (|TBT-slo|/slo, |u-1|, |TTFT-slo|/slo) over the candidates of the tile.
+ */
+void orc_eval_tile(const orc_profile *p, const orc_space *sp, const int32_t *row, const double *weight,
+                   int32_t c, double load, double *E, double *tbt_out, double *pow_out, double *u_out,
+                   double *margin) {
+    const int32_t T = p->T, R = p->R, M = p->M, F = sp->F;
+    double mg = INFINITY;
+    for (int32_t n = 1; n <= sp->Nmax; ++n) {
+        for (int32_t t = 0; t < T; ++t) {
+            for (int32_t q = 0; q < F; ++q) {
+                const size_t j = ((size_t)(n - 1) * T + t) * F + q;
+                const size_t ct = ((size_t)c * T + t) * R;
+                const int32_t r = row[q];
+                const double om = weight[q];
+                const double ttft = lerp((double)p->ttft[ct + r], (double)p->ttft[ct + r + 1], om);
+                const double cap = lerp((double)p->cap[ct + r], (double)p->cap[ct + r + 1], om);
+                const double l = load / (double)n;                 /* fair share per instance */
+                const double u = l / cap;                          /* utilisation */
+                const double x = fmin(u, 1.0) * (double)(M - 1);
+                int32_t m = (int32_t)floor(x);
+                if (m > M - 2) m = M - 2;
+                const double nu = x - (double)m;
+                const double tbt = table_at(p->tbt + ct * M, M, r, om, m, nu);
+                const double pw = table_at(p->pw + ct * M, M, r, om, m, nu);
+                const double slo_a = (double)sp->slo_ttft[c], slo_b = (double)sp->slo_tbt[c];
+                int ok = (ttft <= slo_a) && (tbt <= slo_b) && (u <= 1.0);
+                if (sp->gpu_budget > 0 && n * p->tp[t] > sp->gpu_budget) ok = 0;
+                E[j] = ok ? (double)n * pw * (double)sp->window_s / 3600.0 : INFINITY;
+                if (tbt_out) tbt_out[j] = tbt;
+                if (pow_out) pow_out[j] = pw;
+                if (u_out) u_out[j] = u;
+                double d1 = fabs(tbt - slo_b) / slo_b, d2 = fabs(u - 1.0), d3 = fabs(ttft - slo_a) / slo_a;
+                if (d1 < mg) mg = d1;
+                if (d2 < mg) mg = d2;
+                if (d3 < mg) mg = d3;
+            }
+        }
+    }
+    if (margin) *margin = mg;
+}
+
+/* ---- stage (c): masked argmin, totals ----------------------------------------------------- */
+
+/* smallest j attaining the minimum of E[0..J); -1 if the minimum is +inf.  *E2 = minimum over
+   the other indices (+inf if none). */
+void orc_select_row(const double *E, int64_t J, int32_t *best_idx, double *best_E, double *E2) {
+    int64_t jb = -1;
+    double eb = INFINITY;
+    for (int64_t j = 0; j < J; ++j)
+        if (E[j] < eb) { eb = E[j]; jb = j; }
+    double e2 = INFINITY;
+    for (int64_t j = 0; j < J; ++j)
+        if (j != jb && E[j] < e2) e2 = E[j];
+    *best_idx = (int32_t)jb;
+    *best_E = eb;
+    if (E2) *E2 = e2;
+}
+
+/* E tensor [S][W][C][J] for loads [S][W][C] */
+int orc_eval_configs(const orc_profile *p, const orc_space *sp, const float *load, int64_t S, int64_t W,
+                     double *E) {
+    const int32_t C = p->C;
+    const int64_t J = (int64_t)sp->Nmax * p->T * sp->F;
+    int32_t *row = (int32_t *)malloc(sizeof(int32_t) * (size_t)sp->F);
+    double *wt = (double *)malloc(sizeof(double) * (size_t)sp->F);
+    int rc = orc_resolve(p->f_grid, p->R, sp->f_cand, sp->F, row, wt);
+    if (rc == ORC_OK) {
+        const int64_t tiles = S * W * C;
+#pragma omp parallel for schedule(static)
+        for (int64_t i = 0; i < tiles; ++i)
+            orc_eval_tile(p, sp, row, wt, (int32_t)(i % C), (double)load[i], E + i * J, NULL, NULL, NULL, NULL);
+    }
+    free(row); free(wt);
+    return rc;
+}
+
+/* per tile: argmin of a materialised E tensor */
+void orc_select(const double *E, int64_t tiles, int64_t J, int32_t *best_idx, double *best_E, double *E2) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < tiles; ++i)
+        orc_select_row(E + i * J, J, best_idx + i, best_E + i, E2 ? E2 + i : NULL);
+}
+
+/* evaluate then select, tile by tile (the row of J energies lives only inside the loop body) */
+int orc_eval_select(const orc_profile *p, const orc_space *sp, const float *load, int64_t S, int64_t W,
+                    int32_t *best_idx, double *best_E, double *E2, double *margin) {
+    const int32_t C = p->C;
+    const int64_t J = (int64_t)sp->Nmax * p->T * sp->F;
+    int32_t *row = (int32_t *)malloc(sizeof(int32_t) * (size_t)sp->F);
+    double *wt = (double *)malloc(sizeof(double) * (size_t)sp->F);
+    int rc = orc_resolve(p->f_grid, p->R, sp->f_cand, sp->F, row, wt);
+    if (rc == ORC_OK) {
+        const int64_t tiles = S * W * C;
+#pragma omp parallel
+        {
+            double *Erow = (double *)malloc(sizeof(double) * (size_t)J);
+#pragma omp for schedule(static)
+            for (int64_t i = 0; i < tiles; ++i) {
+                orc_eval_tile(p, sp, row, wt, (int32_t)(i % C), (double)load[i], Erow, NULL, NULL, NULL,
+                              margin ? margin + i : NULL);
+                orc_select_row(Erow, J, best_idx + i, best_E + i, E2 ? E2 + i : NULL);
+            }
+            free(Erow);
+        }
+    }
+    free(row); free(wt);
+    return rc;
+}
+
+/*
+ * Totals per scenario, summed in (w, c) order in fp64 over tiles that have a feasible candidate.
+ * E_window[S][W], hist[S][J], gpus[S][W] optional (NULL to skip); n_of_j / tp_of_j give the
+ * instance count and TP degree of candidate j (needed for gpus only).
+ */
+void orc_totals(const int32_t *best_idx, const double *best_E, int64_t S, int64_t W, int32_t C, int64_t J,
+                const int32_t *n_of_j, const int32_t *tp_of_j,
+                double *E_total, uint32_t *n_infeasible, double *E_window, uint32_t *hist, uint32_t *gpus) {
+    if (hist) memset(hist, 0, sizeof(uint32_t) * (size_t)(S * J));
+    for (int64_t s = 0; s < S; ++s) {
+        double tot = 0.0;
+        uint32_t bad = 0;
+        for (int64_t w = 0; w < W; ++w) {
+            double ew = 0.0;
+            uint32_t g = 0;
+            for (int32_t c = 0; c < C; ++c) {
+                const int64_t i = (s * W + w) * C + c;
+                const int32_t j = best_idx[i];
+                if (j < 0) { ++bad; continue; }
+                tot += best_E[i];
+                ew += best_E[i];
+                if (hist) hist[s * J + j] += 1u;
+                if (gpus && n_of_j && tp_of_j) g += (uint32_t)(n_of_j[j] * tp_of_j[j]);
+            }
+            if (E_window) E_window[s * W + w] = ew;
+            if (gpus) gpus[s * W + w] = g;
+        }
+        E_total[s] = tot;
+        n_infeasible[s] = bad;
+    }
+}
