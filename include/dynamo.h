@@ -1,0 +1,177 @@
+/*
+ * dynamo.h -- C ABI of the B200 configuration-sweep library (libdynamo.so).
+ *
+ * The library evaluates, on one GPU, the search that DynamoLLM (arXiv 2408.00741) states in
+ * Sec. 4.1 / Eq. 1 and Sec. 4.2: for every request class and time window, every candidate
+ * (number of instances N, tensor-parallel degree TP, GPU frequency f) is checked against the
+ * profile-derived latency model and the SLOs, its energy is computed, and the minimum-energy
+ * feasible candidate is chosen.  Three stages:
+ *
+ *   (a) dyn_bin_trace     trace (timestamp, input tokens, output tokens) -> per-(window, class)
+ *                         request counts and loads                      [Sec. 3, Sec. 3.1, Sec. 3.2]
+ *   (b) dyn_eval_configs  loads x candidates -> energy tensor with +inf where a constraint of Eq. 1
+ *                         fails                                         [Sec. 4.1, Eq. 1]
+ *   (c) dyn_select        masked argmin per (window, class) + cluster totals      [Sec. 4.2, Sec. 6]
+ *       dyn_eval_select   (b)+(c) fused, no energy tensor
+ *
+ * Conventions for every call
+ *   - returns DYN_OK (0) or a negative dyn_status; never throws, never aborts, never traps the GPU;
+ *   - work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = default stream) and the
+ *     call returns without synchronising; results are valid once the stream reaches that point;
+ *   - pointers named d_* are DEVICE pointers owned by the caller; all other pointers are HOST
+ *     pointers that are read before the call returns; the library allocates nothing;
+ *   - tensors are dense, row-major, in the index order written in brackets;
+ *   - candidate index  j = ((n-1)*T + t)*F + q  with n = 1..Nmax (slowest), t = TP index, q =
+ *     frequency index (fastest); J = Nmax*T*F.  Ties in energy go to the lowest j.
+ *   - argument errors are detected on the host before anything is enqueued.
+ */
+#ifndef DYNAMO_H_
+#define DYNAMO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DYN_OK = 0,
+    DYN_EINVAL = -1,        /* NULL required pointer, bad size, non-ascending edges / grids, ... */
+    DYN_ECUDA = -2,         /* a CUDA runtime call failed; see dyn_last_cuda_error() */
+    DYN_EUNSUPPORTED = -3,  /* valid request outside the built limits (see each call) */
+    DYN_EWORKSPACE = -4     /* workspace missing, misaligned (256 B) or smaller than dyn_workspace_bytes() */
+} dyn_status;
+
+/* Static, human-readable text for a status code. */
+const char *dyn_strerror(int status);
+
+/* cudaError_t (as int) behind the most recent DYN_ECUDA returned on the calling thread, else 0. */
+int dyn_last_cuda_error(void);
+
+/* Limits the library was built with. */
+#define DYN_MAX_EDGES 15      /* per axis: at most 16 x 16 classes */
+#define DYN_MAX_F 256         /* candidate frequencies */
+#define DYN_MAX_T 16          /* TP degrees */
+
+/* ---------------------------------------------------------------------------------------------
+ * (a) Trace binning.  [Sec. 3: a trace record is (timestamp, #input tokens, #output tokens);
+ *     Sec. 3.1 and its thresholds table: 3 x 3 length classes; Sec. 3.2: load per class over time]
+ *
+ * Request i falls in window w = t_ms[i] / window_ms (unsigned integer division) and class
+ * c = ci*KO + co, where ci = number of in_edges <= in_tok[i], co likewise, KI = n_in_edges+1,
+ * KO = n_out_edges+1, C = KI*KO.  With in_edges {256, 1024} and out_edges {100, 350} this is the
+ * paper's SS, SM, SL, MS, ..., LL order.  Requests with w >= n_windows are counted in *d_dropped.
+ * The trace need not be sorted; a time-sorted trace is the fast case.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+    uint32_t window_ms;          /* > 0 */
+    uint32_t n_windows;          /* W > 0 */
+    int32_t n_in_edges;          /* 0 .. DYN_MAX_EDGES */
+    int32_t n_out_edges;         /* 0 .. DYN_MAX_EDGES */
+    const uint32_t *in_edges;    /* host, strictly ascending */
+    const uint32_t *out_edges;   /* host, strictly ascending */
+} dyn_bin_spec;
+
+/*
+ * d_t_ms, d_in_tok, d_out_tok : device, uint32 [n_req] each (structure of arrays), read only.
+ * d_counts  : device, uint32 [W][C], overwritten (exact counts; W*C must be < 2^31).
+ * d_load    : device, float  [W][C] = (float)count / (window_ms/1000 as float), or NULL to skip.
+ * d_dropped : device, uint64 [1], overwritten.
+ * n_req may be 0.  Errors: DYN_EINVAL (NULL pointer, window_ms or n_windows 0, edges not strictly
+ * ascending, too many edges, W*C >= 2^31), DYN_ECUDA.
+ */
+int dyn_bin_trace(const dyn_bin_spec *spec, const uint32_t *d_t_ms, const uint32_t *d_in_tok,
+                  const uint32_t *d_out_tok, uint64_t n_req, uint32_t *d_counts, float *d_load,
+                  uint64_t *d_dropped, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * (b) Profiles and the candidate space.  [Sec. 4.1 "Generating LLM profiles": the profile maps
+ *     (load, request class, TP, frequency) to energy/power and TTFT/TBT, measured at a few
+ *     frequencies and load levels and interpolated linearly in between.]
+ *
+ * Tables hold, per class c, TP index t and profiled frequency row r:
+ *   ttft[c][t][r]      time to first token (s)
+ *   cap[c][t][r]       largest per-instance load the instance sustains (requests/s), > 0
+ *   tbt[c][t][r][m]    time between tokens (s) at utilisation u_m = m/(M-1), m = 0..M-1
+ *   pow[c][t][r][m]    power of one instance (W) at utilisation u_m
+ * A candidate frequency between two rows is interpolated linearly in f, utilisation linearly in
+ * u (bilinear overall).  NaN table entries give unspecified results.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t C, T, R, M;          /* classes, TP degrees (<= DYN_MAX_T), frequency rows (>= 2), knots (>= 2) */
+    const int32_t *tp;           /* host [T], strictly ascending, > 0 */
+    const float *f_grid_mhz;     /* host [R], strictly ascending */
+    const float *d_ttft;         /* device [C][T][R] */
+    const float *d_cap;          /* device [C][T][R] */
+    const float *d_tbt;          /* device [C][T][R][M] */
+    const float *d_pow;          /* device [C][T][R][M] */
+} dyn_profile;
+
+typedef struct {
+    int32_t F, Nmax;             /* 1 <= F <= DYN_MAX_F; Nmax >= 1; Nmax*T*F < 2^31 */
+    const float *f_cand_mhz;     /* host [F], strictly ascending, inside [f_grid[0], f_grid[R-1]] */
+    const float *slo_ttft_s;     /* host [C] */
+    const float *slo_tbt_s;      /* host [C] */
+    int32_t gpu_budget;          /* Eq. 1 first constraint: n*TP <= gpu_budget; <= 0 means no budget */
+    float window_s;              /* window length in seconds (energy is Wh per window) */
+} dyn_space;
+
+/*
+ * Evaluation of one candidate for a tile (s, w, c) with load L = d_load[s][w][c]   [Eq. 1]:
+ *   l = L/n (fair share),  u = l / cap(c,t,f),  TBT and P interpolated at (f, min(u,1));
+ *   feasible  <=>  TTFT(c,t,f) <= slo_ttft[c]  and  TBT <= slo_tbt[c]  and  u <= 1
+ *                  and (gpu_budget <= 0 or n*TP_t <= gpu_budget);
+ *   E = n * P * window_s / 3600  (Wh)  if feasible, +inf otherwise.
+ * Arithmetic is fp32; results agree with an fp64 evaluation to about 1e-6 relative, and the
+ * feasibility decision can differ where a deciding quantity is within rounding of its bound.
+ */
+
+/* Scratch memory (bytes, multiple of 256) that dyn_eval_configs / dyn_select / dyn_eval_select need
+ * for this problem shape; d_ws must be 256-byte aligned.  The scratch holds the candidate-resolved
+ * tables and partial sums; its contents are meaningless between calls.  Returns 0 on bad input. */
+size_t dyn_workspace_bytes(const dyn_profile *profile, const dyn_space *space, int64_t S, int64_t W);
+
+/*
+ * d_load : device float [S][W][C] (requests/s, >= 0).   d_E : device float [S][W][C][J], overwritten.
+ * Errors: DYN_EINVAL, DYN_EUNSUPPORTED (F > DYN_MAX_F, T > DYN_MAX_T, candidate frequency outside the
+ * grid), DYN_EWORKSPACE, DYN_ECUDA.
+ */
+int dyn_eval_configs(const dyn_profile *profile, const dyn_space *space, const float *d_load,
+                     int64_t S, int64_t W, float *d_E, void *d_ws, size_t ws_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * (c) Selection and totals.  [Sec. 4.2 scale-up/down: drop the settings that violate the SLO, then
+ *     take the one with the least energy; Sec. 6: cluster energy over time, GPUs in use.]
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t *d_best_idx;         /* [S][W][C] chosen j, -1 if no candidate is feasible; required */
+    float *d_best_E;             /* [S][W][C] its energy (Wh), +inf if none; required */
+    double *d_E_total;           /* [S] sum of chosen energies over feasible tiles; required */
+    uint32_t *d_n_infeasible;    /* [S] tiles without a feasible candidate; required */
+    double *d_E_window;          /* [S][W] energy per window, or NULL */
+    uint32_t *d_hist;            /* [S][J] how often each candidate was chosen, or NULL */
+    uint32_t *d_gpus;            /* [S][W] sum over classes of n* x TP*, or NULL */
+} dyn_select_out;
+
+/*
+ * Argmin over a materialised energy tensor d_E [S][W][C][J] (+inf = infeasible).
+ * n_of_j, tp_of_j : host int32 [J], instance count and TP degree of candidate j; needed only when
+ * out->d_gpus is set (else may be NULL).  Sums are fp64, accumulated in a fixed order: results are
+ * bit-identical from run to run.  Workspace: dyn_select_workspace_bytes(S, W, J).
+ */
+size_t dyn_select_workspace_bytes(int64_t S, int64_t W, int64_t J);
+int dyn_select(const float *d_E, int64_t S, int64_t W, int32_t C, int32_t J, const int32_t *n_of_j,
+               const int32_t *tp_of_j, const dyn_select_out *out, void *d_ws, size_t ws_bytes,
+               void *stream);
+
+/* (b)+(c) in one pass: same results as dyn_eval_configs followed by dyn_select, without the
+ * [S][W][C][J] tensor (which need not fit in memory).  Workspace: dyn_workspace_bytes(). */
+int dyn_eval_select(const dyn_profile *profile, const dyn_space *space, const float *d_load,
+                    int64_t S, int64_t W, const dyn_select_out *out, void *d_ws, size_t ws_bytes,
+                    void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DYNAMO_H_ */

@@ -1,0 +1,217 @@
+"""ctypes binding of libdynamo.so: same names as the C ABI, argument marshalling only.
+
+Device buffers are torch CUDA tensors (torch is used for device memory and streams, nothing else);
+host-side descriptors (class edges, TP list, frequency grids, SLOs) are numpy arrays.  Every call
+enqueues on torch's current stream and returns without synchronising.  There is no CPU path: if the
+shared library has not been built the import of this module fails.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "csrc", "libdynamo.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2408_00741_b200.build` "
+                      "(there is no fallback implementation)")
+_lib = C.CDLL(LIB_PATH)
+
+DYN_OK, DYN_EINVAL, DYN_ECUDA, DYN_EUNSUPPORTED, DYN_EWORKSPACE = 0, -1, -2, -3, -4
+EXPORTS = ("dyn_strerror", "dyn_last_cuda_error", "dyn_bin_trace", "dyn_workspace_bytes", "dyn_eval_configs",
+           "dyn_select_workspace_bytes", "dyn_select", "dyn_eval_select")
+
+
+class DynError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = _lib.dyn_strerror(status).decode()
+        if status == DYN_ECUDA:
+            msg += f" [cudaError {_lib.dyn_last_cuda_error()}]"
+        super().__init__(f"{where}: {msg} ({status})")
+
+
+class _BinSpec(C.Structure):
+    _fields_ = [("window_ms", C.c_uint32), ("n_windows", C.c_uint32), ("n_in_edges", C.c_int32),
+                ("n_out_edges", C.c_int32), ("in_edges", C.c_void_p), ("out_edges", C.c_void_p)]
+
+
+class _Profile(C.Structure):
+    _fields_ = [("C", C.c_int32), ("T", C.c_int32), ("R", C.c_int32), ("M", C.c_int32),
+                ("tp", C.c_void_p), ("f_grid_mhz", C.c_void_p), ("d_ttft", C.c_void_p), ("d_cap", C.c_void_p),
+                ("d_tbt", C.c_void_p), ("d_pow", C.c_void_p)]
+
+
+class _Space(C.Structure):
+    _fields_ = [("F", C.c_int32), ("Nmax", C.c_int32), ("f_cand_mhz", C.c_void_p), ("slo_ttft_s", C.c_void_p),
+                ("slo_tbt_s", C.c_void_p), ("gpu_budget", C.c_int32), ("window_s", C.c_float)]
+
+
+class _SelectOut(C.Structure):
+    _fields_ = [("d_best_idx", C.c_void_p), ("d_best_E", C.c_void_p), ("d_E_total", C.c_void_p),
+                ("d_n_infeasible", C.c_void_p), ("d_E_window", C.c_void_p), ("d_hist", C.c_void_p),
+                ("d_gpus", C.c_void_p)]
+
+
+_lib.dyn_strerror.restype = C.c_char_p
+_lib.dyn_strerror.argtypes = [C.c_int]
+_lib.dyn_last_cuda_error.restype = C.c_int
+_lib.dyn_bin_trace.restype = C.c_int
+_lib.dyn_bin_trace.argtypes = [C.POINTER(_BinSpec), C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p,
+                               C.c_void_p, C.c_void_p, C.c_void_p]
+_lib.dyn_workspace_bytes.restype = C.c_size_t
+_lib.dyn_workspace_bytes.argtypes = [C.POINTER(_Profile), C.POINTER(_Space), C.c_int64, C.c_int64]
+_lib.dyn_eval_configs.restype = C.c_int
+_lib.dyn_eval_configs.argtypes = [C.POINTER(_Profile), C.POINTER(_Space), C.c_void_p, C.c_int64, C.c_int64,
+                                  C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+_lib.dyn_select_workspace_bytes.restype = C.c_size_t
+_lib.dyn_select_workspace_bytes.argtypes = [C.c_int64, C.c_int64, C.c_int64]
+_lib.dyn_select.restype = C.c_int
+_lib.dyn_select.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                            C.POINTER(_SelectOut), C.c_void_p, C.c_size_t, C.c_void_p]
+_lib.dyn_eval_select.restype = C.c_int
+_lib.dyn_eval_select.argtypes = [C.POINTER(_Profile), C.POINTER(_Space), C.c_void_p, C.c_int64, C.c_int64,
+                                 C.POINTER(_SelectOut), C.c_void_p, C.c_size_t, C.c_void_p]
+
+
+def _dev(t, dtype, what):
+    if t is None:
+        return None
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError(f"{what}: expected a contiguous CUDA tensor of {dtype}")
+    return t.data_ptr()
+
+
+def _host(a, dtype):
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(rc, where):
+    if rc != DYN_OK:
+        raise DynError(rc, where)
+
+
+class Profile:
+    """Device-resident profile tables plus their host descriptors (mirrors dyn_profile)."""
+
+    def __init__(self, tp, f_grid_mhz, ttft, cap, tbt, pow, device="cuda"):
+        self.tp = _host(tp, np.int32)
+        self.f_grid_mhz = _host(f_grid_mhz, np.float32)
+        as_dev = lambda x: (x if isinstance(x, torch.Tensor) else torch.from_numpy(_host(x, np.float32))).to(
+            device=device, dtype=torch.float32).contiguous()
+        self.d_ttft, self.d_cap, self.d_tbt, self.d_pow = as_dev(ttft), as_dev(cap), as_dev(tbt), as_dev(pow)
+        self.C, self.T, self.R = self.d_ttft.shape
+        self.M = self.d_tbt.shape[3]
+        if (tuple(self.d_tbt.shape) != (self.C, self.T, self.R, self.M) or tuple(self.d_pow.shape) != tuple(self.d_tbt.shape)
+                or tuple(self.d_cap.shape) != (self.C, self.T, self.R) or len(self.tp) != self.T
+                or len(self.f_grid_mhz) != self.R):
+            raise ValueError("profile tables have inconsistent shapes")
+
+    def _struct(self):
+        return _Profile(self.C, self.T, self.R, self.M, self.tp.ctypes.data, self.f_grid_mhz.ctypes.data,
+                        self.d_ttft.data_ptr(), self.d_cap.data_ptr(), self.d_tbt.data_ptr(), self.d_pow.data_ptr())
+
+
+class Space:
+    """Candidate space and SLOs (mirrors dyn_space); host data only."""
+
+    def __init__(self, f_cand_mhz, n_max, slo_ttft_s, slo_tbt_s, window_s, gpu_budget=0):
+        self.f_cand_mhz = _host(f_cand_mhz, np.float32)
+        self.n_max = int(n_max)
+        self.slo_ttft_s = _host(slo_ttft_s, np.float32)
+        self.slo_tbt_s = _host(slo_tbt_s, np.float32)
+        self.window_s = float(window_s)
+        self.gpu_budget = int(gpu_budget)
+
+    @property
+    def F(self):
+        return len(self.f_cand_mhz)
+
+    def _struct(self):
+        return _Space(self.F, self.n_max, self.f_cand_mhz.ctypes.data, self.slo_ttft_s.ctypes.data,
+                      self.slo_tbt_s.ctypes.data, self.gpu_budget, self.window_s)
+
+
+def dyn_bin_trace(window_ms, n_windows, in_edges, out_edges, d_t_ms, d_in_tok, d_out_tok, d_counts, d_load, d_dropped,
+                  n_req=None):
+    """Counts (uint32 viewed as int32 tensor [W][C]), loads (float32 or None), dropped (int64 [1])."""
+    ie, oe = _host(in_edges, np.uint32), _host(out_edges, np.uint32)
+    spec = _BinSpec(int(window_ms), int(n_windows), len(ie), len(oe), ie.ctypes.data, oe.ctypes.data)
+    n = int(d_t_ms.numel() if n_req is None else n_req)
+    rc = _lib.dyn_bin_trace(C.byref(spec), _dev(d_t_ms, torch.int32, "d_t_ms"), _dev(d_in_tok, torch.int32, "d_in_tok"),
+                            _dev(d_out_tok, torch.int32, "d_out_tok"), n, _dev(d_counts, torch.int32, "d_counts"),
+                            _dev(d_load, torch.float32, "d_load"), _dev(d_dropped, torch.int64, "d_dropped"), _stream())
+    _check(rc, "dyn_bin_trace")
+
+
+def dyn_workspace_bytes(profile: Profile, space: Space, S, W) -> int:
+    p, s = profile._struct(), space._struct()
+    return int(_lib.dyn_workspace_bytes(C.byref(p), C.byref(s), int(S), int(W)))
+
+
+def dyn_select_workspace_bytes(S, W, J) -> int:
+    return int(_lib.dyn_select_workspace_bytes(int(S), int(W), int(J)))
+
+
+def _ws(d_ws):
+    if d_ws is None:
+        return None, 0
+    if not (isinstance(d_ws, torch.Tensor) and d_ws.is_cuda and d_ws.is_contiguous()):
+        raise TypeError("d_ws: expected a contiguous CUDA tensor")
+    return d_ws.data_ptr(), d_ws.numel() * d_ws.element_size()
+
+
+def dyn_eval_configs(profile: Profile, space: Space, d_load, d_E, d_ws):
+    S, W, Cn = d_load.shape
+    p, s = profile._struct(), space._struct()
+    ws, nb = _ws(d_ws)
+    rc = _lib.dyn_eval_configs(C.byref(p), C.byref(s), _dev(d_load, torch.float32, "d_load"), S, W,
+                               _dev(d_E, torch.float32, "d_E"), ws, nb, _stream())
+    _check(rc, "dyn_eval_configs")
+
+
+class SelectOut:
+    """Output buffers of the selection stage (mirrors dyn_select_out)."""
+
+    def __init__(self, S, W, Cn, J, device="cuda", windows=True, hist=True, gpus=True):
+        self.best_idx = torch.empty((S, W, Cn), dtype=torch.int32, device=device)
+        self.best_E = torch.empty((S, W, Cn), dtype=torch.float32, device=device)
+        self.E_total = torch.empty((S,), dtype=torch.float64, device=device)
+        self.n_infeasible = torch.empty((S,), dtype=torch.int32, device=device)
+        self.E_window = torch.empty((S, W), dtype=torch.float64, device=device) if windows else None
+        self.hist = torch.empty((S, J), dtype=torch.int32, device=device) if hist else None
+        self.gpus = torch.empty((S, W), dtype=torch.int32, device=device) if gpus else None
+
+    def _struct(self):
+        ptr = lambda t: t.data_ptr() if t is not None else None
+        return _SelectOut(ptr(self.best_idx), ptr(self.best_E), ptr(self.E_total), ptr(self.n_infeasible),
+                          ptr(self.E_window), ptr(self.hist), ptr(self.gpus))
+
+
+def dyn_select(d_E, out: SelectOut, d_ws, n_of_j=None, tp_of_j=None):
+    S, W, Cn, J = d_E.shape
+    nj = _host(n_of_j, np.int32) if n_of_j is not None else None
+    tj = _host(tp_of_j, np.int32) if tp_of_j is not None else None
+    o = out._struct()
+    ws, nb = _ws(d_ws)
+    rc = _lib.dyn_select(_dev(d_E, torch.float32, "d_E"), S, W, Cn, J, nj.ctypes.data if nj is not None else None,
+                         tj.ctypes.data if tj is not None else None, C.byref(o), ws, nb, _stream())
+    _check(rc, "dyn_select")
+
+
+def dyn_eval_select(profile: Profile, space: Space, d_load, out: SelectOut, d_ws):
+    S, W, Cn = d_load.shape
+    p, s = profile._struct(), space._struct()
+    o = out._struct()
+    ws, nb = _ws(d_ws)
+    rc = _lib.dyn_eval_select(C.byref(p), C.byref(s), _dev(d_load, torch.float32, "d_load"), S, W, C.byref(o), ws, nb,
+                              _stream())
+    _check(rc, "dyn_eval_select")

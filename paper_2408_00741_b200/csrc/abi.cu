@@ -1,0 +1,240 @@
+// Host side of the C ABI declared in include/dynamo.h: argument validation and launch sequencing.
+// Every step of the path runs in the kernels of this library; nothing here computes results.
+#include "dyn_internal.cuh"
+
+#include <cmath>
+#include <cstring>
+
+namespace dyn {
+
+static thread_local int tls_cuda_error = 0;
+void set_last_cuda_error(cudaError_t e) { tls_cuda_error = int(e); }
+
+int sm_count() {
+    // per device, cached on first use
+    static thread_local int cached_dev = -1, cached = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (dev != cached_dev) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+        cached = v;
+        cached_dev = dev;
+    }
+    return cached;
+}
+
+namespace {
+
+bool strictly_ascending_u32(const uint32_t *v, int n) {
+    for (int i = 1; i < n; ++i)
+        if (!(v[i - 1] < v[i])) return false;
+    return true;
+}
+
+bool strictly_ascending_f32(const float *v, int n) {
+    for (int i = 0; i < n; ++i)
+        if (!std::isfinite(v[i])) return false;
+    for (int i = 1; i < n; ++i)
+        if (!(v[i - 1] < v[i])) return false;
+    return true;
+}
+
+// shape checks shared by the evaluation entry points; fills the resolve parameters
+int check_problem(const dyn_profile *p, const dyn_space *sp, int64_t S, int64_t W, ResolveParams *rp) {
+    if (!p || !sp) return DYN_EINVAL;
+    if (p->C < 1 || p->T < 1 || p->R < 2 || p->M < 2 || sp->F < 1 || sp->Nmax < 1) return DYN_EINVAL;
+    if (S < 0 || W < 0) return DYN_EINVAL;
+    if (!p->tp || !p->f_grid_mhz || !p->d_ttft || !p->d_cap || !p->d_tbt || !p->d_pow) return DYN_EINVAL;
+    if (!sp->f_cand_mhz || !sp->slo_ttft_s || !sp->slo_tbt_s) return DYN_EINVAL;
+    if (!(sp->window_s > 0.f) || !std::isfinite(sp->window_s)) return DYN_EINVAL;
+    if (p->T > DYN_MAX_T || sp->F > DYN_MAX_F || p->C > 256 || sp->Nmax > 256 || p->M > 4096 || p->R > 32767)
+        return DYN_EUNSUPPORTED;
+    for (int t = 0; t < p->T; ++t) {
+        if (p->tp[t] <= 0) return DYN_EINVAL;
+        if (t > 0 && !(p->tp[t - 1] < p->tp[t])) return DYN_EINVAL;
+    }
+    if (!strictly_ascending_f32(p->f_grid_mhz, p->R) || !strictly_ascending_f32(sp->f_cand_mhz, sp->F))
+        return DYN_EINVAL;
+    const int64_t J = int64_t(sp->Nmax) * p->T * sp->F;
+    if (J >= (int64_t(1) << 31)) return DYN_EINVAL;
+    if (S > 0 && W > 0 && (S > (int64_t(1) << 40) / W || S * W > (int64_t(1) << 40) / p->C)) return DYN_EINVAL;
+    if (sp->f_cand_mhz[0] < p->f_grid_mhz[0] || sp->f_cand_mhz[sp->F - 1] > p->f_grid_mhz[p->R - 1])
+        return DYN_EUNSUPPORTED;
+    if (!rp) return DYN_OK;
+
+    std::memset(rp, 0, sizeof(*rp));
+    rp->C = p->C; rp->T = p->T; rp->R = p->R; rp->M = p->M; rp->F = sp->F;
+    rp->d_ttft = p->d_ttft; rp->d_cap = p->d_cap; rp->d_tbt = p->d_tbt; rp->d_pow = p->d_pow;
+    rp->window_s = sp->window_s;
+    for (int q = 0; q < sp->F; ++q) {
+        // largest row r <= R-2 whose frequency is <= the candidate; weight in [0, 1]
+        const double f = double(sp->f_cand_mhz[q]);
+        int r = 0;
+        for (int i = 0; i <= p->R - 2; ++i)
+            if (double(p->f_grid_mhz[i]) <= f) r = i;
+        rp->row[q] = int16_t(r);
+        rp->weight[q] = float((f - double(p->f_grid_mhz[r])) / (double(p->f_grid_mhz[r + 1]) - double(p->f_grid_mhz[r])));
+    }
+    for (int c = 0; c < p->C; ++c) {
+        rp->slo_ttft[c] = sp->slo_ttft_s[c];
+        rp->slo_tbt[c] = sp->slo_tbt_s[c];
+    }
+    for (int t = 0; t < p->T; ++t) rp->tp[t] = p->tp[t];
+    return DYN_OK;
+}
+
+int check_out(const dyn_select_out *o) {
+    if (!o || !o->d_best_idx || !o->d_best_E || !o->d_E_total || !o->d_n_infeasible) return DYN_EINVAL;
+    return DYN_OK;
+}
+
+SelectOut to_out(const dyn_select_out *o) {
+    SelectOut s;
+    s.best_idx = o->d_best_idx; s.best_E = o->d_best_E; s.E_total = o->d_E_total;
+    s.n_infeasible = o->d_n_infeasible; s.E_window = o->d_E_window; s.hist = o->d_hist; s.gpus = o->d_gpus;
+    return s;
+}
+
+int check_ws(const void *d_ws, size_t ws_bytes, size_t need) {
+    if (need == 0) return DYN_OK;
+    if (!d_ws || (reinterpret_cast<uintptr_t>(d_ws) & 255u) != 0 || ws_bytes < need) return DYN_EWORKSPACE;
+    return DYN_OK;
+}
+
+size_t align256(size_t x) { return (x + 255) / 256 * 256; }
+
+}  // namespace
+}  // namespace dyn
+
+using namespace dyn;
+
+extern "C" {
+
+const char *dyn_strerror(int status) {
+    switch (status) {
+        case DYN_OK: return "success";
+        case DYN_EINVAL: return "invalid argument";
+        case DYN_ECUDA: return "CUDA runtime error (see dyn_last_cuda_error)";
+        case DYN_EUNSUPPORTED: return "request outside the built limits";
+        case DYN_EWORKSPACE: return "workspace missing, misaligned or too small";
+        default: return "unknown status";
+    }
+}
+
+int dyn_last_cuda_error(void) { return tls_cuda_error; }
+
+int dyn_bin_trace(const dyn_bin_spec *spec, const uint32_t *d_t_ms, const uint32_t *d_in_tok,
+                  const uint32_t *d_out_tok, uint64_t n_req, uint32_t *d_counts, float *d_load,
+                  uint64_t *d_dropped, void *stream) {
+    if (!spec || !d_counts || !d_dropped) return DYN_EINVAL;
+    if (n_req > 0 && (!d_t_ms || !d_in_tok || !d_out_tok)) return DYN_EINVAL;
+    if (spec->window_ms == 0 || spec->n_windows == 0) return DYN_EINVAL;
+    if (spec->n_in_edges < 0 || spec->n_out_edges < 0 || spec->n_in_edges > DYN_MAX_EDGES ||
+        spec->n_out_edges > DYN_MAX_EDGES)
+        return DYN_EINVAL;
+    if ((spec->n_in_edges > 0 && !spec->in_edges) || (spec->n_out_edges > 0 && !spec->out_edges)) return DYN_EINVAL;
+    if (!strictly_ascending_u32(spec->in_edges, spec->n_in_edges) ||
+        !strictly_ascending_u32(spec->out_edges, spec->n_out_edges))
+        return DYN_EINVAL;
+    BinParams bp;
+    std::memset(&bp, 0, sizeof(bp));
+    bp.win = make_fastdiv(spec->window_ms);
+    bp.n_windows = spec->n_windows;
+    bp.n_in = spec->n_in_edges;
+    bp.n_out = spec->n_out_edges;
+    bp.C = (bp.n_in + 1) * (bp.n_out + 1);
+    if (uint64_t(spec->n_windows) * uint64_t(bp.C) >= (uint64_t(1) << 31)) return DYN_EINVAL;
+    for (int e = 0; e < bp.n_in; ++e) bp.in_edges[e] = spec->in_edges[e];
+    for (int e = 0; e < bp.n_out; ++e) bp.out_edges[e] = spec->out_edges[e];
+    bp.window_s = float(spec->window_ms) / 1000.0f;
+    DYN_CUDA_TRY(launch_bin_trace(bp, d_t_ms, d_in_tok, d_out_tok, n_req, d_counts, d_load,
+                                  reinterpret_cast<unsigned long long *>(d_dropped),
+                                  static_cast<cudaStream_t>(stream)));
+    return DYN_OK;
+}
+
+size_t dyn_workspace_bytes(const dyn_profile *profile, const dyn_space *space, int64_t S, int64_t W) {
+    if (!profile || !space) return 0;
+    if (profile->C < 1 || profile->T < 1 || profile->M < 2 || space->F < 1 || space->Nmax < 1 || S < 0 || W < 0)
+        return 0;
+    return resolved_layout(profile->C, profile->T, space->F, profile->M, space->Nmax, S, W).total;
+}
+
+int dyn_eval_configs(const dyn_profile *profile, const dyn_space *space, const float *d_load, int64_t S, int64_t W,
+                     float *d_E, void *d_ws, size_t ws_bytes, void *stream) {
+    ResolveParams rp;
+    int rc = check_problem(profile, space, S, W, &rp);
+    if (rc != DYN_OK) return rc;
+    const int64_t tiles = S * W * profile->C;
+    if (tiles > 0 && (!d_load || !d_E)) return DYN_EINVAL;
+    const ResolvedLayout lay = resolved_layout(profile->C, profile->T, space->F, profile->M, space->Nmax, S, W);
+    rc = check_ws(d_ws, ws_bytes, lay.total);
+    if (rc != DYN_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    DYN_CUDA_TRY(launch_resolve(rp, lay, d_ws, st));
+    DYN_CUDA_TRY(launch_eval_configs(lay, d_ws, d_load, tiles, space->gpu_budget, d_E, st));
+    return DYN_OK;
+}
+
+size_t dyn_select_workspace_bytes(int64_t S, int64_t W, int64_t J) {
+    if (S < 0 || W < 0 || J < 0) return 0;
+    const size_t partial = align256(size_t(S) * size_t(totals_chunks(W)) * (sizeof(double) + sizeof(uint32_t)));
+    return partial + 2 * align256(size_t(J) * sizeof(int32_t));
+}
+
+int dyn_select(const float *d_E, int64_t S, int64_t W, int32_t C, int32_t J, const int32_t *n_of_j,
+               const int32_t *tp_of_j, const dyn_select_out *out, void *d_ws, size_t ws_bytes, void *stream) {
+    if (S < 0 || W < 0 || C < 1 || J < 1) return DYN_EINVAL;
+    int rc = check_out(out);
+    if (rc != DYN_OK) return rc;
+    if (out->d_gpus && (!n_of_j || !tp_of_j)) return DYN_EINVAL;
+    if (S > 0 && W > 0 && (S > (int64_t(1) << 40) / W || S * W > (int64_t(1) << 40) / C)) return DYN_EINVAL;
+    const int64_t tiles = S * W * C;
+    if (tiles > 0 && !d_E) return DYN_EINVAL;
+    rc = check_ws(d_ws, ws_bytes, dyn_select_workspace_bytes(S, W, J));
+    if (rc != DYN_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char *ws = static_cast<char *>(d_ws);
+    const int64_t chunks = totals_chunks(W);
+    double *partial = reinterpret_cast<double *>(ws);
+    uint32_t *partial_bad = reinterpret_cast<uint32_t *>(ws + size_t(S) * size_t(chunks) * sizeof(double));
+    const size_t off_nj = align256(size_t(S) * size_t(chunks) * (sizeof(double) + sizeof(uint32_t)));
+    int32_t *d_nj = nullptr, *d_tj = nullptr;
+    if (out->d_gpus) {
+        d_nj = reinterpret_cast<int32_t *>(ws + off_nj);
+        d_tj = reinterpret_cast<int32_t *>(ws + off_nj + align256(size_t(J) * sizeof(int32_t)));
+        // pageable host memory: the copy is staged before the call returns, the arrays may be reused
+        DYN_CUDA_TRY(cudaMemcpyAsync(d_nj, n_of_j, size_t(J) * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+        DYN_CUDA_TRY(cudaMemcpyAsync(d_tj, tp_of_j, size_t(J) * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    }
+    DYN_CUDA_TRY(launch_select(d_E, tiles, J, out->d_best_idx, out->d_best_E, st));
+    DYN_CUDA_TRY(launch_totals(to_out(out), S, W, C, J, d_nj, d_tj, 1, 1, nullptr, partial, partial_bad, st));
+    return DYN_OK;
+}
+
+int dyn_eval_select(const dyn_profile *profile, const dyn_space *space, const float *d_load, int64_t S, int64_t W,
+                    const dyn_select_out *out, void *d_ws, size_t ws_bytes, void *stream) {
+    ResolveParams rp;
+    int rc = check_problem(profile, space, S, W, &rp);
+    if (rc != DYN_OK) return rc;
+    rc = check_out(out);
+    if (rc != DYN_OK) return rc;
+    const int64_t tiles = S * W * profile->C;
+    if (tiles > 0 && !d_load) return DYN_EINVAL;
+    const ResolvedLayout lay = resolved_layout(profile->C, profile->T, space->F, profile->M, space->Nmax, S, W);
+    rc = check_ws(d_ws, ws_bytes, lay.total);
+    if (rc != DYN_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char *ws = static_cast<char *>(d_ws);
+    DYN_CUDA_TRY(launch_resolve(rp, lay, d_ws, st));
+    DYN_CUDA_TRY(launch_eval_select(lay, d_ws, d_load, tiles, space->gpu_budget, out->d_best_idx, out->d_best_E, st));
+    const int64_t chunks = totals_chunks(W);
+    double *partial = reinterpret_cast<double *>(ws + lay.off_partial);
+    uint32_t *partial_bad = reinterpret_cast<uint32_t *>(ws + lay.off_partial + size_t(S) * size_t(chunks) * sizeof(double));
+    DYN_CUDA_TRY(launch_totals(to_out(out), S, W, profile->C, lay.J, nullptr, nullptr, profile->T, space->F,
+                               reinterpret_cast<const int32_t *>(ws + lay.off_tp), partial, partial_bad, st));
+    return DYN_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,113 @@
+// Internal declarations shared by the translation units of libdynamo.so (not installed).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dynamo.h"
+
+namespace dyn {
+
+// ---- error plumbing -----------------------------------------------------------------------
+void set_last_cuda_error(cudaError_t e);
+
+#define DYN_CUDA_TRY(expr)                              \
+    do {                                                \
+        cudaError_t e__ = (expr);                       \
+        if (e__ != cudaSuccess) {                       \
+            ::dyn::set_last_cuda_error(e__);            \
+            return DYN_ECUDA;                           \
+        }                                               \
+    } while (0)
+
+// ---- unsigned division by a run-time invariant (Granlund & Montgomery 1994, Fig. 4.1) -------
+// q = floor(n / d) for every 32-bit n and every d >= 1:
+//   l = ceil(log2 d), m' = floor(2^32 (2^l - d) / d) + 1, t1 = mulhi(m', n),
+//   q = (t1 + ((n - t1) >> min(l,1))) >> max(l-1, 0)
+struct FastDiv {
+    uint32_t mul, sh1, sh2, d;
+};
+
+inline FastDiv make_fastdiv(uint32_t d) {
+    FastDiv f;
+    uint32_t l = 0;
+    while (l < 32 && (uint64_t(1) << l) < d) ++l;
+    f.mul = uint32_t(((uint64_t(1) << 32) * ((uint64_t(1) << l) - d)) / d + 1);
+    f.sh1 = l < 1 ? l : 1;
+    f.sh2 = l > 0 ? l - 1 : 0;
+    f.d = d;
+    return f;
+}
+
+__device__ __forceinline__ uint32_t fastdiv(uint32_t n, const FastDiv &f) {
+    uint32_t t1 = __umulhi(f.mul, n);
+    return (t1 + ((n - t1) >> f.sh1)) >> f.sh2;
+}
+
+// ---- resolved candidate tables (scratch memory) ----------------------------------------------
+// For class c and pair p = t*F + q (P = T*F pairs):
+//   icm[c][p]       (M-1)/cap(c,t,f_q), or +inf when TTFT(c,t,f_q) > slo_ttft[c]
+//   rows[c][p][m]   m = 0..M (M+1 entries), float4 {tbt_a, tbt_d, e_a, e_d} with
+//                   TBT(x) = tbt_a + (x-m)*tbt_d and window energy of ONE instance
+//                   e(x) = e_a + (x-m)*e_d (Wh), x = u*(M-1) in [m, m+1]; entry M repeats knot M-1
+//                   with zero slope (reached only at u == 1).
+//   slo[c]          slo_tbt[c]
+struct ResolvedLayout {
+    int32_t C, T, F, P, M, Nmax, J;
+    int32_t row_stride;          // float4 entries per pair row (M+1)
+    size_t off_icm, off_rows, off_slo, off_tp, off_partial, off_njtj, total;
+    size_t class_rows_bytes;     // bytes of rows[c]
+};
+
+ResolvedLayout resolved_layout(int32_t C, int32_t T, int32_t F, int32_t M, int32_t Nmax, int64_t S, int64_t W);
+
+struct ResolveParams {
+    int32_t C, T, R, M, F;
+    const float *d_ttft, *d_cap, *d_tbt, *d_pow;
+    float window_s;
+    int16_t row[DYN_MAX_F];
+    float weight[DYN_MAX_F];
+    float slo_ttft[256], slo_tbt[256];
+    int32_t tp[DYN_MAX_T];
+};
+
+// launchers (each enqueues on `st` and returns the launch error, if any)
+cudaError_t launch_resolve(const ResolveParams &rp, const ResolvedLayout &lay, void *d_ws, cudaStream_t st);
+
+struct SelectOut {
+    int32_t *best_idx;
+    float *best_E;
+    double *E_total;
+    uint32_t *n_infeasible;
+    double *E_window;
+    uint32_t *hist;
+    uint32_t *gpus;
+};
+
+cudaError_t launch_eval_configs(const ResolvedLayout &lay, const void *d_ws, const float *d_load, int64_t tiles,
+                                int32_t gpu_budget, float *d_E, cudaStream_t st);
+cudaError_t launch_eval_select(const ResolvedLayout &lay, const void *d_ws, const float *d_load, int64_t tiles,
+                               int32_t gpu_budget, int32_t *best_idx, float *best_E, cudaStream_t st);
+cudaError_t launch_select(const float *d_E, int64_t tiles, int32_t J, int32_t *best_idx, float *best_E,
+                          cudaStream_t st);
+// n/tp of candidate j: either from device tables (d_nj, d_tj) or, when those are NULL, from
+// j = ((n-1)*T + t)*F + q with the TP list d_tp.
+cudaError_t launch_totals(const SelectOut &o, int64_t S, int64_t W, int32_t C, int32_t J, const int32_t *d_nj,
+                          const int32_t *d_tj, int32_t T, int32_t F, const int32_t *d_tp, double *d_partial,
+                          uint32_t *d_partial_bad, cudaStream_t st);
+int64_t totals_chunks(int64_t W);
+
+struct BinParams {
+    FastDiv win;
+    uint32_t n_windows;
+    int32_t n_in, n_out, C;
+    uint32_t in_edges[DYN_MAX_EDGES], out_edges[DYN_MAX_EDGES];
+    float window_s;
+};
+cudaError_t launch_bin_trace(const BinParams &bp, const uint32_t *t_ms, const uint32_t *in_tok, const uint32_t *out_tok,
+                             uint64_t n_req, uint32_t *counts, float *load, unsigned long long *dropped,
+                             cudaStream_t st);
+
+int sm_count();
+
+}  // namespace dyn

@@ -1,0 +1,101 @@
+// Stage (b0): resolve the candidate frequencies against the profile tables.
+//
+// The profile is measured at a few frequencies and load levels and interpolated linearly in between
+// [Sec. 4.1 "Generating LLM profiles"].  Everything that depends only on (class, TP, candidate
+// frequency) is computed here once per call, in fp64, and stored in scratch memory in the form the
+// sweep kernels read: per (class, TP, frequency) pair one row of utilisation segments, each holding
+// value and slope of TBT and of the per-instance window energy, plus (M-1)/cap.  Interpolating in f
+// here and in u inside the sweep equals the bilinear interpolation of the definition.
+#include "dyn_internal.cuh"
+
+namespace dyn {
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int64_t totals_chunks(int64_t W) {
+    const int64_t per = 2048;            // windows per partial sum
+    return (W + per - 1) / per;
+}
+
+ResolvedLayout resolved_layout(int32_t C, int32_t T, int32_t F, int32_t M, int32_t Nmax, int64_t S, int64_t W) {
+    ResolvedLayout l{};
+    l.C = C; l.T = T; l.F = F; l.P = T * F; l.M = M; l.Nmax = Nmax;
+    l.J = Nmax * T * F;
+    l.row_stride = M;
+    size_t off = 0;
+    l.off_rows = off;
+    l.class_rows_bytes = size_t(l.P) * size_t(l.row_stride) * sizeof(float4);
+    off = align_up(off + size_t(C) * l.class_rows_bytes, 256);
+    l.off_icm = off;  off = align_up(off + size_t(C) * size_t(l.P) * sizeof(float), 256);
+    l.off_slo = off;  off = align_up(off + size_t(C) * sizeof(float), 256);
+    l.off_tp = off;   off = align_up(off + size_t(T) * sizeof(int32_t), 256);
+    l.off_partial = off;
+    off = align_up(off + size_t(S) * size_t(totals_chunks(W)) * (sizeof(double) + sizeof(uint32_t)), 256);
+    l.off_njtj = off;
+    l.total = off;
+    return l;
+}
+
+namespace {
+
+__device__ __forceinline__ double lerp64(double a, double b, double w) { return (1.0 - w) * a + w * b; }
+
+__global__ void resolve_kernel(const ResolveParams rp, float4 *__restrict__ rows, float *__restrict__ icm,
+                               float *__restrict__ slo, int32_t *__restrict__ tp) {
+    const int P = rp.T * rp.F;
+    const int M = rp.M;
+    const long long total = (long long)rp.C * P * M;
+    const double scale = double(rp.window_s) / 3600.0;
+    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total;
+         e += (long long)gridDim.x * blockDim.x) {
+        const int m = int(e % M);
+        const long long cp = e / M;
+        const int p = int(cp % P);
+        const int c = int(cp / P);
+        const int t = p / rp.F, q = p - t * rp.F;
+        const int r = rp.row[q];
+        const double w = double(rp.weight[q]);
+        const size_t ct = (size_t(c) * rp.T + t) * rp.R;
+        const float *tb0 = rp.d_tbt + (ct + r) * M, *tb1 = tb0 + M;
+        const float *pw0 = rp.d_pow + (ct + r) * M, *pw1 = pw0 + M;
+        const double tb_m = lerp64(tb0[m], tb1[m], w);
+        const double pw_m = lerp64(pw0[m], pw1[m], w) * scale;
+        float4 v;
+        if (m < M - 1) {
+            const double tb_n = lerp64(tb0[m + 1], tb1[m + 1], w);
+            const double pw_n = lerp64(pw0[m + 1], pw1[m + 1], w) * scale;
+            v = make_float4(float(tb_m), float(tb_n - tb_m), float(pw_m), float(pw_n - pw_m));
+        } else {
+            v = make_float4(float(tb_m), 0.f, float(pw_m), 0.f);     // reached only at u == 1
+        }
+        rows[(size_t(c) * P + p) * M + m] = v;
+        if (m == 0) {
+            const double ttft = lerp64(rp.d_ttft[ct + r], rp.d_ttft[ct + r + 1], w);
+            const double cap = lerp64(rp.d_cap[ct + r], rp.d_cap[ct + r + 1], w);
+            // a non-positive (or NaN) capacity can serve no load: the pair is never feasible
+            const bool ok = (ttft <= double(rp.slo_ttft[c])) && (cap > 0.0);
+            icm[size_t(c) * P + p] = ok ? float(double(M - 1) / cap) : __int_as_float(0x7f800000);
+            if (p == 0) slo[c] = rp.slo_tbt[c];
+            if (c == 0 && p < rp.T) tp[p] = rp.tp[p];
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_resolve(const ResolveParams &rp, const ResolvedLayout &lay, void *d_ws, cudaStream_t st) {
+    char *ws = static_cast<char *>(d_ws);
+    const long long total = (long long)rp.C * lay.P * rp.M;
+    const int threads = 256;
+    long long blocks = (total + threads - 1) / threads;
+    const long long cap = (long long)sm_count() * 8;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    resolve_kernel<<<int(blocks), threads, 0, st>>>(rp, reinterpret_cast<float4 *>(ws + lay.off_rows),
+                                                    reinterpret_cast<float *>(ws + lay.off_icm),
+                                                    reinterpret_cast<float *>(ws + lay.off_slo),
+                                                    reinterpret_cast<int32_t *>(ws + lay.off_tp));
+    return cudaGetLastError();
+}
+
+}  // namespace dyn
