@@ -1,0 +1,413 @@
+#!/usr/bin/env python
+"""Benchmark of the configuration-sweep hot path on B200.
+
+A step is one pass of the whole path over one batch of synthetic input: bin the trace into
+per-(window, class) loads, evaluate every candidate (N, TP, f) of every tile against the profile
+tables and the SLOs, pick the minimum-energy feasible candidate per tile, reduce the totals.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `value` is config-evaluations per second with inputs resident in
+device memory; `e2e` is the same metric through the host-buffer entry point (host->device and
+device->host copies inside the timed region); `roofline` is the sweep kernel alone, timed by CUDA
+events recorded around it on its stream; `cpu_baseline` is the CPU oracle on a bounded sample.
+With N > 1 every rank runs an independent replica of the workload (the path has no exchange step).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+FLOP_PER_EVAL = 20.0            # algorithmic fp32 operations per candidate, counted from the definition
+SM_COUNT, FP32_LANES, SM_MAX_MHZ = 148, 128, 1965.0
+BYTES_PER_REQUEST = 12.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="cfg4", choices=["cfg1", "cfg2", "cfg3", "cfg3code", "cfg4", "cfg5"])
+    ap.add_argument("--scenarios", type=int, default=0, help="override the scenario count S (cfg4 default 4096)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true", help="skip the trace-binning side measurement")
+    return ap.parse_args()
+
+
+def max_over_ranks(x: float, dist, device) -> float:
+    """Largest value of x over all ranks (x itself without a process group)."""
+    if dist is None:
+        return float(x)
+    import torch
+    tt = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return float(tt.item())
+
+
+# ----------------------------------------------------------------------------------------------
+# clocks
+# ----------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+        self.marks = []
+
+    def mark(self):
+        """remember how many samples exist now (start / end of the timed region)"""
+        self.f.flush()
+        try:
+            with open(self.f.name) as fh:
+                self.marks.append(sum(1 for _ in fh))
+        except OSError:
+            self.marks.append(0)
+
+    def stop(self):
+        if self.p is not None:
+            self.p.terminate()
+            try:
+                self.p.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.p.kill()
+        rows = []
+        try:
+            with open(self.f.name) as fh:
+                rows = [[x.strip() for x in line.split(",")] for line in fh if line.strip()]
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        lo, hi = (self.marks + [0, len(rows)])[:2] if len(self.marks) >= 2 else (0, len(rows))
+        sel = rows[max(0, lo - 1):hi + 1] or rows
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in sel:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for k, name in enumerate(names):
+                if len(r) > 4 + k and r[4 + k].lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------------------------
+# workload
+# ----------------------------------------------------------------------------------------------
+def make_inputs(name, S_override=0):
+    import gen
+    wl = gen.workload(name)
+    if S_override:
+        wl.S = S_override
+    t, i, o = gen.make_trace(wl.trace)
+    return wl, (t, i, o), wl.profile(), wl.space()
+
+
+def scenario_loads(wl, base_counts, S_extra, s_begin=1):
+    """Loads of scenarios s_begin .. s_begin+S_extra-1 (Poisson-resampled counts over the window length)."""
+    import gen
+    if S_extra <= 0:
+        return None
+    cs = gen.resample_counts(base_counts, S_extra, wl.scenario_seed, s_begin=s_begin)
+    return (cs.astype(np.float32) / np.float32(wl.window_s)).astype(np.float32)
+
+
+def oracle_step(wl, trace, prof, sp, loads_extra):
+    """One pass of the whole path in the CPU oracle over 1 + len(loads_extra) scenarios."""
+    import gen
+    import oracle
+    t, i, o = trace
+    W = wl.trace.n_windows
+    counts, dropped = oracle.bin_trace(t, i, o, wl.trace.window_ms, W, gen.IN_EDGES, gen.OUT_EDGES)
+    load0 = oracle.load_from_counts(counts, wl.window_s)[None]
+    load = load0 if loads_extra is None else np.concatenate([load0, loads_extra], axis=0)
+    r = oracle.eval_select(prof, sp, load)
+    tot = oracle.totals(r["best_idx"], r["best_E"], wl.J)
+    return load.shape[0], tot
+
+
+def time_oracle(wl, trace, prof, sp, base_counts, target_s=15.0, max_scen=512):
+    """Oracle evaluations/s on a bounded sample of the workload (about target_s of CPU work)."""
+    import oracle
+    W, Cn = wl.trace.n_windows, 9
+    per_scen = W * Cn * wl.J
+    n0 = 1 if wl.S == 1 else min(4, wl.S)
+    ex = scenario_loads(wl, base_counts, n0 - 1)
+    t0 = time.perf_counter(); oracle_step(wl, trace, prof, sp, ex); dt0 = time.perf_counter() - t0
+    n = n0
+    if wl.S > 1:
+        n = int(max(n0, min(max_scen, wl.S, target_s / max(dt0 / n0, 1e-9))))
+    if n > n0:
+        ex = scenario_loads(wl, base_counts, n - 1)
+        t0 = time.perf_counter(); oracle_step(wl, trace, prof, sp, ex); dt = time.perf_counter() - t0
+    else:
+        dt = dt0
+    return {"value": n * per_scen / dt, "unit": "evals/s", "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{n} of {wl.S} scenario(s) of {wl.name}: trace binning + {n * W * Cn} tiles x {wl.J} candidates "
+                      f"in {dt:.2f} s"}, n, dt
+
+
+# ----------------------------------------------------------------------------------------------
+def run_reference(args, rank):
+    """The CPU oracle as it stands, timed on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    wl, trace, prof, sp = make_inputs(args.workload, args.scenarios)
+    import gen
+    import oracle
+    counts, _ = oracle.bin_trace(*trace, wl.trace.window_ms, wl.trace.n_windows, gen.IN_EDGES, gen.OUT_EDGES)
+    W, Cn = wl.trace.n_windows, 9
+    per_scen = W * Cn * wl.J
+    # size one step to roughly 2 s of CPU work
+    t0 = time.perf_counter(); oracle_step(wl, trace, prof, sp, None); dt1 = time.perf_counter() - t0
+    n = 1 if wl.S == 1 else int(max(1, min(wl.S, 64, 2.0 / max(dt1, 1e-9))))
+    ex = scenario_loads(wl, counts, n - 1)
+    for _ in range(args.warmup):
+        oracle_step(wl, trace, prof, sp, ex)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(wl, trace, prof, sp, ex)
+    dt = time.perf_counter() - t0
+    value = args.steps * n * per_scen / dt
+    sample = f"{n} of {wl.S} scenario(s) of {wl.name} per step"
+    print(json.dumps({
+        "impl": "reference", "metric": "config_evaluations_per_s", "value": value, "unit": "evals/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "S": wl.S, "W": W, "C": Cn, "J": wl.J, "requests": int(len(trace[0])),
+                   "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "evals/s", "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": "evals/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def run_ours(args, rank, world, local_rank):
+    import torch
+    import gen
+    import paper_2408_00741_b200 as dyn
+
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    wl, trace, prof, sp = make_inputs(args.workload, args.scenarios)
+    t, i, o = trace
+    n_req, W, Cn, S, J = len(t), wl.trace.n_windows, 9, wl.S, wl.J
+    to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a, np.uint32).view(np.int32)).to(dev)
+    d_t, d_i, d_o = to_dev(t), to_dev(i), to_dev(o)
+    d_counts = torch.empty((W, Cn), dtype=torch.int32, device=dev)
+    d_dropped = torch.empty(1, dtype=torch.int64, device=dev)
+    d_load = torch.zeros((S, W, Cn), dtype=torch.float32, device=dev)
+    P = dyn.Profile(prof.tp, prof.f_grid_mhz, prof.ttft, prof.cap, prof.tbt, prof.pow, device=dev)
+    SP = dyn.Space(sp.f_cand_mhz, sp.n_max, sp.slo_ttft_s, sp.slo_tbt_s, sp.window_s, sp.gpu_budget)
+    out = dyn.SelectOut(S, W, Cn, J, device=dev, windows=False, hist=True, gpus=False)
+    ws = torch.empty(dyn.dyn_workspace_bytes(P, SP, S, W), dtype=torch.uint8, device=dev)
+
+    def step():
+        dyn.dyn_bin_trace(wl.trace.window_ms, W, gen.IN_EDGES, gen.OUT_EDGES, d_t, d_i, d_o, d_counts, d_load[0], d_dropped)
+        dyn.dyn_eval_select(P, SP, d_load, out, ws)
+    launches_per_step = 6        # histogram, counts->load, resolve, sweep, totals partial, totals final
+
+    # scenario loads: the base counts come from our own binning; the resampling is input generation
+    step()
+    torch.cuda.synchronize()
+    base_counts = d_counts.cpu().numpy().view(np.uint32)
+    extra = scenario_loads(wl, base_counts, S - 1)
+    if extra is not None:
+        d_load[1:].copy_(torch.from_numpy(extra))
+    input_bytes = 3 * 4 * n_req + d_load.numel() * 4
+    l2_mode = "inputs_larger_than_L2" if input_bytes > 126 * 2 ** 20 else "flushed"
+    flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev) if l2_mode == "flushed" else None
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    for _ in range(max(args.warmup, 3)):
+        step()
+    K = args.steps
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    for a, b in kev:                       # create the handles
+        a.record(); b.record()
+    barrier()
+    if sampler:
+        sampler.mark()
+    for k in range(K):
+        if flush is not None:
+            flush.fill_(k & 0xff)          # outside the per-step events
+        dyn.dyn_set_timing_events(*kev[k])
+        ev[k][0].record()
+        step()
+        ev[k][1].record()
+    dyn.dyn_set_timing_events(None, None)
+    barrier()
+    if sampler:
+        sampler.mark()
+    step_ms = [a.elapsed_time(b) for a, b in ev]
+    # kev now holds the events of the LAST instrumented call of each step (the sweep of dyn_eval_select)
+    kern_ms = [a.elapsed_time(b) for a, b in kev]
+    total_ms = max_over_ranks(float(sum(step_ms)), dist, dev)
+    clocks = sampler.stop() if sampler else None
+
+    evals_per_step = S * W * Cn * J
+    value = world * K * evals_per_step / (total_ms * 1e-3)
+
+    # ---- end to end through the host-buffer entry point ---------------------------------------
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    h_t, h_i, h_o = pin(t.view(np.int32)), pin(i.view(np.int32)), pin(o.view(np.int32))
+    h_extra = pin(extra) if extra is not None else None
+    hp = dyn.HostPipeline(wl.trace.window_ms, W, gen.IN_EDGES, gen.OUT_EDGES, prof.tp, prof.f_grid_mhz, prof.ttft,
+                          prof.cap, prof.tbt, prof.pow, SP)
+    h_out = {"counts": torch.empty((W, Cn), dtype=torch.int32).pin_memory(),
+             "dropped": torch.empty(1, dtype=torch.int64).pin_memory(),
+             "E_total": torch.empty(S, dtype=torch.float64).pin_memory(),
+             "n_infeasible": torch.empty(S, dtype=torch.int32).pin_memory(),
+             "hist": torch.empty((S, J), dtype=torch.int32).pin_memory()}
+    del out, ws, d_load
+    torch.cuda.empty_cache()
+    arena = torch.empty(hp.arena_bytes(n_req, S), dtype=torch.uint8, device=dev)
+    h2d = 3 * 4 * n_req + sum(x.nbytes for x in hp.tabs) + (h_extra.numel() * 4 if h_extra is not None else 0)
+    d2h = sum(v.numel() * v.element_size() for v in h_out.values())
+    for _ in range(2):
+        hp.run(h_t, h_i, h_o, h_extra, h_out, arena)
+    barrier()
+    KE = max(1, args.e2e_steps)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(KE):
+        hp.run(h_t, h_i, h_o, h_extra, h_out, arena)
+    e1.record()
+    barrier()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), dist, dev)
+    e2e_value = world * KE * evals_per_step / (e2e_ms * 1e-3)
+    E_total_e2e = h_out["E_total"].numpy().copy()
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (the sweep), from events recorded around it ------------
+    k_ms = float(np.mean(kern_ms))
+    fp32_peak = SM_COUNT * FP32_LANES * 2 * SM_MAX_MHZ * 1e6 / 1e12
+    achieved = FLOP_PER_EVAL * evals_per_step / (k_ms * 1e-3) / 1e12
+    roofline = {"bound": "alu", "kernel": "eval_select_kernel", "achieved": achieved, "peak": fp32_peak,
+                "unit": "TFLOP/s", "frac": achieved / fp32_peak, "traffic": None,
+                "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 flop x 1965 MHz (no measured fp32 figure in "
+                               "MEASURED_PEAKS.json)",
+                "flop_per_eval": FLOP_PER_EVAL, "kernel_ms": k_ms, "evals_per_s_kernel": evals_per_step / (k_ms * 1e-3)}
+
+    result = {
+        "metric": "config_evaluations_per_s", "value": value, "unit": "evals/s", "n_gpus": world, "steps": K,
+        "warmup": max(args.warmup, 3), "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "S": S, "W": W, "C": Cn, "J": J, "requests": int(n_req), "l2": l2_mode,
+                   "multi_gpu": "replicas only"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": "evals/s", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                "steps": KE, "ms_per_step": e2e_ms / KE},
+        "gpu_launches": launches_per_step * K,
+        "roofline": roofline,
+        "E_total_scenario0_Wh": float(E_total_e2e[0]),
+    }
+
+    # ---- side measurement: the histogram kernel on the week-long trace (HBM-bound) ---------------
+    if not args.no_secondary and world == 1:
+        try:
+            result["bin_trace"] = measure_bin(dyn, gen, dev)
+        except Exception as exc:                      # never lose the main line
+            result["bin_trace"] = {"error": repr(exc)}
+
+    if not args.no_cpu_baseline and world == 1:
+        cb, _, _ = time_oracle(wl, trace, prof, sp, base_counts)
+        result["cpu_baseline"] = cb
+    print(json.dumps(result))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def measure_bin(dyn, gen, dev):
+    """Requests/s of the trace-binning kernel on the 14M-request week trace (168 MB, larger than L2)."""
+    import torch
+    wl = gen.workload("cfg3")
+    t, i, o = gen.make_trace(wl.trace)
+    W = wl.trace.n_windows
+    to_dev = lambda a: torch.from_numpy(a.view(np.int32)).to(dev)
+    d = [to_dev(x) for x in (t, i, o)]
+    counts = torch.empty((W, 9), dtype=torch.int32, device=dev)
+    load = torch.empty((W, 9), dtype=torch.float32, device=dev)
+    dropped = torch.empty(1, dtype=torch.int64, device=dev)
+    run = lambda: dyn.dyn_bin_trace(wl.trace.window_ms, W, gen.IN_EDGES, gen.OUT_EDGES, d[0], d[1], d[2], counts, load, dropped)
+    for _ in range(3):
+        run()
+    K = 20
+    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    for a, b in kev:
+        a.record(); b.record()
+    torch.cuda.synchronize()
+    for k in range(K):
+        dyn.dyn_set_timing_events(*kev[k])
+        run()
+    dyn.dyn_set_timing_events(None, None)
+    torch.cuda.synchronize()
+    ms = float(np.mean([a.elapsed_time(b) for a, b in kev]))
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except OSError:
+        pass
+    peak = float(peaks.get("hbm_gbs", 6650.0))
+    gbs = BYTES_PER_REQUEST * len(t) / (ms * 1e-3) / 1e9
+    return {"workload": "cfg3", "requests": int(len(t)), "kernel": "bin_trace_kernel", "kernel_ms": ms,
+            "requests_per_s": len(t) / (ms * 1e-3),
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                         "traffic": None,
+                         "peak_source": "measured (MEASURED_PEAKS.json)" if peaks else "fallback 6650 GB/s"}}
+
+
+def main():
+    args = parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

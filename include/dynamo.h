@@ -171,6 +171,65 @@ int dyn_eval_select(const dyn_profile *profile, const dyn_space *space, const fl
                     int64_t S, int64_t W, const dyn_select_out *out, void *d_ws, size_t ws_bytes,
                     void *stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * Whole path from HOST buffers: (a) -> (b) -> (c) in one call.  [Sec. 3 trace -> Sec. 3.2 loads ->
+ * Sec. 4.1 / Eq. 1 evaluation -> Sec. 4.2 selection -> Sec. 6 totals]
+ *
+ * Copies the trace and the profile tables to the device, bins the trace into the loads of scenario 0,
+ * appends S_extra further load scenarios given by the caller (e.g. resampled loads), runs the fused
+ * evaluate+select and the totals, and copies the requested results back.  All device memory comes
+ * from the caller's arena (256-byte aligned, at least dyn_pipeline_arena_bytes()); nothing is
+ * allocated.  Copies are cudaMemcpyAsync on `stream`: with pinned host buffers the call returns before
+ * the results have arrived, so synchronise the stream before reading them; the host input buffers
+ * must stay valid until then.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {                 /* as dyn_profile, with the four tables in HOST memory */
+    int32_t C, T, R, M;
+    const int32_t *tp;
+    const float *f_grid_mhz;
+    const float *ttft, *cap, *tbt, *pow;
+} dyn_profile_host;
+
+typedef struct {
+    const uint32_t *t_ms, *in_tok, *out_tok;   /* host [n_req] each */
+    uint64_t n_req;
+    const float *extra_load;                   /* host [S_extra][W][C] requests/s, or NULL */
+    int64_t S_extra;                           /* scenarios after scenario 0 (the binned trace); S = 1 + S_extra */
+} dyn_host_in;
+
+typedef struct {                 /* host result buffers; any of them may be NULL to skip that copy */
+    uint32_t *counts;            /* [W][C] */
+    uint64_t *dropped;           /* [1] */
+    int32_t *best_idx;           /* [S][W][C] */
+    float *best_E;               /* [S][W][C] */
+    double *E_total;             /* [S] */
+    uint32_t *n_infeasible;      /* [S] */
+    double *E_window;            /* [S][W] */
+    uint32_t *hist;              /* [S][J] */
+    uint32_t *gpus;              /* [S][W] */
+} dyn_host_out;
+
+/* Arena size in bytes for this problem (0 on bad input).  spec->n_windows is W, C must equal
+ * (n_in_edges+1)*(n_out_edges+1), S = 1 + S_extra. */
+size_t dyn_pipeline_arena_bytes(const dyn_bin_spec *spec, const dyn_profile_host *profile, const dyn_space *space,
+                                uint64_t n_req, int64_t S);
+
+/* Errors: as the stage calls, plus DYN_EINVAL when profile->C differs from the class count of spec, and
+ * DYN_EWORKSPACE for a missing, misaligned or short arena. */
+int dyn_pipeline_host(const dyn_bin_spec *spec, const dyn_profile_host *profile, const dyn_space *space,
+                      const dyn_host_in *in, const dyn_host_out *out, void *d_arena, size_t arena_bytes,
+                      void *stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Instrumentation (no counterpart in the paper).  With two non-NULL cudaEvent_t handles (created by
+ * the caller with timing enabled), every later stage call on the calling thread records `start`
+ * right before and `stop` right after its main kernel on the call's stream: the histogram kernel of
+ * dyn_bin_trace, the sweep kernel of dyn_eval_configs / dyn_eval_select, the argmin kernel of
+ * dyn_select.  cudaEventElapsedTime(start, stop) after a synchronise is then that kernel's duration.
+ * Pass NULL, NULL to switch it off (the default).
+ * ------------------------------------------------------------------------------------------- */
+void dyn_set_timing_events(void *start_event, void *stop_event);
+
 #ifdef __cplusplus
 }
 #endif

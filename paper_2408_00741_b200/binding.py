@@ -23,7 +23,8 @@ _lib = C.CDLL(LIB_PATH)
 
 DYN_OK, DYN_EINVAL, DYN_ECUDA, DYN_EUNSUPPORTED, DYN_EWORKSPACE = 0, -1, -2, -3, -4
 EXPORTS = ("dyn_strerror", "dyn_last_cuda_error", "dyn_bin_trace", "dyn_workspace_bytes", "dyn_eval_configs",
-           "dyn_select_workspace_bytes", "dyn_select", "dyn_eval_select")
+           "dyn_select_workspace_bytes", "dyn_select", "dyn_eval_select", "dyn_pipeline_arena_bytes",
+           "dyn_pipeline_host", "dyn_set_timing_events")
 
 
 class DynError(RuntimeError):
@@ -57,6 +58,23 @@ class _SelectOut(C.Structure):
                 ("d_gpus", C.c_void_p)]
 
 
+class _ProfileHost(C.Structure):
+    _fields_ = [("C", C.c_int32), ("T", C.c_int32), ("R", C.c_int32), ("M", C.c_int32),
+                ("tp", C.c_void_p), ("f_grid_mhz", C.c_void_p), ("ttft", C.c_void_p), ("cap", C.c_void_p),
+                ("tbt", C.c_void_p), ("pow", C.c_void_p)]
+
+
+class _HostIn(C.Structure):
+    _fields_ = [("t_ms", C.c_void_p), ("in_tok", C.c_void_p), ("out_tok", C.c_void_p), ("n_req", C.c_uint64),
+                ("extra_load", C.c_void_p), ("S_extra", C.c_int64)]
+
+
+class _HostOut(C.Structure):
+    _fields_ = [("counts", C.c_void_p), ("dropped", C.c_void_p), ("best_idx", C.c_void_p), ("best_E", C.c_void_p),
+                ("E_total", C.c_void_p), ("n_infeasible", C.c_void_p), ("E_window", C.c_void_p),
+                ("hist", C.c_void_p), ("gpus", C.c_void_p)]
+
+
 _lib.dyn_strerror.restype = C.c_char_p
 _lib.dyn_strerror.argtypes = [C.c_int]
 _lib.dyn_last_cuda_error.restype = C.c_int
@@ -76,6 +94,16 @@ _lib.dyn_select.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int32, C.c_int
 _lib.dyn_eval_select.restype = C.c_int
 _lib.dyn_eval_select.argtypes = [C.POINTER(_Profile), C.POINTER(_Space), C.c_void_p, C.c_int64, C.c_int64,
                                  C.POINTER(_SelectOut), C.c_void_p, C.c_size_t, C.c_void_p]
+
+
+_lib.dyn_pipeline_arena_bytes.restype = C.c_size_t
+_lib.dyn_pipeline_arena_bytes.argtypes = [C.POINTER(_BinSpec), C.POINTER(_ProfileHost), C.POINTER(_Space), C.c_uint64,
+                                          C.c_int64]
+_lib.dyn_pipeline_host.restype = C.c_int
+_lib.dyn_pipeline_host.argtypes = [C.POINTER(_BinSpec), C.POINTER(_ProfileHost), C.POINTER(_Space), C.POINTER(_HostIn),
+                                   C.POINTER(_HostOut), C.c_void_p, C.c_size_t, C.c_void_p]
+_lib.dyn_set_timing_events.restype = None
+_lib.dyn_set_timing_events.argtypes = [C.c_void_p, C.c_void_p]
 
 
 def _dev(t, dtype, what):
@@ -215,3 +243,59 @@ def dyn_eval_select(profile: Profile, space: Space, d_load, out: SelectOut, d_ws
     rc = _lib.dyn_eval_select(C.byref(p), C.byref(s), _dev(d_load, torch.float32, "d_load"), S, W, C.byref(o), ws, nb,
                               _stream())
     _check(rc, "dyn_eval_select")
+
+
+def dyn_set_timing_events(start=None, stop=None):
+    """start/stop: torch.cuda.Event(enable_timing=True) that have been recorded once (so that their
+    handles exist), or None, None to switch the instrumentation off."""
+    if start is None or stop is None:
+        _lib.dyn_set_timing_events(None, None)
+    else:
+        _lib.dyn_set_timing_events(C.c_void_p(start.cuda_event), C.c_void_p(stop.cuda_event))
+
+
+class HostPipeline:
+    """Marshals dyn_pipeline_host: host (CPU, ideally pinned) tensors or numpy arrays in and out, one
+    caller-owned device arena.  Shapes: trace uint32 [n]; extra_load float32 [S-1][W][C] or None."""
+
+    def __init__(self, window_ms, n_windows, in_edges, out_edges, tp, f_grid_mhz, ttft, cap, tbt, pow, space: Space):
+        self.ie, self.oe = _host(in_edges, np.uint32), _host(out_edges, np.uint32)
+        self.spec = _BinSpec(int(window_ms), int(n_windows), len(self.ie), len(self.oe), self.ie.ctypes.data,
+                             self.oe.ctypes.data)
+        self.tp, self.fg = _host(tp, np.int32), _host(f_grid_mhz, np.float32)
+        self.tabs = [_host(x, np.float32) for x in (ttft, cap, tbt, pow)]
+        Cn, T, R = self.tabs[0].shape
+        M = self.tabs[2].shape[3]
+        self.prof = _ProfileHost(Cn, T, R, M, self.tp.ctypes.data, self.fg.ctypes.data,
+                                 *[t.ctypes.data for t in self.tabs])
+        self.space = space
+        self.W, self.Cn, self.J = int(n_windows), Cn, space.n_max * T * space.F
+
+    def arena_bytes(self, n_req, S) -> int:
+        sp = self.space._struct()
+        return int(_lib.dyn_pipeline_arena_bytes(C.byref(self.spec), C.byref(self.prof), C.byref(sp), int(n_req), int(S)))
+
+    @staticmethod
+    def _hptr(x):
+        if x is None:
+            return None
+        if isinstance(x, torch.Tensor):
+            assert not x.is_cuda and x.is_contiguous()
+            return x.data_ptr()
+        assert x.flags["C_CONTIGUOUS"]
+        return x.ctypes.data
+
+    def run(self, t_ms, in_tok, out_tok, extra_load, out: dict, d_arena):
+        """out: dict with any of counts, dropped, best_idx, best_E, E_total, n_infeasible, E_window, hist,
+        gpus -> host buffers of the right size.  Enqueues on torch's current stream; synchronise before
+        reading the results."""
+        S_extra = 0 if extra_load is None else int(extra_load.shape[0])
+        n = int(t_ms.shape[0])
+        hin = _HostIn(self._hptr(t_ms), self._hptr(in_tok), self._hptr(out_tok), n, self._hptr(extra_load), S_extra)
+        hout = _HostOut(*[self._hptr(out.get(k)) for k in ("counts", "dropped", "best_idx", "best_E", "E_total",
+                                                          "n_infeasible", "E_window", "hist", "gpus")])
+        sp = self.space._struct()
+        ws, nb = _ws(d_arena)
+        rc = _lib.dyn_pipeline_host(C.byref(self.spec), C.byref(self.prof), C.byref(sp), C.byref(hin), C.byref(hout),
+                                    ws, nb, _stream())
+        _check(rc, "dyn_pipeline_host")

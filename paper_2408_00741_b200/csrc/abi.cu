@@ -10,6 +10,9 @@ namespace dyn {
 static thread_local int tls_cuda_error = 0;
 void set_last_cuda_error(cudaError_t e) { tls_cuda_error = int(e); }
 
+static thread_local TimingEvents tls_events = {nullptr, nullptr};
+TimingEvents timing_events() { return tls_events; }
+
 int sm_count() {
     // per device, cached on first use
     static thread_local int cached_dev = -1, cached = 0;
@@ -84,8 +87,11 @@ int check_problem(const dyn_profile *p, const dyn_space *sp, int64_t S, int64_t 
     return DYN_OK;
 }
 
-int check_out(const dyn_select_out *o) {
-    if (!o || !o->d_best_idx || !o->d_best_E || !o->d_E_total || !o->d_n_infeasible) return DYN_EINVAL;
+// required outputs may be NULL only when they would hold nothing
+int check_out(const dyn_select_out *o, int64_t S, int64_t tiles) {
+    if (!o) return DYN_EINVAL;
+    if (tiles > 0 && (!o->d_best_idx || !o->d_best_E)) return DYN_EINVAL;
+    if (S > 0 && (!o->d_E_total || !o->d_n_infeasible)) return DYN_EINVAL;
     return DYN_OK;
 }
 
@@ -123,6 +129,11 @@ const char *dyn_strerror(int status) {
 }
 
 int dyn_last_cuda_error(void) { return tls_cuda_error; }
+
+void dyn_set_timing_events(void *start_event, void *stop_event) {
+    tls_events.start = static_cast<cudaEvent_t>(start_event);
+    tls_events.stop = static_cast<cudaEvent_t>(stop_event);
+}
 
 int dyn_bin_trace(const dyn_bin_spec *spec, const uint32_t *d_t_ms, const uint32_t *d_in_tok,
                   const uint32_t *d_out_tok, uint64_t n_req, uint32_t *d_counts, float *d_load,
@@ -173,7 +184,9 @@ int dyn_eval_configs(const dyn_profile *profile, const dyn_space *space, const f
     if (rc != DYN_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     DYN_CUDA_TRY(launch_resolve(rp, lay, d_ws, st));
+    DYN_CUDA_TRY(record_start(st));
     DYN_CUDA_TRY(launch_eval_configs(lay, d_ws, d_load, tiles, space->gpu_budget, d_E, st));
+    DYN_CUDA_TRY(record_stop(st));
     return DYN_OK;
 }
 
@@ -185,12 +198,12 @@ size_t dyn_select_workspace_bytes(int64_t S, int64_t W, int64_t J) {
 
 int dyn_select(const float *d_E, int64_t S, int64_t W, int32_t C, int32_t J, const int32_t *n_of_j,
                const int32_t *tp_of_j, const dyn_select_out *out, void *d_ws, size_t ws_bytes, void *stream) {
-    if (S < 0 || W < 0 || C < 1 || J < 1) return DYN_EINVAL;
-    int rc = check_out(out);
-    if (rc != DYN_OK) return rc;
+    if (S < 0 || W < 0 || C < 1 || J < 1 || !out) return DYN_EINVAL;
     if (out->d_gpus && (!n_of_j || !tp_of_j)) return DYN_EINVAL;
     if (S > 0 && W > 0 && (S > (int64_t(1) << 40) / W || S * W > (int64_t(1) << 40) / C)) return DYN_EINVAL;
     const int64_t tiles = S * W * C;
+    int rc = check_out(out, S, tiles);
+    if (rc != DYN_OK) return rc;
     if (tiles > 0 && !d_E) return DYN_EINVAL;
     rc = check_ws(d_ws, ws_bytes, dyn_select_workspace_bytes(S, W, J));
     if (rc != DYN_OK) return rc;
@@ -208,7 +221,9 @@ int dyn_select(const float *d_E, int64_t S, int64_t W, int32_t C, int32_t J, con
         DYN_CUDA_TRY(cudaMemcpyAsync(d_nj, n_of_j, size_t(J) * sizeof(int32_t), cudaMemcpyHostToDevice, st));
         DYN_CUDA_TRY(cudaMemcpyAsync(d_tj, tp_of_j, size_t(J) * sizeof(int32_t), cudaMemcpyHostToDevice, st));
     }
+    DYN_CUDA_TRY(record_start(st));
     DYN_CUDA_TRY(launch_select(d_E, tiles, J, out->d_best_idx, out->d_best_E, st));
+    DYN_CUDA_TRY(record_stop(st));
     DYN_CUDA_TRY(launch_totals(to_out(out), S, W, C, J, d_nj, d_tj, 1, 1, nullptr, partial, partial_bad, st));
     return DYN_OK;
 }
@@ -218,9 +233,9 @@ int dyn_eval_select(const dyn_profile *profile, const dyn_space *space, const fl
     ResolveParams rp;
     int rc = check_problem(profile, space, S, W, &rp);
     if (rc != DYN_OK) return rc;
-    rc = check_out(out);
-    if (rc != DYN_OK) return rc;
     const int64_t tiles = S * W * profile->C;
+    rc = check_out(out, S, tiles);
+    if (rc != DYN_OK) return rc;
     if (tiles > 0 && !d_load) return DYN_EINVAL;
     const ResolvedLayout lay = resolved_layout(profile->C, profile->T, space->F, profile->M, space->Nmax, S, W);
     rc = check_ws(d_ws, ws_bytes, lay.total);
@@ -228,7 +243,9 @@ int dyn_eval_select(const dyn_profile *profile, const dyn_space *space, const fl
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     char *ws = static_cast<char *>(d_ws);
     DYN_CUDA_TRY(launch_resolve(rp, lay, d_ws, st));
+    DYN_CUDA_TRY(record_start(st));
     DYN_CUDA_TRY(launch_eval_select(lay, d_ws, d_load, tiles, space->gpu_budget, out->d_best_idx, out->d_best_E, st));
+    DYN_CUDA_TRY(record_stop(st));
     const int64_t chunks = totals_chunks(W);
     double *partial = reinterpret_cast<double *>(ws + lay.off_partial);
     uint32_t *partial_bad = reinterpret_cast<uint32_t *>(ws + lay.off_partial + size_t(S) * size_t(chunks) * sizeof(double));

@@ -213,6 +213,8 @@ cudaError_t launch_bin_trace(const BinParams &bp, const uint32_t *t_ms, const ui
         const bool vec = ((reinterpret_cast<uintptr_t>(t_ms) | reinterpret_cast<uintptr_t>(in_tok) |
                            reinterpret_cast<uintptr_t>(out_tok)) & 15u) == 0;
         const int g = int(grid);
+        e = record_start(st);
+        if (e != cudaSuccess) return e;
         if (bp.C <= 16) {
             if (bp.n_in == 2 && bp.n_out == 2)
                 e = launch_variant<2, 2, true>(vec, g, bp, t_ms, in_tok, out_tok, n_req, chunk, counts, dropped, st);
@@ -221,6 +223,8 @@ cudaError_t launch_bin_trace(const BinParams &bp, const uint32_t *t_ms, const ui
         } else {
             e = launch_variant<-1, -1, false>(vec, g, bp, t_ms, in_tok, out_tok, n_req, chunk, counts, dropped, st);
         }
+        if (e != cudaSuccess) return e;
+        e = record_stop(st);
         if (e != cudaSuccess) return e;
     }
     if (load) {

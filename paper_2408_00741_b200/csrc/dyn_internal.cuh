@@ -47,14 +47,14 @@ __device__ __forceinline__ uint32_t fastdiv(uint32_t n, const FastDiv &f) {
 // ---- resolved candidate tables (scratch memory) ----------------------------------------------
 // For class c and pair p = t*F + q (P = T*F pairs):
 //   icm[c][p]       (M-1)/cap(c,t,f_q), or +inf when TTFT(c,t,f_q) > slo_ttft[c]
-//   rows[c][p][m]   m = 0..M (M+1 entries), float4 {tbt_a, tbt_d, e_a, e_d} with
-//                   TBT(x) = tbt_a + (x-m)*tbt_d and window energy of ONE instance
-//                   e(x) = e_a + (x-m)*e_d (Wh), x = u*(M-1) in [m, m+1]; entry M repeats knot M-1
-//                   with zero slope (reached only at u == 1).
+//   rows[c][p][m]   m = 0..M-1, float4 {tbt_a, tbt_d, e_a, e_d}: on segment m (x = u*(M-1) in
+//                   [m, m+1]) TBT(x) = tbt_a + (x-m)*tbt_d and the window energy of ONE instance is
+//                   e(x) = e_a + (x-m)*e_d (Wh); entry M-1 holds the last knot with zero slope
+//                   (reached only at u == 1).
 //   slo[c]          slo_tbt[c]
 struct ResolvedLayout {
     int32_t C, T, F, P, M, Nmax, J;
-    int32_t row_stride;          // float4 entries per pair row (M+1)
+    int32_t row_stride;          // float4 entries per pair row (M)
     size_t off_icm, off_rows, off_slo, off_tp, off_partial, off_njtj, total;
     size_t class_rows_bytes;     // bytes of rows[c]
 };
@@ -109,5 +109,17 @@ cudaError_t launch_bin_trace(const BinParams &bp, const uint32_t *t_ms, const ui
                              cudaStream_t st);
 
 int sm_count();
+
+// optional caller-owned events recorded around a stage's main kernel (thread-local; NULL = off)
+struct TimingEvents { cudaEvent_t start, stop; };
+TimingEvents timing_events();
+inline cudaError_t record_start(cudaStream_t st) {
+    const TimingEvents t = timing_events();
+    return (t.start && t.stop) ? cudaEventRecord(t.start, st) : cudaSuccess;
+}
+inline cudaError_t record_stop(cudaStream_t st) {
+    const TimingEvents t = timing_events();
+    return (t.start && t.stop) ? cudaEventRecord(t.stop, st) : cudaSuccess;
+}
 
 }  // namespace dyn
