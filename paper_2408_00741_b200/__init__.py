@@ -1,4 +1,24 @@
-"""B200 configuration-sweep library: Python binding of the C ABI in include/dynamo.h."""
-from .binding import (DYN_ECUDA, DYN_EINVAL, DYN_EUNSUPPORTED, DYN_EWORKSPACE, DYN_OK, EXPORTS, LIB_PATH, DynError,  # noqa: F401
-                      HostPipeline, Profile, SelectOut, Space, dyn_bin_trace, dyn_eval_configs, dyn_eval_select, dyn_select,
-                      dyn_select_workspace_bytes, dyn_set_timing_events, dyn_workspace_bytes)
+"""B200 configuration-sweep library: Python binding of the C ABI in include/dynamo.h.
+
+The binding is loaded on first use, so that `paper_2408_00741_b200.build` can be imported (to compile
+the shared library) before the library exists.  There is no CPU implementation behind these names:
+using any of them without the built library raises ImportError.
+"""
+import importlib
+
+_BINDING_NAMES = ("DYN_ECUDA", "DYN_EINVAL", "DYN_EUNSUPPORTED", "DYN_EWORKSPACE", "DYN_OK", "EXPORTS", "LIB_PATH",
+                  "DynError", "HostPipeline", "Profile", "SelectOut", "Space", "dyn_bin_trace", "dyn_eval_configs",
+                  "dyn_eval_select", "dyn_select", "dyn_select_workspace_bytes", "dyn_set_timing_events",
+                  "dyn_workspace_bytes")
+__all__ = list(_BINDING_NAMES)
+
+
+def __getattr__(name):
+    if name in ("build", "binding"):
+        return importlib.import_module(f"{__name__}.{name}")
+    if name in _BINDING_NAMES:
+        binding = importlib.import_module(f"{__name__}.binding")
+        for n in _BINDING_NAMES:
+            globals()[n] = getattr(binding, n)
+        return globals()[name]
+    raise AttributeError(f"module {__name__!r} has no attribute {name!r}")
