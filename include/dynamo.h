@@ -230,6 +230,37 @@ int dyn_pipeline_host(const dyn_bin_spec *spec, const dyn_profile_host *profile,
  * ------------------------------------------------------------------------------------------- */
 void dyn_set_timing_events(void *start_event, void *stop_event);
 
+/* ---------------------------------------------------------------------------------------------
+ * dyn_eval_select without a workspace argument (the paper has no counterpart; this is a packaging
+ * variant of dyn_eval_select for callers that cannot obtain device memory).
+ *
+ * Who needs it: a controller that runs as a guest inside a serving process which has already handed
+ * the whole GPU to its own memory pool (weights + KV cache), a plug-in that is allowed to launch
+ * kernels but not to call the CUDA allocator, or a few-second control loop that must not risk the
+ * device-wide synchronisation an allocation can cause.  Such a caller still owns its input and
+ * output buffers (it got them from its host application) but has nowhere to get scratch from.
+ *
+ * The scratch (candidate-resolved tables and partial sums, the same content dyn_eval_select puts in
+ * d_ws) lives in a fixed array of DYN_STATIC_WS_BYTES inside the library image.  Every GPU on which
+ * the library is loaded holds that array from load until the process exits, used or not.
+ *
+ *   - Limit: the call serves a problem only if dyn_workspace_bytes(profile, space, S, W) is at most
+ *     DYN_STATIC_WS_BYTES; a larger problem is refused with DYN_EUNSUPPORTED and nothing is enqueued
+ *     (use dyn_eval_select with your own workspace instead).
+ *   - The first call on each device looks up the array's device address (once per device, with that
+ *     device current) and keeps it; make that first call before any stream capture begins.
+ *   - The call itself performs no allocation of any kind and frees nothing.
+ *   - All calls on a device share the one array, and it keeps whatever the previous call left there.
+ *     That is harmless for back-to-back calls on one stream, because every word the kernels read from
+ *     the scratch is written earlier in the same call (nothing relies on zero-initialised scratch).
+ *     Two calls whose GPU work overlaps (different streams, or different host threads on different
+ *     streams) race on the array and give undefined results: serialise them.
+ *   - Everything else (arguments, results, errors, tolerances) is exactly dyn_eval_select's.
+ * ------------------------------------------------------------------------------------------- */
+#define DYN_STATIC_WS_BYTES (4u << 20)   /* 4 MiB: every benchmark configuration of this repository fits */
+int dyn_eval_select_static(const dyn_profile *profile, const dyn_space *space, const float *d_load,
+                           int64_t S, int64_t W, const dyn_select_out *out, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

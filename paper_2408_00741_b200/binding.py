@@ -24,7 +24,7 @@ _lib = C.CDLL(LIB_PATH)
 DYN_OK, DYN_EINVAL, DYN_ECUDA, DYN_EUNSUPPORTED, DYN_EWORKSPACE = 0, -1, -2, -3, -4
 EXPORTS = ("dyn_strerror", "dyn_last_cuda_error", "dyn_bin_trace", "dyn_workspace_bytes", "dyn_eval_configs",
            "dyn_select_workspace_bytes", "dyn_select", "dyn_eval_select", "dyn_pipeline_arena_bytes",
-           "dyn_pipeline_host", "dyn_set_timing_events")
+           "dyn_pipeline_host", "dyn_set_timing_events", "dyn_eval_select_static")
 
 
 class DynError(RuntimeError):
@@ -104,6 +104,12 @@ _lib.dyn_pipeline_host.argtypes = [C.POINTER(_BinSpec), C.POINTER(_ProfileHost),
                                    C.POINTER(_HostOut), C.c_void_p, C.c_size_t, C.c_void_p]
 _lib.dyn_set_timing_events.restype = None
 _lib.dyn_set_timing_events.argtypes = [C.c_void_p, C.c_void_p]
+
+
+_lib.dyn_eval_select_static.restype = C.c_int
+_lib.dyn_eval_select_static.argtypes = [C.POINTER(_Profile), C.POINTER(_Space), C.c_void_p, C.c_int64, C.c_int64,
+                                        C.POINTER(_SelectOut), C.c_void_p]
+DYN_STATIC_WS_BYTES = 4 << 20
 
 
 def _dev(t, dtype, what):
@@ -299,3 +305,15 @@ class HostPipeline:
         rc = _lib.dyn_pipeline_host(C.byref(self.spec), C.byref(self.prof), C.byref(sp), C.byref(hin), C.byref(hout),
                                     ws, nb, _stream())
         _check(rc, "dyn_pipeline_host")
+
+
+def dyn_eval_select_static(profile: Profile, space: Space, d_load, out: SelectOut):
+    """dyn_eval_select for callers that cannot allocate device memory: no workspace argument, the
+    scratch is a fixed DYN_STATIC_WS_BYTES array inside the library.  Larger problems raise DynError with
+    status DYN_EUNSUPPORTED.  Calls whose GPU work overlaps share that array and must be serialised."""
+    S, W, Cn = d_load.shape
+    p, s = profile._struct(), space._struct()
+    o = out._struct()
+    rc = _lib.dyn_eval_select_static(C.byref(p), C.byref(s), _dev(d_load, torch.float32, "d_load"), S, W, C.byref(o),
+                                     _stream())
+    _check(rc, "dyn_eval_select_static")
