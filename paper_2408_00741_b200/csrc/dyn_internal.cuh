@@ -45,16 +45,17 @@ __device__ __forceinline__ uint32_t fastdiv(uint32_t n, const FastDiv &f) {
 }
 
 // ---- resolved candidate tables (scratch memory) ----------------------------------------------
-// For class c and pair p = t*F + q (P = T*F pairs):
-//   icm[c][p]       (M-1)/cap(c,t,f_q), or +inf when TTFT(c,t,f_q) > slo_ttft[c]
-//   rows[c][p][m]   m = 0..M-1, float4 {tbt_a, tbt_d, e_a, e_d}: on segment m (x = u*(M-1) in
-//                   [m, m+1]) TBT(x) = tbt_a + (x-m)*tbt_d and the window energy of ONE instance is
-//                   e(x) = e_a + (x-m)*e_d (Wh); entry M-1 holds the last knot with zero slope
-//                   (reached only at u == 1).
+// For class c and pair p = t*F + q (P = T*F pairs), with x = u*(M-1) the table position:
+//   icv[c][p]       (M-1)/(M*cap(c,t,f_q)): x = sat(L/n * icv) * M; 0 for a pair that is never feasible
+//   rows[c][p][m]   m = 0..M, float4 {tbt_a, -tbt_d, e_a, -e_d}: on segment m (x in [m, m+1])
+//                   TBT(x) = tbt_a + (x-m)*tbt_d and the window energy of ONE instance is
+//                   e(x) = e_a + (x-m)*e_d (Wh); slopes are stored negated.  Entry M-1 is the last knot with a huge TBT slope and
+//                   entry M has TBT = +inf, so u > 1 shows up as an SLO violation; a pair whose TTFT
+//                   misses its SLO has TBT = +inf everywhere.
 //   slo[c]          slo_tbt[c]
 struct ResolvedLayout {
     int32_t C, T, F, P, M, Nmax, J;
-    int32_t row_stride;          // float4 entries per pair row (M)
+    int32_t row_stride;          // float4 entries per pair row (M + 1)
     size_t off_icm, off_rows, off_slo, off_tp, off_partial, off_njtj, total;
     size_t class_rows_bytes;     // bytes of rows[c]
 };

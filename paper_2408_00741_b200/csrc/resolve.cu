@@ -4,8 +4,9 @@
 // [Sec. 4.1 "Generating LLM profiles"].  Everything that depends only on (class, TP, candidate
 // frequency) is computed here once per call, in fp64, and stored in scratch memory in the form the
 // sweep kernels read: per (class, TP, frequency) pair one row of utilisation segments, each holding
-// value and slope of TBT and of the per-instance window energy, plus (M-1)/cap.  Interpolating in f
-// here and in u inside the sweep equals the bilinear interpolation of the definition.
+// value and slope of TBT and of the per-instance window energy, plus the scale from per-instance load
+// to table position.  Interpolating in f here and in u inside the sweep equals the bilinear
+// interpolation of the definition.
 #include "dyn_internal.cuh"
 
 namespace dyn {
@@ -21,7 +22,7 @@ ResolvedLayout resolved_layout(int32_t C, int32_t T, int32_t F, int32_t M, int32
     ResolvedLayout l{};
     l.C = C; l.T = T; l.F = F; l.P = T * F; l.M = M; l.Nmax = Nmax;
     l.J = Nmax * T * F;
-    l.row_stride = M;
+    l.row_stride = M + 1;
     size_t off = 0;
     l.off_rows = off;
     l.class_rows_bytes = size_t(l.P) * size_t(l.row_stride) * sizeof(float4);
@@ -40,16 +41,25 @@ namespace {
 
 __device__ __forceinline__ double lerp64(double a, double b, double w) { return (1.0 - w) * a + w * b; }
 
-__global__ void resolve_kernel(const ResolveParams rp, float4 *__restrict__ rows, float *__restrict__ icm,
+// One thread per table entry (class c, pair p = t*F + q, entry m = 0..M):
+//   m <= M-2  segment m: value and NEGATED slope of TBT and of the per-instance window energy (the
+//             sweep multiplies them by minus the fraction)
+//   m == M-1  the last knot, reached with nu == 0 only at u == 1; its TBT slope is huge, so that any
+//             x above M-1 (u > 1) reads as an SLO violation without a separate capacity test
+//   m == M    x saturated (u >= M/(M-1)): TBT = +inf
+// A pair whose TTFT misses its SLO, or whose capacity is not positive, gets TBT = +inf in every entry.
+__global__ void resolve_kernel(const ResolveParams rp, float4 *__restrict__ rows, float *__restrict__ icv,
                                float *__restrict__ slo, int32_t *__restrict__ tp) {
     const int P = rp.T * rp.F;
     const int M = rp.M;
-    const long long total = (long long)rp.C * P * M;
+    const int RS = M + 1;
+    const long long total = (long long)rp.C * P * RS;
     const double scale = double(rp.window_s) / 3600.0;
+    const float kInf = __int_as_float(0x7f800000);
     for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total;
          e += (long long)gridDim.x * blockDim.x) {
-        const int m = int(e % M);
-        const long long cp = e / M;
+        const int m = int(e % RS);
+        const long long cp = e / RS;
         const int p = int(cp % P);
         const int c = int(cp / P);
         const int t = p / rp.F, q = p - t * rp.F;
@@ -58,23 +68,28 @@ __global__ void resolve_kernel(const ResolveParams rp, float4 *__restrict__ rows
         const size_t ct = (size_t(c) * rp.T + t) * rp.R;
         const float *tb0 = rp.d_tbt + (ct + r) * M, *tb1 = tb0 + M;
         const float *pw0 = rp.d_pow + (ct + r) * M, *pw1 = pw0 + M;
-        const double tb_m = lerp64(tb0[m], tb1[m], w);
-        const double pw_m = lerp64(pw0[m], pw1[m], w) * scale;
+        const double ttft = lerp64(rp.d_ttft[ct + r], rp.d_ttft[ct + r + 1], w);
+        const double cap = lerp64(rp.d_cap[ct + r], rp.d_cap[ct + r + 1], w);
+        // a non-positive (or NaN) capacity can serve no load: the pair is never feasible
+        const bool pair_ok = (ttft <= double(rp.slo_ttft[c])) && (cap > 0.0);
+        const int mk = m < M ? m : M - 1;
+        const double tb_m = lerp64(tb0[mk], tb1[mk], w);
+        const double pw_m = lerp64(pw0[mk], pw1[mk], w) * scale;
         float4 v;
         if (m < M - 1) {
             const double tb_n = lerp64(tb0[m + 1], tb1[m + 1], w);
             const double pw_n = lerp64(pw0[m + 1], pw1[m + 1], w) * scale;
-            v = make_float4(float(tb_m), float(tb_n - tb_m), float(pw_m), float(pw_n - pw_m));
+            v = make_float4(float(tb_m), float(tb_m - tb_n), float(pw_m), float(pw_m - pw_n));
+        } else if (m == M - 1) {
+            v = make_float4(float(tb_m), -1e30f, float(pw_m), 0.f);
         } else {
-            v = make_float4(float(tb_m), 0.f, float(pw_m), 0.f);     // reached only at u == 1
+            v = make_float4(kInf, 0.f, float(pw_m), 0.f);
         }
-        rows[(size_t(c) * P + p) * M + m] = v;
+        if (!pair_ok) v.x = kInf;
+        rows[(size_t(c) * P + p) * RS + m] = v;
         if (m == 0) {
-            const double ttft = lerp64(rp.d_ttft[ct + r], rp.d_ttft[ct + r + 1], w);
-            const double cap = lerp64(rp.d_cap[ct + r], rp.d_cap[ct + r + 1], w);
-            // a non-positive (or NaN) capacity can serve no load: the pair is never feasible
-            const bool ok = (ttft <= double(rp.slo_ttft[c])) && (cap > 0.0);
-            icm[size_t(c) * P + p] = ok ? float(double(M - 1) / cap) : __int_as_float(0x7f800000);
+            // x = u*(M-1) is formed as sat(L/n * icv) * M, so that saturation at 1 means x = M
+            icv[size_t(c) * P + p] = pair_ok ? float(double(M - 1) / (double(M) * cap)) : 0.f;
             if (p == 0) slo[c] = rp.slo_tbt[c];
             if (c == 0 && p < rp.T) tp[p] = rp.tp[p];
         }
@@ -85,7 +100,7 @@ __global__ void resolve_kernel(const ResolveParams rp, float4 *__restrict__ rows
 
 cudaError_t launch_resolve(const ResolveParams &rp, const ResolvedLayout &lay, void *d_ws, cudaStream_t st) {
     char *ws = static_cast<char *>(d_ws);
-    const long long total = (long long)rp.C * lay.P * rp.M;
+    const long long total = (long long)rp.C * lay.P * (rp.M + 1);
     const int threads = 256;
     long long blocks = (total + threads - 1) / threads;
     const long long cap = (long long)sm_count() * 8;

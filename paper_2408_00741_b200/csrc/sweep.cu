@@ -2,14 +2,22 @@
 // tile against the latency/power profile and the SLOs [Sec. 4.1, Eq. 1], and keep the
 // minimum-energy feasible one [Sec. 4.2].
 //
-// Work is plain fp32 arithmetic (no dense contraction, so no tensor cores).  A warp owns one tile at
-// a time: lanes hold instance counts n (several per lane when Nmax > 32), the (TP, f) pairs are the
-// inner loop, so the per-pair constants and the table row are warp-uniform and the per-lane work is
-// one multiply, one table lookup indexed by floor(x), two fused multiply-adds, the feasibility
-// compares and the running minimum.  floor(x) comes from adding 2^23 with round-toward-zero: the low
-// mantissa bits are the segment number, and subtracting 2^23 gives it back as a float, so no
-// float-to-int conversion is issued.  The resolved tables of all classes are staged in shared memory
-// once per CTA when they fit; larger tables are read through L1.
+// Work is plain fp32 arithmetic (no dense contraction, so no tensor cores); the kernel is bound by
+// instruction issue, and within that by the half-rate pipe that executes compares, selects and
+// min/max.  The design keeps work off that pipe:
+//   * a warp owns tiles of ONE class; lanes hold instance counts n (several per lane when Nmax > 32),
+//     the (TP, f) pairs are the inner loop, so per-pair constants and the table row are warp-uniform
+//     and shared by all candidates of the pair;
+//   * table position x = u*(M-1) = sat(L/n * icv) * M: the saturating multiply clamps for free, and
+//     u > 1 is not tested: the table rows end in sentinel entries whose TBT breaks any SLO;
+//   * floor(x) comes from a fused multiply-add with 2^23 rounded toward zero: the low mantissa bits
+//     are the segment number (no float-to-int conversion), and the fraction is a second FMA; these
+//     run two candidates at a time on the packed two-wide fp32 instructions of sm_100;
+//   * one 16-byte shared-memory lookup, addressed in 32 bits straight from those mantissa bits,
+//     gives value and slope of TBT and of the window energy;
+//   * per candidate the half-rate pipe sees: TBT <= SLO, E < best, two selects.
+// The resolved tables of all classes are staged in shared memory once per CTA when they fit; larger
+// tables are read through L1.
 #include "dyn_internal.cuh"
 
 #include <math_constants.h>
@@ -22,79 +30,146 @@ constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr unsigned kFull = 0xffffffffu;
 constexpr float kTwo23 = 8388608.0f;
+constexpr int kTwo23Bits = 0x4b000000;
 
 struct SweepArgs {
-    const float4 *rows;      // [C][P][M]
-    const float *icm;        // [C][P]
+    const float4 *rows;      // [C][P][M+1]
+    const float *icv;        // [C][P]
     const float *slo;        // [C]
     const int32_t *tp;       // [T]
-    const float *load;       // [tiles]
+    const float *load;       // [rows_total][C]
     int64_t tiles;
+    int64_t rows_total;      // S*W
+    int64_t rows_per_warp;   // multiple of the tiles a warp takes per pass
+    int64_t blocks;          // row blocks; work units = blocks * C
     int32_t C, T, F, P, M, Nmax, J;
     int32_t budget;          // <= 0: none
     int32_t ln_log2;         // lanes per n-group = 1 << ln_log2
-    int64_t tiles_per_warp;
-    size_t stage_bytes;      // bytes of [rows | icm | slo] staged in shared memory (0: read from global)
-    size_t off_icm, off_slo; // offsets of icm / slo inside the staged block
+    int32_t stage_bytes;     // bytes of [rows | icv | slo] staged in shared memory (0: read from global)
+    int32_t off_icv, off_slo;  // byte offsets of icv / slo inside the staged block
 };
 
-// order-preserving map float -> uint32 (smaller float <=> smaller key), and back
+// order-preserving map float -> uint32 (smaller float <=> smaller key)
 __device__ __forceinline__ uint32_t float_key(float v) {
     const uint32_t b = __float_as_uint(v);
     return b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
 }
 
-// one candidate: x = u*(M-1); returns energy of the whole pool (n instances) and its feasibility
-__device__ __forceinline__ void eval_one(const float4 *__restrict__ row, float x, float mm1, float slo, float nf,
-                                         float &E, bool &ok) {
-    const float xc = fminf(x, mm1);                       // NaN/inf -> last entry: a safe address
-    const float y = __fadd_rz(xc, kTwo23);                // 2^23 + floor(xc), exactly
-    const int m = __float_as_int(y) - 0x4b000000;
-    const float nu = xc - (y - kTwo23);
-    const float4 e = row[m];
-    const float tbt = fmaf(nu, e.y, e.x);
-    const float ew = fmaf(nu, e.w, e.z);
-    ok = (x <= mm1) && (tbt <= slo);                      // u <= 1 and TBT within its SLO
-    E = nf * ew;
+// Table lookup.  In shared memory the entry address is formed in 32 bits (one multiply-add from the
+// bit pattern of y); `base` is then the byte address of the pair's row minus 16 * bits(2^23).
+// Read through L1 otherwise; `base` is then the entry index of the row minus bits(2^23).
+template <bool SMEM>
+__device__ __forceinline__ float4 table_entry(const float4 *__restrict__ grows, uint32_t base, float y) {
+    if (SMEM) {
+        const uint32_t addr = __float_as_uint(y) * 16u + base;
+        float4 r;
+        asm("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "r"(addr));
+        return r;
+    }
+    return __ldg(grows + int(__float_as_uint(y) + base));
+}
+
+template <bool SMEM>
+__device__ __forceinline__ uint32_t row_base(int row_index) {
+    if (SMEM) {
+        extern __shared__ float4 smem[];
+        return uint32_t(__cvta_generic_to_shared(smem)) + uint32_t(row_index) * 16u - uint32_t(kTwo23Bits) * 16u;
+    }
+    return uint32_t(row_index) - uint32_t(kTwo23Bits);
+}
+
+// best = min(best, E) if ok: one compare and one predicated min on the half-rate pipe
+__device__ __forceinline__ void min_if_within_slo(float &best, float tbt, float slo, float E) {
+    asm("{\n\t.reg .pred p;\n\tsetp.le.f32 p, %1, %2;\n\t@p min.f32 %0, %0, %3;\n\t}"
+        : "+f"(best) : "f"(tbt), "f"(slo), "f"(E));
+}
+
+// Two candidates of one (TP, f) pair at once, on the packed two-wide fp32 instructions of sm_100.
+// ln = L/n per candidate, ic = (M-1)/(M*cap).  v = sat(ln*ic) is the table position over M; y =
+// 2^23 + floor(v*M) (fused multiply-add rounded toward zero), whose low mantissa bits index the row;
+// nnu = floor(v*M) - v*M = -(fraction).  Table entries hold {TBT, -slope, energy, -slope}.  The pool
+// energy n*e enters the running minimum of its chain when TBT meets the SLO (u > 1 and never-feasible
+// pairs show up as TBT = huge or +inf through the sentinel entries).  Which pair attained the minimum
+// is not tracked here: it is recovered once per tile (see recover_pair).
+template <bool SMEM>
+__device__ __forceinline__ void eval_two(const float4 *__restrict__ grows, uint32_t base, float lnA, float lnB,
+                                         float ic, float2 M2, float2 negM2, float2 two23, float2 neg23, float slo,
+                                         float2 nf2, bool allowA, bool allowB, float &bestA, float &bestB) {
+    const float2 v = make_float2(__saturatef(lnA * ic), __saturatef(lnB * ic));   // NaN -> 0, > 1 -> 1
+    const float2 y = __ffma2_rz(v, M2, two23);
+    const float2 fm = __fadd2_rn(y, neg23);
+    const float2 nnu = __ffma2_rn(v, negM2, fm);
+    const float4 eA = table_entry<SMEM>(grows, base, y.x);
+    const float4 eB = table_entry<SMEM>(grows, base, y.y);
+    const float tbtA = fmaf(nnu.x, eA.y, eA.x), tbtB = fmaf(nnu.y, eB.y, eB.x);
+    const float2 ew = make_float2(fmaf(nnu.x, eA.w, eA.z), fmaf(nnu.y, eB.w, eB.z));
+    const float2 E = __fmul2_rn(ew, nf2);
+    if (allowA) min_if_within_slo(bestA, tbtA, slo, E.x);     // allow*: GPU budget (compile-time true without one)
+    if (allowB) min_if_within_slo(bestB, tbtB, slo, E.y);
+}
+
+// scalar form of the same evaluation, bit-identical to eval_two (evaluate-only kernel, pair recovery)
+template <bool SMEM>
+__device__ __forceinline__ void eval_one(const float4 *__restrict__ grows, uint32_t base, float ln, float ic, float Mf,
+                                         float slo, float nf, float &E, bool &ok) {
+    const float v = __saturatef(ln * ic);
+    const float y = __fmaf_rz(v, Mf, kTwo23);
+    const float nnu = fmaf(v, -Mf, y - kTwo23);
+    const float4 e = table_entry<SMEM>(grows, base, y);
+    ok = fmaf(nnu, e.y, e.x) <= slo;
+    E = nf * fmaf(nnu, e.w, e.z);
+}
+
+template <bool SMEM>
+__device__ __forceinline__ void stage_tables(const SweepArgs &a, const float *&icv, const float *&slo) {
+    extern __shared__ float4 smem[];
+    icv = a.icv;
+    slo = a.slo;
+    if (SMEM) {
+        // the staged block has the layout of the scratch block: rows, then icv, then slo
+        const float4 *src = a.rows;
+        const int n16 = a.stage_bytes / 16;
+        for (int i = threadIdx.x; i < n16; i += kThreads) smem[i] = src[i];
+        __syncthreads();
+        icv = reinterpret_cast<const float *>(reinterpret_cast<const char *>(smem) + a.off_icv);
+        slo = reinterpret_cast<const float *>(reinterpret_cast<const char *>(smem) + a.off_slo);
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
 // fused evaluate + select
+//   NPL  instance counts per lane (Nmax <= 32*NPL)
+//   TT   tiles (rows of the same class) a warp evaluates per pass over the pairs
 // ---------------------------------------------------------------------------------------------
-template <int NPL, bool BUDGET, bool SMEM>
-__global__ void __launch_bounds__(kThreads)
+template <int NPL, int TT, bool BUDGET, bool SMEM>
+__global__ void __launch_bounds__(kThreads, (NPL <= 2 ? 4 : 2))
 eval_select_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__restrict__ best_E) {
-    extern __shared__ float4 smem[];
-    const float4 *rows = a.rows;
-    const float *icm = a.icm;
-    const float *slo = a.slo;
-    if (SMEM) {
-        // the staged block has the layout of the scratch block: rows, then icm, then slo
-        const float4 *src = a.rows;
-        const int n16 = int(a.stage_bytes / 16);
-        for (int i = threadIdx.x; i < n16; i += kThreads) smem[i] = src[i];
-        __syncthreads();
-        rows = smem;
-        icm = reinterpret_cast<const float *>(reinterpret_cast<const char *>(smem) + a.off_icm);
-        slo = reinterpret_cast<const float *>(reinterpret_cast<const char *>(smem) + a.off_slo);
-    }
+    const float *icv, *slo;
+    stage_tables<SMEM>(a, icv, slo);
 
     const int lane = threadIdx.x & 31;
-    const int64_t gwarp = int64_t(blockIdx.x) * kWarps + (threadIdx.x >> 5);
+    const int64_t unit = int64_t(blockIdx.x) * kWarps + (threadIdx.x >> 5);
+    if (unit >= a.blocks * a.C) return;
+    const int c = int(unit % a.C);
+    const int64_t r_begin = (unit / a.C) * a.rows_per_warp;
+    const int64_t r_end = r_begin + a.rows_per_warp < a.rows_total ? r_begin + a.rows_per_warp : a.rows_total;
+
     const int LN = 1 << a.ln_log2;
-    const int G = 32 >> a.ln_log2;                  // pair groups inside the warp
+    const int G = 32 >> a.ln_log2;                  // pair groups inside the warp (Nmax < 32)
     const int nl = lane & (LN - 1);
     const int g = lane >> a.ln_log2;
-    const int P = a.P, M = a.M;
-    const float mm1 = float(M - 1);
+    const int P = a.P, RS = a.M + 1, C = a.C;
+    const float Mf = float(a.M);
 
     float nf[NPL], rn[NPL];
     int pmax[NPL];
+    bool valid_n[NPL];
 #pragma unroll
     for (int k = 0; k < NPL; ++k) {
         const int n = nl + 1 + LN * k;
+        valid_n[k] = n <= a.Nmax;
         nf[k] = float(n);
-        rn[k] = n <= a.Nmax ? 1.0f / float(n) : CUDART_INF_F;     // n beyond Nmax: never feasible
+        rn[k] = valid_n[k] ? 1.0f / float(n) : 0.f;
         pmax[k] = P;
         if (BUDGET) {
             int nt = 0;
@@ -103,110 +178,128 @@ eval_select_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__r
         }
     }
 
-    int64_t i = gwarp * a.tiles_per_warp;
-    int64_t i_end = i + a.tiles_per_warp;
-    if (i_end > a.tiles) i_end = a.tiles;
-    if (i >= i_end) return;
-    int c = int(i % a.C);
+    // class constants
+    const float *cicv = icv + c * P;
+    const float slo_c = slo[c];
+    const uint32_t cbase = row_base<SMEM>(c * P * RS);
+    const uint32_t pstep = SMEM ? uint32_t(RS) * 16u : uint32_t(RS);
+    const float2 M2 = make_float2(Mf, Mf), negM2 = make_float2(-Mf, -Mf);
+    const float2 two23 = make_float2(kTwo23, kTwo23), neg23 = make_float2(-kTwo23, -kTwo23);
+    constexpr int NCH = TT * NPL;                    // candidates per lane and pair, an even number
+    static_assert(NCH % 2 == 0, "candidates are evaluated two at a time");
 
-    for (; i < i_end; ++i) {
-        const float L = fmaxf(a.load[i], 0.f);      // negative or NaN load counts as zero
-        const float4 *crow = rows + size_t(c) * P * M;
-        const float *cicm = icm + size_t(c) * P;
-        const float slo_c = slo[c];
-        float Ln[NPL], best[NPL];
-        int bp[NPL];
+    for (int64_t r = r_begin; r < r_end; r += TT) {
+        // chain q = t*NPL + k: tile t of this pass, k-th instance count of the lane
+        float ln[NCH], best[NCH], Lt[TT];
 #pragma unroll
-        for (int k = 0; k < NPL; ++k) {
-            Ln[k] = L * rn[k];
-            best[k] = CUDART_INF_F;
-            bp[k] = 0;
+        for (int t = 0; t < TT; ++t) {
+            Lt[t] = (r + t < r_end) ? fmaxf(a.load[(r + t) * C + c], 0.f) : 0.f;   // negative / NaN -> 0
+#pragma unroll
+            for (int k = 0; k < NPL; ++k) {
+                ln[t * NPL + k] = Lt[t] * rn[k];
+                best[t * NPL + k] = CUDART_INF_F;
+            }
         }
 #pragma unroll 4
         for (int p = g; p < P; p += G) {
-            const float ic = cicm[p];
-            const float4 *row = crow + size_t(p) * M;
+            const float ic = cicv[p];
+            const uint32_t base = cbase + uint32_t(p) * pstep;
+#pragma unroll
+            for (int q = 0; q < NCH; q += 2)
+                eval_two<SMEM>(a.rows, base, ln[q], ln[q + 1], ic, M2, negM2, two23, neg23, slo_c,
+                               make_float2(nf[q % NPL], nf[(q + 1) % NPL]), !BUDGET || p < pmax[q % NPL],
+                               !BUDGET || p < pmax[(q + 1) % NPL], best[q], best[q + 1]);
+        }
+#pragma unroll
+        for (int t = 0; t < TT; ++t) {
+            if (r + t >= r_end) break;               // warp-uniform
+            // the lane's chains in ascending n: strict compare keeps the lower n on ties
+            float E = CUDART_INF_F;
+            int n = 0x7fffffff;
 #pragma unroll
             for (int k = 0; k < NPL; ++k) {
-                float E;
-                bool ok;
-                eval_one(row, Ln[k] * ic, mm1, slo_c, nf[k], E, ok);
-                if (BUDGET) ok = ok && (p < pmax[k]);
-                if (ok && E < best[k]) {            // strict: keeps the lowest pair index on ties
-                    best[k] = E;
-                    bp[k] = p;
+                const float Ek = valid_n[k] ? best[t * NPL + k] + 0.f : CUDART_INF_F;   // -0 -> +0: keys order like floats
+                if (Ek < E) {
+                    E = Ek;
+                    n = nl + 1 + LN * k;
                 }
             }
-        }
-        // the lane's chains in ascending n: strict compare keeps the lower n on ties
-        float E = best[0] + 0.f;                    // -0 -> +0 so that keys order like floats
-        int j = nl * P + bp[0];
-#pragma unroll
-        for (int k = 1; k < NPL; ++k) {
-            const float Ek = best[k] + 0.f;
-            if (Ek < E) {
-                E = Ek;
-                j = (nl + LN * k) * P + bp[k];
+            // warp argmin on (E, n): smallest energy, then fewest instances (lowest index: n is the
+            // slowest digit of j); lanes of different pair groups may hold the same n
+            const uint32_t key = float_key(E);
+            const uint32_t kmin = __reduce_min_sync(kFull, key);
+            const uint32_t nmin = __reduce_min_sync(kFull, key == kmin ? uint32_t(n) : 0xffffffffu);
+            const int64_t i = (r + t) * C + c;
+            if (kmin == float_key(CUDART_INF_F)) {                  // no feasible candidate
+                if (lane == 0) {
+                    best_idx[i] = -1;
+                    best_E[i] = CUDART_INF_F;
+                }
+                continue;
+            }
+            // recover the pair: lanes re-evaluate (nmin, p) for 32 pairs at a time, same arithmetic,
+            // and the first pair that reproduces the minimum bit for bit is the lowest-index one
+            const float Emin = __uint_as_float(kmin ^ ((kmin >> 31) ? 0x80000000u : 0xffffffffu));
+            const float nfm = float(nmin);
+            const float lnm = Lt[t] * (1.0f / nfm);
+            int pm = -1;
+            if (BUDGET) {
+                int nt = 0;
+                for (int tt = 0; tt < a.T; ++tt) nt += (int64_t(nmin) * a.tp[tt] <= int64_t(a.budget)) ? 1 : 0;
+                pm = nt * a.F;
+            }
+            int pstar = -1;
+            for (int p0 = 0; p0 < P && pstar < 0; p0 += 32) {
+                const int pp = p0 + lane;
+                bool hit = false;
+                if (pp < P && (!BUDGET || pp < pm)) {
+                    float Ep;
+                    bool ok;
+                    eval_one<SMEM>(a.rows, cbase + uint32_t(pp) * pstep, lnm, cicv[pp], Mf, slo_c, nfm, Ep, ok);
+                    hit = ok && (Ep + 0.f == Emin);
+                }
+                const unsigned m = __ballot_sync(kFull, hit);
+                if (m) pstar = p0 + __ffs(m) - 1;
+            }
+            if (lane == 0) {
+                best_idx[i] = pstar >= 0 ? int32_t((nmin - 1) * uint32_t(P) + uint32_t(pstar)) : -1;
+                best_E[i] = Emin;
             }
         }
-        // warp argmin on (E, j): smallest energy, then smallest index
-        const uint32_t key = float_key(E);
-        const uint32_t kmin = __reduce_min_sync(kFull, key);
-        const uint32_t jmin = __reduce_min_sync(kFull, key == kmin ? uint32_t(j) : 0xffffffffu);
-        if (kmin != float_key(CUDART_INF_F)) {
-            if (key == kmin && uint32_t(j) == jmin) {           // exactly one lane: j is unique per lane
-                best_idx[i] = j;
-                best_E[i] = E;
-            }
-        } else if (lane == 0) {                                 // no feasible candidate
-            best_idx[i] = -1;
-            best_E[i] = CUDART_INF_F;
-        }
-        if (++c == a.C) c = 0;
     }
 }
 
 // ---------------------------------------------------------------------------------------------
-// evaluate only: E[tile][j]
+// evaluate only: E[tile][j].  A CTA takes whole tiles; threads stride over j so that the row of E
+// is written coalesced; (n, pair) of a thread's next candidate follow by increments, no division.
 // ---------------------------------------------------------------------------------------------
 template <bool SMEM>
 __global__ void __launch_bounds__(kThreads)
-eval_configs_kernel(const SweepArgs a, const FastDiv divP, float *__restrict__ E_out) {
-    extern __shared__ float4 smem[];
-    const float4 *rows = a.rows;
-    const float *icm = a.icm;
-    const float *slo = a.slo;
-    if (SMEM) {
-        const float4 *src = a.rows;
-        const int n16 = int(a.stage_bytes / 16);
-        for (int i = threadIdx.x; i < n16; i += kThreads) smem[i] = src[i];
-        __syncthreads();
-        rows = smem;
-        icm = reinterpret_cast<const float *>(reinterpret_cast<const char *>(smem) + a.off_icm);
-        slo = reinterpret_cast<const float *>(reinterpret_cast<const char *>(smem) + a.off_slo);
-    }
-    const int P = a.P, M = a.M, J = a.J;
-    const float mm1 = float(M - 1);
-    // a CTA takes whole tiles; threads stride over j so that the row of E is written coalesced
+eval_configs_kernel(const SweepArgs a, const int dn, const int dp, float *__restrict__ E_out) {
+    const float *icv, *slo;
+    stage_tables<SMEM>(a, icv, slo);
+    const int P = a.P, RS = a.M + 1, J = a.J;
+    const float Mf = float(a.M);
+    const int n1_0 = int(threadIdx.x) / P, p_0 = int(threadIdx.x) - n1_0 * P;
     for (int64_t i = blockIdx.x; i < a.tiles; i += gridDim.x) {
         const int c = int(i % a.C);
         const float L = fmaxf(a.load[i], 0.f);
-        const float4 *crow = rows + size_t(c) * P * M;
-        const float *cicm = icm + size_t(c) * P;
+        const float *cicv = icv + c * P;
         const float slo_c = slo[c];
+        const uint32_t cbase = row_base<SMEM>(c * P * RS);
+        const uint32_t pstep = SMEM ? uint32_t(RS) * 16u : uint32_t(RS);
         float *out = E_out + size_t(i) * size_t(J);
+        int n1 = n1_0, p = p_0;                       // n - 1 and pair of candidate j
         for (int j = threadIdx.x; j < J; j += kThreads) {
-            const int n1 = int(fastdiv(uint32_t(j), divP));      // n - 1
-            const int p = j - n1 * P;
             const float nf = float(n1 + 1);
             float E;
             bool ok;
-            eval_one(crow + size_t(p) * M, (L / nf) * cicm[p], mm1, slo_c, nf, E, ok);
-            if (a.budget > 0) {
-                const int t = p / a.F;
-                ok = ok && (int64_t(n1 + 1) * a.tp[t] <= int64_t(a.budget));
-            }
+            eval_one<SMEM>(a.rows, cbase + uint32_t(p) * pstep, __fdividef(L, nf), cicv[p], Mf, slo_c, nf, E, ok);
+            if (a.budget > 0) ok = ok && (int64_t(n1 + 1) * a.tp[p / a.F] <= int64_t(a.budget));
             out[j] = ok ? E : CUDART_INF_F;
+            n1 += dn;
+            p += dp;
+            if (p >= P) { p -= P; ++n1; }
         }
     }
 }
@@ -226,41 +319,54 @@ SweepArgs make_args(const ResolvedLayout &lay, const void *d_ws, const float *d_
     const char *ws = static_cast<const char *>(d_ws);
     SweepArgs a{};
     a.rows = reinterpret_cast<const float4 *>(ws + lay.off_rows);
-    a.icm = reinterpret_cast<const float *>(ws + lay.off_icm);
+    a.icv = reinterpret_cast<const float *>(ws + lay.off_icm);
     a.slo = reinterpret_cast<const float *>(ws + lay.off_slo);
     a.tp = reinterpret_cast<const int32_t *>(ws + lay.off_tp);
     a.load = d_load;
     a.tiles = tiles;
+    a.rows_total = tiles / lay.C;
     a.C = lay.C; a.T = lay.T; a.F = lay.F; a.P = lay.P; a.M = lay.M; a.Nmax = lay.Nmax; a.J = lay.J;
     a.budget = budget;
-    // rows, icm and slo are consecutive in the scratch block: stage them as one piece when it fits
+    // rows, icv and slo are consecutive in the scratch block: stage them as one piece when it fits
     const size_t block = lay.off_tp - lay.off_rows;
-    a.stage_bytes = block <= 96 * 1024 && block <= smem_limit() ? block : 0;
-    a.off_icm = lay.off_icm - lay.off_rows;
-    a.off_slo = lay.off_slo - lay.off_rows;
+    a.stage_bytes = block <= 96 * 1024 && block <= smem_limit() ? int32_t(block) : 0;
+    a.off_icv = int32_t(lay.off_icm - lay.off_rows);
+    a.off_slo = int32_t(lay.off_slo - lay.off_rows);
     return a;
 }
 
-template <int NPL>
-cudaError_t launch_es(const SweepArgs &a, int grid, int32_t *best_idx, float *best_E, cudaStream_t st) {
+template <int NPL, int TT, bool B, bool S>
+cudaError_t launch_es_variant(SweepArgs &a, int32_t *best_idx, float *best_E, cudaStream_t st) {
+    auto kernel = eval_select_kernel<NPL, TT, B, S>;
+    cudaError_t e = cudaSuccess;
+    if (S) {
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, a.stage_bytes);
+        if (e != cudaSuccess) return e;
+    }
+    int resident = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kernel, kThreads, S ? size_t(a.stage_bytes) : 0);
+    if (e != cudaSuccess) return e;
+    if (resident < 1) resident = 1;
+    // about four work units per resident warp: all units cost the same, so the tail is short
+    const int64_t want_units = int64_t(sm_count()) * resident * kWarps * 4;
+    int64_t rpw = (a.tiles + want_units - 1) / want_units;          // rows of one class per unit
+    rpw = (rpw + TT - 1) / TT * TT;
+    a.rows_per_warp = rpw;
+    a.blocks = (a.rows_total + rpw - 1) / rpw;
+    const int64_t units = a.blocks * a.C;
+    const int64_t grid = (units + kWarps - 1) / kWarps;
+    kernel<<<unsigned(grid), kThreads, S ? size_t(a.stage_bytes) : 0, st>>>(a, best_idx, best_E);
+    return cudaGetLastError();
+}
+
+template <int NPL, int TT>
+cudaError_t launch_es(SweepArgs &a, int32_t *best_idx, float *best_E, cudaStream_t st) {
     const bool smem = a.stage_bytes > 0;
     const bool budget = a.budget > 0;
-    cudaError_t e = cudaSuccess;
-#define DYN_LAUNCH_ES(B, S)                                                                                       \
-    do {                                                                                                          \
-        if (S) e = cudaFuncSetAttribute(eval_select_kernel<NPL, B, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                        int(a.stage_bytes));                                                      \
-        if (e == cudaSuccess) {                                                                                   \
-            eval_select_kernel<NPL, B, S><<<grid, kThreads, S ? a.stage_bytes : 0, st>>>(a, best_idx, best_E);    \
-            e = cudaGetLastError();                                                                               \
-        }                                                                                                         \
-    } while (0)
-    if (budget && smem) DYN_LAUNCH_ES(true, true);
-    else if (budget) DYN_LAUNCH_ES(true, false);
-    else if (smem) DYN_LAUNCH_ES(false, true);
-    else DYN_LAUNCH_ES(false, false);
-#undef DYN_LAUNCH_ES
-    return e;
+    if (budget && smem) return launch_es_variant<NPL, TT, true, true>(a, best_idx, best_E, st);
+    if (budget) return launch_es_variant<NPL, TT, true, false>(a, best_idx, best_E, st);
+    if (smem) return launch_es_variant<NPL, TT, false, true>(a, best_idx, best_E, st);
+    return launch_es_variant<NPL, TT, false, false>(a, best_idx, best_E, st);
 }
 
 }  // namespace
@@ -274,16 +380,11 @@ cudaError_t launch_eval_select(const ResolvedLayout &lay, const void *d_ws, cons
     while ((1 << ln) < lay.Nmax && ln < 5) ++ln;
     a.ln_log2 = ln;
     const int npl = (lay.Nmax + 31) / 32;           // instance counts per lane
-    // resident CTAs: 4 per SM; each warp takes a contiguous run of tiles
-    int64_t grid = int64_t(sm_count()) * 4;
-    const int64_t need = (tiles + kWarps - 1) / kWarps;
-    if (grid > need) grid = need;
-    a.tiles_per_warp = (tiles + grid * kWarps - 1) / (grid * kWarps);
-    grid = (tiles + a.tiles_per_warp * kWarps - 1) / (a.tiles_per_warp * kWarps);
-    if (npl <= 1) return launch_es<1>(a, int(grid), best_idx, best_E, st);
-    if (npl <= 2) return launch_es<2>(a, int(grid), best_idx, best_E, st);
-    if (npl <= 4) return launch_es<4>(a, int(grid), best_idx, best_E, st);
-    if (npl <= 8) return launch_es<8>(a, int(grid), best_idx, best_E, st);
+    // four candidates per lane share each pair's constants
+    if (npl <= 1) return launch_es<1, 4>(a, best_idx, best_E, st);
+    if (npl <= 2) return launch_es<2, 2>(a, best_idx, best_E, st);
+    if (npl <= 4) return launch_es<4, 1>(a, best_idx, best_E, st);
+    if (npl <= 8) return launch_es<8, 1>(a, best_idx, best_E, st);
     return cudaErrorInvalidValue;                   // Nmax > 256 is rejected by the caller
 }
 
@@ -293,15 +394,14 @@ cudaError_t launch_eval_configs(const ResolvedLayout &lay, const void *d_ws, con
     SweepArgs a = make_args(lay, d_ws, d_load, tiles, gpu_budget);
     int64_t grid = int64_t(sm_count()) * 8;
     if (grid > tiles) grid = tiles;
-    const FastDiv divP = make_fastdiv(uint32_t(lay.P));
+    const int dn = kThreads / lay.P, dp = kThreads % lay.P;
     cudaError_t e = cudaSuccess;
     if (a.stage_bytes > 0) {
-        e = cudaFuncSetAttribute(eval_configs_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 int(a.stage_bytes));
+        e = cudaFuncSetAttribute(eval_configs_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, a.stage_bytes);
         if (e != cudaSuccess) return e;
-        eval_configs_kernel<true><<<int(grid), kThreads, a.stage_bytes, st>>>(a, divP, d_E);
+        eval_configs_kernel<true><<<int(grid), kThreads, size_t(a.stage_bytes), st>>>(a, dn, dp, d_E);
     } else {
-        eval_configs_kernel<false><<<int(grid), kThreads, 0, st>>>(a, divP, d_E);
+        eval_configs_kernel<false><<<int(grid), kThreads, 0, st>>>(a, dn, dp, d_E);
     }
     return cudaGetLastError();
 }
