@@ -61,7 +61,7 @@ int check_problem(const dyn_profile *p, const dyn_space *sp, int64_t S, int64_t 
         return DYN_EINVAL;
     const int64_t J = int64_t(sp->Nmax) * p->T * sp->F;
     if (J >= (int64_t(1) << 31)) return DYN_EINVAL;
-    if (int64_t(p->C) * p->T * sp->F * (p->M + 1) >= (int64_t(1) << 28)) return DYN_EUNSUPPORTED;   // table entries
+    if (int64_t(p->C) * p->T * sp->F * (p->M + 1) >= (int64_t(1) << 26)) return DYN_EUNSUPPORTED;   // table entries
     if (S > 0 && W > 0 && (S > (int64_t(1) << 40) / W || S * W > (int64_t(1) << 40) / p->C)) return DYN_EINVAL;
     if (sp->f_cand_mhz[0] < p->f_grid_mhz[0] || sp->f_cand_mhz[sp->F - 1] > p->f_grid_mhz[p->R - 1])
         return DYN_EUNSUPPORTED;

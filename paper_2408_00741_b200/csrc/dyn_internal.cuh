@@ -45,19 +45,22 @@ __device__ __forceinline__ uint32_t fastdiv(uint32_t n, const FastDiv &f) {
 }
 
 // ---- resolved candidate tables (scratch memory) ----------------------------------------------
-// For class c and pair p = t*F + q (P = T*F pairs), with x = u*(M-1) the table position:
-//   icv[c][p]       (M-1)/(M*cap(c,t,f_q)): x = sat(L/n * icv) * M; 0 for a pair that is never feasible
+// For class c and pair p = t*F + q (P = T*F pairs), with x = u*(M-1) the table position and
+// v = x/M = sat(L/n * ic):
 //   rows[c][p][m]   m = 0..M, float4 {tbt_a, -tbt_d, e_a, -e_d}: on segment m (x in [m, m+1])
 //                   TBT(x) = tbt_a + (x-m)*tbt_d and the window energy of ONE instance is
-//                   e(x) = e_a + (x-m)*e_d (Wh); slopes are stored negated.  Entry M-1 is the last knot with a huge TBT slope and
-//                   entry M has TBT = +inf, so u > 1 shows up as an SLO violation; a pair whose TTFT
-//                   misses its SLO has TBT = +inf everywhere.
+//                   e(x) = e_a + (x-m)*e_d (Wh); slopes are stored negated.  Entry M-1 is the last
+//                   knot with a huge TBT slope and entry M has TBT = +inf, so u > 1 shows up as an SLO
+//                   violation; a pair whose TTFT misses its SLO has TBT = +inf everywhere.
+//   pairc[c][p]     float2 {ic, vlim}: ic = (M-1)/(M*cap(c,t,f_q)) (0 for a never-feasible pair);
+//                   vlim = largest v with TBT <= slo_tbt[c] and u <= 1 when TBT does not decrease
+//                   along the row (-1 for a never-feasible pair), NaN when it does decrease somewhere.
 //   slo[c]          slo_tbt[c]
+//   rows2[c][p][m]  m = 0..M, float2 {e_a, -e_d}: the energy half of rows, for the threshold path
 struct ResolvedLayout {
     int32_t C, T, F, P, M, Nmax, J;
-    int32_t row_stride;          // float4 entries per pair row (M + 1)
-    size_t off_icm, off_rows, off_slo, off_tp, off_partial, off_njtj, total;
-    size_t class_rows_bytes;     // bytes of rows[c]
+    int32_t row_stride;          // entries per pair row (M + 1)
+    size_t off_rows, off_pairc, off_slo, off_rows2, off_tp, off_partial, total;
 };
 
 ResolvedLayout resolved_layout(int32_t C, int32_t T, int32_t F, int32_t M, int32_t Nmax, int64_t S, int64_t W);

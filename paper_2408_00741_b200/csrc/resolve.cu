@@ -23,16 +23,16 @@ ResolvedLayout resolved_layout(int32_t C, int32_t T, int32_t F, int32_t M, int32
     l.C = C; l.T = T; l.F = F; l.P = T * F; l.M = M; l.Nmax = Nmax;
     l.J = Nmax * T * F;
     l.row_stride = M + 1;
+    const size_t entries = size_t(C) * size_t(l.P) * size_t(l.row_stride);
     size_t off = 0;
-    l.off_rows = off;
-    l.class_rows_bytes = size_t(l.P) * size_t(l.row_stride) * sizeof(float4);
-    off = align_up(off + size_t(C) * l.class_rows_bytes, 256);
-    l.off_icm = off;  off = align_up(off + size_t(C) * size_t(l.P) * sizeof(float), 256);
-    l.off_slo = off;  off = align_up(off + size_t(C) * sizeof(float), 256);
-    l.off_tp = off;   off = align_up(off + size_t(T) * sizeof(int32_t), 256);
+    // rows | pairc | slo | rows2 are contiguous: the sweep stages rows..slo or pairc..rows2 as one piece
+    l.off_rows = off;   off = align_up(off + entries * sizeof(float4), 256);
+    l.off_pairc = off;  off = align_up(off + size_t(C) * size_t(l.P) * sizeof(float2), 256);
+    l.off_slo = off;    off = align_up(off + size_t(C) * sizeof(float), 256);
+    l.off_rows2 = off;  off = align_up(off + entries * sizeof(float2), 256);
+    l.off_tp = off;     off = align_up(off + size_t(T) * sizeof(int32_t), 256);
     l.off_partial = off;
     off = align_up(off + size_t(S) * size_t(totals_chunks(W)) * (sizeof(double) + sizeof(uint32_t)), 256);
-    l.off_njtj = off;
     l.total = off;
     return l;
 }
@@ -48,8 +48,8 @@ __device__ __forceinline__ double lerp64(double a, double b, double w) { return 
 //             x above M-1 (u > 1) reads as an SLO violation without a separate capacity test
 //   m == M    x saturated (u >= M/(M-1)): TBT = +inf
 // A pair whose TTFT misses its SLO, or whose capacity is not positive, gets TBT = +inf in every entry.
-__global__ void resolve_kernel(const ResolveParams rp, float4 *__restrict__ rows, float *__restrict__ icv,
-                               float *__restrict__ slo, int32_t *__restrict__ tp) {
+__global__ void resolve_kernel(const ResolveParams rp, float4 *__restrict__ rows, float2 *__restrict__ pairc,
+                               float *__restrict__ slo, float2 *__restrict__ rows2, int32_t *__restrict__ tp) {
     const int P = rp.T * rp.F;
     const int M = rp.M;
     const int RS = M + 1;
@@ -87,9 +87,26 @@ __global__ void resolve_kernel(const ResolveParams rp, float4 *__restrict__ rows
         }
         if (!pair_ok) v.x = kInf;
         rows[(size_t(c) * P + p) * RS + m] = v;
+        rows2[(size_t(c) * P + p) * RS + m] = make_float2(v.z, v.w);
         if (m == 0) {
-            // x = u*(M-1) is formed as sat(L/n * icv) * M, so that saturation at 1 means x = M
-            icv[size_t(c) * P + p] = pair_ok ? float(double(M - 1) / (double(M) * cap)) : 0.f;
+            // Load threshold of the pair: if TBT never decreases along the row, "TBT <= slo and u <= 1"
+            // holds exactly for x in [0, xlim].  NaN marks a row without that property.
+            const double slo_c = double(rp.slo_tbt[c]);
+            double vlim = -1.0;
+            bool monotone = true;
+            double prev = lerp64(tb0[0], tb1[0], w);
+            double xlim = prev <= slo_c ? 0.0 : -1.0;
+            for (int k = 1; k < M; ++k) {
+                const double cur = lerp64(tb0[k], tb1[k], w);
+                if (!(cur >= prev)) monotone = false;
+                if (cur <= slo_c) xlim = double(k);
+                else if (prev <= slo_c) xlim = double(k - 1) + (slo_c - prev) / (cur - prev);
+                prev = cur;
+            }
+            if (pair_ok && xlim >= 0.0) vlim = xlim / double(M);
+            // x = u*(M-1) is formed as sat(L/n * ic) * M, so that saturation at 1 means x = M
+            pairc[size_t(c) * P + p] = make_float2(pair_ok ? float(double(M - 1) / (double(M) * cap)) : 0.f,
+                                                   monotone ? float(vlim) : __int_as_float(0x7fc00000));
             if (p == 0) slo[c] = rp.slo_tbt[c];
             if (c == 0 && p < rp.T) tp[p] = rp.tp[p];
         }
@@ -107,8 +124,9 @@ cudaError_t launch_resolve(const ResolveParams &rp, const ResolvedLayout &lay, v
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     resolve_kernel<<<int(blocks), threads, 0, st>>>(rp, reinterpret_cast<float4 *>(ws + lay.off_rows),
-                                                    reinterpret_cast<float *>(ws + lay.off_icm),
+                                                    reinterpret_cast<float2 *>(ws + lay.off_pairc),
                                                     reinterpret_cast<float *>(ws + lay.off_slo),
+                                                    reinterpret_cast<float2 *>(ws + lay.off_rows2),
                                                     reinterpret_cast<int32_t *>(ws + lay.off_tp));
     return cudaGetLastError();
 }

@@ -3,19 +3,23 @@
 // minimum-energy feasible one [Sec. 4.2].
 //
 // Work is plain fp32 arithmetic (no dense contraction, so no tensor cores); the kernel is bound by
-// instruction issue, and within that by the half-rate pipe that executes compares, selects and
-// min/max.  The design keeps work off that pipe:
+// instruction issue and by shared-memory lookups.  The design keeps both low:
 //   * a warp owns tiles of ONE class; lanes hold instance counts n (several per lane when Nmax > 32),
 //     the (TP, f) pairs are the inner loop, so per-pair constants and the table row are warp-uniform
 //     and shared by all candidates of the pair;
-//   * table position x = u*(M-1) = sat(L/n * icv) * M: the saturating multiply clamps for free, and
+//   * table position x = u*(M-1) = sat(L/n * ic) * M: the saturating multiply clamps for free, and
 //     u > 1 is not tested: the table rows end in sentinel entries whose TBT breaks any SLO;
 //   * floor(x) comes from a fused multiply-add with 2^23 rounded toward zero: the low mantissa bits
 //     are the segment number (no float-to-int conversion), and the fraction is a second FMA; these
 //     run two candidates at a time on the packed two-wide fp32 instructions of sm_100;
-//   * one 16-byte shared-memory lookup, addressed in 32 bits straight from those mantissa bits,
-//     gives value and slope of TBT and of the window energy;
-//   * per candidate the half-rate pipe sees: TBT <= SLO, E < best, two selects.
+//   * one shared-memory lookup, addressed in 32 bits straight from those mantissa bits;
+//   * only the running minimum is kept per candidate chain (one compare, one predicated min); the
+//     pair that attained it is recovered once per tile by re-evaluating that instance count for 32
+//     pairs at a time with bit-identical arithmetic;
+//   * when TBT never decreases with load in any table row (the resolve step checks), "TBT <= SLO and
+//     u <= 1" is a threshold on the table position (the largest load an instance sustains within the
+//     SLO, cf. ML in Sec. 4.2), so TBT is not interpolated per candidate and the lookup shrinks from
+//     16 to 8 bytes; otherwise the general path interpolates TBT for every candidate.
 // The resolved tables of all classes are staged in shared memory once per CTA when they fit; larger
 // tables are read through L1.
 #include "dyn_internal.cuh"
@@ -30,14 +34,12 @@ constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr unsigned kFull = 0xffffffffu;
 constexpr float kTwo23 = 8388608.0f;
-constexpr int kTwo23Bits = 0x4b000000;
+constexpr uint32_t kTwo23Bits = 0x4b000000u;
 
 struct SweepArgs {
-    const float4 *rows;      // [C][P][M+1]
-    const float *icv;        // [C][P]
-    const float *slo;        // [C]
-    const int32_t *tp;       // [T]
+    const char *ws;          // scratch block: rows (float4) | pairc (float2) | slo | rows2 (float2) | tp ...
     const float *load;       // [rows_total][C]
+    const int32_t *tp;       // [T]
     int64_t tiles;
     int64_t rows_total;      // S*W
     int64_t rows_per_warp;   // multiple of the tiles a warp takes per pass
@@ -45,8 +47,13 @@ struct SweepArgs {
     int32_t C, T, F, P, M, Nmax, J;
     int32_t budget;          // <= 0: none
     int32_t ln_log2;         // lanes per n-group = 1 << ln_log2
-    int32_t stage_bytes;     // bytes of [rows | icv | slo] staged in shared memory (0: read from global)
-    int32_t off_icv, off_slo;  // byte offsets of icv / slo inside the staged block
+    int32_t off_rows, off_pairc, off_slo, off_rows2, off_end;   // byte offsets inside ws
+    int32_t smem_bytes;      // dynamic shared memory of the launch (0: tables are read from global)
+};
+
+// where the tables of this CTA live: byte offsets from `smem` when staged, else from a.ws
+struct Tables {
+    uint32_t rows, pairc, slo, rows2;
 };
 
 // order-preserving map float -> uint32 (smaller float <=> smaller key)
@@ -55,85 +62,119 @@ __device__ __forceinline__ uint32_t float_key(float v) {
     return b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
 }
 
-// Table lookup.  In shared memory the entry address is formed in 32 bits (one multiply-add from the
-// bit pattern of y); `base` is then the byte address of the pair's row minus 16 * bits(2^23).
-// Read through L1 otherwise; `base` is then the entry index of the row minus bits(2^23).
+// ---- table access -----------------------------------------------------------------------------
+// `base` is the byte address of the pair's row minus ESZ * bits(2^23): the entry address is one
+// multiply-add away from the bit pattern of y = 2^23 + floor(x).  Shared memory is addressed in 32 bits.
 template <bool SMEM>
-__device__ __forceinline__ float4 table_entry(const float4 *__restrict__ grows, uint32_t base, float y) {
+__device__ __forceinline__ float4 entry16(const char *__restrict__ ws, uint32_t base, float y) {
+    const uint32_t addr = __float_as_uint(y) * 16u + base;
     if (SMEM) {
-        const uint32_t addr = __float_as_uint(y) * 16u + base;
         float4 r;
         asm("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "r"(addr));
         return r;
     }
-    return __ldg(grows + int(__float_as_uint(y) + base));
+    return __ldg(reinterpret_cast<const float4 *>(ws + addr));
 }
-
 template <bool SMEM>
-__device__ __forceinline__ uint32_t row_base(int row_index) {
+__device__ __forceinline__ float2 entry8(const char *__restrict__ ws, uint32_t base, float y) {
+    const uint32_t addr = __float_as_uint(y) * 8u + base;
+    if (SMEM) {
+        float2 r;
+        asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(r.x), "=f"(r.y) : "r"(addr));
+        return r;
+    }
+    return __ldg(reinterpret_cast<const float2 *>(ws + addr));
+}
+template <bool SMEM>
+__device__ __forceinline__ float2 pair_consts(const char *__restrict__ ws, uint32_t addr) {   // {ic, vlim}
+    if (SMEM) {
+        float2 r;
+        asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(r.x), "=f"(r.y) : "r"(addr));
+        return r;
+    }
+    return __ldg(reinterpret_cast<const float2 *>(ws + addr));
+}
+template <bool SMEM>
+__device__ __forceinline__ uint32_t table_origin() {
     if (SMEM) {
         extern __shared__ float4 smem[];
-        return uint32_t(__cvta_generic_to_shared(smem)) + uint32_t(row_index) * 16u - uint32_t(kTwo23Bits) * 16u;
+        return uint32_t(__cvta_generic_to_shared(smem));
     }
-    return uint32_t(row_index) - uint32_t(kTwo23Bits);
+    return 0u;
 }
 
-// best = min(best, E) if ok: one compare and one predicated min on the half-rate pipe
-__device__ __forceinline__ void min_if_within_slo(float &best, float tbt, float slo, float E) {
+// best = min(best, E) if a <= b: one compare and one predicated min
+__device__ __forceinline__ void min_if_le(float &best, float a, float b, float E) {
     asm("{\n\t.reg .pred p;\n\tsetp.le.f32 p, %1, %2;\n\t@p min.f32 %0, %0, %3;\n\t}"
-        : "+f"(best) : "f"(tbt), "f"(slo), "f"(E));
+        : "+f"(best) : "f"(a), "f"(b), "f"(E));
 }
 
-// Two candidates of one (TP, f) pair at once, on the packed two-wide fp32 instructions of sm_100.
-// ln = L/n per candidate, ic = (M-1)/(M*cap).  v = sat(ln*ic) is the table position over M; y =
-// 2^23 + floor(v*M) (fused multiply-add rounded toward zero), whose low mantissa bits index the row;
-// nnu = floor(v*M) - v*M = -(fraction).  Table entries hold {TBT, -slope, energy, -slope}.  The pool
-// energy n*e enters the running minimum of its chain when TBT meets the SLO (u > 1 and never-feasible
-// pairs show up as TBT = huge or +inf through the sentinel entries).  Which pair attained the minimum
-// is not tracked here: it is recovered once per tile (see recover_pair).
-template <bool SMEM>
-__device__ __forceinline__ void eval_two(const float4 *__restrict__ grows, uint32_t base, float lnA, float lnB,
-                                         float ic, float2 M2, float2 negM2, float2 two23, float2 neg23, float slo,
-                                         float2 nf2, bool allowA, bool allowB, float &bestA, float &bestB) {
+struct Consts2 {            // the same constant in both halves of a register pair
+    float2 M, negM, two23, neg23;
+};
+
+// Two candidates of one (TP, f) pair at once.  ln = L/n per candidate, ic = (M-1)/(M*cap).
+// v = sat(ln*ic) is the table position over M; y = 2^23 + floor(v*M); nnu = floor(v*M) - v*M.
+// FAST: entries {energy, -slope}, feasible iff v <= vlim.  General: entries {TBT, -slope, energy,
+// -slope}, feasible iff TBT <= slo (u > 1 and never-feasible pairs read as TBT = huge or +inf through
+// the sentinel entries).  The pool energy n*e enters the running minimum of its chain when feasible.
+template <bool SMEM, bool FAST>
+__device__ __forceinline__ void eval_two(const char *__restrict__ ws, uint32_t base, float lnA, float lnB, float ic,
+                                         float lim, const Consts2 &k, float2 nf2, bool allowA, bool allowB,
+                                         float &bestA, float &bestB) {
     const float2 v = make_float2(__saturatef(lnA * ic), __saturatef(lnB * ic));   // NaN -> 0, > 1 -> 1
-    const float2 y = __ffma2_rz(v, M2, two23);
-    const float2 fm = __fadd2_rn(y, neg23);
-    const float2 nnu = __ffma2_rn(v, negM2, fm);
-    const float4 eA = table_entry<SMEM>(grows, base, y.x);
-    const float4 eB = table_entry<SMEM>(grows, base, y.y);
-    const float tbtA = fmaf(nnu.x, eA.y, eA.x), tbtB = fmaf(nnu.y, eB.y, eB.x);
-    const float2 ew = make_float2(fmaf(nnu.x, eA.w, eA.z), fmaf(nnu.y, eB.w, eB.z));
-    const float2 E = __fmul2_rn(ew, nf2);
-    if (allowA) min_if_within_slo(bestA, tbtA, slo, E.x);     // allow*: GPU budget (compile-time true without one)
-    if (allowB) min_if_within_slo(bestB, tbtB, slo, E.y);
+    const float2 y = __ffma2_rz(v, k.M, k.two23);
+    const float2 fm = __fadd2_rn(y, k.neg23);
+    const float2 nnu = __ffma2_rn(v, k.negM, fm);
+    if (FAST) {
+        const float2 eA = entry8<SMEM>(ws, base, y.x);
+        const float2 eB = entry8<SMEM>(ws, base, y.y);
+        const float2 E = __fmul2_rn(make_float2(fmaf(nnu.x, eA.y, eA.x), fmaf(nnu.y, eB.y, eB.x)), nf2);
+        if (allowA) min_if_le(bestA, v.x, lim, E.x);          // allow*: GPU budget (always true without one)
+        if (allowB) min_if_le(bestB, v.y, lim, E.y);
+    } else {
+        const float4 eA = entry16<SMEM>(ws, base, y.x);
+        const float4 eB = entry16<SMEM>(ws, base, y.y);
+        const float tbtA = fmaf(nnu.x, eA.y, eA.x), tbtB = fmaf(nnu.y, eB.y, eB.x);
+        const float2 E = __fmul2_rn(make_float2(fmaf(nnu.x, eA.w, eA.z), fmaf(nnu.y, eB.w, eB.z)), nf2);
+        if (allowA) min_if_le(bestA, tbtA, lim, E.x);
+        if (allowB) min_if_le(bestB, tbtB, lim, E.y);
+    }
 }
 
 // scalar form of the same evaluation, bit-identical to eval_two (evaluate-only kernel, pair recovery)
-template <bool SMEM>
-__device__ __forceinline__ void eval_one(const float4 *__restrict__ grows, uint32_t base, float ln, float ic, float Mf,
-                                         float slo, float nf, float &E, bool &ok) {
+template <bool SMEM, bool FAST>
+__device__ __forceinline__ void eval_one(const char *__restrict__ ws, uint32_t base, float ln, float ic, float lim,
+                                         float Mf, float nf, float &E, bool &ok) {
     const float v = __saturatef(ln * ic);
     const float y = __fmaf_rz(v, Mf, kTwo23);
-    const float nnu = fmaf(v, -Mf, y - kTwo23);
-    const float4 e = table_entry<SMEM>(grows, base, y);
-    ok = fmaf(nnu, e.y, e.x) <= slo;
-    E = nf * fmaf(nnu, e.w, e.z);
+    const float nnu = fmaf(v, -Mf, y + (-kTwo23));
+    if (FAST) {
+        const float2 e = entry8<SMEM>(ws, base, y);
+        ok = v <= lim;
+        E = fmaf(nnu, e.y, e.x) * nf;
+    } else {
+        const float4 e = entry16<SMEM>(ws, base, y);
+        ok = fmaf(nnu, e.y, e.x) <= lim;
+        E = fmaf(nnu, e.w, e.z) * nf;
+    }
 }
 
-template <bool SMEM>
-__device__ __forceinline__ void stage_tables(const SweepArgs &a, const float *&icv, const float *&slo) {
+// copy [ws + from, ws + to) into shared memory (16-byte pieces)
+__device__ __forceinline__ void stage(const SweepArgs &a, int from, int to) {
     extern __shared__ float4 smem[];
-    icv = a.icv;
-    slo = a.slo;
-    if (SMEM) {
-        // the staged block has the layout of the scratch block: rows, then icv, then slo
-        const float4 *src = a.rows;
-        const int n16 = a.stage_bytes / 16;
-        for (int i = threadIdx.x; i < n16; i += kThreads) smem[i] = src[i];
-        __syncthreads();
-        icv = reinterpret_cast<const float *>(reinterpret_cast<const char *>(smem) + a.off_icv);
-        slo = reinterpret_cast<const float *>(reinterpret_cast<const char *>(smem) + a.off_slo);
-    }
+    const float4 *src = reinterpret_cast<const float4 *>(a.ws + from);
+    const int n16 = (to - from) / 16;
+    for (int i = threadIdx.x; i < n16; i += kThreads) smem[i] = src[i];
+    __syncthreads();
+}
+
+// true when every pair row has a load threshold (vlim is NaN for a row whose TBT decreases somewhere)
+__device__ __forceinline__ bool all_rows_monotone(const SweepArgs &a) {
+    const float2 *pc = reinterpret_cast<const float2 *>(a.ws + a.off_pairc);
+    int bad = 0;
+    for (int i = threadIdx.x; i < a.C * a.P; i += kThreads) bad |= isnan(__ldg(pc + i).y) ? 1 : 0;
+    return __syncthreads_or(bad) == 0;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -141,12 +182,9 @@ __device__ __forceinline__ void stage_tables(const SweepArgs &a, const float *&i
 //   NPL  instance counts per lane (Nmax <= 32*NPL)
 //   TT   tiles (rows of the same class) a warp evaluates per pass over the pairs
 // ---------------------------------------------------------------------------------------------
-template <int NPL, int TT, bool BUDGET, bool SMEM>
-__global__ void __launch_bounds__(kThreads, (NPL <= 2 ? 4 : 2))
-eval_select_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__restrict__ best_E) {
-    const float *icv, *slo;
-    stage_tables<SMEM>(a, icv, slo);
-
+template <int NPL, int TT, bool BUDGET, bool SMEM, bool FAST>
+__device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, int32_t *__restrict__ best_idx,
+                                           float *__restrict__ best_E) {
     const int lane = threadIdx.x & 31;
     const int64_t unit = int64_t(blockIdx.x) * kWarps + (threadIdx.x >> 5);
     if (unit >= a.blocks * a.C) return;
@@ -160,6 +198,7 @@ eval_select_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__r
     const int g = lane >> a.ln_log2;
     const int P = a.P, RS = a.M + 1, C = a.C;
     const float Mf = float(a.M);
+    const char *ws = a.ws;
 
     float nf[NPL], rn[NPL];
     int pmax[NPL];
@@ -179,12 +218,26 @@ eval_select_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__r
     }
 
     // class constants
-    const float *cicv = icv + c * P;
-    const float slo_c = slo[c];
-    const uint32_t cbase = row_base<SMEM>(c * P * RS);
-    const uint32_t pstep = SMEM ? uint32_t(RS) * 16u : uint32_t(RS);
-    const float2 M2 = make_float2(Mf, Mf), negM2 = make_float2(-Mf, -Mf);
-    const float2 two23 = make_float2(kTwo23, kTwo23), neg23 = make_float2(-kTwo23, -kTwo23);
+    constexpr uint32_t ESZ = FAST ? 8u : 16u;
+    uint32_t origin = table_origin<SMEM>();
+    // every table address below derives from `origin`: this keeps the (side-effect free) inline-assembly
+    // loads from being scheduled ahead of the barrier that ends the staging
+    asm volatile("" : "+r"(origin) : : "memory");
+    const uint32_t cpair = origin + tb.pairc + uint32_t(c * P) * 8u;
+    const uint32_t cbase = origin + (FAST ? tb.rows2 : tb.rows) + uint32_t(c * P * RS) * ESZ - kTwo23Bits * ESZ;
+    const uint32_t pstep = uint32_t(RS) * ESZ;
+    float slo_c;
+    if (SMEM) {
+        extern __shared__ float4 smem[];
+        slo_c = reinterpret_cast<const float *>(reinterpret_cast<const char *>(smem) + tb.slo)[c];
+    } else {
+        slo_c = __ldg(reinterpret_cast<const float *>(ws + tb.slo) + c);
+    }
+    Consts2 k2;
+    k2.M = make_float2(Mf, Mf);
+    k2.negM = make_float2(-Mf, -Mf);
+    k2.two23 = make_float2(kTwo23, kTwo23);
+    k2.neg23 = make_float2(-kTwo23, -kTwo23);
     constexpr int NCH = TT * NPL;                    // candidates per lane and pair, an even number
     static_assert(NCH % 2 == 0, "candidates are evaluated two at a time");
 
@@ -202,13 +255,14 @@ eval_select_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__r
         }
 #pragma unroll 4
         for (int p = g; p < P; p += G) {
-            const float ic = cicv[p];
+            const float2 pc = pair_consts<SMEM>(ws, cpair + uint32_t(p) * 8u);
             const uint32_t base = cbase + uint32_t(p) * pstep;
+            const float lim = FAST ? pc.y : slo_c;
 #pragma unroll
             for (int q = 0; q < NCH; q += 2)
-                eval_two<SMEM>(a.rows, base, ln[q], ln[q + 1], ic, M2, negM2, two23, neg23, slo_c,
-                               make_float2(nf[q % NPL], nf[(q + 1) % NPL]), !BUDGET || p < pmax[q % NPL],
-                               !BUDGET || p < pmax[(q + 1) % NPL], best[q], best[q + 1]);
+                eval_two<SMEM, FAST>(ws, base, ln[q], ln[q + 1], pc.x, lim, k2,
+                                     make_float2(nf[q % NPL], nf[(q + 1) % NPL]), !BUDGET || p < pmax[q % NPL],
+                                     !BUDGET || p < pmax[(q + 1) % NPL], best[q], best[q + 1]);
         }
 #pragma unroll
         for (int t = 0; t < TT; ++t) {
@@ -242,20 +296,21 @@ eval_select_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__r
             const float Emin = __uint_as_float(kmin ^ ((kmin >> 31) ? 0x80000000u : 0xffffffffu));
             const float nfm = float(nmin);
             const float lnm = Lt[t] * (1.0f / nfm);
-            int pm = -1;
+            int pm = P;
             if (BUDGET) {
                 int nt = 0;
                 for (int tt = 0; tt < a.T; ++tt) nt += (int64_t(nmin) * a.tp[tt] <= int64_t(a.budget)) ? 1 : 0;
                 pm = nt * a.F;
             }
             int pstar = -1;
-            for (int p0 = 0; p0 < P && pstar < 0; p0 += 32) {
+            for (int p0 = 0; p0 < pm && pstar < 0; p0 += 32) {
                 const int pp = p0 + lane;
                 bool hit = false;
-                if (pp < P && (!BUDGET || pp < pm)) {
+                if (pp < pm) {
+                    const float2 pc = pair_consts<SMEM>(ws, cpair + uint32_t(pp) * 8u);
                     float Ep;
                     bool ok;
-                    eval_one<SMEM>(a.rows, cbase + uint32_t(pp) * pstep, lnm, cicv[pp], Mf, slo_c, nfm, Ep, ok);
+                    eval_one<SMEM, FAST>(ws, cbase + uint32_t(pp) * pstep, lnm, pc.x, FAST ? pc.y : slo_c, Mf, nfm, Ep, ok);
                     hit = ok && (Ep + 0.f == Emin);
                 }
                 const unsigned m = __ballot_sync(kFull, hit);
@@ -269,32 +324,71 @@ eval_select_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__r
     }
 }
 
+template <int NPL, int TT, bool BUDGET, bool SMEM>
+__global__ void __launch_bounds__(kThreads, (NPL <= 2 ? 4 : 2))
+eval_select_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__restrict__ best_E) {
+    Tables tb;
+    if (all_rows_monotone(a)) {                      // uniform over the grid: every CTA reads the same flags
+        if (SMEM) {
+            stage(a, a.off_pairc, a.off_end);        // pairc | slo | rows2
+            tb.pairc = 0; tb.slo = a.off_slo - a.off_pairc; tb.rows2 = a.off_rows2 - a.off_pairc; tb.rows = 0;
+        } else {
+            tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.rows2 = a.off_rows2;
+        }
+        sweep_body<NPL, TT, BUDGET, SMEM, true>(a, tb, best_idx, best_E);
+    } else {
+        if (SMEM) {
+            stage(a, a.off_rows, a.off_rows2);       // rows | pairc | slo
+            tb.rows = 0; tb.pairc = a.off_pairc - a.off_rows; tb.slo = a.off_slo - a.off_rows; tb.rows2 = 0;
+        } else {
+            tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.rows2 = a.off_rows2;
+        }
+        sweep_body<NPL, TT, BUDGET, SMEM, false>(a, tb, best_idx, best_E);
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // evaluate only: E[tile][j].  A CTA takes whole tiles; threads stride over j so that the row of E
 // is written coalesced; (n, pair) of a thread's next candidate follow by increments, no division.
+// Always the general path (the kernel is bound by the 4 bytes it writes per candidate).
 // ---------------------------------------------------------------------------------------------
 template <bool SMEM>
 __global__ void __launch_bounds__(kThreads)
 eval_configs_kernel(const SweepArgs a, const int dn, const int dp, float *__restrict__ E_out) {
-    const float *icv, *slo;
-    stage_tables<SMEM>(a, icv, slo);
+    Tables tb;
+    if (SMEM) {
+        stage(a, a.off_rows, a.off_rows2);
+        tb.rows = 0; tb.pairc = a.off_pairc - a.off_rows; tb.slo = a.off_slo - a.off_rows; tb.rows2 = 0;
+    } else {
+        tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.rows2 = a.off_rows2;
+    }
     const int P = a.P, RS = a.M + 1, J = a.J;
     const float Mf = float(a.M);
+    uint32_t origin = table_origin<SMEM>();
+    asm volatile("" : "+r"(origin) : : "memory");        // as in sweep_body: table loads stay behind the staging barrier
+    const char *ws = a.ws;
     const int n1_0 = int(threadIdx.x) / P, p_0 = int(threadIdx.x) - n1_0 * P;
     for (int64_t i = blockIdx.x; i < a.tiles; i += gridDim.x) {
         const int c = int(i % a.C);
         const float L = fmaxf(a.load[i], 0.f);
-        const float *cicv = icv + c * P;
-        const float slo_c = slo[c];
-        const uint32_t cbase = row_base<SMEM>(c * P * RS);
-        const uint32_t pstep = SMEM ? uint32_t(RS) * 16u : uint32_t(RS);
+        float slo_c;
+        if (SMEM) {
+            extern __shared__ float4 smem[];
+            slo_c = reinterpret_cast<const float *>(reinterpret_cast<const char *>(smem) + tb.slo)[c];
+        } else {
+            slo_c = __ldg(reinterpret_cast<const float *>(ws + tb.slo) + c);
+        }
+        const uint32_t cpair = origin + tb.pairc + uint32_t(c * P) * 8u;
+        const uint32_t cbase = origin + tb.rows + uint32_t(c * P * RS) * 16u - kTwo23Bits * 16u;
+        const uint32_t pstep = uint32_t(RS) * 16u;
         float *out = E_out + size_t(i) * size_t(J);
         int n1 = n1_0, p = p_0;                       // n - 1 and pair of candidate j
         for (int j = threadIdx.x; j < J; j += kThreads) {
             const float nf = float(n1 + 1);
+            const float2 pc = pair_consts<SMEM>(ws, cpair + uint32_t(p) * 8u);
             float E;
             bool ok;
-            eval_one<SMEM>(a.rows, cbase + uint32_t(p) * pstep, __fdividef(L, nf), cicv[p], Mf, slo_c, nf, E, ok);
+            eval_one<SMEM, false>(ws, cbase + uint32_t(p) * pstep, __fdividef(L, nf), pc.x, slo_c, Mf, nf, E, ok);
             if (a.budget > 0) ok = ok && (int64_t(n1 + 1) * a.tp[p / a.F] <= int64_t(a.budget));
             out[j] = ok ? E : CUDART_INF_F;
             n1 += dn;
@@ -316,22 +410,22 @@ size_t smem_limit() {
 }
 
 SweepArgs make_args(const ResolvedLayout &lay, const void *d_ws, const float *d_load, int64_t tiles, int32_t budget) {
-    const char *ws = static_cast<const char *>(d_ws);
     SweepArgs a{};
-    a.rows = reinterpret_cast<const float4 *>(ws + lay.off_rows);
-    a.icv = reinterpret_cast<const float *>(ws + lay.off_icm);
-    a.slo = reinterpret_cast<const float *>(ws + lay.off_slo);
-    a.tp = reinterpret_cast<const int32_t *>(ws + lay.off_tp);
+    a.ws = static_cast<const char *>(d_ws);
+    a.tp = reinterpret_cast<const int32_t *>(a.ws + lay.off_tp);
     a.load = d_load;
     a.tiles = tiles;
     a.rows_total = tiles / lay.C;
     a.C = lay.C; a.T = lay.T; a.F = lay.F; a.P = lay.P; a.M = lay.M; a.Nmax = lay.Nmax; a.J = lay.J;
     a.budget = budget;
-    // rows, icv and slo are consecutive in the scratch block: stage them as one piece when it fits
-    const size_t block = lay.off_tp - lay.off_rows;
-    a.stage_bytes = block <= 96 * 1024 && block <= smem_limit() ? int32_t(block) : 0;
-    a.off_icv = int32_t(lay.off_icm - lay.off_rows);
-    a.off_slo = int32_t(lay.off_slo - lay.off_rows);
+    a.off_rows = int32_t(lay.off_rows);
+    a.off_pairc = int32_t(lay.off_pairc);
+    a.off_slo = int32_t(lay.off_slo);
+    a.off_rows2 = int32_t(lay.off_rows2);
+    a.off_end = int32_t(lay.off_tp);
+    // the general path stages rows | pairc | slo, the threshold path pairc | slo | rows2: one piece each
+    const size_t general = lay.off_rows2 - lay.off_rows;
+    a.smem_bytes = general <= 96 * 1024 && general <= smem_limit() ? int32_t(general) : 0;
     return a;
 }
 
@@ -340,11 +434,11 @@ cudaError_t launch_es_variant(SweepArgs &a, int32_t *best_idx, float *best_E, cu
     auto kernel = eval_select_kernel<NPL, TT, B, S>;
     cudaError_t e = cudaSuccess;
     if (S) {
-        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, a.stage_bytes);
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, a.smem_bytes);
         if (e != cudaSuccess) return e;
     }
     int resident = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kernel, kThreads, S ? size_t(a.stage_bytes) : 0);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kernel, kThreads, S ? size_t(a.smem_bytes) : 0);
     if (e != cudaSuccess) return e;
     if (resident < 1) resident = 1;
     // about four work units per resident warp: all units cost the same, so the tail is short
@@ -355,13 +449,13 @@ cudaError_t launch_es_variant(SweepArgs &a, int32_t *best_idx, float *best_E, cu
     a.blocks = (a.rows_total + rpw - 1) / rpw;
     const int64_t units = a.blocks * a.C;
     const int64_t grid = (units + kWarps - 1) / kWarps;
-    kernel<<<unsigned(grid), kThreads, S ? size_t(a.stage_bytes) : 0, st>>>(a, best_idx, best_E);
+    kernel<<<unsigned(grid), kThreads, S ? size_t(a.smem_bytes) : 0, st>>>(a, best_idx, best_E);
     return cudaGetLastError();
 }
 
 template <int NPL, int TT>
 cudaError_t launch_es(SweepArgs &a, int32_t *best_idx, float *best_E, cudaStream_t st) {
-    const bool smem = a.stage_bytes > 0;
+    const bool smem = a.smem_bytes > 0;
     const bool budget = a.budget > 0;
     if (budget && smem) return launch_es_variant<NPL, TT, true, true>(a, best_idx, best_E, st);
     if (budget) return launch_es_variant<NPL, TT, true, false>(a, best_idx, best_E, st);
@@ -396,10 +490,10 @@ cudaError_t launch_eval_configs(const ResolvedLayout &lay, const void *d_ws, con
     if (grid > tiles) grid = tiles;
     const int dn = kThreads / lay.P, dp = kThreads % lay.P;
     cudaError_t e = cudaSuccess;
-    if (a.stage_bytes > 0) {
-        e = cudaFuncSetAttribute(eval_configs_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, a.stage_bytes);
+    if (a.smem_bytes > 0) {
+        e = cudaFuncSetAttribute(eval_configs_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, a.smem_bytes);
         if (e != cudaSuccess) return e;
-        eval_configs_kernel<true><<<int(grid), kThreads, size_t(a.stage_bytes), st>>>(a, dn, dp, d_E);
+        eval_configs_kernel<true><<<int(grid), kThreads, size_t(a.smem_bytes), st>>>(a, dn, dp, d_E);
     } else {
         eval_configs_kernel<false><<<int(grid), kThreads, 0, st>>>(a, dn, dp, d_E);
     }

@@ -126,6 +126,40 @@ def test_eval_configs_then_select_small(dyn, case):
     assert np.array_equal(o["gpus"].astype(np.int64), tot["gpus"].astype(np.int64))
 
 
+def _random_tables(seed, monotone_tbt):
+    """Free-form tables (not the closed forms): TBT rises and falls with load unless monotone_tbt."""
+    rng = np.random.default_rng(seed)
+    Cn, T, R, M = 9, 3, 5, 6
+    tp = np.array([1, 2, 8], np.int32)
+    fg = np.array([800, 1000, 1300, 1700, 1980], np.float32)
+    ttft = (0.2 + 0.9 * rng.random((Cn, T, R))).astype(np.float32)
+    cap = (1.0 + 6.0 * rng.random((Cn, T, R))).astype(np.float32)
+    tbt = (0.04 + 0.1 * rng.random((Cn, T, R, M)))
+    if monotone_tbt:
+        tbt = np.sort(tbt, axis=-1)
+        tbt[:, :, :, 3] = tbt[:, :, :, 2]                 # a flat segment is still "never decreases"
+    pw = (150 + 600 * rng.random((Cn, T, R, M)))
+    prof = gen.Profile(tp, fg, ttft, cap, tbt.astype(np.float32), pw.astype(np.float32))
+    cand = np.array([800, 850, 1000, 1111, 1500, 1700, 1979, 1980], np.float32)
+    sp = gen.make_space(cand, 40, 60.0, slo_ttft=0.8, slo_tbt=0.1)
+    return prof, sp
+
+
+@pytest.mark.parametrize("monotone", [False, True], ids=["tbt-rises-and-falls", "tbt-never-decreases"])
+def test_eval_select_free_form_tables(dyn, monotone):
+    """Both evaluation paths of the fused kernel: per-candidate TBT interpolation when some table row
+    decreases with load, the load-threshold path when none does."""
+    prof, sp = _random_tables(17, monotone)
+    load = gen.random_loads((2, 37, 9), seed=5, mean=6.0)
+    J = sp.n_max * prof.T * sp.F
+    ref = oracle.eval_select(prof, sp, load)
+    out = out_to_host(gpu_eval_select(dyn, prof, sp, load))
+    fixed, n_ex = check_selection(prof, sp, load, out["best_idx"], out["best_E"], ref)
+    _check_totals(sp, prof, out, ref, fixed, J)
+    feas = (ref["best_idx"] >= 0).mean()
+    assert 0.2 < feas <= 1.0
+
+
 def test_select_ties_infeasible_and_odd_sizes(dyn):
     """dyn_select alone: exact duplicates -> lowest index; all +inf -> -1; J not a multiple of 4."""
     rng = np.random.default_rng(0)
