@@ -182,7 +182,7 @@ __device__ __forceinline__ bool all_rows_monotone(const SweepArgs &a) {
 //   NPL  instance counts per lane (Nmax <= 32*NPL)
 //   TT   tiles (rows of the same class) a warp evaluates per pass over the pairs
 // ---------------------------------------------------------------------------------------------
-template <int NPL, int TT, bool BUDGET, bool SMEM, bool FAST>
+template <int NPL, int TT, bool BUDGET, bool SMEM, bool FAST, bool FULL>
 __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, int32_t *__restrict__ best_idx,
                                            float *__restrict__ best_E) {
     const int lane = threadIdx.x & 31;
@@ -192,10 +192,12 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
     const int64_t r_begin = (unit / a.C) * a.rows_per_warp;
     const int64_t r_end = r_begin + a.rows_per_warp < a.rows_total ? r_begin + a.rows_per_warp : a.rows_total;
 
-    const int LN = 1 << a.ln_log2;
-    const int G = 32 >> a.ln_log2;                  // pair groups inside the warp (Nmax < 32)
+    // FULL: lanes are 32 instance counts and every lane walks all pairs (compile-time stride 1);
+    // otherwise (Nmax < 32) the warp splits into G groups that take every G-th pair
+    const int LN = FULL ? 32 : 1 << a.ln_log2;
+    const int G = FULL ? 1 : 32 >> a.ln_log2;
     const int nl = lane & (LN - 1);
-    const int g = lane >> a.ln_log2;
+    const int g = FULL ? 0 : lane >> a.ln_log2;
     const int P = a.P, RS = a.M + 1, C = a.C;
     const float Mf = float(a.M);
     const char *ws = a.ws;
@@ -243,17 +245,17 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
 
     for (int64_t r = r_begin; r < r_end; r += TT) {
         // chain q = t*NPL + k: tile t of this pass, k-th instance count of the lane
-        float ln[NCH], best[NCH], Lt[TT];
+        float ln[NCH], best[NCH];
 #pragma unroll
         for (int t = 0; t < TT; ++t) {
-            Lt[t] = (r + t < r_end) ? fmaxf(a.load[(r + t) * C + c], 0.f) : 0.f;   // negative / NaN -> 0
+            const float L = (r + t < r_end) ? fmaxf(a.load[(r + t) * C + c], 0.f) : 0.f;   // negative / NaN -> 0
 #pragma unroll
             for (int k = 0; k < NPL; ++k) {
-                ln[t * NPL + k] = Lt[t] * rn[k];
+                ln[t * NPL + k] = L * rn[k];
                 best[t * NPL + k] = CUDART_INF_F;
             }
         }
-#pragma unroll 4
+#pragma unroll 8
         for (int p = g; p < P; p += G) {
             const float2 pc = pair_consts<SMEM>(ws, cpair + uint32_t(p) * 8u);
             const uint32_t base = cbase + uint32_t(p) * pstep;
@@ -295,7 +297,12 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
             // and the first pair that reproduces the minimum bit for bit is the lowest-index one
             const float Emin = __uint_as_float(kmin ^ ((kmin >> 31) ? 0x80000000u : 0xffffffffu));
             const float nfm = float(nmin);
-            const float lnm = Lt[t] * (1.0f / nfm);
+            // L/n of the winning instance count, from the lane that holds it (bit-identical by construction)
+            const int kstar = int(nmin - 1) >> (FULL ? 5 : a.ln_log2);
+            float lnk = ln[t * NPL];
+#pragma unroll
+            for (int k = 1; k < NPL; ++k) lnk = (k == kstar) ? ln[t * NPL + k] : lnk;
+            const float lnm = __shfl_sync(kFull, lnk, int(nmin - 1) & (LN - 1));
             int pm = P;
             if (BUDGET) {
                 int nt = 0;
@@ -324,8 +331,8 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
     }
 }
 
-template <int NPL, int TT, bool BUDGET, bool SMEM>
-__global__ void __launch_bounds__(kThreads, (NPL <= 2 ? 4 : 2))
+template <int NPL, int TT, bool BUDGET, bool SMEM, bool FULL>
+__global__ void __launch_bounds__(kThreads, (NPL <= 2 ? 5 : 2))
 eval_select_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__restrict__ best_E) {
     Tables tb;
     if (all_rows_monotone(a)) {                      // uniform over the grid: every CTA reads the same flags
@@ -335,7 +342,7 @@ eval_select_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__r
         } else {
             tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.rows2 = a.off_rows2;
         }
-        sweep_body<NPL, TT, BUDGET, SMEM, true>(a, tb, best_idx, best_E);
+        sweep_body<NPL, TT, BUDGET, SMEM, true, FULL>(a, tb, best_idx, best_E);
     } else {
         if (SMEM) {
             stage(a, a.off_rows, a.off_rows2);       // rows | pairc | slo
@@ -343,7 +350,7 @@ eval_select_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__r
         } else {
             tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.rows2 = a.off_rows2;
         }
-        sweep_body<NPL, TT, BUDGET, SMEM, false>(a, tb, best_idx, best_E);
+        sweep_body<NPL, TT, BUDGET, SMEM, false, FULL>(a, tb, best_idx, best_E);
     }
 }
 
@@ -429,9 +436,9 @@ SweepArgs make_args(const ResolvedLayout &lay, const void *d_ws, const float *d_
     return a;
 }
 
-template <int NPL, int TT, bool B, bool S>
+template <int NPL, int TT, bool B, bool S, bool FULL>
 cudaError_t launch_es_variant(SweepArgs &a, int32_t *best_idx, float *best_E, cudaStream_t st) {
-    auto kernel = eval_select_kernel<NPL, TT, B, S>;
+    auto kernel = eval_select_kernel<NPL, TT, B, S, FULL>;
     cudaError_t e = cudaSuccess;
     if (S) {
         e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, a.smem_bytes);
@@ -457,10 +464,17 @@ template <int NPL, int TT>
 cudaError_t launch_es(SweepArgs &a, int32_t *best_idx, float *best_E, cudaStream_t st) {
     const bool smem = a.smem_bytes > 0;
     const bool budget = a.budget > 0;
-    if (budget && smem) return launch_es_variant<NPL, TT, true, true>(a, best_idx, best_E, st);
-    if (budget) return launch_es_variant<NPL, TT, true, false>(a, best_idx, best_E, st);
-    if (smem) return launch_es_variant<NPL, TT, false, true>(a, best_idx, best_E, st);
-    return launch_es_variant<NPL, TT, false, false>(a, best_idx, best_E, st);
+    constexpr bool FULL = NPL > 1;                   // more than 32 instance counts: one pair group
+    if (NPL == 1 && a.ln_log2 == 5) {                // exactly 17..32 instance counts
+        if (budget && smem) return launch_es_variant<NPL, TT, true, true, true>(a, best_idx, best_E, st);
+        if (budget) return launch_es_variant<NPL, TT, true, false, true>(a, best_idx, best_E, st);
+        if (smem) return launch_es_variant<NPL, TT, false, true, true>(a, best_idx, best_E, st);
+        return launch_es_variant<NPL, TT, false, false, true>(a, best_idx, best_E, st);
+    }
+    if (budget && smem) return launch_es_variant<NPL, TT, true, true, FULL>(a, best_idx, best_E, st);
+    if (budget) return launch_es_variant<NPL, TT, true, false, FULL>(a, best_idx, best_E, st);
+    if (smem) return launch_es_variant<NPL, TT, false, true, FULL>(a, best_idx, best_E, st);
+    return launch_es_variant<NPL, TT, false, false, FULL>(a, best_idx, best_E, st);
 }
 
 }  // namespace
