@@ -4,13 +4,16 @@
 // KI x KO length classes of the thresholds table [Sec. 3.1]; the per-class load over time [Sec. 3.2]
 // is the count per (window, class) divided by the window length.
 //
-// Memory-bound: 12 bytes are read per request and nothing else scales with the trace.  A CTA owns a
-// contiguous slice of the trace; on a time-sorted trace that slice covers few windows, so its bins
-// live in shared memory.  A warp takes 128 consecutive requests (one 16-byte load per lane and
-// array), reduces the requests of one window to per-class counts with packed 8-bit counters and
-// warp-wide integer reductions, and issues at most C shared-memory atomics per window present.
-// Requests outside the CTA's window range (unsorted input) go to global atomics, so the counts are
-// exact for any order.
+// Memory-bound: 12 bytes are read per request and nothing else scales with the trace, so the kernel
+// is written for few instructions per request.  A CTA owns a contiguous slice of the trace; on a
+// time-sorted trace that slice covers few windows, so its bins live in shared memory, four copies of
+// each bin side by side (lane l adds to copy l mod 4) so that the lanes of one warp instruction that
+// hit the same (window, class) spread over four banks.  A warp takes 128 consecutive requests (one
+// 16-byte load per lane and array, two batches in flight).  When a lane's four timestamps are in order
+// and both ends fall inside the CTA's window range (the rule on a sorted trace) nothing has to be
+// tested per request, and two divisions serve all four unless a window boundary falls among them; the
+// window is a multiply-shift division by the invariant window length.  Requests outside the CTA's
+// window range (unsorted input) go to global atomics, so the counts are exact for any order.
 #include "dyn_internal.cuh"
 
 namespace dyn {
@@ -19,9 +22,9 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
-constexpr int kSmemBins = 4096;       // uint32 bins per CTA
+constexpr int kCopies = 4;            // copies of every shared-memory bin
+constexpr int kSmemBins = 6144;       // uint32 words of bins per CTA (copies included)
 constexpr int kBatch = 128;           // requests per warp step (4 per lane)
-constexpr int kMaxRounds = 4;         // distinct windows reduced per batch before falling back
 constexpr unsigned kFull = 0xffffffffu;
 
 template <int NI, int NO>
@@ -41,14 +44,13 @@ __device__ __forceinline__ uint32_t classify(const BinParams &bp, uint32_t in, u
 }
 
 // NI/NO: compile-time edge counts (or -1: read them from the parameters).
-// PACKED: C <= 16, per-class counts of a window travel as 4 x 8-bit fields in up to 4 words.
 // VEC: the three arrays are 16-byte aligned.
-template <int NI, int NO, bool PACKED, bool VEC>
+template <int NI, int NO, bool VEC>
 __global__ void __launch_bounds__(kThreads)
 bin_trace_kernel(const BinParams bp, const uint32_t *__restrict__ t_ms, const uint32_t *__restrict__ in_tok,
                  const uint32_t *__restrict__ out_tok, const uint64_t n_req, const uint64_t chunk,
                  uint32_t *__restrict__ counts, unsigned long long *__restrict__ dropped) {
-    __shared__ uint32_t sbins[kSmemBins];
+    __shared__ __align__(16) uint32_t sbins[kSmemBins];
 
     const uint64_t begin = uint64_t(blockIdx.x) * chunk;
     if (begin >= n_req) return;
@@ -57,6 +59,7 @@ bin_trace_kernel(const BinParams bp, const uint32_t *__restrict__ t_ms, const ui
     const uint32_t W = bp.n_windows;
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
+    const uint32_t copy = uint32_t(lane) & (kCopies - 1);
 
     // window range kept in shared memory: starts at the window of the slice's first (or last,
     // if that is earlier) request
@@ -66,105 +69,84 @@ bin_trace_kernel(const BinParams bp, const uint32_t *__restrict__ t_ms, const ui
     uint32_t nwin = 0;
     if (w_lo < W) {
         const uint32_t span = (wa < wb ? wb - wa : wa - wb) + 1u;
-        const uint32_t cap = uint32_t(kSmemBins) / C;
+        const uint32_t cap = uint32_t(kSmemBins / kCopies) / C;
         nwin = span < cap ? span : cap;
         if (nwin > W - w_lo) nwin = W - w_lo;
     }
-    const uint32_t nbins = nwin * C;
-    for (uint32_t i = threadIdx.x; i < nbins; i += kThreads) sbins[i] = 0u;
+    const uint32_t nbins = nwin * C;                         // distinct bins held here
+    for (uint32_t i = threadIdx.x; i < nbins * kCopies; i += kThreads) sbins[i] = 0u;
     __syncthreads();
 
-    auto add_bin = [&](uint32_t w, uint32_t c, uint32_t v) {
+    // any request, any order: window by division, dropped / shared / global by range
+    auto count_one = [&](uint32_t t, uint32_t a, uint32_t b, uint32_t &ndrop) {
+        const uint32_t w = fastdiv(t, bp.win);
+        if (w >= W) {
+            ++ndrop;
+            return;
+        }
+        const uint32_t c = classify<NI, NO>(bp, a, b);
         const uint32_t rel = w - w_lo;                       // wraps for w < w_lo: then rel >= nwin
-        if (rel < nwin) atomicAdd(&sbins[rel * C + c], v);
-        else atomicAdd(&counts[size_t(w) * C + c], v);
+        if (rel < nwin) atomicAdd(&sbins[(rel * C + c) * kCopies + copy], 1u);
+        else atomicAdd(&counts[size_t(w) * C + c], 1u);
+    };
+
+    // four consecutive requests of one lane
+    auto count_four = [&](const uint4 vt, const uint4 va, const uint4 vb, uint32_t &ndrop) {
+        // the rule on a sorted trace: timestamps in order and both ends inside the CTA's window range;
+        // then no request is dropped or out of range, and the middle windows are the end windows
+        // unless a window boundary falls between the lane's four requests
+        const uint32_t w0 = fastdiv(vt.x, bp.win), w3 = fastdiv(vt.w, bp.win);
+        const uint32_t r0 = w0 - w_lo, r3 = w3 - w_lo;
+        const bool fast = (vt.x <= vt.y) && (vt.y <= vt.z) && (vt.z <= vt.w) && (r0 < nwin) && (r3 < nwin);
+        if (fast) {
+            uint32_t r1 = r0, r2 = r0;
+            if (r0 != r3) {
+                r1 = fastdiv(vt.y, bp.win) - w_lo;
+                r2 = fastdiv(vt.z, bp.win) - w_lo;
+            }
+            uint32_t *row = sbins + copy;
+            const uint32_t stride = C * kCopies;
+            atomicAdd(row + r0 * stride + classify<NI, NO>(bp, va.x, vb.x) * kCopies, 1u);
+            atomicAdd(row + r1 * stride + classify<NI, NO>(bp, va.y, vb.y) * kCopies, 1u);
+            atomicAdd(row + r2 * stride + classify<NI, NO>(bp, va.z, vb.z) * kCopies, 1u);
+            atomicAdd(row + r3 * stride + classify<NI, NO>(bp, va.w, vb.w) * kCopies, 1u);
+        } else {
+            count_one(vt.x, va.x, vb.x, ndrop);
+            count_one(vt.y, va.y, vb.y, ndrop);
+            count_one(vt.z, va.z, vb.z, ndrop);
+            count_one(vt.w, va.w, vb.w, ndrop);
+        }
     };
 
     uint32_t my_dropped = 0;
-    for (uint64_t base = begin + uint64_t(warp) * kBatch; base < end; base += uint64_t(kWarps) * kBatch) {
+    const uint64_t step = uint64_t(kWarps) * kBatch;
+    uint64_t base = begin + uint64_t(warp) * kBatch;
+    if (VEC) {
+        // two full batches per pass: six 16-byte loads in flight per lane before any of them is used
+        for (; base + step + kBatch <= end; base += 2 * step) {
+            const uint64_t i0 = base + uint64_t(lane) * 4, i1 = i0 + step;
+            const uint4 t0 = __ldcs(reinterpret_cast<const uint4 *>(t_ms + i0));
+            const uint4 a0 = __ldcs(reinterpret_cast<const uint4 *>(in_tok + i0));
+            const uint4 b0 = __ldcs(reinterpret_cast<const uint4 *>(out_tok + i0));
+            const uint4 t1 = __ldcs(reinterpret_cast<const uint4 *>(t_ms + i1));
+            const uint4 a1 = __ldcs(reinterpret_cast<const uint4 *>(in_tok + i1));
+            const uint4 b1 = __ldcs(reinterpret_cast<const uint4 *>(out_tok + i1));
+            count_four(t0, a0, b0, my_dropped);
+            count_four(t1, a1, b1, my_dropped);
+        }
+        for (; base + kBatch <= end; base += step) {
+            const uint64_t i0 = base + uint64_t(lane) * 4;
+            count_four(__ldcs(reinterpret_cast<const uint4 *>(t_ms + i0)),
+                       __ldcs(reinterpret_cast<const uint4 *>(in_tok + i0)),
+                       __ldcs(reinterpret_cast<const uint4 *>(out_tok + i0)), my_dropped);
+        }
+    }
+    // ragged tail of the slice (and everything, when the arrays are not 16-byte aligned)
+    for (; base < end; base += step) {
         const uint64_t i0 = base + uint64_t(lane) * 4;
-        uint32_t t[4], a[4], b[4];
-        uint32_t live = 0;
-        if (VEC && i0 + 4 <= end) {
-            const uint4 vt = *reinterpret_cast<const uint4 *>(t_ms + i0);
-            const uint4 va = *reinterpret_cast<const uint4 *>(in_tok + i0);
-            const uint4 vb = *reinterpret_cast<const uint4 *>(out_tok + i0);
-            t[0] = vt.x; t[1] = vt.y; t[2] = vt.z; t[3] = vt.w;
-            a[0] = va.x; a[1] = va.y; a[2] = va.z; a[3] = va.w;
-            b[0] = vb.x; b[1] = vb.y; b[2] = vb.z; b[3] = vb.w;
-            live = 0xfu;
-        } else {
 #pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                t[r] = a[r] = b[r] = 0u;
-                if (i0 + r < end) {
-                    t[r] = t_ms[i0 + r];
-                    a[r] = in_tok[i0 + r];
-                    b[r] = out_tok[i0 + r];
-                    live |= 1u << r;
-                }
-            }
-        }
-        uint32_t w[4], c[4];
-        uint32_t ndrop = 0;
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            w[r] = fastdiv(t[r], bp.win);
-            c[r] = classify<NI, NO>(bp, a[r], b[r]);
-            if ((live >> r & 1u) && w[r] >= W) {
-                live &= ~(1u << r);
-                ++ndrop;
-            }
-        }
-        my_dropped += ndrop;
-
-        if (PACKED) {
-            // one round per distinct window present in the batch, earliest first
-            for (int round = 0; round < kMaxRounds; ++round) {
-                uint32_t wmin = 0xffffffffu;
-#pragma unroll
-                for (int r = 0; r < 4; ++r)
-                    if (live >> r & 1u) wmin = w[r] < wmin ? w[r] : wmin;
-                wmin = __reduce_min_sync(kFull, wmin);
-                if (wmin == 0xffffffffu) break;              // warp-uniform
-                uint32_t pk0 = 0, pk1 = 0, pk2 = 0, pk3 = 0;
-#pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    if ((live >> r & 1u) && w[r] == wmin) {
-                        const uint32_t inc = 1u << ((c[r] & 3u) * 8u);
-                        const uint32_t g = c[r] >> 2;
-                        pk0 += g == 0 ? inc : 0u;
-                        pk1 += g == 1 ? inc : 0u;
-                        pk2 += g == 2 ? inc : 0u;
-                        pk3 += g == 3 ? inc : 0u;
-                        live &= ~(1u << r);
-                    }
-                }
-                // at most 4 requests x 32 lanes = 128 per 8-bit field: no carry between fields
-                uint32_t s0 = __reduce_add_sync(kFull, pk0), s1 = 0, s2 = 0, s3 = 0;
-                if (C > 4) s1 = __reduce_add_sync(kFull, pk1);
-                if (C > 8) s2 = __reduce_add_sync(kFull, pk2);
-                if (C > 12) s3 = __reduce_add_sync(kFull, pk3);
-                if (uint32_t(lane) < C) {
-                    const uint32_t g = uint32_t(lane) >> 2;
-                    const uint32_t word = g == 0 ? s0 : g == 1 ? s1 : g == 2 ? s2 : s3;
-                    const uint32_t cnt = (word >> ((uint32_t(lane) & 3u) * 8u)) & 0xffu;
-                    if (cnt) add_bin(wmin, uint32_t(lane), cnt);
-                }
-            }
-#pragma unroll
-            for (int r = 0; r < 4; ++r)
-                if (live >> r & 1u) add_bin(w[r], c[r], 1u);
-        } else {
-            // many classes: lanes holding the same bin elect one leader that adds the group size
-#pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                const bool on = live >> r & 1u;
-                const uint32_t key = on ? w[r] * C + c[r] : (0x80000000u | uint32_t(lane));
-                const unsigned peers = __match_any_sync(kFull, key);
-                if (on && lane == __ffs(peers) - 1) add_bin(w[r], c[r], uint32_t(__popc(peers)));
-            }
-        }
+        for (int r = 0; r < 4; ++r)
+            if (i0 + r < end) count_one(t_ms[i0 + r], in_tok[i0 + r], out_tok[i0 + r], my_dropped);
     }
 
     my_dropped = __reduce_add_sync(kFull, my_dropped);
@@ -172,8 +154,9 @@ bin_trace_kernel(const BinParams bp, const uint32_t *__restrict__ t_ms, const ui
 
     __syncthreads();
     for (uint32_t i = threadIdx.x; i < nbins; i += kThreads) {
-        const uint32_t v = sbins[i];
-        if (v) atomicAdd(&counts[size_t(w_lo) * C + i], v);
+        const uint4 v = *reinterpret_cast<const uint4 *>(&sbins[i * kCopies]);
+        const uint32_t sum = v.x + v.y + v.z + v.w;
+        if (sum) atomicAdd(&counts[size_t(w_lo) * C + i], sum);
     }
 }
 
@@ -183,12 +166,12 @@ __global__ void counts_to_load_kernel(const uint32_t *__restrict__ counts, float
         load[i] = __fdiv_rn(float(counts[i]), window_s);
 }
 
-template <int NI, int NO, bool PACKED>
+template <int NI, int NO>
 cudaError_t launch_variant(bool vec, int grid, const BinParams &bp, const uint32_t *t, const uint32_t *a,
                            const uint32_t *b, uint64_t n, uint64_t chunk, uint32_t *counts,
                            unsigned long long *dropped, cudaStream_t st) {
-    if (vec) bin_trace_kernel<NI, NO, PACKED, true><<<grid, kThreads, 0, st>>>(bp, t, a, b, n, chunk, counts, dropped);
-    else bin_trace_kernel<NI, NO, PACKED, false><<<grid, kThreads, 0, st>>>(bp, t, a, b, n, chunk, counts, dropped);
+    if (vec) bin_trace_kernel<NI, NO, true><<<grid, kThreads, 0, st>>>(bp, t, a, b, n, chunk, counts, dropped);
+    else bin_trace_kernel<NI, NO, false><<<grid, kThreads, 0, st>>>(bp, t, a, b, n, chunk, counts, dropped);
     return cudaGetLastError();
 }
 
@@ -215,14 +198,10 @@ cudaError_t launch_bin_trace(const BinParams &bp, const uint32_t *t_ms, const ui
         const int g = int(grid);
         e = record_start(st);
         if (e != cudaSuccess) return e;
-        if (bp.C <= 16) {
-            if (bp.n_in == 2 && bp.n_out == 2)
-                e = launch_variant<2, 2, true>(vec, g, bp, t_ms, in_tok, out_tok, n_req, chunk, counts, dropped, st);
-            else
-                e = launch_variant<-1, -1, true>(vec, g, bp, t_ms, in_tok, out_tok, n_req, chunk, counts, dropped, st);
-        } else {
-            e = launch_variant<-1, -1, false>(vec, g, bp, t_ms, in_tok, out_tok, n_req, chunk, counts, dropped, st);
-        }
+        if (bp.n_in == 2 && bp.n_out == 2)
+            e = launch_variant<2, 2>(vec, g, bp, t_ms, in_tok, out_tok, n_req, chunk, counts, dropped, st);
+        else
+            e = launch_variant<-1, -1>(vec, g, bp, t_ms, in_tok, out_tok, n_req, chunk, counts, dropped, st);
         if (e != cudaSuccess) return e;
         e = record_stop(st);
         if (e != cudaSuccess) return e;
