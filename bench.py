@@ -350,6 +350,10 @@ def run_ours(args, rank, world, local_rank):
             result["bin_trace"] = measure_bin(dyn, gen, dev)
         except Exception as exc:                      # never lose the main line
             result["bin_trace"] = {"error": repr(exc)}
+        try:
+            result["materialised"] = measure_materialised(dyn, gen, dev)
+        except Exception as exc:
+            result["materialised"] = {"error": repr(exc)}
 
     if not args.no_cpu_baseline and world == 1:
         cb, _, _ = time_oracle(wl, trace, prof, sp, base_counts)
@@ -396,6 +400,51 @@ def measure_bin(dyn, gen, dev):
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
                          "traffic": None,
                          "peak_source": "measured (MEASURED_PEAKS.json)" if peaks else "fallback 6650 GB/s"}}
+
+
+def _hbm_peak():
+    try:
+        return float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["hbm_gbs"]), "measured (MEASURED_PEAKS.json)"
+    except (OSError, KeyError, ValueError):
+        return 6650.0, "fallback 6650 GB/s"
+
+
+def measure_materialised(dyn, gen, dev, S=16):
+    """The unfused stages on the 1-day shape with S scenarios: dyn_eval_configs writes the energy tensor
+    (4 bytes per candidate), dyn_select reads it back (4 bytes per candidate); both HBM-bound."""
+    import torch
+    wl = gen.workload("cfg2")
+    prof, sp = wl.profile(), wl.space()
+    W, Cn, J = wl.trace.n_windows, 9, wl.J
+    load = torch.from_numpy(gen.random_loads((S, W, Cn), seed=9, mean=2.5)).to(dev)
+    P = dyn.Profile(prof.tp, prof.f_grid_mhz, prof.ttft, prof.cap, prof.tbt, prof.pow, device=dev)
+    SP = dyn.Space(sp.f_cand_mhz, sp.n_max, sp.slo_ttft_s, sp.slo_tbt_s, sp.window_s, sp.gpu_budget)
+    E = torch.empty((S, W, Cn, J), dtype=torch.float32, device=dev)          # 1.7 GB at S = 16: larger than L2
+    ws = torch.empty(dyn.dyn_workspace_bytes(P, SP, S, W), dtype=torch.uint8, device=dev)
+    ws2 = torch.empty(dyn.dyn_select_workspace_bytes(S, W, J), dtype=torch.uint8, device=dev)
+    out = dyn.SelectOut(S, W, Cn, J, device=dev, windows=False, hist=False, gpus=False)
+    peak, src = _hbm_peak()
+    res = {"workload": f"cfg2 shape x {S} scenarios", "candidates": int(E.numel()), "tensor_bytes": int(E.numel() * 4)}
+    for name, call in (("eval_configs_kernel", lambda: dyn.dyn_eval_configs(P, SP, load, E, ws)),
+                       ("select_kernel", lambda: dyn.dyn_select(E, out, ws2))):
+        for _ in range(3):
+            call()
+        K = 10
+        kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        for a, b in kev:
+            a.record(); b.record()
+        torch.cuda.synchronize()
+        for k in range(K):
+            dyn.dyn_set_timing_events(*kev[k])
+            call()
+        dyn.dyn_set_timing_events(None, None)
+        torch.cuda.synchronize()
+        ms = float(np.mean([a.elapsed_time(b) for a, b in kev]))
+        gbs = E.numel() * 4 / (ms * 1e-3) / 1e9
+        res[name] = {"kernel_ms": ms, "evals_per_s": E.numel() / (ms * 1e-3),
+                     "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                                  "traffic": None, "peak_source": src}}
+    return res
 
 
 def main():
