@@ -44,7 +44,9 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-secondary", action="store_true", help="skip the trace-binning side measurement")
+    ap.add_argument("--no-secondary", action="store_true", help="skip the side measurements of the other kernels")
+    ap.add_argument("--secondary-only", action="store_true",
+                    help="run only the side measurements (trace binning, unfused stages) and print them")
     return ap.parse_args()
 
 
@@ -454,6 +456,14 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.secondary_only:
+        import torch
+        import gen
+        import paper_2408_00741_b200 as dyn
+        dev = torch.device("cuda", local_rank)
+        torch.cuda.set_device(dev)
+        print(json.dumps({"bin_trace": measure_bin(dyn, gen, dev), "materialised": measure_materialised(dyn, gen, dev)}))
         return
     run_ours(args, rank, world, local_rank)
 

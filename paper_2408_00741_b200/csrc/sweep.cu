@@ -355,28 +355,45 @@ eval_select_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__r
 }
 
 // ---------------------------------------------------------------------------------------------
-// evaluate only: E[tile][j].  A CTA takes whole tiles; threads stride over j so that the row of E
-// is written coalesced; (n, pair) of a thread's next candidate follow by increments, no division.
-// Always the general path (the kernel is bound by the 4 bytes it writes per candidate).
+// evaluate only: E[tile][j], j = (n-1)*P + p.  A warp takes one tile and 32 consecutive pairs: lanes
+// are pairs (their constants stay in registers), the loop runs over n two at a time, and each pass
+// writes two coalesced runs of 32 energies.  Always the general path: the kernel is bound by the 4
+// bytes it writes per candidate.
 // ---------------------------------------------------------------------------------------------
-template <bool SMEM>
+template <bool BUDGET, bool SMEM>
 __global__ void __launch_bounds__(kThreads)
-eval_configs_kernel(const SweepArgs a, const int dn, const int dp, float *__restrict__ E_out) {
+eval_configs_kernel(const SweepArgs a, const int64_t units, float *__restrict__ E_out) {
+    __shared__ __align__(16) float2 s_n[258];         // {n, 1/n} for n = 1..Nmax (Nmax <= 256), padded to even
+    for (int n1 = threadIdx.x; n1 < a.Nmax + 1; n1 += kThreads) s_n[n1] = make_float2(float(n1 + 1), 1.0f / float(n1 + 1));
     Tables tb;
     if (SMEM) {
         stage(a, a.off_rows, a.off_rows2);
         tb.rows = 0; tb.pairc = a.off_pairc - a.off_rows; tb.slo = a.off_slo - a.off_rows; tb.rows2 = 0;
     } else {
+        __syncthreads();
         tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.rows2 = a.off_rows2;
     }
-    const int P = a.P, RS = a.M + 1, J = a.J;
+    const int lane = threadIdx.x & 31;
+    const int P = a.P, RS = a.M + 1, Nmax = a.Nmax;
+    const int PG = (P + 31) / 32;                     // pair groups per tile
     const float Mf = float(a.M);
     uint32_t origin = table_origin<SMEM>();
     asm volatile("" : "+r"(origin) : : "memory");        // as in sweep_body: table loads stay behind the staging barrier
     const char *ws = a.ws;
-    const int n1_0 = int(threadIdx.x) / P, p_0 = int(threadIdx.x) - n1_0 * P;
-    for (int64_t i = blockIdx.x; i < a.tiles; i += gridDim.x) {
+    Consts2 k2;
+    k2.M = make_float2(Mf, Mf);
+    k2.negM = make_float2(-Mf, -Mf);
+    k2.two23 = make_float2(kTwo23, kTwo23);
+    k2.neg23 = make_float2(-kTwo23, -kTwo23);
+    const float4 *s_n4 = reinterpret_cast<const float4 *>(s_n);
+
+    const int64_t nwarps = int64_t(gridDim.x) * kWarps;
+    for (int64_t u = int64_t(blockIdx.x) * kWarps + (threadIdx.x >> 5); u < units; u += nwarps) {
+        const int64_t i = u / PG;
+        const int p = int(u - i * PG) * 32 + lane;
         const int c = int(i % a.C);
+        const bool active = p < P;
+        const int pp = active ? p : 0;
         const float L = fmaxf(a.load[i], 0.f);
         float slo_c;
         if (SMEM) {
@@ -385,22 +402,31 @@ eval_configs_kernel(const SweepArgs a, const int dn, const int dp, float *__rest
         } else {
             slo_c = __ldg(reinterpret_cast<const float *>(ws + tb.slo) + c);
         }
-        const uint32_t cpair = origin + tb.pairc + uint32_t(c * P) * 8u;
-        const uint32_t cbase = origin + tb.rows + uint32_t(c * P * RS) * 16u - kTwo23Bits * 16u;
-        const uint32_t pstep = uint32_t(RS) * 16u;
-        float *out = E_out + size_t(i) * size_t(J);
-        int n1 = n1_0, p = p_0;                       // n - 1 and pair of candidate j
-        for (int j = threadIdx.x; j < J; j += kThreads) {
-            const float nf = float(n1 + 1);
-            const float2 pc = pair_consts<SMEM>(ws, cpair + uint32_t(p) * 8u);
-            float E;
-            bool ok;
-            eval_one<SMEM, false>(ws, cbase + uint32_t(p) * pstep, __fdividef(L, nf), pc.x, slo_c, Mf, nf, E, ok);
-            if (a.budget > 0) ok = ok && (int64_t(n1 + 1) * a.tp[p / a.F] <= int64_t(a.budget));
-            out[j] = ok ? E : CUDART_INF_F;
-            n1 += dn;
-            p += dp;
-            if (p >= P) { p -= P; ++n1; }
+        const float2 pc = pair_consts<SMEM>(ws, origin + tb.pairc + uint32_t(c * P + pp) * 8u);
+        const uint32_t base = origin + tb.rows + uint32_t((c * P + pp) * RS) * 16u - kTwo23Bits * 16u;
+        int nlim = Nmax;                              // Eq. 1 GPU budget: n * TP <= budget
+        if (BUDGET) {
+            const int64_t q = int64_t(a.budget) / a.tp[pp / a.F];
+            nlim = q < Nmax ? int(q) : Nmax;
+        }
+        float *out = E_out + size_t(i) * size_t(a.J) + p;
+        for (int n1 = 0; n1 < Nmax; n1 += 2) {
+            const float4 nn = s_n4[n1 >> 1];                       // {n, 1/n, n+1, 1/(n+1)}
+            const float2 v = make_float2(__saturatef(L * nn.y * pc.x), __saturatef(L * nn.w * pc.x));
+            const float2 y = __ffma2_rz(v, k2.M, k2.two23);
+            const float2 fm = __fadd2_rn(y, k2.neg23);
+            const float2 nnu = __ffma2_rn(v, k2.negM, fm);
+            const float4 eA = entry16<SMEM>(ws, base, y.x);
+            const float4 eB = entry16<SMEM>(ws, base, y.y);
+            const float tbtA = fmaf(nnu.x, eA.y, eA.x), tbtB = fmaf(nnu.y, eB.y, eB.x);
+            const float2 E = __fmul2_rn(make_float2(fmaf(nnu.x, eA.w, eA.z), fmaf(nnu.y, eB.w, eB.z)),
+                                        make_float2(nn.x, nn.z));
+            const bool okA = tbtA <= slo_c && (!BUDGET || n1 + 1 <= nlim);
+            const bool okB = tbtB <= slo_c && (!BUDGET || n1 + 2 <= nlim);
+            if (active) {
+                __stcs(out + size_t(n1) * P, okA ? E.x : CUDART_INF_F);
+                if (n1 + 1 < Nmax) __stcs(out + size_t(n1 + 1) * P, okB ? E.y : CUDART_INF_F);
+            }
         }
     }
 }
@@ -500,18 +526,28 @@ cudaError_t launch_eval_configs(const ResolvedLayout &lay, const void *d_ws, con
                                 int32_t gpu_budget, float *d_E, cudaStream_t st) {
     if (tiles == 0) return cudaSuccess;
     SweepArgs a = make_args(lay, d_ws, d_load, tiles, gpu_budget);
+    const int64_t units = tiles * ((lay.P + 31) / 32);          // (tile, group of 32 pairs) per warp
     int64_t grid = int64_t(sm_count()) * 8;
-    if (grid > tiles) grid = tiles;
-    const int dn = kThreads / lay.P, dp = kThreads % lay.P;
+    const int64_t need = (units + kWarps - 1) / kWarps;
+    if (grid > need) grid = need;
+    const bool smem = a.smem_bytes > 0, budget = gpu_budget > 0;
+    const size_t dyn_smem = smem ? size_t(a.smem_bytes) : 0;
     cudaError_t e = cudaSuccess;
-    if (a.smem_bytes > 0) {
-        e = cudaFuncSetAttribute(eval_configs_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, a.smem_bytes);
-        if (e != cudaSuccess) return e;
-        eval_configs_kernel<true><<<int(grid), kThreads, size_t(a.smem_bytes), st>>>(a, dn, dp, d_E);
-    } else {
-        eval_configs_kernel<false><<<int(grid), kThreads, 0, st>>>(a, dn, dp, d_E);
-    }
-    return cudaGetLastError();
+#define DYN_LAUNCH_EC(B, S)                                                                                        \
+    do {                                                                                                           \
+        if (S) e = cudaFuncSetAttribute(eval_configs_kernel<B, S>, cudaFuncAttributeMaxDynamicSharedMemorySize,     \
+                                        a.smem_bytes);                                                             \
+        if (e == cudaSuccess) {                                                                                    \
+            eval_configs_kernel<B, S><<<int(grid), kThreads, dyn_smem, st>>>(a, units, d_E);                       \
+            e = cudaGetLastError();                                                                                \
+        }                                                                                                          \
+    } while (0)
+    if (budget && smem) DYN_LAUNCH_EC(true, true);
+    else if (budget) DYN_LAUNCH_EC(true, false);
+    else if (smem) DYN_LAUNCH_EC(false, true);
+    else DYN_LAUNCH_EC(false, false);
+#undef DYN_LAUNCH_EC
+    return e;
 }
 
 }  // namespace dyn
