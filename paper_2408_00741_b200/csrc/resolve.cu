@@ -14,7 +14,7 @@ namespace dyn {
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 int64_t totals_chunks(int64_t W) {
-    const int64_t per = 2048;            // windows per partial sum
+    const int64_t per = 256;             // windows per partial sum (one CTA, one window per thread)
     return (W + per - 1) / per;
 }
 

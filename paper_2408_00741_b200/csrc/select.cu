@@ -7,8 +7,8 @@
 //
 // select: one warp per tile, lanes stride over the candidates with 16-byte streaming loads, each
 // lane keeps its first minimum, then two warp-wide integer min-reductions pick (energy, index).
-// totals: fp64 sums in a fixed order (thread: its windows in order, classes in order; block: a
-// fixed tree; scenario: chunks in order), so results repeat bit for bit.
+// totals: fp64 sums in a fixed order (thread: the classes of its window in order; block: a fixed tree
+// over 256 windows; scenario: chunks in order), so results repeat bit for bit.
 #include "dyn_internal.cuh"
 
 #include <math_constants.h>
@@ -20,7 +20,7 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr unsigned kFull = 0xffffffffu;
-constexpr int kChunkWindows = 2048;          // must match totals_chunks()
+constexpr int kChunkWindows = 256;           // one window per thread; must match totals_chunks()
 
 __device__ __forceinline__ uint32_t float_key(float v) {
     const uint32_t b = __float_as_uint(v);
@@ -81,35 +81,43 @@ struct TotalsArgs {
     uint32_t *partial_bad;
 };
 
+// One CTA per (scenario, chunk of kChunkWindows windows), one window per thread.
 __global__ void __launch_bounds__(kThreads) totals_partial_kernel(const TotalsArgs a) {
     __shared__ double s_sum[kThreads];
     __shared__ uint32_t s_bad[kThreads];
     const int64_t s = blockIdx.x / a.chunks;
     const int64_t ch = blockIdx.x % a.chunks;
-    const int64_t w0 = ch * kChunkWindows;
-    const int64_t w1 = (w0 + kChunkWindows < a.W) ? w0 + kChunkWindows : a.W;
+    const int64_t w = ch * kChunkWindows + threadIdx.x;
+    const bool have = threadIdx.x < kChunkWindows && w < a.W;
+    const int lane = threadIdx.x & 31;
     const int TF = a.T * a.F;
-    double sum = 0.0;
-    uint32_t bad = 0;
-    for (int64_t w = w0 + threadIdx.x; w < w1; w += kThreads) {
-        const size_t base = size_t(s * a.W + w) * size_t(a.C);
-        double ew = 0.0;
-        uint32_t g = 0;
-        for (int c = 0; c < a.C; ++c) {
-            const int32_t j = a.o.best_idx[base + c];
-            if (j < 0) { ++bad; continue; }
-            ew += double(a.o.best_E[base + c]);
-            if (a.o.hist) atomicAdd(&a.o.hist[size_t(s) * size_t(a.J) + size_t(j)], 1u);
-            if (a.o.gpus) {
-                if (a.nj) g += uint32_t(a.nj[j] * a.tj[j]);
-                else g += uint32_t((j / TF + 1) * a.tp[(j / a.F) % a.T]);
-            }
+    const size_t base = size_t(s * a.W + (have ? w : 0)) * size_t(a.C);
+    double ew = 0.0;
+    uint32_t bad = 0, g = 0;
+    for (int c = 0; c < a.C; ++c) {                 // every lane takes every trip: the match below is warp-wide
+        int32_t j = -1;
+        if (have) {
+            j = a.o.best_idx[base + c];
+            if (j < 0) ++bad;
+            else ew += double(a.o.best_E[base + c]);
         }
-        sum += ew;
+        if (a.o.hist) {
+            // neighbouring windows of a class often choose the same candidate: one atomic per distinct
+            // candidate in the warp, by the lowest lane that holds it
+            const unsigned peers = __match_any_sync(kFull, j);
+            if (j >= 0 && lane == __ffs(peers) - 1)
+                atomicAdd(&a.o.hist[size_t(s) * size_t(a.J) + size_t(j)], uint32_t(__popc(peers)));
+        }
+        if (a.o.gpus && j >= 0) {
+            if (a.nj) g += uint32_t(a.nj[j] * a.tj[j]);
+            else g += uint32_t((j / TF + 1) * a.tp[(j / a.F) % a.T]);
+        }
+    }
+    if (have) {
         if (a.o.E_window) a.o.E_window[s * a.W + w] = ew;
         if (a.o.gpus) a.o.gpus[s * a.W + w] = g;
     }
-    s_sum[threadIdx.x] = sum;
+    s_sum[threadIdx.x] = ew;
     s_bad[threadIdx.x] = bad;
     __syncthreads();
     for (int h = kThreads / 2; h > 0; h >>= 1) {
