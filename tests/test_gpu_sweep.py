@@ -160,6 +160,71 @@ def test_eval_select_free_form_tables(dyn, monotone):
     assert 0.2 < feas <= 1.0
 
 
+def test_limits_of_the_candidate_space(dyn):
+    """Largest built shape per axis (256 instance counts, 16 TP degrees) and the smallest tables
+    (two frequency rows, two load knots); the GPU budget cuts the space unevenly."""
+    rng = np.random.default_rng(3)
+    Cn, T, R, M = 9, 16, 2, 2
+    tp = np.arange(1, T + 1, dtype=np.int32)
+    fg = np.array([800.0, 1980.0], np.float32)
+    ttft = (0.1 + 0.5 * rng.random((Cn, T, R))).astype(np.float32)
+    cap = (0.5 + 2.0 * rng.random((Cn, T, R))).astype(np.float32)
+    tbt = np.sort(0.05 + 0.08 * rng.random((Cn, T, R, M)), axis=-1).astype(np.float32)
+    pw = (100 + 50 * tp[None, :, None, None] * (1 + rng.random((Cn, T, R, M)))).astype(np.float32)
+    prof = gen.Profile(tp, fg, ttft, cap, tbt, pw)
+    cand = np.linspace(800, 1980, 16).astype(np.float32)
+    for budget in (0, 300):
+        sp = gen.make_space(cand, 256, 5.0, slo_ttft=0.5, slo_tbt=0.1, gpu_budget=budget)
+        load = gen.random_loads((1, 7, 9), seed=2, mean=40.0)
+        J = 256 * T * 16
+        ref = oracle.eval_select(prof, sp, load)
+        out = out_to_host(gpu_eval_select(dyn, prof, sp, load))
+        fixed, _ = check_selection(prof, sp, load, out["best_idx"], out["best_E"], ref)
+        _check_totals(sp, prof, out, ref, fixed, J)
+        assert (ref["best_idx"] >= 0).all()
+
+
+def test_loads_that_are_not_valid_numbers_count_as_zero(dyn):
+    wl, prof, sp, load = _small("cfg1", W=6, seed=12)
+    bad = load.copy()
+    bad[0, 2, 0] = -3.0
+    bad[0, 2, 1] = np.nan
+    bad[0, 3, 4] = -np.inf
+    clean = bad.copy()
+    clean[0, 2, 0] = clean[0, 2, 1] = clean[0, 3, 4] = 0.0
+    a = out_to_host(gpu_eval_select(dyn, prof, sp, bad))
+    b = out_to_host(gpu_eval_select(dyn, prof, sp, clean))
+    assert np.array_equal(a["best_idx"], b["best_idx"]) and np.array_equal(a["best_E"], b["best_E"])
+    ref = oracle.eval_select(prof, sp, clean)
+    check_selection(prof, sp, clean, a["best_idx"], a["best_E"], ref)
+
+
+def test_kernel_timing_events(dyn):
+    """The instrumentation hook brackets the sweep kernel: a positive time, shorter than the whole call."""
+    wl, prof, sp, load = _small("cfg2", W=300, S=2, seed=13)
+    p, s = gpu_profile_space(dyn, prof, sp)
+    d_load = torch.from_numpy(load).cuda()
+    out = dyn.SelectOut(2, 300, 9, wl.J)
+    ws = torch.empty(dyn.dyn_workspace_bytes(p, s, 2, 300), dtype=torch.uint8, device="cuda")
+    k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    k0.record(); k1.record()
+    dyn.dyn_eval_select(p, s, d_load, out, ws)                 # warm-up
+    torch.cuda.synchronize()
+    dyn.dyn_set_timing_events(k0, k1)
+    c0.record()
+    dyn.dyn_eval_select(p, s, d_load, out, ws)
+    c1.record()
+    dyn.dyn_set_timing_events(None, None)
+    torch.cuda.synchronize()
+    assert 0.0 < k0.elapsed_time(k1) <= c0.elapsed_time(c1)
+    # switched off again: a later call leaves the events alone
+    before = k0.elapsed_time(k1)
+    dyn.dyn_eval_select(p, s, d_load, out, ws)
+    torch.cuda.synchronize()
+    assert k0.elapsed_time(k1) == before
+
+
 def test_select_ties_infeasible_and_odd_sizes(dyn):
     """dyn_select alone: exact duplicates -> lowest index; all +inf -> -1; J not a multiple of 4."""
     rng = np.random.default_rng(0)
