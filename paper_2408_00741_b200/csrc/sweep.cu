@@ -165,7 +165,7 @@ __device__ __forceinline__ void stage(const SweepArgs &a, int from, int to) {
     extern __shared__ float4 smem[];
     const float4 *src = reinterpret_cast<const float4 *>(a.ws + from);
     const int n16 = (to - from) / 16;
-    for (int i = threadIdx.x; i < n16; i += kThreads) smem[i] = src[i];
+    for (int i = threadIdx.x; i < n16; i += blockDim.x) smem[i] = src[i];
     __syncthreads();
 }
 
@@ -173,7 +173,7 @@ __device__ __forceinline__ void stage(const SweepArgs &a, int from, int to) {
 __device__ __forceinline__ bool all_rows_monotone(const SweepArgs &a) {
     const float2 *pc = reinterpret_cast<const float2 *>(a.ws + a.off_pairc);
     int bad = 0;
-    for (int i = threadIdx.x; i < a.C * a.P; i += kThreads) bad |= isnan(__ldg(pc + i).y) ? 1 : 0;
+    for (int i = threadIdx.x; i < a.C * a.P; i += blockDim.x) bad |= isnan(__ldg(pc + i).y) ? 1 : 0;
     return __syncthreads_or(bad) == 0;
 }
 
@@ -182,14 +182,15 @@ __device__ __forceinline__ bool all_rows_monotone(const SweepArgs &a) {
 //   NPL  instance counts per lane (Nmax <= 32*NPL)
 //   TT   tiles (rows of the same class) a warp evaluates per pass over the pairs
 // ---------------------------------------------------------------------------------------------
-template <int NPL, int TT, bool BUDGET, bool SMEM, bool FAST, bool FULL>
+//   CLS  the CTA serves one class (blockIdx.y) and `tb` points at that class's tables alone
+template <int NPL, int TT, bool BUDGET, bool SMEM, bool FAST, bool FULL, bool CLS = false>
 __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, int32_t *__restrict__ best_idx,
                                            float *__restrict__ best_E) {
     const int lane = threadIdx.x & 31;
-    const int64_t unit = int64_t(blockIdx.x) * kWarps + (threadIdx.x >> 5);
-    if (unit >= a.blocks * a.C) return;
-    const int c = int(unit % a.C);
-    const int64_t r_begin = (unit / a.C) * a.rows_per_warp;
+    const int64_t unit = int64_t(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (unit >= (CLS ? a.blocks : a.blocks * a.C)) return;
+    const int c = CLS ? int(blockIdx.y) : int(unit % a.C);
+    const int64_t r_begin = (CLS ? unit : unit / a.C) * a.rows_per_warp;
     const int64_t r_end = r_begin + a.rows_per_warp < a.rows_total ? r_begin + a.rows_per_warp : a.rows_total;
 
     // FULL: lanes are 32 instance counts and every lane walks all pairs (compile-time stride 1);
@@ -225,15 +226,16 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
     // every table address below derives from `origin`: this keeps the (side-effect free) inline-assembly
     // loads from being scheduled ahead of the barrier that ends the staging
     asm volatile("" : "+r"(origin) : : "memory");
-    const uint32_t cpair = origin + tb.pairc + uint32_t(c * P) * 8u;
-    const uint32_t cbase = origin + (FAST ? tb.rows2 : tb.rows) + uint32_t(c * P * RS) * ESZ - kTwo23Bits * ESZ;
+    const int ct = CLS ? 0 : c;                      // class offset inside the tables `tb` points at
+    const uint32_t cpair = origin + tb.pairc + uint32_t(ct * P) * 8u;
+    const uint32_t cbase = origin + (FAST ? tb.rows2 : tb.rows) + uint32_t(ct * P * RS) * ESZ - kTwo23Bits * ESZ;
     const uint32_t pstep = uint32_t(RS) * ESZ;
     float slo_c;
-    if (SMEM) {
+    if (SMEM && !CLS) {
         extern __shared__ float4 smem[];
         slo_c = reinterpret_cast<const float *>(reinterpret_cast<const char *>(smem) + tb.slo)[c];
     } else {
-        slo_c = __ldg(reinterpret_cast<const float *>(ws + tb.slo) + c);
+        slo_c = __ldg(reinterpret_cast<const float *>(ws + a.off_slo) + c);
     }
     Consts2 k2;
     k2.M = make_float2(Mf, Mf);
@@ -351,6 +353,34 @@ eval_select_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__r
             tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.rows2 = a.off_rows2;
         }
         sweep_body<NPL, TT, BUDGET, SMEM, false, FULL>(a, tb, best_idx, best_E);
+    }
+}
+
+// Tables too large to stage for all classes at once (fine frequency grids): a CTA serves ONE class
+// (blockIdx.y) and stages that class's threshold tables, pairc_c | rows2_c, in shared memory; one CTA
+// of 16 warps per SM.  When some row is not monotone the general path reads the full tables through L1.
+template <int NPL, int TT, bool BUDGET>
+__global__ void __launch_bounds__(512, 1)
+eval_select_class_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__restrict__ best_E) {
+    Tables tb;
+    if (all_rows_monotone(a)) {
+        extern __shared__ float4 smem[];
+        const int c = blockIdx.y;
+        const int pair_bytes = a.P * 8, rows2_bytes = a.P * (a.M + 1) * 8;
+        const float4 *src_p = reinterpret_cast<const float4 *>(a.ws + a.off_pairc + size_t(c) * pair_bytes);
+        const float4 *src_r = reinterpret_cast<const float4 *>(a.ws + a.off_rows2 + size_t(c) * rows2_bytes);
+        const int np16 = (pair_bytes + 15) / 16, nr16 = (rows2_bytes + 15) / 16;   // rounding up stays inside the scratch block
+        for (int i = threadIdx.x; i < np16; i += blockDim.x) smem[i] = src_p[i];
+        for (int i = threadIdx.x; i < nr16; i += blockDim.x) smem[np16 + i] = src_r[i];
+        __syncthreads();
+        tb.pairc = 0; tb.rows2 = uint32_t(np16) * 16u; tb.rows = 0; tb.slo = 0;
+        sweep_body<NPL, TT, BUDGET, true, true, true, true>(a, tb, best_idx, best_E);
+    } else {
+        const int c = blockIdx.y;
+        tb.rows = a.off_rows + uint32_t(c) * uint32_t(a.P * (a.M + 1)) * 16u;
+        tb.pairc = a.off_pairc + uint32_t(c) * uint32_t(a.P) * 8u;
+        tb.slo = a.off_slo; tb.rows2 = 0;
+        sweep_body<NPL, TT, BUDGET, false, false, true, true>(a, tb, best_idx, best_E);
     }
 }
 
@@ -486,10 +516,35 @@ cudaError_t launch_es_variant(SweepArgs &a, int32_t *best_idx, float *best_E, cu
     return cudaGetLastError();
 }
 
+// one class per CTA, 512 threads, the class's threshold tables in shared memory
+template <int NPL, int TT, bool B>
+cudaError_t launch_es_class(SweepArgs &a, size_t class_bytes, int32_t *best_idx, float *best_E, cudaStream_t st) {
+    auto kernel = eval_select_class_kernel<NPL, TT, B>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(class_bytes));
+    if (e != cudaSuccess) return e;
+    const int warps = 16;
+    // about four work units per resident warp
+    const int64_t want_units = int64_t(sm_count()) * warps * 4;
+    int64_t rpw = (a.tiles + want_units - 1) / want_units;          // rows of one class per unit
+    rpw = (rpw + TT - 1) / TT * TT;
+    a.rows_per_warp = rpw;
+    a.blocks = (a.rows_total + rpw - 1) / rpw;                      // units per class
+    const int64_t gx = (a.blocks + warps - 1) / warps;
+    kernel<<<dim3(unsigned(gx), unsigned(a.C)), warps * 32, class_bytes, st>>>(a, best_idx, best_E);
+    return cudaGetLastError();
+}
+
 template <int NPL, int TT>
 cudaError_t launch_es(SweepArgs &a, int32_t *best_idx, float *best_E, cudaStream_t st) {
     const bool smem = a.smem_bytes > 0;
     const bool budget = a.budget > 0;
+    if (!smem && NPL > 1) {
+        // pairc_c and rows2_c, each rounded up to 16 bytes
+        const size_t class_bytes = (size_t(a.P) * 8 + 15) / 16 * 16 + (size_t(a.P) * size_t(a.M + 1) * 8 + 15) / 16 * 16;
+        if (a.P % 2 == 0 && class_bytes + 1024 <= smem_limit())       // even P: class blocks stay 16-byte aligned
+            return budget ? launch_es_class<NPL, TT, true>(a, class_bytes, best_idx, best_E, st)
+                          : launch_es_class<NPL, TT, false>(a, class_bytes, best_idx, best_E, st);
+    }
     constexpr bool FULL = NPL > 1;                   // more than 32 instance counts: one pair group
     if (NPL == 1 && a.ln_log2 == 5) {                // exactly 17..32 instance counts
         if (budget && smem) return launch_es_variant<NPL, TT, true, true, true>(a, best_idx, best_E, st);
