@@ -387,26 +387,16 @@ eval_select_class_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, floa
 // ---------------------------------------------------------------------------------------------
 // evaluate only: E[tile][j], j = (n-1)*P + p.  A warp takes one tile and 32 consecutive pairs: lanes
 // are pairs (their constants stay in registers), the loop runs over n two at a time, and each pass
-// writes two coalesced runs of 32 energies.  Always the general path: the kernel is bound by the 4
-// bytes it writes per candidate.
+// writes two coalesced runs of 32 energies.  Threshold or general path as in the fused kernel.
 // ---------------------------------------------------------------------------------------------
-template <bool BUDGET, bool SMEM>
-__global__ void __launch_bounds__(kThreads)
-eval_configs_kernel(const SweepArgs a, const int64_t units, float *__restrict__ E_out) {
-    __shared__ __align__(16) float2 s_n[258];         // {n, 1/n} for n = 1..Nmax (Nmax <= 256), padded to even
-    for (int n1 = threadIdx.x; n1 < a.Nmax + 1; n1 += kThreads) s_n[n1] = make_float2(float(n1 + 1), 1.0f / float(n1 + 1));
-    Tables tb;
-    if (SMEM) {
-        stage(a, a.off_rows, a.off_rows2);
-        tb.rows = 0; tb.pairc = a.off_pairc - a.off_rows; tb.slo = a.off_slo - a.off_rows; tb.rows2 = 0;
-    } else {
-        __syncthreads();
-        tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.rows2 = a.off_rows2;
-    }
+template <bool BUDGET, bool SMEM, bool FAST>
+__device__ __forceinline__ void configs_body(const SweepArgs &a, const Tables tb, const float2 *s_n, const int64_t units,
+                                             float *__restrict__ E_out) {
     const int lane = threadIdx.x & 31;
     const int P = a.P, RS = a.M + 1, Nmax = a.Nmax;
     const int PG = (P + 31) / 32;                     // pair groups per tile
     const float Mf = float(a.M);
+    constexpr uint32_t ESZ = FAST ? 8u : 16u;
     uint32_t origin = table_origin<SMEM>();
     asm volatile("" : "+r"(origin) : : "memory");        // as in sweep_body: table loads stay behind the staging barrier
     const char *ws = a.ws;
@@ -425,39 +415,74 @@ eval_configs_kernel(const SweepArgs a, const int64_t units, float *__restrict__ 
         const bool active = p < P;
         const int pp = active ? p : 0;
         const float L = fmaxf(a.load[i], 0.f);
-        float slo_c;
-        if (SMEM) {
-            extern __shared__ float4 smem[];
-            slo_c = reinterpret_cast<const float *>(reinterpret_cast<const char *>(smem) + tb.slo)[c];
-        } else {
-            slo_c = __ldg(reinterpret_cast<const float *>(ws + tb.slo) + c);
-        }
+        const float slo_c = __ldg(reinterpret_cast<const float *>(ws + a.off_slo) + c);
         const float2 pc = pair_consts<SMEM>(ws, origin + tb.pairc + uint32_t(c * P + pp) * 8u);
-        const uint32_t base = origin + tb.rows + uint32_t((c * P + pp) * RS) * 16u - kTwo23Bits * 16u;
+        const uint32_t base = origin + (FAST ? tb.rows2 : tb.rows) + uint32_t((c * P + pp) * RS) * ESZ - kTwo23Bits * ESZ;
+        const float lic = L * pc.x;                   // per-instance table position is lic / n
+        const float lim = FAST ? pc.y : slo_c;
         int nlim = Nmax;                              // Eq. 1 GPU budget: n * TP <= budget
         if (BUDGET) {
             const int64_t q = int64_t(a.budget) / a.tp[pp / a.F];
             nlim = q < Nmax ? int(q) : Nmax;
         }
         float *out = E_out + size_t(i) * size_t(a.J) + p;
-        for (int n1 = 0; n1 < Nmax; n1 += 2) {
+        int off = 0;                                  // (n - 1) * P, below J < 2^31
+        for (int n1 = 0; n1 < Nmax; n1 += 2, off += 2 * P) {
             const float4 nn = s_n4[n1 >> 1];                       // {n, 1/n, n+1, 1/(n+1)}
-            const float2 v = make_float2(__saturatef(L * nn.y * pc.x), __saturatef(L * nn.w * pc.x));
+            const float2 v = make_float2(__saturatef(lic * nn.y), __saturatef(lic * nn.w));
             const float2 y = __ffma2_rz(v, k2.M, k2.two23);
             const float2 fm = __fadd2_rn(y, k2.neg23);
             const float2 nnu = __ffma2_rn(v, k2.negM, fm);
-            const float4 eA = entry16<SMEM>(ws, base, y.x);
-            const float4 eB = entry16<SMEM>(ws, base, y.y);
-            const float tbtA = fmaf(nnu.x, eA.y, eA.x), tbtB = fmaf(nnu.y, eB.y, eB.x);
-            const float2 E = __fmul2_rn(make_float2(fmaf(nnu.x, eA.w, eA.z), fmaf(nnu.y, eB.w, eB.z)),
-                                        make_float2(nn.x, nn.z));
-            const bool okA = tbtA <= slo_c && (!BUDGET || n1 + 1 <= nlim);
-            const bool okB = tbtB <= slo_c && (!BUDGET || n1 + 2 <= nlim);
+            float2 ew;
+            bool okA, okB;
+            if (FAST) {
+                const float2 eA = entry8<SMEM>(ws, base, y.x);
+                const float2 eB = entry8<SMEM>(ws, base, y.y);
+                ew = make_float2(fmaf(nnu.x, eA.y, eA.x), fmaf(nnu.y, eB.y, eB.x));
+                okA = v.x <= lim;
+                okB = v.y <= lim;
+            } else {
+                const float4 eA = entry16<SMEM>(ws, base, y.x);
+                const float4 eB = entry16<SMEM>(ws, base, y.y);
+                ew = make_float2(fmaf(nnu.x, eA.w, eA.z), fmaf(nnu.y, eB.w, eB.z));
+                okA = fmaf(nnu.x, eA.y, eA.x) <= lim;
+                okB = fmaf(nnu.y, eB.y, eB.x) <= lim;
+            }
+            const float2 E = __fmul2_rn(ew, make_float2(nn.x, nn.z));
+            if (BUDGET) {
+                okA = okA && n1 + 1 <= nlim;
+                okB = okB && n1 + 2 <= nlim;
+            }
             if (active) {
-                __stcs(out + size_t(n1) * P, okA ? E.x : CUDART_INF_F);
-                if (n1 + 1 < Nmax) __stcs(out + size_t(n1 + 1) * P, okB ? E.y : CUDART_INF_F);
+                __stcs(out + off, okA ? E.x : CUDART_INF_F);
+                if (n1 + 1 < Nmax) __stcs(out + off + P, okB ? E.y : CUDART_INF_F);
             }
         }
+    }
+}
+
+template <bool BUDGET, bool SMEM>
+__global__ void __launch_bounds__(kThreads)
+eval_configs_kernel(const SweepArgs a, const int64_t units, float *__restrict__ E_out) {
+    __shared__ __align__(16) float2 s_n[258];         // {n, 1/n} for n = 1..Nmax (Nmax <= 256), padded to even
+    for (int n1 = threadIdx.x; n1 < a.Nmax + 1; n1 += kThreads) s_n[n1] = make_float2(float(n1 + 1), 1.0f / float(n1 + 1));
+    Tables tb;
+    if (all_rows_monotone(a)) {                      // load-threshold path: 8-byte lookups (also a barrier for s_n)
+        if (SMEM) {
+            stage(a, a.off_pairc, a.off_end);
+            tb.pairc = 0; tb.slo = a.off_slo - a.off_pairc; tb.rows2 = a.off_rows2 - a.off_pairc; tb.rows = 0;
+        } else {
+            tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.rows2 = a.off_rows2;
+        }
+        configs_body<BUDGET, SMEM, true>(a, tb, s_n, units, E_out);
+    } else {
+        if (SMEM) {
+            stage(a, a.off_rows, a.off_rows2);
+            tb.rows = 0; tb.pairc = a.off_pairc - a.off_rows; tb.slo = a.off_slo - a.off_rows; tb.rows2 = 0;
+        } else {
+            tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.rows2 = a.off_rows2;
+        }
+        configs_body<BUDGET, SMEM, false>(a, tb, s_n, units, E_out);
     }
 }
 
