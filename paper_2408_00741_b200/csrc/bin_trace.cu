@@ -45,31 +45,48 @@ __device__ __forceinline__ uint32_t classify(const BinParams &bp, uint32_t in, u
 
 // NI/NO: compile-time edge counts (or -1: read them from the parameters).
 // VEC: the three arrays are 16-byte aligned.
-template <int NI, int NO, bool VEC>
+// PIECES: a slice may be taken in several pieces (chosen by the host for long slices); without it the
+// slice is one piece and the code is the plain straight-line form.
+template <int NI, int NO, bool VEC, bool PIECES>
 __global__ void __launch_bounds__(kThreads)
 bin_trace_kernel(const BinParams bp, const uint32_t *__restrict__ t_ms, const uint32_t *__restrict__ in_tok,
                  const uint32_t *__restrict__ out_tok, const uint64_t n_req, const uint64_t chunk,
                  uint32_t *__restrict__ counts, unsigned long long *__restrict__ dropped) {
     __shared__ __align__(16) uint32_t sbins[kSmemBins];
 
-    const uint64_t begin = uint64_t(blockIdx.x) * chunk;
-    if (begin >= n_req) return;
-    const uint64_t end = (begin + chunk < n_req) ? begin + chunk : n_req;
+    const uint64_t cta_begin = uint64_t(blockIdx.x) * chunk;
+    if (cta_begin >= n_req) return;
+    const uint64_t cta_end = (cta_begin + chunk < n_req) ? cta_begin + chunk : n_req;
     const uint32_t C = uint32_t(bp.C);
     const uint32_t W = bp.n_windows;
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const uint32_t copy = uint32_t(lane) & (kCopies - 1);
+    const uint32_t cap = uint32_t(kSmemBins / kCopies) / C;  // windows whose bins fit in shared memory
+    const uint64_t step = uint64_t(kWarps) * kBatch;
 
-    // window range kept in shared memory: starts at the window of the slice's first (or last,
+    // A slice that spans more windows than fit (a long sparse trace) is taken in pieces sized from its
+    // average density; whatever still falls outside a piece's window range goes to global atomics.
+    uint64_t piece = cta_end - cta_begin;
+    const uint32_t cta_wa = fastdiv(t_ms[cta_begin], bp.win), cta_wb = fastdiv(t_ms[cta_end - 1], bp.win);
+    {
+        const uint32_t wa = cta_wa, wb = cta_wb;
+        const uint64_t span = uint64_t(wa < wb ? wb - wa : wa - wb) + 1u;
+        if (PIECES && span > cap) {
+            piece = piece * cap / span * 3 / 4;
+            piece = piece / (2 * step) * (2 * step);         // whole double-batch passes of the CTA
+            if (piece < 2 * step) piece = 2 * step;
+        }
+    }
+    uint32_t my_dropped = 0;
+
+    auto run_piece = [&](const uint64_t begin, const uint64_t end, const uint32_t wa, const uint32_t wb) {
+    // window range kept in shared memory: starts at the window of the piece's first (or last,
     // if that is earlier) request
-    const uint32_t wa = fastdiv(t_ms[begin], bp.win);
-    const uint32_t wb = fastdiv(t_ms[end - 1], bp.win);
     const uint32_t w_lo = wa < wb ? wa : wb;
     uint32_t nwin = 0;
     if (w_lo < W) {
         const uint32_t span = (wa < wb ? wb - wa : wa - wb) + 1u;
-        const uint32_t cap = uint32_t(kSmemBins / kCopies) / C;
         nwin = span < cap ? span : cap;
         if (nwin > W - w_lo) nwin = W - w_lo;
     }
@@ -118,8 +135,6 @@ bin_trace_kernel(const BinParams bp, const uint32_t *__restrict__ t_ms, const ui
         }
     };
 
-    uint32_t my_dropped = 0;
-    const uint64_t step = uint64_t(kWarps) * kBatch;
     uint64_t base = begin + uint64_t(warp) * kBatch;
     if (VEC) {
         // two full batches per pass: six 16-byte loads in flight per lane before any of them is used
@@ -149,15 +164,26 @@ bin_trace_kernel(const BinParams bp, const uint32_t *__restrict__ t_ms, const ui
             if (i0 + r < end) count_one(t_ms[i0 + r], in_tok[i0 + r], out_tok[i0 + r], my_dropped);
     }
 
-    my_dropped = __reduce_add_sync(kFull, my_dropped);
-    if (lane == 0 && my_dropped) atomicAdd(dropped, (unsigned long long)my_dropped);
-
     __syncthreads();
     for (uint32_t i = threadIdx.x; i < nbins; i += kThreads) {
         const uint4 v = *reinterpret_cast<const uint4 *>(&sbins[i * kCopies]);
         const uint32_t sum = v.x + v.y + v.z + v.w;
         if (sum) atomicAdd(&counts[size_t(w_lo) * C + i], sum);
     }
+    };   // run_piece
+
+    if (!PIECES || piece == cta_end - cta_begin) {           // one piece, ends already read
+        run_piece(cta_begin, cta_end, cta_wa, cta_wb);
+    } else {
+        for (uint64_t begin = cta_begin; begin < cta_end; begin += piece) {
+            const uint64_t end = (begin + piece < cta_end) ? begin + piece : cta_end;
+            run_piece(begin, end, fastdiv(t_ms[begin], bp.win), fastdiv(t_ms[end - 1], bp.win));
+            __syncthreads();                                 // the bins are cleared again for the next piece
+        }
+    }
+
+    my_dropped = __reduce_add_sync(kFull, my_dropped);
+    if (lane == 0 && my_dropped) atomicAdd(dropped, (unsigned long long)my_dropped);
 }
 
 __global__ void counts_to_load_kernel(const uint32_t *__restrict__ counts, float *__restrict__ load, uint64_t n,
@@ -170,8 +196,12 @@ template <int NI, int NO>
 cudaError_t launch_variant(bool vec, int grid, const BinParams &bp, const uint32_t *t, const uint32_t *a,
                            const uint32_t *b, uint64_t n, uint64_t chunk, uint32_t *counts,
                            unsigned long long *dropped, cudaStream_t st) {
-    if (vec) bin_trace_kernel<NI, NO, true><<<grid, kThreads, 0, st>>>(bp, t, a, b, n, chunk, counts, dropped);
-    else bin_trace_kernel<NI, NO, false><<<grid, kThreads, 0, st>>>(bp, t, a, b, n, chunk, counts, dropped);
+    // slices longer than this may span more windows than the shared-memory bins hold
+    const bool pieces = chunk > 12288;
+    if (vec && pieces) bin_trace_kernel<NI, NO, true, true><<<grid, kThreads, 0, st>>>(bp, t, a, b, n, chunk, counts, dropped);
+    else if (vec) bin_trace_kernel<NI, NO, true, false><<<grid, kThreads, 0, st>>>(bp, t, a, b, n, chunk, counts, dropped);
+    else if (pieces) bin_trace_kernel<NI, NO, false, true><<<grid, kThreads, 0, st>>>(bp, t, a, b, n, chunk, counts, dropped);
+    else bin_trace_kernel<NI, NO, false, false><<<grid, kThreads, 0, st>>>(bp, t, a, b, n, chunk, counts, dropped);
     return cudaGetLastError();
 }
 

@@ -54,6 +54,19 @@ def test_unsorted_trace_and_few_windows(dyn):
     _check(dyn, t, i, o, 86_400_000, 1)                                     # one window
 
 
+@pytest.mark.parametrize("n,per_window", [(3_000_000, 0.7), (20_000_000, 12.0)])
+def test_long_sparse_trace(dyn, n, per_window):
+    """Many windows per request slice: a CTA's slice no longer fits its shared-memory bins and is taken in
+    pieces (long slices, 12 requests per window) or spills to global atomics (fewer than one per window)."""
+    rng = np.random.default_rng(7)
+    W = int(n / per_window)
+    wm = 3
+    t = np.sort(rng.integers(0, W * wm, n)).astype(np.uint32)
+    i = rng.integers(1, 3000, n).astype(np.uint32)
+    o = rng.integers(1, 1200, n).astype(np.uint32)
+    _check(dyn, t, i, o, wm, W)
+
+
 def test_window_edges_and_large_timestamps(dyn):
     for wm in (1, 7, 1000, 5000, 60_000, 65_536, 86_400_000, 4_294_967_295):
         ks = np.arange(0, 40, dtype=np.uint64)
