@@ -209,3 +209,28 @@ def totals(best_idx, best_E, J, n_of_j=None, tp_of_j=None):
     _load().orc_totals(_p(idx), _p(be), C.c_int64(S), C.c_int64(W), C.c_int32(Cn), C.c_int64(int(J)),
                        _p(nj), _p(tj), _p(et), _p(bad), _p(ew), _p(hist), _p(gp))
     return dict(E_total=et, n_infeasible=bad, E_window=ew, hist=hist, gpus=gp)
+
+
+def hier_select(profile, space, e1, e2, load):
+    """Hierarchical selection (nodes per pool -> sharding -> frequency): dict(nodes[S][K1][C],
+    shard[S][K2][C], best_idx, best_E [S][W][C], max_load[C]) plus the diagnostics nodes_frac,
+    shard_margin, shard_gap, freq_margin, freq_gap used for parity exemptions."""
+    lib = _load()
+    p, s, keep = _structs(profile, space)
+    load = _arr(load, np.float32)
+    S, W, Cn = load.shape
+    assert Cn == p.C
+    if int(e1) < 1 or int(e2) < 1 or int(e1) % int(e2) != 0:
+        raise ValueError("orc_hier_select: epochs must be >= 1 and e1 a multiple of e2")
+    K1, K2 = -(-W // int(e1)), -(-W // int(e2))
+    out = dict(nodes=np.empty((S, K1, Cn), np.int32), shard=np.empty((S, K2, Cn), np.int32),
+               best_idx=np.empty((S, W, Cn), np.int32), best_E=np.empty((S, W, Cn)),
+               max_load=np.empty(Cn), nodes_frac=np.empty((S, K1, Cn)), shard_margin=np.empty((S, K2, Cn)),
+               shard_gap=np.empty((S, K2, Cn)), freq_margin=np.empty((S, W, Cn)), freq_gap=np.empty((S, W, Cn)))
+    rc = lib.orc_hier_select(C.byref(p), C.byref(s), C.c_int32(int(e1)), C.c_int32(int(e2)), _p(load),
+                             C.c_int64(S), C.c_int64(W), _p(out["nodes"]), _p(out["shard"]), _p(out["best_idx"]),
+                             _p(out["best_E"]), _p(out["max_load"]), _p(out["nodes_frac"]), _p(out["shard_margin"]),
+                             _p(out["shard_gap"]), _p(out["freq_margin"]), _p(out["freq_gap"]))
+    if rc != 0:
+        raise ValueError("orc_hier_select: invalid argument (epochs must be >= 1 and e1 a multiple of e2)")
+    return out

@@ -24,6 +24,9 @@
  *                     runner-up energy (for near-tie exemptions in parity tests).
  *   orc_totals        cluster energy per scenario and per window, GPUs in use per window, histogram
  *                     of chosen configurations [Sec. 6 cluster-level energy, GPUs per sharding].
+ *   orc_hier_select   the controller hierarchy of Sec. 4.2 on the same models: nodes per pool from the
+ *                     epoch's peak load and the per-node maximum load (ceil(PL/ML)), sharding at the
+ *                     highest frequency within those GPUs, then the frequency per window.
  *
  * Readings of points the paper leaves open: class = number of edges <= value; window =
  * t_ms / window_ms (unsigned integer division); utilisation u = (L/n)/cap with u > 1 infeasible; tables sampled at u_m = m/(M-1);
@@ -287,4 +290,158 @@ void orc_totals(const int32_t *best_idx, const double *best_E, int64_t S, int64_
         E_total[s] = tot;
         n_infeasible[s] = bad;
     }
+}
+
+/* ---- hierarchical control (Sec. 4.2): nodes per pool, then sharding, then frequency ---------- */
+
+/*
+ * One candidate of class c at total load `load`: energy (+inf if infeasible) and the smallest
+ * relative distance of a deciding quantity to its bound.  Same arithmetic as orc_eval_tile.
+ */
+static double eval_candidate(const orc_profile *p, const orc_space *sp, const int32_t *row, const double *weight,
+                             int32_t c, double load, int32_t n, int32_t t, int32_t q, int32_t budget, double *margin) {
+    const int32_t R = p->R, M = p->M;
+    const size_t ct = ((size_t)c * p->T + t) * R;
+    const int32_t r = row[q];
+    const double om = weight[q];
+    const double ttft = lerp((double)p->ttft[ct + r], (double)p->ttft[ct + r + 1], om);
+    const double cap = lerp((double)p->cap[ct + r], (double)p->cap[ct + r + 1], om);
+    const double u = load / (double)n / cap;
+    const double x = fmin(u, 1.0) * (double)(M - 1);
+    int32_t m = (int32_t)floor(x);
+    if (m > M - 2) m = M - 2;
+    const double nu = x - (double)m;
+    const double tbt = table_at(p->tbt + ct * M, M, r, om, m, nu);
+    const double pw = table_at(p->pw + ct * M, M, r, om, m, nu);
+    const double slo_a = (double)sp->slo_ttft[c], slo_b = (double)sp->slo_tbt[c];
+    int ok = (ttft <= slo_a) && (tbt <= slo_b) && (u <= 1.0);
+    if (budget > 0 && n * p->tp[t] > budget) ok = 0;
+    if (margin) {
+        double d = fabs(tbt - slo_b) / slo_b;
+        if (fabs(u - 1.0) < d) d = fabs(u - 1.0);
+        if (d < *margin) *margin = d;
+    }
+    return ok ? (double)n * pw * (double)sp->window_s / 3600.0 : INFINITY;
+}
+
+/*
+ * ML of class c: the largest load one instance of the highest-performance configuration (largest TP,
+ * highest candidate frequency) sustains with TTFT, TBT and capacity within bounds [Sec. 4.2
+ * scale-out/in].  TBT is piecewise linear in the utilisation, so the largest feasible utilisation is
+ * found segment by segment from the top.  0 if no load is feasible.
+ */
+double orc_max_load(const orc_profile *p, const orc_space *sp, const int32_t *row, const double *weight, int32_t c) {
+    const int32_t t = p->T - 1, q = sp->F - 1, R = p->R, M = p->M;
+    const size_t ct = ((size_t)c * p->T + t) * R;
+    const int32_t r = row[q];
+    const double om = weight[q];
+    const double ttft = lerp((double)p->ttft[ct + r], (double)p->ttft[ct + r + 1], om);
+    const double cap = lerp((double)p->cap[ct + r], (double)p->cap[ct + r + 1], om);
+    const double slo_b = (double)sp->slo_tbt[c];
+    if (!(ttft <= (double)sp->slo_ttft[c]) || !(cap > 0.0)) return 0.0;
+    for (int32_t m = M - 2; m >= 0; --m) {
+        const double a = table_at(p->tbt + ct * M, M, r, om, m, 0.0);
+        const double b = table_at(p->tbt + ct * M, M, r, om, m, 1.0);
+        if (b <= slo_b) return (double)(m + 1) / (double)(M - 1) * cap;
+        if (a <= slo_b) return ((double)m + (slo_b - a) / (b - a)) / (double)(M - 1) * cap;
+    }
+    return 0.0;
+}
+
+/*
+ * Hierarchical selection for loads [S][W][C].  Epoch lengths in windows: e1 (nodes per pool), e2
+ * (sharding), 1 (frequency); e1 must be a multiple of e2.  The load predictor is the epoch's own peak.
+ *   nodes[s][k1][c]  = max(1, ceil(PL / ML_c)), PL = peak load of the scale epoch; -1 if ML_c == 0
+ *   shard[s][k2][c]  = (n-1)*T + t minimising the energy at the highest candidate frequency and the
+ *                      shard epoch's peak load, over n*TP <= nodes*TP_max (and the space's own GPU
+ *                      budget), lowest index on ties; -1 if none is feasible
+ *   best_idx/best_E  per window: with (n, t) of its shard epoch, the feasible frequency of least
+ *                      energy at the window's load (lowest on ties); -1 / +inf if none
+ * Optional diagnostics for parity tests (NULL to skip): nodes_frac = PL/ML; shard_margin / shard_gap =
+ * margin and relative runner-up gap of the sharding decision; freq_margin / freq_gap likewise per tile.
+ */
+int orc_hier_select(const orc_profile *p, const orc_space *sp, int32_t e1, int32_t e2, const float *load,
+                    int64_t S, int64_t W, int32_t *nodes, int32_t *shard, int32_t *best_idx, double *best_E,
+                    double *max_load, double *nodes_frac, double *shard_margin, double *shard_gap,
+                    double *freq_margin, double *freq_gap) {
+    if (e1 < 1 || e2 < 1 || e1 % e2 != 0) return ORC_EINVAL;
+    const int32_t C = p->C, T = p->T, F = sp->F;
+    int32_t *row = (int32_t *)malloc(sizeof(int32_t) * (size_t)F);
+    double *wt = (double *)malloc(sizeof(double) * (size_t)F);
+    int rc = orc_resolve(p->f_grid, p->R, sp->f_cand, F, row, wt);
+    if (rc != ORC_OK) { free(row); free(wt); return rc; }
+    const int64_t K1 = (W + e1 - 1) / e1, K2 = (W + e2 - 1) / e2;
+    const int32_t gpus_per_node = p->tp[T - 1];
+    double *ml = (double *)malloc(sizeof(double) * (size_t)C);
+    for (int32_t c = 0; c < C; ++c) {
+        ml[c] = orc_max_load(p, sp, row, wt, c);
+        if (max_load) max_load[c] = ml[c];
+    }
+#pragma omp parallel for schedule(static) collapse(2)
+    for (int64_t s = 0; s < S; ++s) {
+        for (int32_t c = 0; c < C; ++c) {
+            for (int64_t k1 = 0; k1 < K1; ++k1) {
+                /* scale-out/in: nodes for the peak of the epoch */
+                const int64_t w1a = k1 * e1, w1b = (w1a + e1 < W) ? w1a + e1 : W;
+                double PL = 0.0;
+                for (int64_t w = w1a; w < w1b; ++w) {
+                    const double L = (double)load[(s * W + w) * C + c];
+                    if (L > PL) PL = L;
+                }
+                int32_t nn = -1;
+                if (ml[c] > 0.0) {
+                    nn = (int32_t)ceil(PL / ml[c]);
+                    if (nn < 1) nn = 1;
+                }
+                nodes[(s * K1 + k1) * C + c] = nn;
+                if (nodes_frac) nodes_frac[(s * K1 + k1) * C + c] = ml[c] > 0.0 ? PL / ml[c] : INFINITY;
+                int32_t budget = nn > 0 ? nn * gpus_per_node : 0;
+                if (sp->gpu_budget > 0 && budget > sp->gpu_budget) budget = sp->gpu_budget;
+
+                /* shard-up/down: instances x TP at the highest frequency, peak of the shard epoch */
+                for (int64_t w2a = w1a; w2a < w1b; w2a += e2) {
+                    const int64_t k2 = w2a / e2, w2b = (w2a + e2 < w1b) ? w2a + e2 : w1b;
+                    double PL2 = 0.0;
+                    for (int64_t w = w2a; w < w2b; ++w) {
+                        const double L = (double)load[(s * W + w) * C + c];
+                        if (L > PL2) PL2 = L;
+                    }
+                    int32_t best_nt = -1;
+                    double eb = INFINITY, e2nd = INFINITY, mg = INFINITY;
+                    if (nn > 0) {
+                        for (int32_t n = 1; n <= sp->Nmax; ++n)
+                            for (int32_t t = 0; t < T; ++t) {
+                                const double E = eval_candidate(p, sp, row, wt, c, PL2, n, t, F - 1, budget, &mg);
+                                if (E < eb) { e2nd = eb; eb = E; best_nt = (n - 1) * T + t; }
+                                else if (E < e2nd) e2nd = E;
+                            }
+                    }
+                    shard[(s * K2 + k2) * C + c] = best_nt;
+                    if (shard_margin) shard_margin[(s * K2 + k2) * C + c] = mg;
+                    if (shard_gap) shard_gap[(s * K2 + k2) * C + c] = best_nt >= 0 ? (e2nd - eb) / eb : INFINITY;
+
+                    /* scale-up/down: frequency per window for the chosen sharding */
+                    for (int64_t w = w2a; w < w2b; ++w) {
+                        const int64_t i = (s * W + w) * C + c;
+                        int32_t bq = -1;
+                        double fb = INFINITY, f2 = INFINITY, fm = INFINITY;
+                        if (best_nt >= 0) {
+                            const int32_t n = best_nt / T + 1, t = best_nt % T;
+                            for (int32_t q = 0; q < F; ++q) {
+                                const double E = eval_candidate(p, sp, row, wt, c, (double)load[i], n, t, q, 0, &fm);
+                                if (E < fb) { f2 = fb; fb = E; bq = q; }
+                                else if (E < f2) f2 = E;
+                            }
+                        }
+                        best_idx[i] = bq >= 0 ? best_nt * F + bq : -1;
+                        best_E[i] = fb;
+                        if (freq_margin) freq_margin[i] = fm;
+                        if (freq_gap) freq_gap[i] = bq >= 0 ? (f2 - fb) / fb : INFINITY;
+                    }
+                }
+            }
+        }
+    }
+    free(row); free(wt); free(ml);
+    return ORC_OK;
 }
