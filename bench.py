@@ -359,6 +359,10 @@ def run_ours(args, rank, world, local_rank):
             result["materialised"] = measure_materialised(dyn, gen, dev)
         except Exception as exc:
             result["materialised"] = {"error": repr(exc)}
+        try:
+            result["hierarchical"] = measure_hier(dyn, gen, dev)
+        except Exception as exc:
+            result["hierarchical"] = {"error": repr(exc)}
 
     if not args.no_cpu_baseline and world == 1:
         cb, _, _ = time_oracle(wl, trace, prof, sp, base_counts)
@@ -452,6 +456,53 @@ def measure_materialised(dyn, gen, dev, S=16):
     return res
 
 
+def measure_hier(dyn, gen, dev, S=2048):
+    """Hierarchical selection (nodes per 30 min, sharding per 5 min, frequency per 1-min window) on S
+    day-long scenarios, whole call; and its energy against the joint optimum on the first 8 scenarios."""
+    import torch
+    wl = gen.workload("cfg2")
+    prof, sp = wl.profile(), wl.space()
+    W, Cn, J = wl.trace.n_windows, 9, wl.J
+    e1, e2 = 30, 5
+    load = torch.from_numpy(gen.random_loads((S, W, Cn), seed=10, mean=2.5)).to(dev)
+    P = dyn.Profile(prof.tp, prof.f_grid_mhz, prof.ttft, prof.cap, prof.tbt, prof.pow, device=dev)
+    SP = dyn.Space(sp.f_cand_mhz, sp.n_max, sp.slo_ttft_s, sp.slo_tbt_s, sp.window_s, sp.gpu_budget)
+    nodes = torch.empty((S, -(-W // e1), Cn), dtype=torch.int32, device=dev)
+    shard = torch.empty((S, -(-W // e2), Cn), dtype=torch.int32, device=dev)
+    out = dyn.SelectOut(S, W, Cn, J, device=dev, windows=False, hist=False, gpus=False)
+    ws = torch.empty(dyn.dyn_hier_workspace_bytes(P, SP, S, W), dtype=torch.uint8, device=dev)
+    call = lambda: dyn.dyn_hier_select(P, SP, e1, e2, load, nodes, shard, out, ws)
+    for _ in range(3):
+        call()
+    K = 10
+    e0, e1_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(K):
+        call()
+    e1_.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1_) / K
+    tiles = S * W * Cn
+    # candidates of the two restricted searches: (n, TP) per shard epoch, f per window; the node budget
+    # prunes part of the first, so this is an upper bound of what was evaluated
+    K2 = -(-W // e2)
+    cands = S * Cn * (K2 * sp.n_max * len(prof.tp) + W * len(sp.f_cand_mhz))
+    fp32_peak = SM_COUNT * FP32_LANES * 2 * SM_MAX_MHZ * 1e6 / 1e12
+    tfl = FLOP_PER_EVAL * cands / (ms * 1e-3) / 1e12
+    hier_total = float(out.E_total[:8].sum().item())
+    jout = dyn.SelectOut(8, W, Cn, J, device=dev, windows=False, hist=False, gpus=False)
+    jws = torch.empty(dyn.dyn_workspace_bytes(P, SP, 8, W), dtype=torch.uint8, device=dev)
+    dyn.dyn_eval_select(P, SP, load[:8].contiguous(), jout, jws)
+    torch.cuda.synchronize()
+    joint_total = float(jout.E_total.sum().item())
+    return {"workload": f"cfg2 shape x {S} scenarios, epochs {e1}/{e2}/1 windows", "tiles": int(tiles), "call_ms": ms,
+            "tiles_per_s": tiles / (ms * 1e-3), "candidates_upper_bound": int(cands),
+            "roofline": {"bound": "alu", "achieved": tfl, "peak": fp32_peak, "unit": "TFLOP/s", "frac": tfl / fp32_peak,
+                         "traffic": None, "peak_source": "derived fp32 peak; candidates are an upper bound (node budget prunes)"},
+            "energy_over_joint_optimum": hier_total / joint_total}
+
+
 def main():
     args = parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -466,7 +517,8 @@ def main():
         import paper_2408_00741_b200 as dyn
         dev = torch.device("cuda", local_rank)
         torch.cuda.set_device(dev)
-        print(json.dumps({"bin_trace": measure_bin(dyn, gen, dev), "materialised": measure_materialised(dyn, gen, dev)}))
+        print(json.dumps({"bin_trace": measure_bin(dyn, gen, dev), "materialised": measure_materialised(dyn, gen, dev),
+                          "hierarchical": measure_hier(dyn, gen, dev)}))
         return
     run_ours(args, rank, world, local_rank)
 

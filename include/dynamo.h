@@ -172,6 +172,37 @@ int dyn_eval_select(const dyn_profile *profile, const dyn_space *space, const fl
                     void *stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Hierarchical control.  [Sec. 4.2: instead of the joint search, three controllers set one knob each
+ * at their own time scale -- scale-out/in: the number of nodes of a pool for the epoch's peak load PL,
+ * ceil(PL / ML) with ML the largest load one node sustains in the highest-performance configuration;
+ * shard-up/down: how the machine's GPUs are split into instances x TP, decided at the highest frequency;
+ * scale-up/down: the frequency, per window, among those that keep the SLO.]
+ *
+ * Epoch lengths are in windows: scale_epoch_windows (nodes), shard_epoch_windows (sharding), 1
+ * (frequency); scale_epoch_windows must be a multiple of shard_epoch_windows.  The load "prediction"
+ * of an epoch is its own peak.  A node has TP_max = tp[T-1] GPUs.  Per scenario s and class c:
+ *   d_nodes[s][k1][c] = max(1, ceil(PL / ML_c)), PL = max load over scale epoch k1; -1 if no load is
+ *                       feasible at (TP_max, highest candidate frequency);
+ *   d_shard[s][k2][c] = (n-1)*T + t of least energy at the highest candidate frequency and the peak
+ *                       load of shard epoch k2, over n*TP_t <= nodes*TP_max (and space->gpu_budget when
+ *                       set), lowest index on ties; -1 if none is feasible;
+ *   out->d_best_idx / d_best_E [s][w][c]: for that (n, t), the feasible frequency of least energy at
+ *                       the window's load (lowest on ties), as candidate index j; -1 / +inf if none.
+ * The totals in `out` are as in dyn_select.  K1 = ceil(W / scale_epoch_windows), K2 likewise.
+ * Workspace: dyn_hier_workspace_bytes().  Errors: as dyn_eval_select, plus DYN_EINVAL for bad epochs
+ * or NULL d_nodes / d_shard.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t scale_epoch_windows;
+    int32_t shard_epoch_windows;
+} dyn_hier_spec;
+
+size_t dyn_hier_workspace_bytes(const dyn_profile *profile, const dyn_space *space, int64_t S, int64_t W);
+int dyn_hier_select(const dyn_profile *profile, const dyn_space *space, const dyn_hier_spec *hier,
+                    const float *d_load, int64_t S, int64_t W, int32_t *d_nodes, int32_t *d_shard,
+                    const dyn_select_out *out, void *d_ws, size_t ws_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Whole path from HOST buffers: (a) -> (b) -> (c) in one call.  [Sec. 3 trace -> Sec. 3.2 loads ->
  * Sec. 4.1 / Eq. 1 evaluation -> Sec. 4.2 selection -> Sec. 6 totals]
  *

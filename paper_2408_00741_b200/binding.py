@@ -24,7 +24,8 @@ _lib = C.CDLL(LIB_PATH)
 DYN_OK, DYN_EINVAL, DYN_ECUDA, DYN_EUNSUPPORTED, DYN_EWORKSPACE = 0, -1, -2, -3, -4
 EXPORTS = ("dyn_strerror", "dyn_last_cuda_error", "dyn_bin_trace", "dyn_workspace_bytes", "dyn_eval_configs",
            "dyn_select_workspace_bytes", "dyn_select", "dyn_eval_select", "dyn_pipeline_arena_bytes",
-           "dyn_pipeline_host", "dyn_set_timing_events", "dyn_eval_select_static")
+           "dyn_pipeline_host", "dyn_set_timing_events", "dyn_eval_select_static", "dyn_hier_workspace_bytes",
+           "dyn_hier_select")
 
 
 class DynError(RuntimeError):
@@ -106,6 +107,16 @@ _lib.dyn_set_timing_events.restype = None
 _lib.dyn_set_timing_events.argtypes = [C.c_void_p, C.c_void_p]
 
 
+class _HierSpec(C.Structure):
+    _fields_ = [("scale_epoch_windows", C.c_int32), ("shard_epoch_windows", C.c_int32)]
+
+
+_lib.dyn_hier_workspace_bytes.restype = C.c_size_t
+_lib.dyn_hier_workspace_bytes.argtypes = [C.POINTER(_Profile), C.POINTER(_Space), C.c_int64, C.c_int64]
+_lib.dyn_hier_select.restype = C.c_int
+_lib.dyn_hier_select.argtypes = [C.POINTER(_Profile), C.POINTER(_Space), C.POINTER(_HierSpec), C.c_void_p, C.c_int64,
+                                 C.c_int64, C.c_void_p, C.c_void_p, C.POINTER(_SelectOut), C.c_void_p, C.c_size_t,
+                                 C.c_void_p]
 _lib.dyn_eval_select_static.restype = C.c_int
 _lib.dyn_eval_select_static.argtypes = [C.POINTER(_Profile), C.POINTER(_Space), C.c_void_p, C.c_int64, C.c_int64,
                                         C.POINTER(_SelectOut), C.c_void_p]
@@ -317,3 +328,22 @@ def dyn_eval_select_static(profile: Profile, space: Space, d_load, out: SelectOu
     rc = _lib.dyn_eval_select_static(C.byref(p), C.byref(s), _dev(d_load, torch.float32, "d_load"), S, W, C.byref(o),
                                      _stream())
     _check(rc, "dyn_eval_select_static")
+
+
+def dyn_hier_workspace_bytes(profile: Profile, space: Space, S, W) -> int:
+    p, s = profile._struct(), space._struct()
+    return int(_lib.dyn_hier_workspace_bytes(C.byref(p), C.byref(s), int(S), int(W)))
+
+
+def dyn_hier_select(profile: Profile, space: Space, scale_epoch_windows, shard_epoch_windows, d_load, d_nodes, d_shard,
+                    out: SelectOut, d_ws):
+    """Hierarchical selection: d_nodes int32 [S][K1][C], d_shard int32 [S][K2][C], per-window choice in `out`."""
+    S, W, Cn = d_load.shape
+    p, s = profile._struct(), space._struct()
+    h = _HierSpec(int(scale_epoch_windows), int(shard_epoch_windows))
+    o = out._struct()
+    ws, nb = _ws(d_ws)
+    rc = _lib.dyn_hier_select(C.byref(p), C.byref(s), C.byref(h), _dev(d_load, torch.float32, "d_load"), S, W,
+                              _dev(d_nodes, torch.int32, "d_nodes"), _dev(d_shard, torch.int32, "d_shard"), C.byref(o),
+                              ws, nb, _stream())
+    _check(rc, "dyn_hier_select")

@@ -255,4 +255,40 @@ int dyn_eval_select(const dyn_profile *profile, const dyn_space *space, const fl
     return DYN_OK;
 }
 
+size_t dyn_hier_workspace_bytes(const dyn_profile *profile, const dyn_space *space, int64_t S, int64_t W) {
+    const size_t base = dyn_workspace_bytes(profile, space, S, W);
+    return base ? base + align256(size_t(profile->C) * sizeof(double)) : 0;
+}
+
+int dyn_hier_select(const dyn_profile *profile, const dyn_space *space, const dyn_hier_spec *hier,
+                    const float *d_load, int64_t S, int64_t W, int32_t *d_nodes, int32_t *d_shard,
+                    const dyn_select_out *out, void *d_ws, size_t ws_bytes, void *stream) {
+    ResolveParams rp;
+    int rc = check_problem(profile, space, S, W, &rp);
+    if (rc != DYN_OK) return rc;
+    if (!hier || hier->scale_epoch_windows < 1 || hier->shard_epoch_windows < 1 ||
+        hier->scale_epoch_windows % hier->shard_epoch_windows != 0)
+        return DYN_EINVAL;
+    if (W * profile->C >= (int64_t(1) << 31)) return DYN_EUNSUPPORTED;      // 32-bit indices inside a scenario
+    const int64_t tiles = S * W * profile->C;
+    rc = check_out(out, S, tiles);
+    if (rc != DYN_OK) return rc;
+    if (tiles > 0 && (!d_load || !d_nodes || !d_shard)) return DYN_EINVAL;
+    const ResolvedLayout lay = resolved_layout(profile->C, profile->T, space->F, profile->M, space->Nmax, S, W);
+    rc = check_ws(d_ws, ws_bytes, lay.total + align256(size_t(profile->C) * sizeof(double)));
+    if (rc != DYN_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char *ws = static_cast<char *>(d_ws);
+    DYN_CUDA_TRY(launch_resolve(rp, lay, d_ws, st));
+    DYN_CUDA_TRY(launch_hier(rp, lay, d_ws, lay.total, d_load, S, W, hier->scale_epoch_windows,
+                             hier->shard_epoch_windows, space->gpu_budget, d_nodes, d_shard, out->d_best_idx,
+                             out->d_best_E, st));
+    const int64_t chunks = totals_chunks(W);
+    double *partial = reinterpret_cast<double *>(ws + lay.off_partial);
+    uint32_t *partial_bad = reinterpret_cast<uint32_t *>(ws + lay.off_partial + size_t(S) * size_t(chunks) * sizeof(double));
+    DYN_CUDA_TRY(launch_totals(to_out(out), S, W, profile->C, lay.J, nullptr, nullptr, profile->T, space->F,
+                               reinterpret_cast<const int32_t *>(ws + lay.off_tp), partial, partial_bad, st));
+    return DYN_OK;
+}
+
 }  // extern "C"

@@ -100,6 +100,9 @@ cudaError_t launch_totals(const SelectOut &o, int64_t S, int64_t W, int32_t C, i
                           const int32_t *d_tj, int32_t T, int32_t F, const int32_t *d_tp, double *d_partial,
                           uint32_t *d_partial_bad, cudaStream_t st);
 int64_t totals_chunks(int64_t W);
+cudaError_t launch_hier(const ResolveParams &rp, const ResolvedLayout &lay, void *d_ws, size_t off_ml, const float *d_load,
+                        int64_t S, int64_t W, int32_t e1, int32_t e2, int32_t space_budget, int32_t *d_nodes,
+                        int32_t *d_shard, int32_t *best_idx, float *best_E, cudaStream_t st);
 
 struct BinParams {
     FastDiv win;
