@@ -334,7 +334,7 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
 }
 
 template <int NPL, int TT, bool BUDGET, bool SMEM, bool FULL>
-__global__ void __launch_bounds__(kThreads, (NPL <= 2 ? 5 : 2))
+__global__ void __launch_bounds__(kThreads, (NPL * TT <= 4 ? 5 : (NPL * TT <= 8 && NPL <= 2 ? 4 : 2)))
 eval_select_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__restrict__ best_E) {
     Tables tb;
     if (all_rows_monotone(a)) {                      // uniform over the grid: every CTA reads the same flags
@@ -596,7 +596,7 @@ cudaError_t launch_eval_select(const ResolvedLayout &lay, const void *d_ws, cons
     const int npl = (lay.Nmax + 31) / 32;           // instance counts per lane
     // four candidates per lane share each pair's constants
     if (npl <= 1) return launch_es<1, 4>(a, best_idx, best_E, st);
-    if (npl <= 2) return launch_es<2, 2>(a, best_idx, best_E, st);
+    if (npl <= 2) return launch_es<2, 4>(a, best_idx, best_E, st);
     if (npl <= 4) return launch_es<4, 1>(a, best_idx, best_E, st);
     if (npl <= 8) return launch_es<8, 1>(a, best_idx, best_E, st);
     return cudaErrorInvalidValue;                   // Nmax > 256 is rejected by the caller
