@@ -327,8 +327,8 @@ def run_ours(args, rank, world, local_rank):
     fp32_peak = SM_COUNT * FP32_LANES * 2 * SM_MAX_MHZ * 1e6 / 1e12
     achieved = FLOP_PER_EVAL * evals_per_step / (k_ms * 1e-3) / 1e12
     # DRAM bytes per launch from the ncu capture summarised in profiles/eval_select_kernel_cfg4_S64.md
-    # (3.38 MB read, 0 written at S = 64; grows in proportion to S); null for other shapes
-    traffic = 3.38e6 * S / 64 if (wl.name == "cfg4" and J == 2048) else None
+    # (3.40 MB read, 0 written at S = 64; grows in proportion to S); null for other shapes
+    traffic = 3.40e6 * S / 64 if (wl.name == "cfg4" and J == 2048) else None
     roofline = {"bound": "alu", "kernel": "eval_select_kernel", "achieved": achieved, "peak": fp32_peak,
                 "unit": "TFLOP/s", "frac": achieved / fp32_peak, "traffic": traffic,
                 "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 flop x 1965 MHz (no measured fp32 figure in "
