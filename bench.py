@@ -168,9 +168,17 @@ def time_oracle(wl, trace, prof, sp, base_counts, target_s=15.0, max_scen=512):
         t0 = time.perf_counter(); oracle_step(wl, trace, prof, sp, ex); dt = time.perf_counter() - t0
     else:
         dt = dt0
-    return {"value": n * per_scen / dt, "unit": "evals/s", "cores": oracle.num_threads(), "kind": "oracle",
+    cores = oracle.num_threads()
+    # the same oracle on one thread, on a smaller sample (about a fifth of the time)
+    n1 = max(1, min(n, int(round(n / max(cores, 1) / 5)) or 1))
+    ex1 = scenario_loads(wl, base_counts, n1 - 1)
+    oracle.set_num_threads(1)
+    t0 = time.perf_counter(); oracle_step(wl, trace, prof, sp, ex1); dt1 = time.perf_counter() - t0
+    oracle.set_num_threads(cores)
+    return {"value": n * per_scen / dt, "unit": "evals/s", "cores": cores, "kind": "oracle",
             "sample": f"{n} of {wl.S} scenario(s) of {wl.name}: trace binning + {n * W * Cn} tiles x {wl.J} candidates "
-                      f"in {dt:.2f} s"}, n, dt
+                      f"in {dt:.2f} s",
+            "single_thread_value": n1 * per_scen / dt1, "single_thread_sample": f"{n1} scenario(s) in {dt1:.2f} s"}, n, dt
 
 
 # ----------------------------------------------------------------------------------------------
@@ -373,42 +381,45 @@ def run_ours(args, rank, world, local_rank):
 
 
 def measure_bin(dyn, gen, dev):
-    """Requests/s of the trace-binning kernel on the 14M-request week trace (168 MB, larger than L2)."""
+    """Requests/s of the trace-binning kernel on the 14M-request week trace (168 MB, larger than L2), and
+    on the same trace repeated 8 times (1.3 GB) to show what the kernel sustains on a long trace."""
     import torch
     wl = gen.workload("cfg3")
     t, i, o = gen.make_trace(wl.trace)
     W = wl.trace.n_windows
-    to_dev = lambda a: torch.from_numpy(a.view(np.int32)).to(dev)
-    d = [to_dev(x) for x in (t, i, o)]
+    peak, src = _hbm_peak()
     counts = torch.empty((W, 9), dtype=torch.int32, device=dev)
     load = torch.empty((W, 9), dtype=torch.float32, device=dev)
     dropped = torch.empty(1, dtype=torch.int64, device=dev)
-    run = lambda: dyn.dyn_bin_trace(wl.trace.window_ms, W, gen.IN_EDGES, gen.OUT_EDGES, d[0], d[1], d[2], counts, load, dropped)
-    for _ in range(3):
-        run()
-    K = 20
-    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
-    for a, b in kev:
-        a.record(); b.record()
-    torch.cuda.synchronize()
-    for k in range(K):
-        dyn.dyn_set_timing_events(*kev[k])
-        run()
-    dyn.dyn_set_timing_events(None, None)
-    torch.cuda.synchronize()
-    ms = float(np.mean([a.elapsed_time(b) for a, b in kev]))
-    peaks = {}
-    try:
-        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
-    except OSError:
-        pass
-    peak = float(peaks.get("hbm_gbs", 6650.0))
-    gbs = BYTES_PER_REQUEST * len(t) / (ms * 1e-3) / 1e9
-    return {"workload": "cfg3", "requests": int(len(t)), "kernel": "bin_trace_kernel", "kernel_ms": ms,
-            "requests_per_s": len(t) / (ms * 1e-3),
-            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
-                         "traffic": None,
-                         "peak_source": "measured (MEASURED_PEAKS.json)" if peaks else "fallback 6650 GB/s"}}
+    out = {}
+    for rep in (1, 8):
+        d = [torch.from_numpy(np.tile(x, rep).view(np.int32)).to(dev) for x in (t, i, o)]
+        n = int(d[0].numel())
+        run = lambda: dyn.dyn_bin_trace(wl.trace.window_ms, W, gen.IN_EDGES, gen.OUT_EDGES, d[0], d[1], d[2], counts, load, dropped)
+        for _ in range(3):
+            run()
+        K = 20 if rep == 1 else 5
+        kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        for a, b in kev:
+            a.record(); b.record()
+        torch.cuda.synchronize()
+        for k in range(K):
+            dyn.dyn_set_timing_events(*kev[k])
+            run()
+        dyn.dyn_set_timing_events(None, None)
+        torch.cuda.synchronize()
+        assert int(counts.sum().item()) + int(dropped.item()) == n
+        ms = float(np.mean([a.elapsed_time(b) for a, b in kev]))
+        gbs = BYTES_PER_REQUEST * n / (ms * 1e-3) / 1e9
+        r = {"requests": n, "kernel_ms": ms, "requests_per_s": n / (ms * 1e-3),
+             "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                          "traffic": None, "peak_source": src}}
+        if rep == 1:
+            out = {"workload": "cfg3", "kernel": "bin_trace_kernel", **r}
+        else:
+            out["long_trace_x8"] = r
+        del d
+    return out
 
 
 def _hbm_peak():
