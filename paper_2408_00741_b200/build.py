@@ -15,7 +15,7 @@ HEADERS = [os.path.join(CSRC, "dyn_internal.cuh"), os.path.join(ROOT, "include",
 
 def nvcc_command(verbose_ptxas: bool = False):
     cmd = ["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
-           "-shared", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
+           "-shared", "-Xcompiler", "-fPIC", "--threads", "0", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
     if verbose_ptxas:
         cmd += ["-Xptxas", "-v"]
     cmd += [os.path.join(CSRC, s) for s in SOURCES] + ["-o", LIB]

@@ -56,7 +56,8 @@ __device__ __forceinline__ uint32_t fastdiv(uint32_t n, const FastDiv &f) {
 //                   vlim = largest v with TBT <= slo_tbt[c] and u <= 1 when TBT does not decrease
 //                   along the row (-1 for a never-feasible pair), NaN when it does decrease somewhere.
 //   slo[c]          slo_tbt[c]
-//   rows2[c][p][m]  m = 0..M, float2 {e_a, -e_d}: the energy half of rows, for the threshold path
+//   rows2[c][p][m]  m = 0..M, float2 {a, b}: the energy line of segment m in v, e = a + v*b (a = e_a - m*e_d,
+//                   b = M*e_d; flat at the last knot's energy for m >= M-1), for the threshold path
 struct ResolvedLayout {
     int32_t C, T, F, P, M, Nmax, J;
     int32_t row_stride;          // entries per pair row (M + 1)

@@ -87,7 +87,15 @@ __global__ void resolve_kernel(const ResolveParams rp, float4 *__restrict__ rows
         }
         if (!pair_ok) v.x = kInf;
         rows[(size_t(c) * P + p) * RS + m] = v;
-        rows2[(size_t(c) * P + p) * RS + m] = make_float2(v.z, v.w);
+        // threshold path: the same energy line as intercept and slope in v = x/M, e(v) = a + v*b
+        // (the lines of neighbouring segments meet at the knots, so a position that rounding puts on
+        // either side of a knot gets the same value)
+        float2 line = make_float2(float(pw_m), 0.f);
+        if (m < M - 1) {
+            const double d = lerp64(pw0[m + 1], pw1[m + 1], w) * scale - pw_m;
+            line = make_float2(float(pw_m - double(m) * d), float(d * double(M)));
+        }
+        rows2[(size_t(c) * P + p) * RS + m] = line;
         if (m == 0) {
             // Load threshold of the pair: if TBT never decreases along the row, "TBT <= slo and u <= 1"
             // holds exactly for x in [0, xlim].  NaN marks a row without that property.

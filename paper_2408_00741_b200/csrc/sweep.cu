@@ -10,16 +10,18 @@
 //   * table position x = u*(M-1) = sat(L/n * ic) * M: the saturating multiply clamps for free, and
 //     u > 1 is not tested: the table rows end in sentinel entries whose TBT breaks any SLO;
 //   * floor(x) comes from a fused multiply-add with 2^23 rounded toward zero: the low mantissa bits
-//     are the segment number (no float-to-int conversion), and the fraction is a second FMA; these
-//     run two candidates at a time on the packed two-wide fp32 instructions of sm_100;
+//     are the segment number (no float-to-int conversion); it runs two candidates at a time on the
+//     packed two-wide fp32 instructions of sm_100;
 //   * one shared-memory lookup, addressed in 32 bits straight from those mantissa bits;
 //   * only the running minimum is kept per candidate chain (one compare, one predicated min); the
 //     pair that attained it is recovered once per tile by re-evaluating that instance count for 32
 //     pairs at a time with bit-identical arithmetic;
 //   * when TBT never decreases with load in any table row (the resolve step checks), "TBT <= SLO and
 //     u <= 1" is a threshold on the table position (the largest load an instance sustains within the
-//     SLO, cf. ML in Sec. 4.2), so TBT is not interpolated per candidate and the lookup shrinks from
-//     16 to 8 bytes; otherwise the general path interpolates TBT for every candidate.
+//     SLO, cf. ML in Sec. 4.2), so TBT is not interpolated per candidate, the lookup shrinks from
+//     16 to 8 bytes, and the entry holds the segment's energy line as intercept and slope in v, so
+//     that one FMA on v gives the energy (no fraction); otherwise the general path interpolates TBT
+//     and energy from the segment's left knot for every candidate.
 // The resolved tables of all classes are staged in shared memory once per CTA when they fit; larger
 // tables are read through L1.
 #include "dyn_internal.cuh"
@@ -115,24 +117,26 @@ struct Consts2 {            // the same constant in both halves of a register pa
 
 // Two candidates of one (TP, f) pair at once.  ln = L/n per candidate, ic = (M-1)/(M*cap).
 // v = sat(ln*ic) is the table position over M; y = 2^23 + floor(v*M); nnu = floor(v*M) - v*M.
-// FAST: entries {energy, -slope}, feasible iff v <= vlim.  General: entries {TBT, -slope, energy,
-// -slope}, feasible iff TBT <= slo (u > 1 and never-feasible pairs read as TBT = huge or +inf through
-// the sentinel entries).  The pool energy n*e enters the running minimum of its chain when feasible.
+// FAST: entries {a, b} hold the segment's line e(v) = a + v*b, feasible iff v <= vlim.  General: entries
+// {TBT, -slope, energy, -slope} at the segment's left knot, feasible iff TBT <= slo (u > 1 and
+// never-feasible pairs read as TBT = huge or +inf through the sentinel entries).  The pool energy n*e
+// enters the running minimum of its chain when feasible.
 template <bool SMEM, bool FAST>
 __device__ __forceinline__ void eval_two(const char *__restrict__ ws, uint32_t base, float lnA, float lnB, float ic,
                                          float lim, const Consts2 &k, float2 nf2, bool allowA, bool allowB,
                                          float &bestA, float &bestB) {
     const float2 v = make_float2(__saturatef(lnA * ic), __saturatef(lnB * ic));   // NaN -> 0, > 1 -> 1
     const float2 y = __ffma2_rz(v, k.M, k.two23);
-    const float2 fm = __fadd2_rn(y, k.neg23);
-    const float2 nnu = __ffma2_rn(v, k.negM, fm);
     if (FAST) {
+        // the segment's line in intercept form: no fraction is needed
         const float2 eA = entry8<SMEM>(ws, base, y.x);
         const float2 eB = entry8<SMEM>(ws, base, y.y);
-        const float2 E = __fmul2_rn(make_float2(fmaf(nnu.x, eA.y, eA.x), fmaf(nnu.y, eB.y, eB.x)), nf2);
+        const float2 E = __fmul2_rn(make_float2(fmaf(v.x, eA.y, eA.x), fmaf(v.y, eB.y, eB.x)), nf2);
         if (allowA) min_if_le(bestA, v.x, lim, E.x);          // allow*: GPU budget (always true without one)
         if (allowB) min_if_le(bestB, v.y, lim, E.y);
     } else {
+        const float2 fm = __fadd2_rn(y, k.neg23);
+        const float2 nnu = __ffma2_rn(v, k.negM, fm);
         const float4 eA = entry16<SMEM>(ws, base, y.x);
         const float4 eB = entry16<SMEM>(ws, base, y.y);
         const float tbtA = fmaf(nnu.x, eA.y, eA.x), tbtB = fmaf(nnu.y, eB.y, eB.x);
@@ -148,12 +152,12 @@ __device__ __forceinline__ void eval_one(const char *__restrict__ ws, uint32_t b
                                          float Mf, float nf, float &E, bool &ok) {
     const float v = __saturatef(ln * ic);
     const float y = __fmaf_rz(v, Mf, kTwo23);
-    const float nnu = fmaf(v, -Mf, y + (-kTwo23));
     if (FAST) {
         const float2 e = entry8<SMEM>(ws, base, y);
         ok = v <= lim;
-        E = fmaf(nnu, e.y, e.x) * nf;
+        E = fmaf(v, e.y, e.x) * nf;
     } else {
+        const float nnu = fmaf(v, -Mf, y + (-kTwo23));
         const float4 e = entry16<SMEM>(ws, base, y);
         ok = fmaf(nnu, e.y, e.x) <= lim;
         E = fmaf(nnu, e.w, e.z) * nf;
@@ -431,17 +435,17 @@ __device__ __forceinline__ void configs_body(const SweepArgs &a, const Tables tb
             const float4 nn = s_n4[n1 >> 1];                       // {n, 1/n, n+1, 1/(n+1)}
             const float2 v = make_float2(__saturatef(lic * nn.y), __saturatef(lic * nn.w));
             const float2 y = __ffma2_rz(v, k2.M, k2.two23);
-            const float2 fm = __fadd2_rn(y, k2.neg23);
-            const float2 nnu = __ffma2_rn(v, k2.negM, fm);
             float2 ew;
             bool okA, okB;
             if (FAST) {
                 const float2 eA = entry8<SMEM>(ws, base, y.x);
                 const float2 eB = entry8<SMEM>(ws, base, y.y);
-                ew = make_float2(fmaf(nnu.x, eA.y, eA.x), fmaf(nnu.y, eB.y, eB.x));
+                ew = make_float2(fmaf(v.x, eA.y, eA.x), fmaf(v.y, eB.y, eB.x));
                 okA = v.x <= lim;
                 okB = v.y <= lim;
             } else {
+                const float2 fm = __fadd2_rn(y, k2.neg23);
+                const float2 nnu = __ffma2_rn(v, k2.negM, fm);
                 const float4 eA = entry16<SMEM>(ws, base, y.x);
                 const float4 eB = entry16<SMEM>(ws, base, y.y);
                 ew = make_float2(fmaf(nnu.x, eA.w, eA.z), fmaf(nnu.y, eB.w, eB.z));
