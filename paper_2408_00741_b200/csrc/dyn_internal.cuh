@@ -56,12 +56,15 @@ __device__ __forceinline__ uint32_t fastdiv(uint32_t n, const FastDiv &f) {
 //                   vlim = largest v with TBT <= slo_tbt[c] and u <= 1 when TBT does not decrease
 //                   along the row (-1 for a never-feasible pair), NaN when it does decrease somewhere.
 //   slo[c]          slo_tbt[c]
-//   rows2[c][p][m]  m = 0..M, float2 {a, b}: the energy line of segment m in v, e = a + v*b (a = e_a - m*e_d,
-//                   b = M*e_d; flat at the last knot's energy for m >= M-1), for the threshold path
+//   pair2[c][p]     float4 {icm, icm, llim, 0} for the threshold path: icm = (M-1)/cap, the table position per
+//                   unit of per-instance load l (x = l*icm); llim = largest l with TBT <= slo_tbt[c] and
+//                   u <= 1 (-1 for a never-feasible pair)
+//   rows2[c][p][m]  m = 0..M, float2 {a, b}: the energy line of segment m in l, e = a + l*b (a = e_a - m*e_d,
+//                   b = e_d*(M-1)/cap; flat at the last knot's energy for m >= M-1), for the threshold path
 struct ResolvedLayout {
     int32_t C, T, F, P, M, Nmax, J;
     int32_t row_stride;          // entries per pair row (M + 1)
-    size_t off_rows, off_pairc, off_slo, off_rows2, off_tp, off_partial, total;
+    size_t off_rows, off_pairc, off_slo, off_pair2, off_rows2, off_tp, off_partial, total;
 };
 
 ResolvedLayout resolved_layout(int32_t C, int32_t T, int32_t F, int32_t M, int32_t Nmax, int64_t S, int64_t W);

@@ -25,10 +25,11 @@ ResolvedLayout resolved_layout(int32_t C, int32_t T, int32_t F, int32_t M, int32
     l.row_stride = M + 1;
     const size_t entries = size_t(C) * size_t(l.P) * size_t(l.row_stride);
     size_t off = 0;
-    // rows | pairc | slo | rows2 are contiguous: the sweep stages rows..slo or pairc..rows2 as one piece
+    // rows | pairc | slo and pair2 | rows2 are contiguous: the sweep stages one or the other as one piece
     l.off_rows = off;   off = align_up(off + entries * sizeof(float4), 256);
     l.off_pairc = off;  off = align_up(off + size_t(C) * size_t(l.P) * sizeof(float2), 256);
     l.off_slo = off;    off = align_up(off + size_t(C) * sizeof(float), 256);
+    l.off_pair2 = off;  off = align_up(off + size_t(C) * size_t(l.P) * sizeof(float4), 256);
     l.off_rows2 = off;  off = align_up(off + entries * sizeof(float2), 256);
     l.off_tp = off;     off = align_up(off + size_t(T) * sizeof(int32_t), 256);
     l.off_partial = off;
@@ -49,7 +50,8 @@ __device__ __forceinline__ double lerp64(double a, double b, double w) { return 
 //   m == M    x saturated (u >= M/(M-1)): TBT = +inf
 // A pair whose TTFT misses its SLO, or whose capacity is not positive, gets TBT = +inf in every entry.
 __global__ void resolve_kernel(const ResolveParams rp, float4 *__restrict__ rows, float2 *__restrict__ pairc,
-                               float *__restrict__ slo, float2 *__restrict__ rows2, int32_t *__restrict__ tp) {
+                               float *__restrict__ slo, float4 *__restrict__ pair2, float2 *__restrict__ rows2,
+                               int32_t *__restrict__ tp) {
     const int P = rp.T * rp.F;
     const int M = rp.M;
     const int RS = M + 1;
@@ -87,13 +89,13 @@ __global__ void resolve_kernel(const ResolveParams rp, float4 *__restrict__ rows
         }
         if (!pair_ok) v.x = kInf;
         rows[(size_t(c) * P + p) * RS + m] = v;
-        // threshold path: the same energy line as intercept and slope in v = x/M, e(v) = a + v*b
-        // (the lines of neighbouring segments meet at the knots, so a position that rounding puts on
-        // either side of a knot gets the same value)
+        // threshold path: the same energy as a line in the per-instance load l, e(l) = a + l*b (x = l*(M-1)/cap);
+        // the lines of neighbouring segments meet at the knots, so a position that rounding puts on
+        // either side of a knot gets the same value
         float2 line = make_float2(float(pw_m), 0.f);
-        if (m < M - 1) {
+        if (m < M - 1 && pair_ok) {
             const double d = lerp64(pw0[m + 1], pw1[m + 1], w) * scale - pw_m;
-            line = make_float2(float(pw_m - double(m) * d), float(d * double(M)));
+            line = make_float2(float(pw_m - double(m) * d), float(d * double(M - 1) / cap));
         }
         rows2[(size_t(c) * P + p) * RS + m] = line;
         if (m == 0) {
@@ -115,6 +117,11 @@ __global__ void resolve_kernel(const ResolveParams rp, float4 *__restrict__ rows
             // x = u*(M-1) is formed as sat(L/n * ic) * M, so that saturation at 1 means x = M
             pairc[size_t(c) * P + p] = make_float2(pair_ok ? float(double(M - 1) / (double(M) * cap)) : 0.f,
                                                    monotone ? float(vlim) : __int_as_float(0x7fc00000));
+            // threshold path: table position per unit of per-instance load (twice: the sweep uses it as a
+            // packed pair) and the largest per-instance load within the SLO and the capacity
+            const float icm = pair_ok ? float(double(M - 1) / cap) : 0.f;
+            const float llim = (pair_ok && xlim >= 0.0) ? float(xlim / double(M - 1) * cap) : -1.f;
+            pair2[size_t(c) * P + p] = make_float4(icm, icm, llim, 0.f);
             if (p == 0) slo[c] = rp.slo_tbt[c];
             if (c == 0 && p < rp.T) tp[p] = rp.tp[p];
         }
@@ -134,6 +141,7 @@ cudaError_t launch_resolve(const ResolveParams &rp, const ResolvedLayout &lay, v
     resolve_kernel<<<int(blocks), threads, 0, st>>>(rp, reinterpret_cast<float4 *>(ws + lay.off_rows),
                                                     reinterpret_cast<float2 *>(ws + lay.off_pairc),
                                                     reinterpret_cast<float *>(ws + lay.off_slo),
+                                                    reinterpret_cast<float4 *>(ws + lay.off_pair2),
                                                     reinterpret_cast<float2 *>(ws + lay.off_rows2),
                                                     reinterpret_cast<int32_t *>(ws + lay.off_tp));
     return cudaGetLastError();

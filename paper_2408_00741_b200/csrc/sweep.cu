@@ -3,27 +3,31 @@
 // minimum-energy feasible one [Sec. 4.2].
 //
 // Work is plain fp32 arithmetic (no dense contraction, so no tensor cores); the kernel is bound by
-// instruction issue and by shared-memory lookups.  The design keeps both low:
+// instruction issue.  The design keeps the instructions per candidate low:
 //   * a warp owns tiles of ONE class; lanes hold instance counts n (several per lane when Nmax > 32),
 //     the (TP, f) pairs are the inner loop, so per-pair constants and the table row are warp-uniform
 //     and shared by all candidates of the pair;
-//   * table position x = u*(M-1) = sat(L/n * ic) * M: the saturating multiply clamps for free, and
-//     u > 1 is not tested: the table rows end in sentinel entries whose TBT breaks any SLO;
-//   * floor(x) comes from a fused multiply-add with 2^23 rounded toward zero: the low mantissa bits
-//     are the segment number (no float-to-int conversion); it runs two candidates at a time on the
-//     packed two-wide fp32 instructions of sm_100;
-//   * one shared-memory lookup, addressed in 32 bits straight from those mantissa bits;
-//   * only the running minimum is kept per candidate chain (one compare, one predicated min); the
-//     pair that attained it is recovered once per tile by re-evaluating that instance count for 32
-//     pairs at a time with bit-identical arithmetic;
+//   * within one (tile, n) chain the instance count is fixed, so the running minimum is kept on the
+//     energy of ONE instance and multiplied by n once per chain after the pair loop (rounding is
+//     monotone, so the minimum of the products is the product of the minimum, bit for bit);
 //   * when TBT never decreases with load in any table row (the resolve step checks), "TBT <= SLO and
-//     u <= 1" is a threshold on the table position (the largest load an instance sustains within the
-//     SLO, cf. ML in Sec. 4.2), so TBT is not interpolated per candidate, the lookup shrinks from
-//     16 to 8 bytes, and the entry holds the segment's energy line as intercept and slope in v, so
-//     that one FMA on v gives the energy (no fraction); otherwise the general path interpolates TBT
-//     and energy from the segment's left knot for every candidate.
+//     u <= 1" is a threshold on the per-instance load l = L/n (the largest load an instance sustains
+//     within the SLO, cf. ML in Sec. 4.2): one compare, no TBT interpolation.  The energy of the
+//     segment is stored as a line in l (intercept, slope), so one FMA on l gives it and no fraction is
+//     formed.  The segment number is floor(l*icm), taken from a fused multiply-add with 2^23 rounded
+//     toward zero (the low mantissa bits are the integer; no float-to-int conversion); a second fused
+//     multiply-add by 2^-146 with a per-pair offset turns 2^23 + m into the subnormal number whose bit
+//     pattern IS the shared-memory byte address of entry m of the pair's row (subnormal floats count
+//     in units of 2^-149, entries are 8 bytes apart).  Both run two candidates at a time on the packed
+//     two-wide fp32 instructions of sm_100.  Per candidate that leaves: compare, 2 x half a packed
+//     FMA, lookup, FMA, predicated min.  Infeasible candidates skip the lookup (same predicate), so
+//     no clamp of the table position is needed;
+//   * otherwise the general path interpolates TBT and energy from the segment's left knot for every
+//     candidate (16-byte lookups, saturating multiply as clamp, sentinel entries for u > 1);
+//   * only the running minimum is kept; the pair that attained it is recovered once per tile by
+//     re-evaluating that instance count for 32 pairs at a time with bit-identical arithmetic.
 // The resolved tables of all classes are staged in shared memory once per CTA when they fit; larger
-// tables are read through L1.
+// tables are read through L1 or staged per class.
 #include "dyn_internal.cuh"
 
 #include <math_constants.h>
@@ -32,6 +36,17 @@ namespace dyn {
 
 namespace {
 
+#ifndef DYN_SW_UNROLL
+#define DYN_SW_UNROLL 8
+#endif
+constexpr int kPairUnroll = DYN_SW_UNROLL;
+#ifndef DYN_SW_MINB4
+#define DYN_SW_MINB4 5
+#endif
+#ifndef DYN_SW_MINB8
+#define DYN_SW_MINB8 4
+#endif
+
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr unsigned kFull = 0xffffffffu;
@@ -39,7 +54,7 @@ constexpr float kTwo23 = 8388608.0f;
 constexpr uint32_t kTwo23Bits = 0x4b000000u;
 
 struct SweepArgs {
-    const char *ws;          // scratch block: rows (float4) | pairc (float2) | slo | rows2 (float2) | tp ...
+    const char *ws;          // scratch block: rows (float4) | pairc (float2) | slo | pair2 (float4) | rows2 (float2) | tp ...
     const float *load;       // [rows_total][C]
     const int32_t *tp;       // [T]
     int64_t tiles;
@@ -49,13 +64,13 @@ struct SweepArgs {
     int32_t C, T, F, P, M, Nmax, J;
     int32_t budget;          // <= 0: none
     int32_t ln_log2;         // lanes per n-group = 1 << ln_log2
-    int32_t off_rows, off_pairc, off_slo, off_rows2, off_end;   // byte offsets inside ws
+    int32_t off_rows, off_pairc, off_slo, off_pair2, off_rows2, off_end;   // byte offsets inside ws
     int32_t smem_bytes;      // dynamic shared memory of the launch (0: tables are read from global)
 };
 
 // where the tables of this CTA live: byte offsets from `smem` when staged, else from a.ws
 struct Tables {
-    uint32_t rows, pairc, slo, rows2;
+    uint32_t rows, pairc, slo, pair2, rows2;
 };
 
 // order-preserving map float -> uint32 (smaller float <=> smaller key)
@@ -65,8 +80,8 @@ __device__ __forceinline__ uint32_t float_key(float v) {
 }
 
 // ---- table access -----------------------------------------------------------------------------
-// `base` is the byte address of the pair's row minus ESZ * bits(2^23): the entry address is one
-// multiply-add away from the bit pattern of y = 2^23 + floor(x).  Shared memory is addressed in 32 bits.
+// General path: `base` is the byte address of the pair's row minus 16 * bits(2^23): the entry address is
+// one multiply-add away from the bit pattern of y = 2^23 + floor(x).  Shared memory is addressed in 32 bits.
 template <bool SMEM>
 __device__ __forceinline__ float4 entry16(const char *__restrict__ ws, uint32_t base, float y) {
     const uint32_t addr = __float_as_uint(y) * 16u + base;
@@ -77,9 +92,9 @@ __device__ __forceinline__ float4 entry16(const char *__restrict__ ws, uint32_t 
     }
     return __ldg(reinterpret_cast<const float4 *>(ws + addr));
 }
+// 8-byte entry / 16-byte pair constants at byte address (shared) or byte offset (scratch block) `addr`
 template <bool SMEM>
-__device__ __forceinline__ float2 entry8(const char *__restrict__ ws, uint32_t base, float y) {
-    const uint32_t addr = __float_as_uint(y) * 8u + base;
+__device__ __forceinline__ float2 load8(const char *__restrict__ ws, uint32_t addr) {
     if (SMEM) {
         float2 r;
         asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(r.x), "=f"(r.y) : "r"(addr));
@@ -88,13 +103,13 @@ __device__ __forceinline__ float2 entry8(const char *__restrict__ ws, uint32_t b
     return __ldg(reinterpret_cast<const float2 *>(ws + addr));
 }
 template <bool SMEM>
-__device__ __forceinline__ float2 pair_consts(const char *__restrict__ ws, uint32_t addr) {   // {ic, vlim}
+__device__ __forceinline__ float4 load16(const char *__restrict__ ws, uint32_t addr) {
     if (SMEM) {
-        float2 r;
-        asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(r.x), "=f"(r.y) : "r"(addr));
+        float4 r;
+        asm("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "r"(addr));
         return r;
     }
-    return __ldg(reinterpret_cast<const float2 *>(ws + addr));
+    return __ldg(reinterpret_cast<const float4 *>(ws + addr));
 }
 template <bool SMEM>
 __device__ __forceinline__ uint32_t table_origin() {
@@ -111,57 +126,114 @@ __device__ __forceinline__ void min_if_le(float &best, float a, float b, float E
         : "+f"(best) : "f"(a), "f"(b), "f"(E));
 }
 
+// ---- packed fp32 pairs held in 64-bit registers ---------------------------------------------------
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ float half_of(uint64_t v, int hi) {
+    float lo, up;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(up) : "l"(v));
+    return hi ? up : lo;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
+// A subnormal float with bit pattern k has the value k * 2^-149 ("k units").
+__device__ __forceinline__ float units(uint32_t k) { return __uint_as_float(k); }
+
+// (bytes - 2^26) units as a float.  Added to (2^23 + m) * 2^-146 = (2^26 + 8m) units it leaves bytes + 8m
+// units, a subnormal number whose bit pattern is the integer bytes + 8m.  `bytes` is a multiple of 8
+// below 2^23, so every value involved is exactly representable and the arithmetic is exact.
+__device__ __forceinline__ float row_offset_units(uint32_t bytes) {
+    return -float(int(67108864u - bytes)) * units(1u);
+}
+
+// ---- threshold path, tables in shared memory: two candidates of one (TP, f) pair ---------------------
+// ln2 = per-instance loads {lA, lB}; icm2 = {icm, icm}; off2 = row offset in units, twice; limA/limB =
+// load limit of the pair (or -1 where the GPU budget excludes the candidate).  Per candidate:
+//   feasible = l <= lim;  y = rz(l*icm + 2^23);  z = y*2^-146 + off  (bits(z) = address of the entry);
+//   if feasible: {a, b} = entry;  best = min(best, a + l*b).
+__device__ __forceinline__ void fast_two(uint64_t ln2, uint64_t icm2, uint64_t off2, uint64_t two23_2, uint64_t eight2,
+                                         float limA, float limB, float &bestA, float &bestB) {
+    // The lookups are predicated and land in the registers that held y and z: those are defined on every
+    // path, so nothing stays live around the pair loop for the sake of a skipped load (an infeasible
+    // candidate forms a meaningless energy from them, which its predicated min ignores).
+    asm("{\n\t"
+        ".reg .pred pA, pB;\n\t"
+        ".reg .f32 lA, lB, a0, b0, a1, b1, eA, eB;\n\t"
+        ".reg .b32 zA, zB;\n\t"
+        ".reg .b64 y, z;\n\t"
+        "mov.b64 {lA, lB}, %2;\n\t"
+        "setp.le.f32 pA, lA, %7;\n\t"
+        "setp.le.f32 pB, lB, %8;\n\t"
+        "fma.rz.f32x2 y, %2, %3, %5;\n\t"
+        "fma.rn.f32x2 z, y, %6, %4;\n\t"
+        "mov.b64 {zA, zB}, z;\n\t"
+        "@pA ld.shared.b64 y, [zA];\n\t"
+        "@pB ld.shared.b64 z, [zB];\n\t"
+        "mov.b64 {a0, b0}, y;\n\t"
+        "mov.b64 {a1, b1}, z;\n\t"
+        "fma.rn.f32 eA, lA, b0, a0;\n\t"
+        "fma.rn.f32 eB, lB, b1, a1;\n\t"
+        "@pA min.f32 %0, %0, eA;\n\t"
+        "@pB min.f32 %1, %1, eB;\n\t"
+        "}"
+        : "+f"(bestA), "+f"(bestB)
+        : "l"(ln2), "l"(icm2), "l"(off2), "l"(two23_2), "l"(eight2), "f"(limA), "f"(limB));
+}
+
+// the same evaluation for one candidate with ordinary address arithmetic (tables in shared memory or
+// read through L1), bit-identical to fast_two: e = a + l*b of segment floor(l*icm), ok = l <= lim.
+// `row` is the byte address / offset of the pair's row.  An infeasible candidate reads entry 0.
+template <bool SMEM>
+__device__ __forceinline__ void fast_one(const char *__restrict__ ws, uint32_t row, float l, float icm, float lim,
+                                         float &e, bool &ok) {
+    ok = l <= lim;
+    const float y = __fmaf_rz(l, icm, kTwo23);
+    const uint32_t m = ok ? __float_as_uint(y) - kTwo23Bits : 0u;
+    const float2 en = load8<SMEM>(ws, row + m * 8u);
+    e = fmaf(l, en.y, en.x);
+}
+
 struct Consts2 {            // the same constant in both halves of a register pair
     float2 M, negM, two23, neg23;
 };
 
-// Two candidates of one (TP, f) pair at once.  ln = L/n per candidate, ic = (M-1)/(M*cap).
+// General path: two candidates of one (TP, f) pair.  ln = L/n per candidate, ic = (M-1)/(M*cap).
 // v = sat(ln*ic) is the table position over M; y = 2^23 + floor(v*M); nnu = floor(v*M) - v*M.
-// FAST: entries {a, b} hold the segment's line e(v) = a + v*b, feasible iff v <= vlim.  General: entries
-// {TBT, -slope, energy, -slope} at the segment's left knot, feasible iff TBT <= slo (u > 1 and
-// never-feasible pairs read as TBT = huge or +inf through the sentinel entries).  The pool energy n*e
-// enters the running minimum of its chain when feasible.
-template <bool SMEM, bool FAST>
-__device__ __forceinline__ void eval_two(const char *__restrict__ ws, uint32_t base, float lnA, float lnB, float ic,
-                                         float lim, const Consts2 &k, float2 nf2, bool allowA, bool allowB,
-                                         float &bestA, float &bestB) {
+// Entries {TBT, -slope, energy, -slope} at the segment's left knot, feasible iff TBT <= slo (u > 1 and
+// never-feasible pairs read as TBT = huge or +inf through the sentinel entries).  The energy of one
+// instance enters the running minimum of its chain when feasible.
+template <bool SMEM>
+__device__ __forceinline__ void general_two(const char *__restrict__ ws, uint32_t base, float lnA, float lnB, float ic,
+                                            float slo, const Consts2 &k, bool allowA, bool allowB, float &bestA,
+                                            float &bestB) {
     const float2 v = make_float2(__saturatef(lnA * ic), __saturatef(lnB * ic));   // NaN -> 0, > 1 -> 1
     const float2 y = __ffma2_rz(v, k.M, k.two23);
-    if (FAST) {
-        // the segment's line in intercept form: no fraction is needed
-        const float2 eA = entry8<SMEM>(ws, base, y.x);
-        const float2 eB = entry8<SMEM>(ws, base, y.y);
-        const float2 E = __fmul2_rn(make_float2(fmaf(v.x, eA.y, eA.x), fmaf(v.y, eB.y, eB.x)), nf2);
-        if (allowA) min_if_le(bestA, v.x, lim, E.x);          // allow*: GPU budget (always true without one)
-        if (allowB) min_if_le(bestB, v.y, lim, E.y);
-    } else {
-        const float2 fm = __fadd2_rn(y, k.neg23);
-        const float2 nnu = __ffma2_rn(v, k.negM, fm);
-        const float4 eA = entry16<SMEM>(ws, base, y.x);
-        const float4 eB = entry16<SMEM>(ws, base, y.y);
-        const float tbtA = fmaf(nnu.x, eA.y, eA.x), tbtB = fmaf(nnu.y, eB.y, eB.x);
-        const float2 E = __fmul2_rn(make_float2(fmaf(nnu.x, eA.w, eA.z), fmaf(nnu.y, eB.w, eB.z)), nf2);
-        if (allowA) min_if_le(bestA, tbtA, lim, E.x);
-        if (allowB) min_if_le(bestB, tbtB, lim, E.y);
-    }
+    const float2 fm = __fadd2_rn(y, k.neg23);
+    const float2 nnu = __ffma2_rn(v, k.negM, fm);
+    const float4 eA = entry16<SMEM>(ws, base, y.x);
+    const float4 eB = entry16<SMEM>(ws, base, y.y);
+    const float tbtA = fmaf(nnu.x, eA.y, eA.x), tbtB = fmaf(nnu.y, eB.y, eB.x);
+    if (allowA) min_if_le(bestA, tbtA, slo, fmaf(nnu.x, eA.w, eA.z));     // allow*: GPU budget (always true without one)
+    if (allowB) min_if_le(bestB, tbtB, slo, fmaf(nnu.y, eB.w, eB.z));
 }
 
-// scalar form of the same evaluation, bit-identical to eval_two (evaluate-only kernel, pair recovery)
-template <bool SMEM, bool FAST>
-__device__ __forceinline__ void eval_one(const char *__restrict__ ws, uint32_t base, float ln, float ic, float lim,
-                                         float Mf, float nf, float &E, bool &ok) {
+// scalar form of the same evaluation, bit-identical to general_two (evaluate-only kernel, pair recovery)
+template <bool SMEM>
+__device__ __forceinline__ void general_one(const char *__restrict__ ws, uint32_t base, float ln, float ic, float slo,
+                                            float Mf, float &e, bool &ok) {
     const float v = __saturatef(ln * ic);
     const float y = __fmaf_rz(v, Mf, kTwo23);
-    if (FAST) {
-        const float2 e = entry8<SMEM>(ws, base, y);
-        ok = v <= lim;
-        E = fmaf(v, e.y, e.x) * nf;
-    } else {
-        const float nnu = fmaf(v, -Mf, y + (-kTwo23));
-        const float4 e = entry16<SMEM>(ws, base, y);
-        ok = fmaf(nnu, e.y, e.x) <= lim;
-        E = fmaf(nnu, e.w, e.z) * nf;
-    }
+    const float nnu = fmaf(v, -Mf, y + (-kTwo23));
+    const float4 en = entry16<SMEM>(ws, base, y);
+    ok = fmaf(nnu, en.y, en.x) <= slo;
+    e = fmaf(nnu, en.w, en.z);
 }
 
 // copy [ws + from, ws + to) into shared memory (16-byte pieces)
@@ -185,8 +257,8 @@ __device__ __forceinline__ bool all_rows_monotone(const SweepArgs &a) {
 // fused evaluate + select
 //   NPL  instance counts per lane (Nmax <= 32*NPL)
 //   TT   tiles (rows of the same class) a warp evaluates per pass over the pairs
-// ---------------------------------------------------------------------------------------------
 //   CLS  the CTA serves one class (blockIdx.y) and `tb` points at that class's tables alone
+// ---------------------------------------------------------------------------------------------
 template <int NPL, int TT, bool BUDGET, bool SMEM, bool FAST, bool FULL, bool CLS = false>
 __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, int32_t *__restrict__ best_idx,
                                            float *__restrict__ best_E) {
@@ -231,56 +303,101 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
     // loads from being scheduled ahead of the barrier that ends the staging
     asm volatile("" : "+r"(origin) : : "memory");
     const int ct = CLS ? 0 : c;                      // class offset inside the tables `tb` points at
-    const uint32_t cpair = origin + tb.pairc + uint32_t(ct * P) * 8u;
-    const uint32_t cbase = origin + (FAST ? tb.rows2 : tb.rows) + uint32_t(ct * P * RS) * ESZ - kTwo23Bits * ESZ;
+    // pair constants: threshold path pair2 (16 bytes), general path pairc (8 bytes)
+    const uint32_t cpair = origin + (FAST ? tb.pair2 + uint32_t(ct * P) * 16u : tb.pairc + uint32_t(ct * P) * 8u);
+    const uint32_t crow = origin + (FAST ? tb.rows2 : tb.rows) + uint32_t(ct * P * RS) * ESZ;   // row of pair 0
     const uint32_t pstep = uint32_t(RS) * ESZ;
-    float slo_c;
-    if (SMEM && !CLS) {
-        extern __shared__ float4 smem[];
-        slo_c = reinterpret_cast<const float *>(reinterpret_cast<const char *>(smem) + tb.slo)[c];
-    } else {
-        slo_c = __ldg(reinterpret_cast<const float *>(ws + a.off_slo) + c);
+    float slo_c = 0.f;
+    if (!FAST) {
+        if (SMEM && !CLS) {
+            extern __shared__ float4 smem[];
+            slo_c = reinterpret_cast<const float *>(reinterpret_cast<const char *>(smem) + tb.slo)[c];
+        } else {
+            slo_c = __ldg(reinterpret_cast<const float *>(ws + a.off_slo) + c);
+        }
     }
     Consts2 k2;
     k2.M = make_float2(Mf, Mf);
     k2.negM = make_float2(-Mf, -Mf);
     k2.two23 = make_float2(kTwo23, kTwo23);
     k2.neg23 = make_float2(-kTwo23, -kTwo23);
+    // threshold path with staged tables: row offsets as subnormal floats (see fast_two)
+    const uint64_t two23_2 = pack2(kTwo23, kTwo23);
+    const uint64_t eight2 = pack2(units(8u), units(8u));
+    const float off0 = row_offset_units(crow + uint32_t(g) * pstep);
+    const float offs = float(int(uint32_t(G) * pstep)) * units(1u);
+    const uint64_t off2_first = pack2(off0, off0), off2_step = pack2(offs, offs);
     constexpr int NCH = TT * NPL;                    // candidates per lane and pair, an even number
     static_assert(NCH % 2 == 0, "candidates are evaluated two at a time");
 
     for (int64_t r = r_begin; r < r_end; r += TT) {
-        // chain q = t*NPL + k: tile t of this pass, k-th instance count of the lane
-        float ln[NCH], best[NCH];
+        // chain q = t*NPL + k: tile t of this pass, k-th instance count of the lane; `best` is the least
+        // energy of ONE instance over the feasible pairs of the chain
+        float best[NCH];
+        uint64_t ln2[NCH / 2];                       // per-instance loads L/n of chains (q, q+1), packed
+        {
+            float ln[NCH];
 #pragma unroll
-        for (int t = 0; t < TT; ++t) {
-            const float L = (r + t < r_end) ? fmaxf(a.load[(r + t) * C + c], 0.f) : 0.f;   // negative / NaN -> 0
+            for (int t = 0; t < TT; ++t) {
+                const float L = (r + t < r_end) ? fmaxf(a.load[(r + t) * C + c], 0.f) : 0.f;   // negative / NaN -> 0
 #pragma unroll
-            for (int k = 0; k < NPL; ++k) {
-                ln[t * NPL + k] = L * rn[k];
-                best[t * NPL + k] = CUDART_INF_F;
+                for (int k = 0; k < NPL; ++k) {
+                    ln[t * NPL + k] = L * rn[k];
+                    best[t * NPL + k] = CUDART_INF_F;
+                }
             }
-        }
-#pragma unroll 8
-        for (int p = g; p < P; p += G) {
-            const float2 pc = pair_consts<SMEM>(ws, cpair + uint32_t(p) * 8u);
-            const uint32_t base = cbase + uint32_t(p) * pstep;
-            const float lim = FAST ? pc.y : slo_c;
 #pragma unroll
-            for (int q = 0; q < NCH; q += 2)
-                eval_two<SMEM, FAST>(ws, base, ln[q], ln[q + 1], pc.x, lim, k2,
-                                     make_float2(nf[q % NPL], nf[(q + 1) % NPL]), !BUDGET || p < pmax[q % NPL],
-                                     !BUDGET || p < pmax[(q + 1) % NPL], best[q], best[q + 1]);
+            for (int q = 0; q < NCH; q += 2) ln2[q / 2] = pack2(ln[q], ln[q + 1]);
+        }
+#define DYN_LN(q) half_of(ln2[(q) / 2], (q) & 1)
+        if (FAST && SMEM) {
+            uint64_t off2 = off2_first;
+#pragma unroll kPairUnroll
+            for (int p = g; p < P; p += G) {
+                uint64_t icm2, lim2;
+                asm("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(icm2), "=l"(lim2) : "r"(cpair + uint32_t(p) * 16u));
+                const float lim = __uint_as_float(uint32_t(lim2));
+#pragma unroll
+                for (int q = 0; q < NCH; q += 2)
+                    fast_two(ln2[q / 2], icm2, off2, two23_2, eight2,
+                             (!BUDGET || p < pmax[q % NPL]) ? lim : -1.f,
+                             (!BUDGET || p < pmax[(q + 1) % NPL]) ? lim : -1.f, best[q], best[q + 1]);
+                off2 = add2(off2, off2_step);
+            }
+        } else if (FAST) {
+#pragma unroll 4
+            for (int p = g; p < P; p += G) {
+                const float4 pc = load16<SMEM>(ws, cpair + uint32_t(p) * 16u);
+                const uint32_t row = crow + uint32_t(p) * pstep;
+#pragma unroll
+                for (int q = 0; q < NCH; ++q) {
+                    float e;
+                    bool ok;
+                    fast_one<SMEM>(ws, row, DYN_LN(q), pc.x, pc.z, e, ok);
+                    if (ok && (!BUDGET || p < pmax[q % NPL])) best[q] = fminf(best[q], e);
+                }
+            }
+        } else {
+#pragma unroll 8
+            for (int p = g; p < P; p += G) {
+                const float2 pc = load8<SMEM>(ws, cpair + uint32_t(p) * 8u);
+                const uint32_t base = crow + uint32_t(p) * pstep - kTwo23Bits * 16u;
+#pragma unroll
+                for (int q = 0; q < NCH; q += 2)
+                    general_two<SMEM>(ws, base, DYN_LN(q), DYN_LN(q + 1), pc.x, slo_c, k2, !BUDGET || p < pmax[q % NPL],
+                                      !BUDGET || p < pmax[(q + 1) % NPL], best[q], best[q + 1]);
+            }
         }
 #pragma unroll
         for (int t = 0; t < TT; ++t) {
             if (r + t >= r_end) break;               // warp-uniform
-            // the lane's chains in ascending n: strict compare keeps the lower n on ties
+            // the lane's chains in ascending n: strict compare keeps the lower n on ties.  Pool energy =
+            // n * (energy of one instance); + 0 turns -0 into +0 so that the keys order like the floats
             float E = CUDART_INF_F;
             int n = 0x7fffffff;
 #pragma unroll
             for (int k = 0; k < NPL; ++k) {
-                const float Ek = valid_n[k] ? best[t * NPL + k] + 0.f : CUDART_INF_F;   // -0 -> +0: keys order like floats
+                const float Ek = valid_n[k] ? best[t * NPL + k] * nf[k] + 0.f : CUDART_INF_F;
                 if (Ek < E) {
                     E = Ek;
                     n = nl + 1 + LN * k;
@@ -305,9 +422,9 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
             const float nfm = float(nmin);
             // L/n of the winning instance count, from the lane that holds it (bit-identical by construction)
             const int kstar = int(nmin - 1) >> (FULL ? 5 : a.ln_log2);
-            float lnk = ln[t * NPL];
+            float lnk = DYN_LN(t * NPL);
 #pragma unroll
-            for (int k = 1; k < NPL; ++k) lnk = (k == kstar) ? ln[t * NPL + k] : lnk;
+            for (int k = 1; k < NPL; ++k) lnk = (k == kstar) ? DYN_LN(t * NPL + k) : lnk;
             const float lnm = __shfl_sync(kFull, lnk, int(nmin - 1) & (LN - 1));
             int pm = P;
             if (BUDGET) {
@@ -320,11 +437,16 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
                 const int pp = p0 + lane;
                 bool hit = false;
                 if (pp < pm) {
-                    const float2 pc = pair_consts<SMEM>(ws, cpair + uint32_t(pp) * 8u);
-                    float Ep;
+                    float e;
                     bool ok;
-                    eval_one<SMEM, FAST>(ws, cbase + uint32_t(pp) * pstep, lnm, pc.x, FAST ? pc.y : slo_c, Mf, nfm, Ep, ok);
-                    hit = ok && (Ep + 0.f == Emin);
+                    if (FAST) {
+                        const float4 pc = load16<SMEM>(ws, cpair + uint32_t(pp) * 16u);
+                        fast_one<SMEM>(ws, crow + uint32_t(pp) * pstep, lnm, pc.x, pc.z, e, ok);
+                    } else {
+                        const float2 pc = load8<SMEM>(ws, cpair + uint32_t(pp) * 8u);
+                        general_one<SMEM>(ws, crow + uint32_t(pp) * pstep - kTwo23Bits * 16u, lnm, pc.x, slo_c, Mf, e, ok);
+                    }
+                    hit = ok && (e * nfm + 0.f == Emin);
                 }
                 const unsigned m = __ballot_sync(kFull, hit);
                 if (m) pstar = p0 + __ffs(m) - 1;
@@ -337,53 +459,53 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
     }
 }
 
+#undef DYN_LN
+
 template <int NPL, int TT, bool BUDGET, bool SMEM, bool FULL>
-__global__ void __launch_bounds__(kThreads, (NPL * TT <= 4 ? 5 : (NPL * TT <= 8 && NPL <= 2 ? 4 : 2)))
+__global__ void __launch_bounds__(kThreads, (NPL * TT <= 4 ? DYN_SW_MINB4 : (NPL * TT <= 8 && NPL <= 2 ? DYN_SW_MINB8 : 2)))
 eval_select_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__restrict__ best_E) {
     Tables tb;
+    tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.pair2 = a.off_pair2; tb.rows2 = a.off_rows2;
     if (all_rows_monotone(a)) {                      // uniform over the grid: every CTA reads the same flags
         if (SMEM) {
-            stage(a, a.off_pairc, a.off_end);        // pairc | slo | rows2
-            tb.pairc = 0; tb.slo = a.off_slo - a.off_pairc; tb.rows2 = a.off_rows2 - a.off_pairc; tb.rows = 0;
-        } else {
-            tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.rows2 = a.off_rows2;
+            stage(a, a.off_pair2, a.off_end);        // pair2 | rows2
+            tb.pair2 = 0; tb.rows2 = a.off_rows2 - a.off_pair2;
         }
         sweep_body<NPL, TT, BUDGET, SMEM, true, FULL>(a, tb, best_idx, best_E);
     } else {
         if (SMEM) {
-            stage(a, a.off_rows, a.off_rows2);       // rows | pairc | slo
-            tb.rows = 0; tb.pairc = a.off_pairc - a.off_rows; tb.slo = a.off_slo - a.off_rows; tb.rows2 = 0;
-        } else {
-            tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.rows2 = a.off_rows2;
+            stage(a, a.off_rows, a.off_pair2);       // rows | pairc | slo
+            tb.rows = 0; tb.pairc = a.off_pairc - a.off_rows; tb.slo = a.off_slo - a.off_rows;
         }
         sweep_body<NPL, TT, BUDGET, SMEM, false, FULL>(a, tb, best_idx, best_E);
     }
 }
 
 // Tables too large to stage for all classes at once (fine frequency grids): a CTA serves ONE class
-// (blockIdx.y) and stages that class's threshold tables, pairc_c | rows2_c, in shared memory; one CTA
+// (blockIdx.y) and stages that class's threshold tables, pair2_c | rows2_c, in shared memory; one CTA
 // of 16 warps per SM.  When some row is not monotone the general path reads the full tables through L1.
 template <int NPL, int TT, bool BUDGET>
 __global__ void __launch_bounds__(512, 1)
 eval_select_class_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__restrict__ best_E) {
     Tables tb;
+    tb.rows = tb.pairc = tb.slo = tb.pair2 = tb.rows2 = 0;
     if (all_rows_monotone(a)) {
         extern __shared__ float4 smem[];
         const int c = blockIdx.y;
-        const int pair_bytes = a.P * 8, rows2_bytes = a.P * (a.M + 1) * 8;
-        const float4 *src_p = reinterpret_cast<const float4 *>(a.ws + a.off_pairc + size_t(c) * pair_bytes);
+        const int pair_bytes = a.P * 16, rows2_bytes = a.P * (a.M + 1) * 8;
+        const float4 *src_p = reinterpret_cast<const float4 *>(a.ws + a.off_pair2 + size_t(c) * pair_bytes);
         const float4 *src_r = reinterpret_cast<const float4 *>(a.ws + a.off_rows2 + size_t(c) * rows2_bytes);
-        const int np16 = (pair_bytes + 15) / 16, nr16 = (rows2_bytes + 15) / 16;   // rounding up stays inside the scratch block
+        const int np16 = pair_bytes / 16, nr16 = (rows2_bytes + 15) / 16;   // rounding up stays inside the scratch block
         for (int i = threadIdx.x; i < np16; i += blockDim.x) smem[i] = src_p[i];
         for (int i = threadIdx.x; i < nr16; i += blockDim.x) smem[np16 + i] = src_r[i];
         __syncthreads();
-        tb.pairc = 0; tb.rows2 = uint32_t(np16) * 16u; tb.rows = 0; tb.slo = 0;
+        tb.pair2 = 0; tb.rows2 = uint32_t(pair_bytes);
         sweep_body<NPL, TT, BUDGET, true, true, true, true>(a, tb, best_idx, best_E);
     } else {
         const int c = blockIdx.y;
         tb.rows = a.off_rows + uint32_t(c) * uint32_t(a.P * (a.M + 1)) * 16u;
         tb.pairc = a.off_pairc + uint32_t(c) * uint32_t(a.P) * 8u;
-        tb.slo = a.off_slo; tb.rows2 = 0;
+        tb.slo = a.off_slo;
         sweep_body<NPL, TT, BUDGET, false, false, true, true>(a, tb, best_idx, best_E);
     }
 }
@@ -391,10 +513,11 @@ eval_select_class_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, floa
 // ---------------------------------------------------------------------------------------------
 // evaluate only: E[tile][j], j = (n-1)*P + p.  A warp takes one tile and 32 consecutive pairs: lanes
 // are pairs (their constants stay in registers), the loop runs over n two at a time, and each pass
-// writes two coalesced runs of 32 energies.  Threshold or general path as in the fused kernel.
+// writes two coalesced runs of 32 energies.  Threshold or general path as in the fused kernel, with
+// the same arithmetic per candidate.
 // ---------------------------------------------------------------------------------------------
 template <bool BUDGET, bool SMEM, bool FAST>
-__device__ __forceinline__ void configs_body(const SweepArgs &a, const Tables tb, const float2 *s_n, const int64_t units,
+__device__ __forceinline__ void configs_body(const SweepArgs &a, const Tables tb, const float2 *s_n, const int64_t units_total,
                                              float *__restrict__ E_out) {
     const int lane = threadIdx.x & 31;
     const int P = a.P, RS = a.M + 1, Nmax = a.Nmax;
@@ -404,15 +527,10 @@ __device__ __forceinline__ void configs_body(const SweepArgs &a, const Tables tb
     uint32_t origin = table_origin<SMEM>();
     asm volatile("" : "+r"(origin) : : "memory");        // as in sweep_body: table loads stay behind the staging barrier
     const char *ws = a.ws;
-    Consts2 k2;
-    k2.M = make_float2(Mf, Mf);
-    k2.negM = make_float2(-Mf, -Mf);
-    k2.two23 = make_float2(kTwo23, kTwo23);
-    k2.neg23 = make_float2(-kTwo23, -kTwo23);
     const float4 *s_n4 = reinterpret_cast<const float4 *>(s_n);
 
     const int64_t nwarps = int64_t(gridDim.x) * kWarps;
-    for (int64_t u = int64_t(blockIdx.x) * kWarps + (threadIdx.x >> 5); u < units; u += nwarps) {
+    for (int64_t u = int64_t(blockIdx.x) * kWarps + (threadIdx.x >> 5); u < units_total; u += nwarps) {
         const int64_t i = u / PG;
         const int p = int(u - i * PG) * 32 + lane;
         const int c = int(i % a.C);
@@ -420,10 +538,16 @@ __device__ __forceinline__ void configs_body(const SweepArgs &a, const Tables tb
         const int pp = active ? p : 0;
         const float L = fmaxf(a.load[i], 0.f);
         const float slo_c = __ldg(reinterpret_cast<const float *>(ws + a.off_slo) + c);
-        const float2 pc = pair_consts<SMEM>(ws, origin + tb.pairc + uint32_t(c * P + pp) * 8u);
-        const uint32_t base = origin + (FAST ? tb.rows2 : tb.rows) + uint32_t((c * P + pp) * RS) * ESZ - kTwo23Bits * ESZ;
-        const float lic = L * pc.x;                   // per-instance table position is lic / n
-        const float lim = FAST ? pc.y : slo_c;
+        const uint32_t row = origin + (FAST ? tb.rows2 : tb.rows) + uint32_t((c * P + pp) * RS) * ESZ;
+        float ic, lim;                                // threshold path: {icm, llim}; general: {ic, slo}
+        if (FAST) {
+            const float4 pc = load16<SMEM>(ws, origin + tb.pair2 + uint32_t(c * P + pp) * 16u);
+            ic = pc.x;
+            lim = pc.z;
+        } else {
+            ic = load8<SMEM>(ws, origin + tb.pairc + uint32_t(c * P + pp) * 8u).x;
+            lim = slo_c;
+        }
         int nlim = Nmax;                              // Eq. 1 GPU budget: n * TP <= budget
         if (BUDGET) {
             const int64_t q = int64_t(a.budget) / a.tp[pp / a.F];
@@ -433,33 +557,23 @@ __device__ __forceinline__ void configs_body(const SweepArgs &a, const Tables tb
         int off = 0;                                  // (n - 1) * P, below J < 2^31
         for (int n1 = 0; n1 < Nmax; n1 += 2, off += 2 * P) {
             const float4 nn = s_n4[n1 >> 1];                       // {n, 1/n, n+1, 1/(n+1)}
-            const float2 v = make_float2(__saturatef(lic * nn.y), __saturatef(lic * nn.w));
-            const float2 y = __ffma2_rz(v, k2.M, k2.two23);
-            float2 ew;
+            const float lnA = L * nn.y, lnB = L * nn.w;
+            float eA, eB;
             bool okA, okB;
             if (FAST) {
-                const float2 eA = entry8<SMEM>(ws, base, y.x);
-                const float2 eB = entry8<SMEM>(ws, base, y.y);
-                ew = make_float2(fmaf(v.x, eA.y, eA.x), fmaf(v.y, eB.y, eB.x));
-                okA = v.x <= lim;
-                okB = v.y <= lim;
+                fast_one<SMEM>(ws, row, lnA, ic, lim, eA, okA);
+                fast_one<SMEM>(ws, row, lnB, ic, lim, eB, okB);
             } else {
-                const float2 fm = __fadd2_rn(y, k2.neg23);
-                const float2 nnu = __ffma2_rn(v, k2.negM, fm);
-                const float4 eA = entry16<SMEM>(ws, base, y.x);
-                const float4 eB = entry16<SMEM>(ws, base, y.y);
-                ew = make_float2(fmaf(nnu.x, eA.w, eA.z), fmaf(nnu.y, eB.w, eB.z));
-                okA = fmaf(nnu.x, eA.y, eA.x) <= lim;
-                okB = fmaf(nnu.y, eB.y, eB.x) <= lim;
+                general_one<SMEM>(ws, row - kTwo23Bits * 16u, lnA, ic, lim, Mf, eA, okA);
+                general_one<SMEM>(ws, row - kTwo23Bits * 16u, lnB, ic, lim, Mf, eB, okB);
             }
-            const float2 E = __fmul2_rn(ew, make_float2(nn.x, nn.z));
             if (BUDGET) {
                 okA = okA && n1 + 1 <= nlim;
                 okB = okB && n1 + 2 <= nlim;
             }
             if (active) {
-                __stcs(out + off, okA ? E.x : CUDART_INF_F);
-                if (n1 + 1 < Nmax) __stcs(out + off + P, okB ? E.y : CUDART_INF_F);
+                __stcs(out + off, okA ? eA * nn.x : CUDART_INF_F);
+                if (n1 + 1 < Nmax) __stcs(out + off + P, okB ? eB * nn.z : CUDART_INF_F);
             }
         }
     }
@@ -467,26 +581,23 @@ __device__ __forceinline__ void configs_body(const SweepArgs &a, const Tables tb
 
 template <bool BUDGET, bool SMEM>
 __global__ void __launch_bounds__(kThreads)
-eval_configs_kernel(const SweepArgs a, const int64_t units, float *__restrict__ E_out) {
+eval_configs_kernel(const SweepArgs a, const int64_t units_total, float *__restrict__ E_out) {
     __shared__ __align__(16) float2 s_n[258];         // {n, 1/n} for n = 1..Nmax (Nmax <= 256), padded to even
     for (int n1 = threadIdx.x; n1 < a.Nmax + 1; n1 += kThreads) s_n[n1] = make_float2(float(n1 + 1), 1.0f / float(n1 + 1));
     Tables tb;
+    tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.pair2 = a.off_pair2; tb.rows2 = a.off_rows2;
     if (all_rows_monotone(a)) {                      // load-threshold path: 8-byte lookups (also a barrier for s_n)
         if (SMEM) {
-            stage(a, a.off_pairc, a.off_end);
-            tb.pairc = 0; tb.slo = a.off_slo - a.off_pairc; tb.rows2 = a.off_rows2 - a.off_pairc; tb.rows = 0;
-        } else {
-            tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.rows2 = a.off_rows2;
+            stage(a, a.off_pair2, a.off_end);
+            tb.pair2 = 0; tb.rows2 = a.off_rows2 - a.off_pair2;
         }
-        configs_body<BUDGET, SMEM, true>(a, tb, s_n, units, E_out);
+        configs_body<BUDGET, SMEM, true>(a, tb, s_n, units_total, E_out);
     } else {
         if (SMEM) {
-            stage(a, a.off_rows, a.off_rows2);
-            tb.rows = 0; tb.pairc = a.off_pairc - a.off_rows; tb.slo = a.off_slo - a.off_rows; tb.rows2 = 0;
-        } else {
-            tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.rows2 = a.off_rows2;
+            stage(a, a.off_rows, a.off_pair2);
+            tb.rows = 0; tb.pairc = a.off_pairc - a.off_rows; tb.slo = a.off_slo - a.off_rows;
         }
-        configs_body<BUDGET, SMEM, false>(a, tb, s_n, units, E_out);
+        configs_body<BUDGET, SMEM, false>(a, tb, s_n, units_total, E_out);
     }
 }
 
@@ -513,10 +624,11 @@ SweepArgs make_args(const ResolvedLayout &lay, const void *d_ws, const float *d_
     a.off_rows = int32_t(lay.off_rows);
     a.off_pairc = int32_t(lay.off_pairc);
     a.off_slo = int32_t(lay.off_slo);
+    a.off_pair2 = int32_t(lay.off_pair2);
     a.off_rows2 = int32_t(lay.off_rows2);
     a.off_end = int32_t(lay.off_tp);
-    // the general path stages rows | pairc | slo, the threshold path pairc | slo | rows2: one piece each
-    const size_t general = lay.off_rows2 - lay.off_rows;
+    // the general path stages rows | pairc | slo, the threshold path pair2 | rows2 (smaller): one piece each
+    const size_t general = lay.off_pair2 - lay.off_rows;
     a.smem_bytes = general <= 96 * 1024 && general <= smem_limit() ? int32_t(general) : 0;
     return a;
 }
@@ -568,8 +680,8 @@ cudaError_t launch_es(SweepArgs &a, int32_t *best_idx, float *best_E, cudaStream
     const bool smem = a.smem_bytes > 0;
     const bool budget = a.budget > 0;
     if (!smem && NPL > 1) {
-        // pairc_c and rows2_c, each rounded up to 16 bytes
-        const size_t class_bytes = (size_t(a.P) * 8 + 15) / 16 * 16 + (size_t(a.P) * size_t(a.M + 1) * 8 + 15) / 16 * 16;
+        // pair2_c and rows2_c (rounded up to 16 bytes)
+        const size_t class_bytes = size_t(a.P) * 16 + (size_t(a.P) * size_t(a.M + 1) * 8 + 15) / 16 * 16;
         if (a.P % 2 == 0 && class_bytes + 1024 <= smem_limit())       // even P: class blocks stay 16-byte aligned
             return budget ? launch_es_class<NPL, TT, true>(a, class_bytes, best_idx, best_E, st)
                           : launch_es_class<NPL, TT, false>(a, class_bytes, best_idx, best_E, st);
