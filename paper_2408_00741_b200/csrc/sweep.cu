@@ -73,10 +73,11 @@ struct Tables {
     uint32_t rows, pairc, slo, pair2, rows2;
 };
 
-// order-preserving map float -> uint32 (smaller float <=> smaller key)
-__device__ __forceinline__ uint32_t float_key(float v) {
-    const uint32_t b = __float_as_uint(v);
-    return b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
+// smallest value over the warp (no NaNs here)
+__device__ __forceinline__ float warp_min(float v) {
+    float r;
+    asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
+    return r;
 }
 
 // ---- table access -----------------------------------------------------------------------------
@@ -279,15 +280,19 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
     const float Mf = float(a.M);
     const char *ws = a.ws;
 
+    // chain k of the lane evaluates n = nl + 1 + LN*k.  A lane whose n exceeds Nmax: on the threshold path its
+    // per-instance load is made +inf (or NaN), which no pair accepts; on the general path it is dropped
+    // after the pair loop
     float nf[NPL], rn[NPL];
     int pmax[NPL];
-    bool valid_n[NPL];
+    bool keep[NPL];
 #pragma unroll
     for (int k = 0; k < NPL; ++k) {
         const int n = nl + 1 + LN * k;
-        valid_n[k] = n <= a.Nmax;
+        const bool valid = n <= a.Nmax;
+        keep[k] = FAST || valid;
         nf[k] = float(n);
-        rn[k] = valid_n[k] ? 1.0f / float(n) : 0.f;
+        rn[k] = valid ? 1.0f / float(n) : (FAST ? CUDART_INF_F : 0.f);
         pmax[k] = P;
         if (BUDGET) {
             int nt = 0;
@@ -330,7 +335,15 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
     constexpr int NCH = TT * NPL;                    // candidates per lane and pair, an even number
     static_assert(NCH % 2 == 0, "candidates are evaluated two at a time");
 
-    for (int64_t r = r_begin; r < r_end; r += TT) {
+    // per-lane constants of the pair recovery: lane p re-evaluates pair p0 + p
+    const uint32_t cpair_lane = cpair + uint32_t(lane) * (FAST ? 16u : 8u);
+    const uint32_t crow_lane = crow + uint32_t(lane) * pstep;
+    const int sh_n = FULL ? 5 : a.ln_log2;           // n - 1 = (chain number << sh_n) + lane number
+    const float *lp = a.load + (r_begin * C + c);    // load of the pass's first tile; tiles are C floats apart
+    int64_t oi = r_begin * C + c;                    // its index in the outputs
+
+    for (int64_t r = r_begin; r < r_end; r += TT, lp += TT * C, oi += int64_t(TT) * C) {
+        const int nt = r_end - r < TT ? int(r_end - r) : TT;          // tiles of this pass (warp-uniform)
         // chain q = t*NPL + k: tile t of this pass, k-th instance count of the lane; `best` is the least
         // energy of ONE instance over the feasible pairs of the chain
         float best[NCH];
@@ -339,7 +352,7 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
             float ln[NCH];
 #pragma unroll
             for (int t = 0; t < TT; ++t) {
-                const float L = (r + t < r_end) ? fmaxf(a.load[(r + t) * C + c], 0.f) : 0.f;   // negative / NaN -> 0
+                const float L = t < nt ? fmaxf(lp[t * C], 0.f) : 0.f;   // negative / NaN -> 0
 #pragma unroll
                 for (int k = 0; k < NPL; ++k) {
                     ln[t * NPL + k] = L * rn[k];
@@ -388,73 +401,74 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
                                       !BUDGET || p < pmax[(q + 1) % NPL], best[q], best[q + 1]);
             }
         }
+        // per tile: warp argmin on (pool energy, n), then the pair; lane t keeps the result of tile t
+        int32_t my_idx = -1;
+        float my_E = CUDART_INF_F;
 #pragma unroll
         for (int t = 0; t < TT; ++t) {
-            if (r + t >= r_end) break;               // warp-uniform
+            if (t >= nt) break;                      // warp-uniform
             // the lane's chains in ascending n: strict compare keeps the lower n on ties.  Pool energy =
-            // n * (energy of one instance); + 0 turns -0 into +0 so that the keys order like the floats
-            float E = CUDART_INF_F;
-            int n = 0x7fffffff;
+            // n * (energy of one instance); the zero addend turns -0 into +0, so equal energies have equal bits
+            float E = keep[0] ? fmaf(best[t * NPL], nf[0], 0.f) : CUDART_INF_F;
+            int kk = 0;
 #pragma unroll
-            for (int k = 0; k < NPL; ++k) {
-                const float Ek = valid_n[k] ? best[t * NPL + k] * nf[k] + 0.f : CUDART_INF_F;
+            for (int k = 1; k < NPL; ++k) {
+                const float Ek = keep[k] ? fmaf(best[t * NPL + k], nf[k], 0.f) : CUDART_INF_F;
                 if (Ek < E) {
                     E = Ek;
-                    n = nl + 1 + LN * k;
+                    kk = k;
                 }
             }
-            // warp argmin on (E, n): smallest energy, then fewest instances (lowest index: n is the
+            // smallest energy of the tile, then the fewest instances that attain it (lowest index: n is the
             // slowest digit of j); lanes of different pair groups may hold the same n
-            const uint32_t key = float_key(E);
-            const uint32_t kmin = __reduce_min_sync(kFull, key);
-            const uint32_t nmin = __reduce_min_sync(kFull, key == kmin ? uint32_t(n) : 0xffffffffu);
-            const int64_t i = (r + t) * C + c;
-            if (kmin == float_key(CUDART_INF_F)) {                  // no feasible candidate
-                if (lane == 0) {
-                    best_idx[i] = -1;
-                    best_E[i] = CUDART_INF_F;
-                }
-                continue;
-            }
-            // recover the pair: lanes re-evaluate (nmin, p) for 32 pairs at a time, same arithmetic,
-            // and the first pair that reproduces the minimum bit for bit is the lowest-index one
-            const float Emin = __uint_as_float(kmin ^ ((kmin >> 31) ? 0x80000000u : 0xffffffffu));
-            const float nfm = float(nmin);
+            const float Emin = warp_min(E);
+            if (Emin == CUDART_INF_F) continue;      // no feasible candidate: -1 / +inf
+            const uint32_t n1 = uint32_t(kk << sh_n) + uint32_t(nl);              // n - 1
+            const uint32_t n1min = __reduce_min_sync(kFull, E == Emin ? n1 : 0xffffffffu);
+            const float nfm = float(n1min + 1u);
             // L/n of the winning instance count, from the lane that holds it (bit-identical by construction)
-            const int kstar = int(nmin - 1) >> (FULL ? 5 : a.ln_log2);
+            const int kstar = int(n1min >> sh_n);
             float lnk = DYN_LN(t * NPL);
 #pragma unroll
             for (int k = 1; k < NPL; ++k) lnk = (k == kstar) ? DYN_LN(t * NPL + k) : lnk;
-            const float lnm = __shfl_sync(kFull, lnk, int(nmin - 1) & (LN - 1));
+            const float lnm = __shfl_sync(kFull, lnk, int(n1min) & (LN - 1));
             int pm = P;
             if (BUDGET) {
-                int nt = 0;
-                for (int tt = 0; tt < a.T; ++tt) nt += (int64_t(nmin) * a.tp[tt] <= int64_t(a.budget)) ? 1 : 0;
-                pm = nt * a.F;
+                int ntp = 0;
+                for (int tt = 0; tt < a.T; ++tt) ntp += (int64_t(n1min + 1u) * a.tp[tt] <= int64_t(a.budget)) ? 1 : 0;
+                pm = ntp * a.F;
             }
+            // recover the pair: lanes re-evaluate (nmin, p) for 32 pairs at a time, same arithmetic, and the
+            // first pair that reproduces the minimum bit for bit is the lowest-index one
             int pstar = -1;
-            for (int p0 = 0; p0 < pm && pstar < 0; p0 += 32) {
-                const int pp = p0 + lane;
+            for (int p0 = 0; p0 < pm; p0 += 32) {
                 bool hit = false;
-                if (pp < pm) {
+                if (p0 + lane < pm) {
                     float e;
                     bool ok;
                     if (FAST) {
-                        const float4 pc = load16<SMEM>(ws, cpair + uint32_t(pp) * 16u);
-                        fast_one<SMEM>(ws, crow + uint32_t(pp) * pstep, lnm, pc.x, pc.z, e, ok);
+                        const float4 pc = load16<SMEM>(ws, cpair_lane + uint32_t(p0) * 16u);
+                        fast_one<SMEM>(ws, crow_lane + uint32_t(p0) * pstep, lnm, pc.x, pc.z, e, ok);
                     } else {
-                        const float2 pc = load8<SMEM>(ws, cpair + uint32_t(pp) * 8u);
-                        general_one<SMEM>(ws, crow + uint32_t(pp) * pstep - kTwo23Bits * 16u, lnm, pc.x, slo_c, Mf, e, ok);
+                        const float2 pc = load8<SMEM>(ws, cpair_lane + uint32_t(p0) * 8u);
+                        general_one<SMEM>(ws, crow_lane + uint32_t(p0) * pstep - kTwo23Bits * 16u, lnm, pc.x, slo_c, Mf, e, ok);
                     }
-                    hit = ok && (e * nfm + 0.f == Emin);
+                    hit = ok && (fmaf(e, nfm, 0.f) == Emin);
                 }
                 const unsigned m = __ballot_sync(kFull, hit);
-                if (m) pstar = p0 + __ffs(m) - 1;
+                if (m) {
+                    pstar = p0 + __ffs(m) - 1;
+                    break;
+                }
             }
-            if (lane == 0) {
-                best_idx[i] = pstar >= 0 ? int32_t((nmin - 1) * uint32_t(P) + uint32_t(pstar)) : -1;
-                best_E[i] = Emin;
+            if (lane == t) {
+                my_idx = pstar >= 0 ? int32_t(n1min * uint32_t(P) + uint32_t(pstar)) : -1;
+                my_E = Emin;
             }
+        }
+        if (lane < nt) {
+            best_idx[oi + lane * C] = my_idx;
+            best_E[oi + lane * C] = my_E;
         }
     }
 }
