@@ -43,6 +43,15 @@ constexpr int kPairUnroll = DYN_SW_UNROLL;
 #ifndef DYN_SW_MINB4
 #define DYN_SW_MINB4 5
 #endif
+#ifndef DYN_SW_TT1
+#define DYN_SW_TT1 8
+#endif
+#ifndef DYN_SW_TT2
+#define DYN_SW_TT2 4
+#endif
+#ifndef DYN_SW_MINB16
+#define DYN_SW_MINB16 2
+#endif
 #ifndef DYN_SW_MINB8
 #define DYN_SW_MINB8 4
 #endif
@@ -476,7 +485,7 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
 #undef DYN_LN
 
 template <int NPL, int TT, bool BUDGET, bool SMEM, bool FULL>
-__global__ void __launch_bounds__(kThreads, (NPL * TT <= 4 ? DYN_SW_MINB4 : (NPL * TT <= 8 && NPL <= 2 ? DYN_SW_MINB8 : 2)))
+__global__ void __launch_bounds__(kThreads, (NPL * TT <= 4 ? DYN_SW_MINB4 : (NPL * TT <= 8 && NPL <= 2 ? DYN_SW_MINB8 : (NPL * TT <= 16 && NPL <= 2 ? DYN_SW_MINB16 : 2))))
 eval_select_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__restrict__ best_E) {
     Tables tb;
     tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.pair2 = a.off_pair2; tb.rows2 = a.off_rows2;
@@ -725,8 +734,8 @@ cudaError_t launch_eval_select(const ResolvedLayout &lay, const void *d_ws, cons
     a.ln_log2 = ln;
     const int npl = (lay.Nmax + 31) / 32;           // instance counts per lane
     // four candidates per lane share each pair's constants
-    if (npl <= 1) return launch_es<1, 4>(a, best_idx, best_E, st);
-    if (npl <= 2) return launch_es<2, 4>(a, best_idx, best_E, st);
+    if (npl <= 1) return launch_es<1, DYN_SW_TT1>(a, best_idx, best_E, st);
+    if (npl <= 2) return launch_es<2, DYN_SW_TT2>(a, best_idx, best_E, st);
     if (npl <= 4) return launch_es<4, 1>(a, best_idx, best_E, st);
     if (npl <= 8) return launch_es<8, 1>(a, best_idx, best_E, st);
     return cudaErrorInvalidValue;                   // Nmax > 256 is rejected by the caller
