@@ -344,9 +344,23 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
     constexpr int NCH = TT * NPL;                    // candidates per lane and pair, an even number
     static_assert(NCH % 2 == 0, "candidates are evaluated two at a time");
 
-    // per-lane constants of the pair recovery: lane p re-evaluates pair p0 + p
+    // per-lane constants of the pair recovery: lane p re-evaluates pair p0 + p.  With at most 32 pairs and
+    // no GPU budget there is one round, and the lane's pair constants stay in registers for all tiles
     const uint32_t cpair_lane = cpair + uint32_t(lane) * (FAST ? 16u : 8u);
     const uint32_t crow_lane = crow + uint32_t(lane) * pstep;
+    const bool one_round = !BUDGET && P <= 32;
+    float rc_ic = 0.f, rc_lim = FAST ? -1.f : -CUDART_INF_F;          // a lane without a pair never hits
+    if (one_round && lane < P) {
+        if (FAST) {
+            const float4 pc = load16<SMEM>(ws, cpair_lane);
+            rc_ic = pc.x;
+            rc_lim = pc.z;
+        } else {
+            rc_ic = load8<SMEM>(ws, cpair_lane).x;
+            rc_lim = slo_c;
+        }
+    }
+    const uint32_t rc_row = (one_round && lane < P) ? crow_lane : crow;
     const int sh_n = FULL ? 5 : a.ln_log2;           // n - 1 = (chain number << sh_n) + lane number
     const float *lp = a.load + (r_begin * C + c);    // load of the pass's first tile; tiles are C floats apart
     int64_t oi = r_begin * C + c;                    // its index in the outputs
@@ -429,45 +443,55 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
                 }
             }
             // smallest energy of the tile, then the fewest instances that attain it (lowest index: n is the
-            // slowest digit of j); lanes of different pair groups may hold the same n
+            // slowest digit of j); lanes of different pair groups may hold the same n.  A tile without a
+            // feasible candidate (minimum +inf) runs through the same steps and finds no pair: -1 / +inf
             const float Emin = warp_min(E);
-            if (Emin == CUDART_INF_F) continue;      // no feasible candidate: -1 / +inf
             const uint32_t n1 = uint32_t(kk << sh_n) + uint32_t(nl);              // n - 1
             const uint32_t n1min = __reduce_min_sync(kFull, E == Emin ? n1 : 0xffffffffu);
             const float nfm = float(n1min + 1u);
             // L/n of the winning instance count, from the lane that holds it (bit-identical by construction)
-            const int kstar = int(n1min >> sh_n);
             float lnk = DYN_LN(t * NPL);
+            if (NPL > 1) {
+                const int kstar = int(n1min >> sh_n);
 #pragma unroll
-            for (int k = 1; k < NPL; ++k) lnk = (k == kstar) ? DYN_LN(t * NPL + k) : lnk;
-            const float lnm = __shfl_sync(kFull, lnk, int(n1min) & (LN - 1));
-            int pm = P;
-            if (BUDGET) {
-                int ntp = 0;
-                for (int tt = 0; tt < a.T; ++tt) ntp += (int64_t(n1min + 1u) * a.tp[tt] <= int64_t(a.budget)) ? 1 : 0;
-                pm = ntp * a.F;
+                for (int k = 1; k < NPL; ++k) lnk = (k == kstar) ? DYN_LN(t * NPL + k) : lnk;
             }
+            const float lnm = __shfl_sync(kFull, lnk, int(n1min) & (LN - 1));
             // recover the pair: lanes re-evaluate (nmin, p) for 32 pairs at a time, same arithmetic, and the
             // first pair that reproduces the minimum bit for bit is the lowest-index one
             int pstar = -1;
-            for (int p0 = 0; p0 < pm; p0 += 32) {
-                bool hit = false;
-                if (p0 + lane < pm) {
-                    float e;
-                    bool ok;
-                    if (FAST) {
-                        const float4 pc = load16<SMEM>(ws, cpair_lane + uint32_t(p0) * 16u);
-                        fast_one<SMEM>(ws, crow_lane + uint32_t(p0) * pstep, lnm, pc.x, pc.z, e, ok);
-                    } else {
-                        const float2 pc = load8<SMEM>(ws, cpair_lane + uint32_t(p0) * 8u);
-                        general_one<SMEM>(ws, crow_lane + uint32_t(p0) * pstep - kTwo23Bits * 16u, lnm, pc.x, slo_c, Mf, e, ok);
-                    }
-                    hit = ok && (fmaf(e, nfm, 0.f) == Emin);
+            if (one_round) {
+                float e;
+                bool ok;
+                if (FAST) fast_one<SMEM>(ws, rc_row, lnm, rc_ic, rc_lim, e, ok);
+                else general_one<SMEM>(ws, rc_row - kTwo23Bits * 16u, lnm, rc_ic, rc_lim, Mf, e, ok);
+                pstar = __ffs(__ballot_sync(kFull, ok && (fmaf(e, nfm, 0.f) == Emin))) - 1;
+            } else {
+                int pm = P;
+                if (BUDGET) {
+                    int ntp = 0;
+                    for (int tt = 0; tt < a.T; ++tt) ntp += (int64_t(n1min + 1u) * a.tp[tt] <= int64_t(a.budget)) ? 1 : 0;
+                    pm = ntp * a.F;
                 }
-                const unsigned m = __ballot_sync(kFull, hit);
-                if (m) {
-                    pstar = p0 + __ffs(m) - 1;
-                    break;
+                for (int p0 = 0; p0 < pm; p0 += 32) {
+                    bool hit = false;
+                    if (p0 + lane < pm) {
+                        float e;
+                        bool ok;
+                        if (FAST) {
+                            const float4 pc = load16<SMEM>(ws, cpair_lane + uint32_t(p0) * 16u);
+                            fast_one<SMEM>(ws, crow_lane + uint32_t(p0) * pstep, lnm, pc.x, pc.z, e, ok);
+                        } else {
+                            const float2 pc = load8<SMEM>(ws, cpair_lane + uint32_t(p0) * 8u);
+                            general_one<SMEM>(ws, crow_lane + uint32_t(p0) * pstep - kTwo23Bits * 16u, lnm, pc.x, slo_c, Mf, e, ok);
+                        }
+                        hit = ok && (fmaf(e, nfm, 0.f) == Emin);
+                    }
+                    const unsigned m = __ballot_sync(kFull, hit);
+                    if (m) {
+                        pstar = p0 + __ffs(m) - 1;
+                        break;
+                    }
                 }
             }
             if (lane == t) {
