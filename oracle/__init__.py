@@ -234,3 +234,21 @@ def hier_select(profile, space, e1, e2, load):
     if rc != 0:
         raise ValueError("orc_hier_select: invalid argument (epochs must be >= 1 and e1 a multiple of e2)")
     return out
+
+
+def mixed_select(profile, space, load):
+    """Pools that mix tensor parallelisms (Eq. 1 in full, by enumeration; needs space.gpu_budget > 0):
+    dict(counts[S][W][C][T], freq[S][W][C][T], tuple_no, best_E, E2, margin [S][W][C])."""
+    lib = _load()
+    p, s, keep = _structs(profile, space)
+    load = _arr(load, np.float32)
+    S, W, Cn = load.shape
+    assert Cn == p.C
+    out = dict(counts=np.empty((S, W, Cn, p.T), np.int32), freq=np.empty((S, W, Cn, p.T), np.int32),
+               tuple_no=np.empty((S, W, Cn), np.int32), best_E=np.empty((S, W, Cn)), E2=np.empty((S, W, Cn)),
+               margin=np.empty((S, W, Cn)))
+    rc = lib.orc_mixed_select(C.byref(p), C.byref(s), _p(load), C.c_int64(S), C.c_int64(W), _p(out["counts"]),
+                              _p(out["freq"]), _p(out["tuple_no"]), _p(out["best_E"]), _p(out["E2"]), _p(out["margin"]))
+    if rc != 0:
+        raise ValueError("orc_mixed_select: invalid argument (a GPU budget > 0 is required)")
+    return out

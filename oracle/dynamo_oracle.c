@@ -24,6 +24,8 @@
  *                     runner-up energy (for near-tie exemptions in parity tests).
  *   orc_totals        cluster energy per scenario and per window, GPUs in use per window, histogram
  *                     of chosen configurations [Sec. 6 cluster-level energy, GPUs per sharding].
+ *   orc_mixed_select  Eq. 1 in full: a pool that mixes tensor parallelisms (counts per TP under a GPU
+ *                     budget, load split by capacity, one frequency per TP), by enumeration.
  *   orc_hier_select   the controller hierarchy of Sec. 4.2 on the same models: nodes per pool from the
  *                     epoch's peak load and the per-node maximum load (ceil(PL/ML)), sharding at the
  *                     highest frequency within those GPUs, then the frequency per window.
@@ -443,5 +445,95 @@ int orc_hier_select(const orc_profile *p, const orc_space *sp, int32_t e1, int32
         }
     }
     free(row); free(wt); free(ml);
+    return ORC_OK;
+}
+
+/* ---- pools that mix tensor parallelisms (Sec. 4.1, Eq. 1 in full) ------------------------------- */
+
+/*
+ * Eq. 1 lets one pool hold instances of several tensor parallelisms at once: counts N^{TP_i}, one
+ * frequency f^{TP_i} per parallelism, a load L^{TP_i} per instance, under the GPU budget
+ * sum_i TP_i * N^{TP_i} <= N, with all the load served and every instance within the SLO; the objective
+ * is sum_i N^{TP_i} * Energy^{TP_i, f_i}(L^{TP_i}).  The paper hands this to a solver; here the count
+ * tuples are enumerated.  Readings (the paper leaves the split and the enumeration open):
+ *   - counts n_t = 0..Nmax per TP index t, not all zero, sum_t n_t*TP_t <= gpu_budget (required > 0);
+ *   - the load is split in proportion to the capacity at the highest candidate frequency: the group
+ *     of type t gets L * n_t*capH_t / A, A = sum_j n_j*capH_j, capH_t = cap(c, t, highest candidate f),
+ *     so every instance runs at the same fraction L/A of its top-frequency capacity;
+ *   - each group then takes, on its own, the feasible frequency of least energy for its share (fair
+ *     share inside the group, TTFT / TBT / capacity as for a single-type pool), lowest q on ties; a
+ *     tuple with a group that has no feasible frequency is infeasible;
+ *   - energy of the tuple = sum over groups in ascending t; the tuple of least energy wins, ties go to
+ *     the lowest tuple number, tuples being numbered in odometer order with n_0 (smallest TP) the
+ *     fastest digit.
+ * Outputs per tile (s, w, c): counts[T], freq[T] (-1 where the count is 0; all -1 and E = +inf if no
+ * tuple is feasible), tuple number (position among the budget-feasible tuples in odometer order, -1 if
+ * none), energy.  Optional diagnostics (NULL to skip): E2 = least energy over the other tuples, margin =
+ * smallest relative distance of a deciding quantity to its bound over everything evaluated for the tile.
+ */
+int orc_mixed_select(const orc_profile *p, const orc_space *sp, const float *load, int64_t S, int64_t W,
+                     int32_t *counts, int32_t *freq, int32_t *tuple_no, double *best_E, double *E2, double *margin) {
+    const int32_t C = p->C, T = p->T, F = sp->F, Nmax = sp->Nmax, B = sp->gpu_budget;
+    if (B <= 0 || T > 8) return ORC_EINVAL;
+    int32_t *row = (int32_t *)malloc(sizeof(int32_t) * (size_t)F);
+    double *wt = (double *)malloc(sizeof(double) * (size_t)F);
+    int rc = orc_resolve(p->f_grid, p->R, sp->f_cand, F, row, wt);
+    if (rc != ORC_OK) { free(row); free(wt); return rc; }
+    const int64_t tiles = S * W * C;
+#pragma omp parallel for schedule(dynamic, 16)
+    for (int64_t i = 0; i < tiles; ++i) {
+        const int32_t c = (int32_t)(i % C);
+        const double L = (double)load[i];
+        double capH[8];
+        for (int32_t t = 0; t < T; ++t) {
+            const size_t ct = ((size_t)c * T + t) * p->R;
+            capH[t] = lerp((double)p->cap[ct + row[F - 1]], (double)p->cap[ct + row[F - 1] + 1], wt[F - 1]);
+        }
+        int32_t n[8] = {0}, bn[8], bq[8];
+        for (int32_t t = 0; t < T; ++t) { bn[t] = -1; bq[t] = -1; }
+        double eb = INFINITY, e2nd = INFINITY, mg = INFINITY;
+        int32_t number = -1, bnum = -1;
+        for (;;) {
+            /* next tuple in odometer order, n_0 fastest */
+            int32_t t = 0;
+            while (t < T && n[t] == Nmax) n[t++] = 0;
+            if (t == T) break;
+            ++n[t];
+            int64_t gpus = 0;
+            for (int32_t k = 0; k < T; ++k) gpus += (int64_t)n[k] * p->tp[k];
+            if (gpus > B) continue;
+            ++number;
+            double A = 0.0;
+            for (int32_t k = 0; k < T; ++k) A += (double)n[k] * capH[k];
+            double E = 0.0;
+            int32_t qs[8];
+            for (int32_t k = 0; k < T; ++k) {
+                qs[k] = -1;
+                if (n[k] == 0) continue;
+                const double share = L * ((double)n[k] * capH[k]) / A;      /* load of the whole group */
+                double eg = INFINITY;
+                for (int32_t q = 0; q < F; ++q) {
+                    const double e = eval_candidate(p, sp, row, wt, c, share, n[k], k, q, 0, &mg);
+                    if (e < eg) { eg = e; qs[k] = q; }
+                }
+                E += eg;                                                     /* +inf if the group has no frequency */
+            }
+            if (E < eb) {
+                e2nd = eb; eb = E; bnum = number;
+                for (int32_t k = 0; k < T; ++k) { bn[k] = n[k]; bq[k] = qs[k]; }
+            } else if (E < e2nd) {
+                e2nd = E;
+            }
+        }
+        for (int32_t k = 0; k < T; ++k) {
+            counts[i * T + k] = bnum >= 0 ? bn[k] : -1;
+            freq[i * T + k] = bnum >= 0 ? bq[k] : -1;
+        }
+        tuple_no[i] = bnum;
+        best_E[i] = eb;
+        if (E2) E2[i] = e2nd;
+        if (margin) margin[i] = mg;
+    }
+    free(row); free(wt);
     return ORC_OK;
 }

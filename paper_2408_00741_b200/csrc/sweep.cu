@@ -509,7 +509,7 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
 #undef DYN_LN
 
 template <int NPL, int TT, bool BUDGET, bool SMEM, bool FULL>
-__global__ void __launch_bounds__(kThreads, (NPL * TT <= 4 ? DYN_SW_MINB4 : (NPL * TT <= 8 && NPL <= 2 ? DYN_SW_MINB8 : (NPL * TT <= 16 && NPL <= 2 ? DYN_SW_MINB16 : 2))))
+__global__ void __launch_bounds__(kThreads, (NPL * TT <= 4 ? DYN_SW_MINB4 : (NPL * TT <= 8 && NPL <= 2 ? (NPL == 1 ? DYN_SW_MINB4 : DYN_SW_MINB8) : (NPL * TT <= 16 && NPL <= 2 ? DYN_SW_MINB16 : 2))))
 eval_select_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__restrict__ best_E) {
     Tables tb;
     tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.pair2 = a.off_pair2; tb.rows2 = a.off_rows2;
