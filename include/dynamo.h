@@ -288,7 +288,8 @@ void dyn_set_timing_events(void *start_event, void *stop_event);
  *     streams) race on the array and give undefined results: serialise them.
  *   - Everything else (arguments, results, errors, tolerances) is exactly dyn_eval_select's.
  * ------------------------------------------------------------------------------------------- */
-#define DYN_STATIC_WS_BYTES (4u << 20)   /* 4 MiB: every benchmark configuration of this repository fits */
+#define DYN_STATIC_WS_BYTES (4u << 20)   /* 4 MiB: coarse frequency grids fit with thousands of scenarios; a
+                                            79-frequency, 64-knot grid (5 MB of resolved tables) does not */
 int dyn_eval_select_static(const dyn_profile *profile, const dyn_space *space, const float *d_load,
                            int64_t S, int64_t W, const dyn_select_out *out, void *stream);
 
