@@ -203,6 +203,41 @@ int dyn_hier_select(const dyn_profile *profile, const dyn_space *space, const dy
                     const dyn_select_out *out, void *d_ws, size_t ws_bytes, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Pools that mix tensor parallelisms.  [Sec. 4.1, Eq. 1 in full: the pool may hold N^{TP_i} instances of
+ * several parallelisms at once, each parallelism at its own frequency f^{TP_i} and with its own per-instance
+ * load L^{TP_i}, under  sum_i TP_i * N^{TP_i} <= N,  sum_i N^{TP_i} * L^{TP_i} >= L  and the SLO for every
+ * instance; the objective is  sum_i N^{TP_i} * Energy^{TP_i, f_i}(L^{TP_i}).]
+ *
+ * The paper leaves the search to a solver; this call enumerates.  Per tile (s, w, c) with load L:
+ *   - count tuples (n_0, ..., n_{T-1}), n_t = 0 .. space->Nmax instances of TP index t, not all zero, with
+ *     sum_t n_t * tp[t] <= space->gpu_budget (the budget is REQUIRED here, > 0);
+ *   - the load is split in proportion to capacity at the highest candidate frequency: the group of TP index t
+ *     serves L * n_t*capH_t / sum_j n_j*capH_j, capH_t = cap(c, t, f_cand[F-1]);
+ *   - every group takes, on its own, the feasible candidate frequency of least energy for its share (fair
+ *     share within the group; TTFT, TBT and capacity as in the single-type evaluation above), lowest
+ *     frequency index on ties; a tuple with a group that has none is infeasible;
+ *   - the tuple's energy is the sum over its groups; the tuple of least energy is chosen, lowest tuple
+ *     number on ties.  Tuples are numbered 0, 1, ... in odometer order with n_0 the fastest digit, counting
+ *     only tuples within the budget.
+ * Limits: T <= 4, Nmax <= 255, at most 2^20 tuples within the budget (else DYN_EUNSUPPORTED).
+ * Workspace: dyn_mixed_workspace_bytes().  Errors: as dyn_eval_select, plus DYN_EINVAL for gpu_budget <= 0.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t *d_counts;           /* [S][W][C][T] chosen n_t; -1 in every slot if no tuple is feasible; required */
+    int32_t *d_freq;             /* [S][W][C][T] chosen frequency index of TP index t, -1 where n_t is 0; required */
+    int32_t *d_tuple;            /* [S][W][C] number of the chosen tuple, -1 if none; required */
+    float *d_best_E;             /* [S][W][C] its energy (Wh), +inf if none; required */
+    double *d_E_total;           /* [S] sum over feasible tiles; required */
+    uint32_t *d_n_infeasible;    /* [S] tiles without a feasible tuple; required */
+} dyn_mixed_out;
+
+size_t dyn_mixed_workspace_bytes(const dyn_profile *profile, const dyn_space *space, int64_t S, int64_t W);
+/* Number of count tuples within the budget (0 on bad input): the work per tile is this times T*F evaluations. */
+int64_t dyn_mixed_tuple_count(const dyn_profile *profile, const dyn_space *space);
+int dyn_mixed_select(const dyn_profile *profile, const dyn_space *space, const float *d_load, int64_t S, int64_t W,
+                     const dyn_mixed_out *out, void *d_ws, size_t ws_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Whole path from HOST buffers: (a) -> (b) -> (c) in one call.  [Sec. 3 trace -> Sec. 3.2 loads ->
  * Sec. 4.1 / Eq. 1 evaluation -> Sec. 4.2 selection -> Sec. 6 totals]
  *

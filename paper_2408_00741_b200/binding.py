@@ -25,7 +25,7 @@ DYN_OK, DYN_EINVAL, DYN_ECUDA, DYN_EUNSUPPORTED, DYN_EWORKSPACE = 0, -1, -2, -3,
 EXPORTS = ("dyn_strerror", "dyn_last_cuda_error", "dyn_bin_trace", "dyn_workspace_bytes", "dyn_eval_configs",
            "dyn_select_workspace_bytes", "dyn_select", "dyn_eval_select", "dyn_pipeline_arena_bytes",
            "dyn_pipeline_host", "dyn_set_timing_events", "dyn_eval_select_static", "dyn_hier_workspace_bytes",
-           "dyn_hier_select")
+           "dyn_hier_select", "dyn_mixed_workspace_bytes", "dyn_mixed_tuple_count", "dyn_mixed_select")
 
 
 class DynError(RuntimeError):
@@ -121,6 +121,19 @@ _lib.dyn_eval_select_static.restype = C.c_int
 _lib.dyn_eval_select_static.argtypes = [C.POINTER(_Profile), C.POINTER(_Space), C.c_void_p, C.c_int64, C.c_int64,
                                         C.POINTER(_SelectOut), C.c_void_p]
 DYN_STATIC_WS_BYTES = 4 << 20
+
+class _MixedOut(C.Structure):
+    _fields_ = [("d_counts", C.c_void_p), ("d_freq", C.c_void_p), ("d_tuple", C.c_void_p), ("d_best_E", C.c_void_p),
+                ("d_E_total", C.c_void_p), ("d_n_infeasible", C.c_void_p)]
+
+
+_lib.dyn_mixed_workspace_bytes.restype = C.c_size_t
+_lib.dyn_mixed_workspace_bytes.argtypes = [C.POINTER(_Profile), C.POINTER(_Space), C.c_int64, C.c_int64]
+_lib.dyn_mixed_tuple_count.restype = C.c_int64
+_lib.dyn_mixed_tuple_count.argtypes = [C.POINTER(_Profile), C.POINTER(_Space)]
+_lib.dyn_mixed_select.restype = C.c_int
+_lib.dyn_mixed_select.argtypes = [C.POINTER(_Profile), C.POINTER(_Space), C.c_void_p, C.c_int64, C.c_int64,
+                                  C.POINTER(_MixedOut), C.c_void_p, C.c_size_t, C.c_void_p]
 
 
 def _dev(t, dtype, what):
@@ -347,3 +360,40 @@ def dyn_hier_select(profile: Profile, space: Space, scale_epoch_windows, shard_e
                               _dev(d_nodes, torch.int32, "d_nodes"), _dev(d_shard, torch.int32, "d_shard"), C.byref(o),
                               ws, nb, _stream())
     _check(rc, "dyn_hier_select")
+
+
+class MixedOut:
+    """Output buffers of dyn_mixed_select (mirrors dyn_mixed_out)."""
+
+    def __init__(self, S, W, Cn, T, device="cuda"):
+        self.counts = torch.empty((S, W, Cn, T), dtype=torch.int32, device=device)
+        self.freq = torch.empty((S, W, Cn, T), dtype=torch.int32, device=device)
+        self.tuple = torch.empty((S, W, Cn), dtype=torch.int32, device=device)
+        self.best_E = torch.empty((S, W, Cn), dtype=torch.float32, device=device)
+        self.E_total = torch.empty((S,), dtype=torch.float64, device=device)
+        self.n_infeasible = torch.empty((S,), dtype=torch.int32, device=device)
+
+    def _struct(self):
+        return _MixedOut(self.counts.data_ptr(), self.freq.data_ptr(), self.tuple.data_ptr(), self.best_E.data_ptr(),
+                         self.E_total.data_ptr(), self.n_infeasible.data_ptr())
+
+
+def dyn_mixed_workspace_bytes(profile: Profile, space: Space, S, W) -> int:
+    p, s = profile._struct(), space._struct()
+    return int(_lib.dyn_mixed_workspace_bytes(C.byref(p), C.byref(s), int(S), int(W)))
+
+
+def dyn_mixed_tuple_count(profile: Profile, space: Space) -> int:
+    p, s = profile._struct(), space._struct()
+    return int(_lib.dyn_mixed_tuple_count(C.byref(p), C.byref(s)))
+
+
+def dyn_mixed_select(profile: Profile, space: Space, d_load, out: MixedOut, d_ws):
+    """Pools that mix tensor parallelisms under space.gpu_budget (> 0): per tile the count tuple of least energy."""
+    S, W, Cn = d_load.shape
+    p, s = profile._struct(), space._struct()
+    o = out._struct()
+    ws, nb = _ws(d_ws)
+    rc = _lib.dyn_mixed_select(C.byref(p), C.byref(s), _dev(d_load, torch.float32, "d_load"), S, W, C.byref(o), ws, nb,
+                               _stream())
+    _check(rc, "dyn_mixed_select")

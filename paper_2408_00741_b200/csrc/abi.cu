@@ -4,6 +4,7 @@
 
 #include <cmath>
 #include <cstring>
+#include <vector>
 
 namespace dyn {
 
@@ -110,6 +111,40 @@ int check_ws(const void *d_ws, size_t ws_bytes, size_t need) {
 }
 
 size_t align256(size_t x) { return (x + 255) / 256 * 256; }
+
+// count tuples within the GPU budget in odometer order (n_0 fastest), 8 bits per TP index; with out == nullptr
+// only counts.  Returns -1 when there are more than `limit` tuples.
+int64_t enumerate_tuples(const dyn_profile *p, const dyn_space *sp, int64_t limit, uint32_t *out) {
+    const int T = p->T, Nmax = sp->Nmax;
+    int n[4] = {0, 0, 0, 0};
+    int64_t K = 0;
+    for (;;) {
+        int t = 0;
+        while (t < T && n[t] == Nmax) n[t++] = 0;
+        if (t == T) break;
+        ++n[t];                                              // the digits below t are zero now
+        int64_t gpus = 0;
+        for (int k = 0; k < T; ++k) gpus += int64_t(n[k]) * p->tp[k];
+        if (gpus > sp->gpu_budget) {
+            n[t] = Nmax;                                     // larger values of this digit only add GPUs: carry next
+            continue;
+        }
+        if (K >= limit) return -1;
+        if (out) out[K] = uint32_t(n[0]) | (uint32_t(n[1]) << 8) | (uint32_t(n[2]) << 16) | (uint32_t(n[3]) << 24);
+        ++K;
+    }
+    return K;
+}
+
+constexpr int64_t kMaxTuples = int64_t(1) << 20;
+
+int check_mixed(const dyn_profile *p, const dyn_space *sp, int64_t S, int64_t W, ResolveParams *rp) {
+    const int rc = check_problem(p, sp, S, W, rp);
+    if (rc != DYN_OK) return rc;
+    if (sp->gpu_budget <= 0) return DYN_EINVAL;
+    if (p->T > 4 || sp->Nmax > 255) return DYN_EUNSUPPORTED;
+    return DYN_OK;
+}
 
 }  // namespace
 }  // namespace dyn
@@ -288,6 +323,55 @@ int dyn_hier_select(const dyn_profile *profile, const dyn_space *space, const dy
     uint32_t *partial_bad = reinterpret_cast<uint32_t *>(ws + lay.off_partial + size_t(S) * size_t(chunks) * sizeof(double));
     DYN_CUDA_TRY(launch_totals(to_out(out), S, W, profile->C, lay.J, nullptr, nullptr, profile->T, space->F,
                                reinterpret_cast<const int32_t *>(ws + lay.off_tp), partial, partial_bad, st));
+    return DYN_OK;
+}
+
+int64_t dyn_mixed_tuple_count(const dyn_profile *profile, const dyn_space *space) {
+    if (check_mixed(profile, space, 0, 0, nullptr) != DYN_OK) return 0;
+    const int64_t K = enumerate_tuples(profile, space, kMaxTuples, nullptr);
+    return K < 0 ? 0 : K;
+}
+
+size_t dyn_mixed_workspace_bytes(const dyn_profile *profile, const dyn_space *space, int64_t S, int64_t W) {
+    const size_t base = dyn_workspace_bytes(profile, space, S, W);
+    const int64_t K = dyn_mixed_tuple_count(profile, space);
+    if (!base || K <= 0) return 0;
+    return base + align256(size_t(K) * sizeof(uint32_t)) + align256(size_t(profile->C) * profile->T * sizeof(float));
+}
+
+int dyn_mixed_select(const dyn_profile *profile, const dyn_space *space, const float *d_load, int64_t S, int64_t W,
+                     const dyn_mixed_out *out, void *d_ws, size_t ws_bytes, void *stream) {
+    ResolveParams rp;
+    int rc = check_mixed(profile, space, S, W, &rp);
+    if (rc != DYN_OK) return rc;
+    const int64_t tiles = S * W * profile->C;
+    if (!out) return DYN_EINVAL;
+    if (tiles > 0 && (!out->d_counts || !out->d_freq || !out->d_tuple || !out->d_best_E || !d_load)) return DYN_EINVAL;
+    if (S > 0 && (!out->d_E_total || !out->d_n_infeasible)) return DYN_EINVAL;
+    const int64_t K = enumerate_tuples(profile, space, kMaxTuples, nullptr);
+    if (K < 0) return DYN_EUNSUPPORTED;
+    if (K == 0) return DYN_EINVAL;                           // the budget admits no instance at all
+    static thread_local std::vector<uint32_t> tuples;        // host list, rebuilt per call (cheap next to the search)
+    tuples.resize(size_t(K));
+    enumerate_tuples(profile, space, K, tuples.data());
+    const ResolvedLayout lay = resolved_layout(profile->C, profile->T, space->F, profile->M, space->Nmax, S, W);
+    const size_t off_tuples = lay.total, off_caph = off_tuples + align256(size_t(K) * sizeof(uint32_t));
+    const size_t need = off_caph + align256(size_t(profile->C) * profile->T * sizeof(float));
+    rc = check_ws(d_ws, ws_bytes, need);
+    if (rc != DYN_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char *ws = static_cast<char *>(d_ws);
+    // pageable host memory: the copy is staged before the call returns
+    DYN_CUDA_TRY(cudaMemcpyAsync(ws + off_tuples, tuples.data(), size_t(K) * sizeof(uint32_t), cudaMemcpyHostToDevice, st));
+    DYN_CUDA_TRY(launch_resolve(rp, lay, d_ws, st));
+    DYN_CUDA_TRY(launch_mixed(lay, d_ws, off_tuples, off_caph, K, d_load, tiles, out->d_counts, out->d_freq,
+                              out->d_tuple, out->d_best_E, st));
+    SelectOut so{};
+    so.best_idx = out->d_tuple; so.best_E = out->d_best_E; so.E_total = out->d_E_total; so.n_infeasible = out->d_n_infeasible;
+    const int64_t chunks = totals_chunks(W);
+    double *partial = reinterpret_cast<double *>(ws + lay.off_partial);
+    uint32_t *partial_bad = reinterpret_cast<uint32_t *>(ws + lay.off_partial + size_t(S) * size_t(chunks) * sizeof(double));
+    DYN_CUDA_TRY(launch_totals(so, S, W, profile->C, 1, nullptr, nullptr, 1, 1, nullptr, partial, partial_bad, st));
     return DYN_OK;
 }
 

@@ -108,6 +108,11 @@ cudaError_t launch_hier(const ResolveParams &rp, const ResolvedLayout &lay, void
                         int64_t S, int64_t W, int32_t e1, int32_t e2, int32_t space_budget, int32_t *d_nodes,
                         int32_t *d_shard, int32_t *best_idx, float *best_E, cudaStream_t st);
 
+// pools that mix tensor parallelisms: `tuples` holds K count tuples, 8 bits per TP index
+cudaError_t launch_mixed(const ResolvedLayout &lay, void *d_ws, size_t off_tuples, size_t off_caph, int64_t K,
+                         const float *d_load, int64_t tiles, int32_t *d_counts, int32_t *d_freq, int32_t *d_tuple,
+                         float *d_best_E, cudaStream_t st);
+
 struct BinParams {
     FastDiv win;
     uint32_t n_windows;
@@ -120,6 +125,21 @@ cudaError_t launch_bin_trace(const BinParams &bp, const uint32_t *t_ms, const ui
                              cudaStream_t st);
 
 int sm_count();
+
+#ifdef __CUDACC__
+// general-path evaluation of one candidate from the resolved rows (used by the small restricted searches)
+// energy of the pool (n instances) for pair row `row` at per-instance load ln; ok = TBT within the SLO
+// (u > 1 and never-feasible pairs read as TBT = huge or +inf through the sentinel entries of the row)
+__device__ __forceinline__ float eval_pair(const float4 *__restrict__ row, float ic, float Mf, float ln, float nf,
+                                           float slo, bool &ok) {
+    const float x = __saturatef(ln * ic) * Mf;
+    const int m = int(x);
+    const float nu = x - float(m);
+    const float4 e = __ldg(row + m);
+    ok = fmaf(-nu, e.y, e.x) <= slo;
+    return nf * fmaf(-nu, e.w, e.z);
+}
+#endif
 
 // optional caller-owned events recorded around a stage's main kernel (thread-local; NULL = off)
 struct TimingEvents { cudaEvent_t start, stop; };

@@ -51,18 +51,6 @@ struct HierArgs {
     float *best_E;
 };
 
-// energy of the pool (n instances) for pair row `row` at per-instance load ln; ok = TBT within the SLO
-// (u > 1 and never-feasible pairs read as TBT = huge or +inf through the sentinel entries of the row)
-__device__ __forceinline__ float eval_pair(const float4 *__restrict__ row, float ic, float Mf, float ln, float nf,
-                                           float slo, bool &ok) {
-    const float x = __saturatef(ln * ic) * Mf;
-    const int m = int(x);
-    const float nu = x - float(m);
-    const float4 e = __ldg(row + m);
-    ok = fmaf(-nu, e.y, e.x) <= slo;
-    return nf * fmaf(-nu, e.w, e.z);
-}
-
 // grid: x over the (epoch or window, class) pairs of one scenario, y over scenarios (strided)
 
 __global__ void __launch_bounds__(256) hier_nodes_kernel(const HierArgs a) {
