@@ -387,6 +387,10 @@ def run_ours(args, rank, world, local_rank):
             result["hierarchical"] = measure_hier(dyn, gen, dev)
         except Exception as exc:
             result["hierarchical"] = {"error": repr(exc)}
+        try:
+            result["mixed_pools"] = measure_mixed(dyn, gen, dev)
+        except Exception as exc:
+            result["mixed_pools"] = {"error": repr(exc)}
 
     if not args.no_cpu_baseline and world == 1:
         cb, _, _ = time_oracle(wl, trace, prof, sp, base_counts)
@@ -530,6 +534,51 @@ def measure_hier(dyn, gen, dev, S=2048):
             "energy_over_joint_optimum": hier_total / joint_total}
 
 
+def measure_mixed(dyn, gen, dev, S=16, n_max=16, budget=16):
+    """Pools that mix tensor parallelisms (Eq. 1 in full, by enumeration) on S day-long scenarios of the 1-day
+    profile: every count tuple within `budget` GPUs, per group every candidate frequency."""
+    import itertools
+    import torch
+    wl = gen.workload("cfg2")
+    prof = wl.profile()
+    sp = gen.make_space(wl.f_cand_mhz, n_max, wl.window_s, gpu_budget=budget)
+    W, Cn, T, F = wl.trace.n_windows, 9, len(prof.tp), len(sp.f_cand_mhz)
+    load = torch.from_numpy(gen.random_loads((S, W, Cn), seed=12, mean=2.5)).to(dev)
+    P = dyn.Profile(prof.tp, prof.f_grid_mhz, prof.ttft, prof.cap, prof.tbt, prof.pow, device=dev)
+    SP = dyn.Space(sp.f_cand_mhz, sp.n_max, sp.slo_ttft_s, sp.slo_tbt_s, sp.window_s, sp.gpu_budget)
+    out = dyn.MixedOut(S, W, Cn, T, device=dev)
+    ws = torch.empty(dyn.dyn_mixed_workspace_bytes(P, SP, S, W), dtype=torch.uint8, device=dev)
+    call = lambda: dyn.dyn_mixed_select(P, SP, load, out, ws)
+    for _ in range(3):
+        call()
+    K = 10
+    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    for a, b in kev:
+        a.record(); b.record()
+    torch.cuda.synchronize()
+    for k in range(K):
+        dyn.dyn_set_timing_events(*kev[k])
+        call()
+    dyn.dyn_set_timing_events(None, None)
+    torch.cuda.synchronize()
+    ms = float(np.mean([a.elapsed_time(b) for a, b in kev]))
+    # single-type evaluations per tile: for every tuple within the budget, F per parallelism in use
+    tuples = [n for n in itertools.product(range(n_max + 1), repeat=T)
+              if 0 < sum(a * int(t) for a, t in zip(n, prof.tp)) <= budget]
+    assert len(tuples) == dyn.dyn_mixed_tuple_count(P, SP)
+    per_tile = F * sum(sum(1 for a in n if a) for n in tuples)
+    evals = S * W * Cn * per_tile
+    fp32_peak = SM_COUNT * FP32_LANES * 2 * SM_MAX_MHZ * 1e6 / 1e12
+    tfl = FLOP_PER_EVAL * evals / (ms * 1e-3) / 1e12
+    mixed_frac = float(((out.counts > 0).sum(dim=3) > 1).float().mean().item())
+    return {"workload": f"cfg2 profile x {S} scenarios, counts 0..{n_max} per TP, {budget} GPUs per pool",
+            "tiles": int(S * W * Cn), "tuples": len(tuples), "evaluations": int(evals), "kernel_ms": ms,
+            "evals_per_s": evals / (ms * 1e-3), "tiles_per_s": S * W * Cn / (ms * 1e-3),
+            "roofline": {"bound": "alu", "achieved": tfl, "peak": fp32_peak, "unit": "TFLOP/s", "frac": tfl / fp32_peak,
+                         "traffic": None, "peak_source": "derived fp32 peak; 20 flop per single-type evaluation"},
+            "tiles_that_mix_parallelisms": mixed_frac}
+
+
 def main():
     args = parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -545,7 +594,7 @@ def main():
         dev = torch.device("cuda", local_rank)
         torch.cuda.set_device(dev)
         print(json.dumps({"bin_trace": measure_bin(dyn, gen, dev), "materialised": measure_materialised(dyn, gen, dev),
-                          "hierarchical": measure_hier(dyn, gen, dev)}))
+                          "hierarchical": measure_hier(dyn, gen, dev), "mixed_pools": measure_mixed(dyn, gen, dev)}))
         return
     run_ours(args, rank, world, local_rank)
 

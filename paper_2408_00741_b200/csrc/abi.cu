@@ -3,6 +3,7 @@
 #include "dyn_internal.cuh"
 
 #include <cmath>
+#include <algorithm>
 #include <cstring>
 #include <vector>
 
@@ -112,9 +113,9 @@ int check_ws(const void *d_ws, size_t ws_bytes, size_t need) {
 
 size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
-// count tuples within the GPU budget in odometer order (n_0 fastest), 8 bits per TP index; with out == nullptr
-// only counts.  Returns -1 when there are more than `limit` tuples.
-int64_t enumerate_tuples(const dyn_profile *p, const dyn_space *sp, int64_t limit, uint32_t *out) {
+// count tuples within the GPU budget in odometer order (n_0 fastest): {counts, 8 bits per TP index; number};
+// with out == nullptr only counts.  Returns -1 when there are more than `limit` tuples.
+int64_t enumerate_tuples(const dyn_profile *p, const dyn_space *sp, int64_t limit, uint2 *out) {
     const int T = p->T, Nmax = sp->Nmax;
     int n[4] = {0, 0, 0, 0};
     int64_t K = 0;
@@ -130,7 +131,8 @@ int64_t enumerate_tuples(const dyn_profile *p, const dyn_space *sp, int64_t limi
             continue;
         }
         if (K >= limit) return -1;
-        if (out) out[K] = uint32_t(n[0]) | (uint32_t(n[1]) << 8) | (uint32_t(n[2]) << 16) | (uint32_t(n[3]) << 24);
+        if (out) out[K] = make_uint2(uint32_t(n[0]) | (uint32_t(n[1]) << 8) | (uint32_t(n[2]) << 16) | (uint32_t(n[3]) << 24),
+                                     uint32_t(K));
         ++K;
     }
     return K;
@@ -336,7 +338,7 @@ size_t dyn_mixed_workspace_bytes(const dyn_profile *profile, const dyn_space *sp
     const size_t base = dyn_workspace_bytes(profile, space, S, W);
     const int64_t K = dyn_mixed_tuple_count(profile, space);
     if (!base || K <= 0) return 0;
-    return base + align256(size_t(K) * sizeof(uint32_t)) + align256(size_t(profile->C) * profile->T * sizeof(float));
+    return base + align256(size_t(K) * sizeof(uint2)) + align256(size_t(profile->C) * profile->T * sizeof(float));
 }
 
 int dyn_mixed_select(const dyn_profile *profile, const dyn_space *space, const float *d_load, int64_t S, int64_t W,
@@ -351,18 +353,24 @@ int dyn_mixed_select(const dyn_profile *profile, const dyn_space *space, const f
     const int64_t K = enumerate_tuples(profile, space, kMaxTuples, nullptr);
     if (K < 0) return DYN_EUNSUPPORTED;
     if (K == 0) return DYN_EINVAL;                           // the budget admits no instance at all
-    static thread_local std::vector<uint32_t> tuples;        // host list, rebuilt per call (cheap next to the search)
+    static thread_local std::vector<uint2> tuples;           // host list, rebuilt per call (cheap next to the search)
     tuples.resize(size_t(K));
     enumerate_tuples(profile, space, K, tuples.data());
+    // group the tuples by the set of TP indices in use (stable: number order inside a group), so that the
+    // tuples a warp evaluates side by side take the same branches
+    auto mask_of = [](const uint2 &u) {
+        return ((u.x & 0xffu) ? 1u : 0u) | ((u.x & 0xff00u) ? 2u : 0u) | ((u.x & 0xff0000u) ? 4u : 0u) | ((u.x >> 24) ? 8u : 0u);
+    };
+    std::stable_sort(tuples.begin(), tuples.end(), [&](const uint2 &x, const uint2 &y) { return mask_of(x) < mask_of(y); });
     const ResolvedLayout lay = resolved_layout(profile->C, profile->T, space->F, profile->M, space->Nmax, S, W);
-    const size_t off_tuples = lay.total, off_caph = off_tuples + align256(size_t(K) * sizeof(uint32_t));
+    const size_t off_tuples = lay.total, off_caph = off_tuples + align256(size_t(K) * sizeof(uint2));
     const size_t need = off_caph + align256(size_t(profile->C) * profile->T * sizeof(float));
     rc = check_ws(d_ws, ws_bytes, need);
     if (rc != DYN_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     char *ws = static_cast<char *>(d_ws);
     // pageable host memory: the copy is staged before the call returns
-    DYN_CUDA_TRY(cudaMemcpyAsync(ws + off_tuples, tuples.data(), size_t(K) * sizeof(uint32_t), cudaMemcpyHostToDevice, st));
+    DYN_CUDA_TRY(cudaMemcpyAsync(ws + off_tuples, tuples.data(), size_t(K) * sizeof(uint2), cudaMemcpyHostToDevice, st));
     DYN_CUDA_TRY(launch_resolve(rp, lay, d_ws, st));
     DYN_CUDA_TRY(launch_mixed(lay, d_ws, off_tuples, off_caph, K, d_load, tiles, out->d_counts, out->d_freq,
                               out->d_tuple, out->d_best_E, st));

@@ -1,15 +1,24 @@
 // Pools that mix tensor parallelisms [Sec. 4.1, Eq. 1 in full]: counts N^{TP_i} per parallelism under the GPU
 // budget sum_i TP_i*N^{TP_i} <= N, one frequency per parallelism, the load shared out over the groups, the
 // objective sum_i N^{TP_i} * Energy^{TP_i, f_i}(L^{TP_i}).  The paper gives this to a solver; here the count
-// tuples are enumerated: the host lists the tuples within the budget (odometer order, smallest TP fastest),
-// a warp takes a tile, its lanes take every 32nd tuple.  For a tuple the load is split in proportion to the
+// tuples are enumerated: the host lists the tuples within the budget (numbered in odometer order, smallest TP
+// fastest) and sorts the list by the set of parallelisms in use, so that the 32 tuples a warp handles at once
+// mostly take the same branches; a warp takes a tile, lane l takes tuples l, l + 32, ... of the sorted list.  For a tuple the load is split in proportion to the
 // groups' capacity at the highest candidate frequency, each group then picks its own feasible frequency of
 // least energy (the single-type evaluation at fixed n and TP), and the tuple's energy is the sum.  The warp
 // keeps the tuple of least energy, lowest tuple number on ties.
 //
-// Work per tile is (tuples) x (TP degrees in use) x F single-type evaluations on the general-path tables,
-// read through L1 (they are a few tens of KB); the loads and results are 4 + 12 + 8T bytes per tile.
+// Work per tile is (tuples) x (TP degrees in use) x F single-type evaluations; the loads and results are
+// 4 + 12 + 8T bytes per tile.  The energy of a group is n x (energy of one instance at its per-instance load l),
+// and l = (L/A) x capH_t, so for one TP degree the 32 x 4 tuples a warp holds are 128 per-instance loads run
+// against that degree's F table rows: the inner loop of the single-type sweep.  When every TBT row is
+// monotone in load (the resolve step's flags) and the threshold tables fit in shared memory, the kernel uses
+// that loop (compare on l, segment address from a subnormal FMA, one FMA per candidate, predicated min) and
+// recovers the frequencies of the winning tuple afterwards with the same arithmetic; otherwise a plain
+// variant evaluates from the general-path tables through L1.  Both are launched; each looks at the flags
+// and only the one they select does the work.
 #include "dyn_internal.cuh"
+#include "eval_dev.cuh"
 
 #include <math_constants.h>
 
@@ -19,14 +28,16 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
-constexpr unsigned kFull = 0xffffffffu;
 
 struct MixedArgs {
     const float4 *rows;       // [C][P][M+1]
     const float2 *pairc;      // [C][P]
+    const char *ws;           // scratch block (threshold tables at off_pair2 .. off_end)
+    int32_t off_pair2, off_rows2, off_end;
+    int32_t use_fast;         // threshold tables fit in shared memory
     const float *slo;         // [C]
     float *caph;              // [C][T] capacity at the highest candidate frequency
-    const uint32_t *tuples;   // [K]
+    const uint2 *tuples;      // [K] {counts, 8 bits per TP index; tuple number}, sorted by the set of TP indices in use
     const float *load;        // [tiles]
     int64_t tiles, K;
     int32_t C, T, F, M;
@@ -43,8 +54,16 @@ __global__ void mixed_caph_kernel(const MixedArgs a) {
     a.caph[i] = ic > 0.f ? float(double(a.M - 1) / (double(a.M) * double(ic))) : 0.f;
 }
 
+// true when every pair row has a load threshold (vlim is NaN for a row whose TBT decreases somewhere)
+__device__ __forceinline__ bool rows_monotone(const MixedArgs &a) {
+    int bad = 0;
+    for (int i = threadIdx.x; i < a.C * a.T * a.F; i += blockDim.x) bad |= isnan(__ldg(a.pairc + i).y) ? 1 : 0;
+    return __syncthreads_or(bad) == 0;
+}
+
 template <int T>
 __global__ void __launch_bounds__(kThreads) mixed_select_kernel(const MixedArgs a) {
+    if (a.use_fast && rows_monotone(a)) return;              // the threshold variant does this call
     const int lane = threadIdx.x & 31;
     const int P = T * a.F, RS = a.M + 1;
     const float Mf = float(a.M);
@@ -57,10 +76,11 @@ __global__ void __launch_bounds__(kThreads) mixed_select_kernel(const MixedArgs 
 #pragma unroll
         for (int t = 0; t < T; ++t) caph[t] = a.caph[c * T + t];
         float best = CUDART_INF_F;
-        int64_t bk = a.K;                                    // tuple number of the lane's best
+        uint32_t bnum = 0xffffffffu, btup = 0;               // number and counts of the lane's best tuple
         uint32_t bq = 0;                                     // its frequencies, 8 bits per TP index
         for (int64_t k = lane; k < a.K; k += 32) {
-            const uint32_t tup = __ldg(a.tuples + k);
+            const uint2 tk = __ldg(a.tuples + k);
+            const uint32_t tup = tk.x;
             float A = 0.f;
 #pragma unroll
             for (int t = 0; t < T; ++t) A = fmaf(float((tup >> (8 * t)) & 255u), caph[t], A);
@@ -87,17 +107,18 @@ __global__ void __launch_bounds__(kThreads) mixed_select_kernel(const MixedArgs 
                 E += eg;                                     // ascending TP index; +inf if the group has no frequency
                 qs |= qg << (8 * t);
             }
-            if (E < best) {                                  // ascending tuple number per lane
+            if (E < best || (E == best && tk.y < bnum)) {    // the list is not in number order: lowest number on ties
                 best = E;
-                bk = k;
+                bnum = tk.y;
+                btup = tup;
                 bq = qs;
             }
         }
         best += 0.f;                                         // -0 -> +0
         float Emin;
         asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(Emin) : "f"(best));
-        // lowest tuple number among the lanes that hold the minimum (numbers fit 32 bits: K <= 2^20)
-        const uint32_t kmin = __reduce_min_sync(kFull, best == Emin ? uint32_t(bk) : 0xffffffffu);
+        // lowest tuple number among the lanes that hold the minimum
+        const uint32_t kmin = __reduce_min_sync(kFull, best == Emin ? bnum : 0xffffffffu);
         if (Emin == CUDART_INF_F) {
             if (lane < T) {
                 a.counts[i * T + lane] = -1;
@@ -109,13 +130,158 @@ __global__ void __launch_bounds__(kThreads) mixed_select_kernel(const MixedArgs 
             }
             continue;
         }
-        if (best == Emin && uint32_t(bk) == kmin) {          // exactly one lane: tuple numbers are distinct
-            const uint32_t tup = __ldg(a.tuples + bk);
+        if (best == Emin && bnum == kmin) {                  // exactly one lane: tuple numbers are distinct
 #pragma unroll
             for (int t = 0; t < T; ++t) {
-                const uint32_t n = (tup >> (8 * t)) & 255u;
+                const uint32_t n = (btup >> (8 * t)) & 255u;
                 a.counts[i * T + t] = int32_t(n);
                 a.freq[i * T + t] = n ? int32_t((bq >> (8 * t)) & 255u) : -1;
+            }
+            a.tuple[i] = int32_t(kmin);
+            a.best_E[i] = Emin;
+        }
+    }
+}
+
+
+// threshold variant: tables of all classes in shared memory, four tuples per lane and pass
+template <int T>
+__global__ void __launch_bounds__(kThreads) mixed_fast_kernel(const MixedArgs a) {
+    if (!rows_monotone(a)) return;                           // the plain variant does this call
+    extern __shared__ float4 smem[];
+    {
+        const float4 *src = reinterpret_cast<const float4 *>(a.ws + a.off_pair2);
+        const int n16 = (a.off_end - a.off_pair2) / 16;
+        for (int i = threadIdx.x; i < n16; i += blockDim.x) smem[i] = src[i];
+        __syncthreads();
+    }
+    uint32_t origin = table_origin<true>();
+    asm volatile("" : "+r"(origin) : : "memory");        // table loads stay behind the staging barrier
+    const int lane = threadIdx.x & 31;
+    const int F = a.F, P = T * F, RS = a.M + 1;
+    const uint32_t pstep = uint32_t(RS) * 8u;
+    const uint32_t rows2 = origin + uint32_t(a.off_rows2 - a.off_pair2);
+    const uint64_t two23_2 = pack2(kTwo23, kTwo23);
+    const uint64_t eight2 = pack2(units(8u), units(8u));
+    const float offs = float(int(pstep)) * units(1u);
+    const uint64_t off2_step = pack2(offs, offs);
+    const int64_t nwarps = int64_t(gridDim.x) * kWarps;
+    for (int64_t i = int64_t(blockIdx.x) * kWarps + (threadIdx.x >> 5); i < a.tiles; i += nwarps) {
+        const int c = int(i % a.C);
+        const float L = fmaxf(a.load[i], 0.f);              // negative / NaN -> 0
+        float caph[T];
+#pragma unroll
+        for (int t = 0; t < T; ++t) caph[t] = a.caph[c * T + t];
+        float best = CUDART_INF_F, bfrac = 0.f;
+        uint32_t bnum = 0xffffffffu, btup = 0;
+        for (int64_t base = 0; base < a.K; base += 128) {
+            uint32_t tup[4], num[4];
+            float frac[4], E[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int64_t k = base + j * 32 + lane;
+                const uint2 tk = k < a.K ? __ldg(a.tuples + k) : make_uint2(0u, 0xffffffffu);
+                tup[j] = tk.x;
+                num[j] = tk.y;
+                float A = 0.f;
+#pragma unroll
+                for (int t = 0; t < T; ++t) A = fmaf(float((tk.x >> (8 * t)) & 255u), caph[t], A);
+                frac[j] = L / A;                             // every instance at this fraction of its top-frequency capacity
+                E[j] = tk.x ? 0.f : CUDART_INF_F;            // a slot past the end of the list never wins
+            }
+#pragma unroll
+            for (int t = 0; t < T; ++t) {
+                uint32_t n[4];
+                float ln[4], e1[4];
+                uint32_t any = 0;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    n[j] = (tup[j] >> (8 * t)) & 255u;
+                    any |= n[j];
+                    ln[j] = n[j] ? frac[j] * caph[t] : CUDART_INF_F;      // no instance of this degree: nothing to serve
+                    e1[j] = CUDART_INF_F;
+                }
+                if (!__any_sync(kFull, any != 0)) continue;              // no tuple of the pass uses this degree
+                const uint64_t lnA = pack2(ln[0], ln[1]), lnB = pack2(ln[2], ln[3]);
+                const uint32_t cpair = origin + uint32_t(c * P + t * F) * 16u;
+                const float off0 = row_offset_units(rows2 + uint32_t((c * P + t * F) * RS) * 8u);
+                uint64_t off2 = pack2(off0, off0);
+#pragma unroll 4
+                for (int q = 0; q < F; ++q) {
+                    uint64_t icm2, lim2;
+                    asm("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(icm2), "=l"(lim2) : "r"(cpair + uint32_t(q) * 16u));
+                    const float lim = __uint_as_float(uint32_t(lim2));
+                    fast_two(lnA, icm2, off2, two23_2, eight2, lim, lim, e1[0], e1[1]);
+                    fast_two(lnB, icm2, off2, two23_2, eight2, lim, lim, e1[2], e1[3]);
+                    off2 = add2(off2, off2_step);
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (n[j]) E[j] += float(n[j]) * e1[j];   // ascending TP index; +inf if the group has no frequency
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (E[j] < best || (E[j] == best && num[j] < bnum)) {     // lowest tuple number on ties
+                    best = E[j];
+                    bnum = num[j];
+                    btup = tup[j];
+                    bfrac = frac[j];
+                }
+        }
+        best += 0.f;                                         // -0 -> +0
+        const float Emin = warp_min(best);
+        const uint32_t kmin = __reduce_min_sync(kFull, best == Emin ? bnum : 0xffffffffu);
+        if (Emin == CUDART_INF_F) {
+            if (lane < T) {
+                a.counts[i * T + lane] = -1;
+                a.freq[i * T + lane] = -1;
+            }
+            if (lane == 0) {
+                a.tuple[i] = -1;
+                a.best_E[i] = CUDART_INF_F;
+            }
+            continue;
+        }
+        // the winning tuple and its load fraction, from the lane that holds it (tuple numbers are distinct)
+        const int wl = __ffs(__ballot_sync(kFull, best == Emin && bnum == kmin)) - 1;
+        const uint32_t wt = __shfl_sync(kFull, btup, wl);
+        const float wf = __shfl_sync(kFull, bfrac, wl);
+        // its frequencies: lane p re-evaluates pair (t, q) = (p / F, p % F) with the same arithmetic; per degree
+        // the least energy, lowest q among equals
+        float gmin[T];
+        int gq[T];
+#pragma unroll
+        for (int t = 0; t < T; ++t) { gmin[t] = CUDART_INF_F; gq[t] = -1; }
+        for (int p0 = 0; p0 < P; p0 += 32) {
+            const int p = p0 + lane;
+            const int tp = p < P ? p / F : 0;
+            float val = CUDART_INF_F;
+            if (p < P && ((wt >> (8 * tp)) & 255u)) {
+                float ctp = caph[0];
+#pragma unroll
+                for (int t = 1; t < T; ++t) ctp = (t == tp) ? caph[t] : ctp;
+                const float4 pc = load16<true>(a.ws, origin + uint32_t(c * P + p) * 16u);
+                float e;
+                bool ok;
+                fast_one<true>(a.ws, rows2 + uint32_t((c * P + p) * RS) * 8u, wf * ctp, pc.x, pc.z, e, ok);
+                if (ok) val = e;
+            }
+#pragma unroll
+            for (int t = 0; t < T; ++t) {
+                const bool mine = p < P && tp == t;
+                const float m = warp_min(mine ? val : CUDART_INF_F);
+                if (m < gmin[t]) {                           // strictly better than the earlier rounds (lower q)
+                    gmin[t] = m;
+                    gq[t] = p0 + __ffs(__ballot_sync(kFull, mine && val == m)) - 1 - t * F;
+                }
+            }
+        }
+        if (lane == 0) {
+#pragma unroll
+            for (int t = 0; t < T; ++t) {
+                const uint32_t n = (wt >> (8 * t)) & 255u;
+                a.counts[i * T + t] = int32_t(n);
+                a.freq[i * T + t] = n ? gq[t] : -1;
             }
             a.tuple[i] = int32_t(kmin);
             a.best_E[i] = Emin;
@@ -134,7 +300,7 @@ cudaError_t launch_mixed(const ResolvedLayout &lay, void *d_ws, size_t off_tuple
     a.pairc = reinterpret_cast<const float2 *>(ws + lay.off_pairc);
     a.slo = reinterpret_cast<const float *>(ws + lay.off_slo);
     a.caph = reinterpret_cast<float *>(ws + off_caph);
-    a.tuples = reinterpret_cast<const uint32_t *>(ws + off_tuples);
+    a.tuples = reinterpret_cast<const uint2 *>(ws + off_tuples);
     a.load = d_load;
     a.tiles = tiles; a.K = K;
     a.C = lay.C; a.T = lay.T; a.F = lay.F; a.M = lay.M;
@@ -145,15 +311,31 @@ cudaError_t launch_mixed(const ResolvedLayout &lay, void *d_ws, size_t off_tuple
     int64_t grid = (tiles + kWarps - 1) / kWarps;
     const int64_t cap = int64_t(sm_count()) * 8;
     if (grid > cap) grid = cap;
+    a.ws = ws;
+    a.off_pair2 = int32_t(lay.off_pair2); a.off_rows2 = int32_t(lay.off_rows2); a.off_end = int32_t(lay.off_tp);
+    const size_t fast_bytes = lay.off_tp - lay.off_pair2;
+    a.use_fast = fast_bytes <= 96 * 1024 ? 1 : 0;
     e = record_start(st);
     if (e != cudaSuccess) return e;
+#define DYN_MIXED_LAUNCH(TT)                                                                                      \
+    do {                                                                                                          \
+        if (a.use_fast) {                                                                                         \
+            e = cudaFuncSetAttribute(mixed_fast_kernel<TT>, cudaFuncAttributeMaxDynamicSharedMemorySize,          \
+                                     int(fast_bytes));                                                            \
+            if (e != cudaSuccess) return e;                                                                       \
+            mixed_fast_kernel<TT><<<int(grid), kThreads, fast_bytes, st>>>(a);                                    \
+            if ((e = cudaGetLastError()) != cudaSuccess) return e;                                                \
+        }                                                                                                         \
+        mixed_select_kernel<TT><<<int(grid), kThreads, 0, st>>>(a);                                               \
+    } while (0)
     switch (lay.T) {
-        case 1: mixed_select_kernel<1><<<int(grid), kThreads, 0, st>>>(a); break;
-        case 2: mixed_select_kernel<2><<<int(grid), kThreads, 0, st>>>(a); break;
-        case 3: mixed_select_kernel<3><<<int(grid), kThreads, 0, st>>>(a); break;
-        case 4: mixed_select_kernel<4><<<int(grid), kThreads, 0, st>>>(a); break;
+        case 1: DYN_MIXED_LAUNCH(1); break;
+        case 2: DYN_MIXED_LAUNCH(2); break;
+        case 3: DYN_MIXED_LAUNCH(3); break;
+        case 4: DYN_MIXED_LAUNCH(4); break;
         default: return cudaErrorInvalidValue;
     }
+#undef DYN_MIXED_LAUNCH
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     return record_stop(st);
