@@ -338,7 +338,8 @@ size_t dyn_mixed_workspace_bytes(const dyn_profile *profile, const dyn_space *sp
     const size_t base = dyn_workspace_bytes(profile, space, S, W);
     const int64_t K = dyn_mixed_tuple_count(profile, space);
     if (!base || K <= 0) return 0;
-    return base + align256(size_t(K) * sizeof(uint2)) + align256(size_t(profile->C) * profile->T * sizeof(float));
+    return base + align256(size_t(K) * sizeof(uint2)) + align256(size_t(profile->C) * profile->T * sizeof(float)) +
+           align256(size_t(profile->C) * size_t(K) * sizeof(float));
 }
 
 int dyn_mixed_select(const dyn_profile *profile, const dyn_space *space, const float *d_load, int64_t S, int64_t W,
@@ -364,7 +365,8 @@ int dyn_mixed_select(const dyn_profile *profile, const dyn_space *space, const f
     std::stable_sort(tuples.begin(), tuples.end(), [&](const uint2 &x, const uint2 &y) { return mask_of(x) < mask_of(y); });
     const ResolvedLayout lay = resolved_layout(profile->C, profile->T, space->F, profile->M, space->Nmax, S, W);
     const size_t off_tuples = lay.total, off_caph = off_tuples + align256(size_t(K) * sizeof(uint2));
-    const size_t need = off_caph + align256(size_t(profile->C) * profile->T * sizeof(float));
+    const size_t off_inva = off_caph + align256(size_t(profile->C) * profile->T * sizeof(float));
+    const size_t need = off_inva + align256(size_t(profile->C) * size_t(K) * sizeof(float));
     rc = check_ws(d_ws, ws_bytes, need);
     if (rc != DYN_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -372,7 +374,7 @@ int dyn_mixed_select(const dyn_profile *profile, const dyn_space *space, const f
     // pageable host memory: the copy is staged before the call returns
     DYN_CUDA_TRY(cudaMemcpyAsync(ws + off_tuples, tuples.data(), size_t(K) * sizeof(uint2), cudaMemcpyHostToDevice, st));
     DYN_CUDA_TRY(launch_resolve(rp, lay, d_ws, st));
-    DYN_CUDA_TRY(launch_mixed(lay, d_ws, off_tuples, off_caph, K, d_load, tiles, out->d_counts, out->d_freq,
+    DYN_CUDA_TRY(launch_mixed(lay, d_ws, off_tuples, off_caph, off_inva, K, d_load, tiles, out->d_counts, out->d_freq,
                               out->d_tuple, out->d_best_E, st));
     SelectOut so{};
     so.best_idx = out->d_tuple; so.best_E = out->d_best_E; so.E_total = out->d_E_total; so.n_infeasible = out->d_n_infeasible;

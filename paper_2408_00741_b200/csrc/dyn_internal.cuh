@@ -109,7 +109,7 @@ cudaError_t launch_hier(const ResolveParams &rp, const ResolvedLayout &lay, void
                         int32_t *d_shard, int32_t *best_idx, float *best_E, cudaStream_t st);
 
 // pools that mix tensor parallelisms: `tuples` holds K count tuples, 8 bits per TP index
-cudaError_t launch_mixed(const ResolvedLayout &lay, void *d_ws, size_t off_tuples, size_t off_caph, int64_t K,
+cudaError_t launch_mixed(const ResolvedLayout &lay, void *d_ws, size_t off_tuples, size_t off_caph, size_t off_inva, int64_t K,
                          const float *d_load, int64_t tiles, int32_t *d_counts, int32_t *d_freq, int32_t *d_tuple,
                          float *d_best_E, cudaStream_t st);
 

@@ -37,6 +37,7 @@ struct MixedArgs {
     int32_t use_fast;         // threshold tables fit in shared memory
     const float *slo;         // [C]
     float *caph;              // [C][T] capacity at the highest candidate frequency
+    float *inva;              // [C][K] 1 / (sum_t n_t * capH_t) of every tuple (threshold variant)
     const uint2 *tuples;      // [K] {counts, 8 bits per TP index; tuple number}, sorted by the set of TP indices in use
     const float *load;        // [tiles]
     int64_t tiles, K;
@@ -59,6 +60,17 @@ __device__ __forceinline__ bool rows_monotone(const MixedArgs &a) {
     int bad = 0;
     for (int i = threadIdx.x; i < a.C * a.T * a.F; i += blockDim.x) bad |= isnan(__ldg(a.pairc + i).y) ? 1 : 0;
     return __syncthreads_or(bad) == 0;
+}
+
+// 1 / A of every (class, tuple): A = sum_t n_t * capH_t, the pool's capacity at the highest candidate frequency
+__global__ void mixed_inva_kernel(const MixedArgs a) {
+    const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= int64_t(a.C) * a.K) return;
+    const int c = int(i / a.K);
+    const uint32_t tup = a.tuples[i - int64_t(c) * a.K].x;
+    double A = 0.0;
+    for (int t = 0; t < a.T; ++t) A += double((tup >> (8 * t)) & 255u) * double(a.caph[c * a.T + t]);
+    a.inva[i] = float(1.0 / A);                              // +inf when no degree of the tuple has capacity: infeasible
 }
 
 template <int T>
@@ -146,7 +158,7 @@ __global__ void __launch_bounds__(kThreads) mixed_select_kernel(const MixedArgs 
 
 // threshold variant: tables of all classes in shared memory, four tuples per lane and pass
 template <int T>
-__global__ void __launch_bounds__(kThreads) mixed_fast_kernel(const MixedArgs a) {
+__global__ void __launch_bounds__(kThreads, 3) mixed_fast_kernel(const MixedArgs a) {
     if (!rows_monotone(a)) return;                           // the plain variant does this call
     extern __shared__ float4 smem[];
     {
@@ -183,10 +195,8 @@ __global__ void __launch_bounds__(kThreads) mixed_fast_kernel(const MixedArgs a)
                 const uint2 tk = k < a.K ? __ldg(a.tuples + k) : make_uint2(0u, 0xffffffffu);
                 tup[j] = tk.x;
                 num[j] = tk.y;
-                float A = 0.f;
-#pragma unroll
-                for (int t = 0; t < T; ++t) A = fmaf(float((tk.x >> (8 * t)) & 255u), caph[t], A);
-                frac[j] = L / A;                             // every instance at this fraction of its top-frequency capacity
+                // every instance runs at this fraction of its top-frequency capacity
+                frac[j] = k < a.K ? L * __ldg(a.inva + int64_t(c) * a.K + k) : 0.f;
                 E[j] = tk.x ? 0.f : CUDART_INF_F;            // a slot past the end of the list never wins
             }
 #pragma unroll
@@ -291,7 +301,7 @@ __global__ void __launch_bounds__(kThreads) mixed_fast_kernel(const MixedArgs a)
 
 }  // namespace
 
-cudaError_t launch_mixed(const ResolvedLayout &lay, void *d_ws, size_t off_tuples, size_t off_caph, int64_t K,
+cudaError_t launch_mixed(const ResolvedLayout &lay, void *d_ws, size_t off_tuples, size_t off_caph, size_t off_inva, int64_t K,
                          const float *d_load, int64_t tiles, int32_t *d_counts, int32_t *d_freq, int32_t *d_tuple,
                          float *d_best_E, cudaStream_t st) {
     char *ws = static_cast<char *>(d_ws);
@@ -300,6 +310,7 @@ cudaError_t launch_mixed(const ResolvedLayout &lay, void *d_ws, size_t off_tuple
     a.pairc = reinterpret_cast<const float2 *>(ws + lay.off_pairc);
     a.slo = reinterpret_cast<const float *>(ws + lay.off_slo);
     a.caph = reinterpret_cast<float *>(ws + off_caph);
+    a.inva = reinterpret_cast<float *>(ws + off_inva);
     a.tuples = reinterpret_cast<const uint2 *>(ws + off_tuples);
     a.load = d_load;
     a.tiles = tiles; a.K = K;
@@ -308,6 +319,8 @@ cudaError_t launch_mixed(const ResolvedLayout &lay, void *d_ws, size_t off_tuple
     mixed_caph_kernel<<<(lay.C * lay.T + 127) / 128, 128, 0, st>>>(a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess || tiles == 0) return e;
+    mixed_inva_kernel<<<unsigned((int64_t(lay.C) * K + 255) / 256), 256, 0, st>>>(a);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
     int64_t grid = (tiles + kWarps - 1) / kWarps;
     const int64_t cap = int64_t(sm_count()) * 8;
     if (grid > cap) grid = cap;
