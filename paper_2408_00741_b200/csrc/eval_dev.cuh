@@ -128,6 +128,41 @@ __device__ __forceinline__ void fast_two(uint64_t ln2, uint64_t icm2, uint64_t o
         : "l"(ln2), "l"(icm2), "l"(off2), "l"(two23_2), "l"(eight2), "f"(limA), "f"(limB));
 }
 
+// fast_two for the evaluate-only kernel: the pool energies n*e of the two candidates, +inf where infeasible
+__device__ __forceinline__ void fast_two_energy(uint64_t ln2, uint64_t icm2, uint64_t off2, uint64_t two23_2,
+                                                uint64_t eight2, float limA, float limB, float nfA, float nfB,
+                                                float &EA, float &EB) {
+    asm("{\n\t"
+        ".reg .pred pA, pB;\n\t"
+        ".reg .f32 lA, lB, a0, b0, a1, b1, eA, eB;\n\t"
+        ".reg .b32 zA, zB;\n\t"
+        ".reg .b64 y, z;\n\t"
+        "mov.b64 {lA, lB}, %2;\n\t"
+        "setp.le.f32 pA, lA, %7;\n\t"
+        "setp.le.f32 pB, lB, %8;\n\t"
+        "fma.rz.f32x2 y, %2, %3, %5;\n\t"
+        "fma.rn.f32x2 z, y, %6, %4;\n\t"
+        "mov.b64 {zA, zB}, z;\n\t"
+        "@pA ld.shared.b64 y, [zA];\n\t"
+        "@pB ld.shared.b64 z, [zB];\n\t"
+        "mov.b64 {a0, b0}, y;\n\t"
+        "mov.b64 {a1, b1}, z;\n\t"
+        "fma.rn.f32 eA, lA, b0, a0;\n\t"
+        "fma.rn.f32 eB, lB, b1, a1;\n\t"
+        "mul.rn.f32 eA, eA, %9;\n\t"
+        "mul.rn.f32 eB, eB, %10;\n\t"
+        "selp.f32 %0, eA, 0f7F800000, pA;\n\t"
+        "selp.f32 %1, eB, 0f7F800000, pB;\n\t"
+        "}"
+        : "=f"(EA), "=f"(EB)
+        : "l"(ln2), "l"(icm2), "l"(off2), "l"(two23_2), "l"(eight2), "f"(limA), "f"(limB), "f"(nfA), "f"(nfB));
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
 // the same evaluation for one candidate with ordinary address arithmetic (tables in shared memory or
 // read through L1), bit-identical to fast_two: e = a + l*b of segment floor(l*icm), ok = l <= lim.
 // `row` is the byte address / offset of the pair's row.  An infeasible candidate reads entry 0.

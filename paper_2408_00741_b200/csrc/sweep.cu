@@ -408,7 +408,8 @@ __device__ __forceinline__ void configs_body(const SweepArgs &a, const Tables tb
     uint32_t origin = table_origin<SMEM>();
     asm volatile("" : "+r"(origin) : : "memory");        // as in sweep_body: table loads stay behind the staging barrier
     const char *ws = a.ws;
-    const float4 *s_n4 = reinterpret_cast<const float4 *>(s_n);
+    const float4 *s_n4 = reinterpret_cast<const float4 *>(s_n);   // per pair of counts: {1/n, 1/(n+1), n, n+1}
+    const uint32_t sn_addr = uint32_t(__cvta_generic_to_shared(s_n));
 
     const int64_t nwarps = int64_t(gridDim.x) * kWarps;
     for (int64_t u = int64_t(blockIdx.x) * kWarps + (threadIdx.x >> 5); u < units_total; u += nwarps) {
@@ -434,11 +435,40 @@ __device__ __forceinline__ void configs_body(const SweepArgs &a, const Tables tb
             const int64_t q = int64_t(a.budget) / a.tp[pp / a.F];
             nlim = q < Nmax ? int(q) : Nmax;
         }
-        float *out = E_out + size_t(i) * size_t(a.J) + p;
-        int off = 0;                                  // (n - 1) * P, below J < 2^31
-        for (int n1 = 0; n1 < Nmax; n1 += 2, off += 2 * P) {
-            const float4 nn = s_n4[n1 >> 1];                       // {n, 1/n, n+1, 1/(n+1)}
-            const float lnA = L * nn.y, lnB = L * nn.w;
+        float *out = E_out + size_t(i) * size_t(a.J) + p;     // candidates of this pair are P floats apart
+        if (FAST && SMEM) {
+            // two instance counts per trip with the packed form of the fused kernel (same arithmetic)
+            const uint64_t L2 = pack2(L, L), icm2 = pack2(ic, ic);
+            const float off = row_offset_units(row);
+            const uint64_t off2 = pack2(off, off);
+            const uint64_t two23_2 = pack2(kTwo23, kTwo23), eight2 = pack2(units(8u), units(8u));
+            const int pairs = Nmax >> 1;
+#pragma unroll 4
+            for (int h = 0; h < pairs; ++h, out += 2 * P) {
+                uint64_t rn2, nf2;                            // {1/n, 1/(n+1)}, {n, n+1}
+                asm("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(rn2), "=l"(nf2) : "r"(sn_addr + uint32_t(h) * 16u));
+                const float limA = (!BUDGET || 2 * h + 1 <= nlim) ? lim : -1.f;
+                const float limB = (!BUDGET || 2 * h + 2 <= nlim) ? lim : -1.f;
+                float EA, EB;
+                fast_two_energy(mul2(L2, rn2), icm2, off2, two23_2, eight2, limA, limB, half_of(nf2, 0), half_of(nf2, 1),
+                                EA, EB);
+                if (active) {
+                    __stcs(out, EA);
+                    __stcs(out + P, EB);
+                }
+            }
+            if (Nmax & 1) {                               // odd count: the last n alone
+                const float4 nn = s_n4[pairs];
+                float e;
+                bool ok;
+                fast_one<SMEM>(ws, row, L * nn.x, ic, (!BUDGET || Nmax <= nlim) ? lim : -1.f, e, ok);
+                if (active) __stcs(out, ok ? e * nn.z : CUDART_INF_F);
+            }
+            continue;
+        }
+        for (int n1 = 0; n1 < Nmax; n1 += 2, out += 2 * P) {
+            const float4 nn = s_n4[n1 >> 1];                       // {1/n, 1/(n+1), n, n+1}
+            const float lnA = L * nn.x, lnB = L * nn.y;
             float eA, eB;
             bool okA, okB;
             if (FAST) {
@@ -453,8 +483,8 @@ __device__ __forceinline__ void configs_body(const SweepArgs &a, const Tables tb
                 okB = okB && n1 + 2 <= nlim;
             }
             if (active) {
-                __stcs(out + off, okA ? eA * nn.x : CUDART_INF_F);
-                if (n1 + 1 < Nmax) __stcs(out + off + P, okB ? eB * nn.z : CUDART_INF_F);
+                __stcs(out, okA ? eA * nn.z : CUDART_INF_F);
+                if (n1 + 1 < Nmax) __stcs(out + P, okB ? eB * nn.w : CUDART_INF_F);
             }
         }
     }
@@ -463,8 +493,13 @@ __device__ __forceinline__ void configs_body(const SweepArgs &a, const Tables tb
 template <bool BUDGET, bool SMEM>
 __global__ void __launch_bounds__(kThreads)
 eval_configs_kernel(const SweepArgs a, const int64_t units_total, float *__restrict__ E_out) {
-    __shared__ __align__(16) float2 s_n[258];         // {n, 1/n} for n = 1..Nmax (Nmax <= 256), padded to even
-    for (int n1 = threadIdx.x; n1 < a.Nmax + 1; n1 += kThreads) s_n[n1] = make_float2(float(n1 + 1), 1.0f / float(n1 + 1));
+    // for the counts (2h+1, 2h+2), h = 0..Nmax/2: {1/n, 1/(n+1), n, n+1} (Nmax <= 256)
+    __shared__ __align__(16) float2 s_n[258];
+    for (int h = threadIdx.x; h <= a.Nmax / 2; h += kThreads) {
+        const float n0 = float(2 * h + 1), n1 = float(2 * h + 2);
+        s_n[2 * h] = make_float2(1.0f / n0, 1.0f / n1);
+        s_n[2 * h + 1] = make_float2(n0, n1);
+    }
     Tables tb;
     tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.pair2 = a.off_pair2; tb.rows2 = a.off_rows2;
     if (all_rows_monotone(a)) {                      // load-threshold path: 8-byte lookups (also a barrier for s_n)
