@@ -219,7 +219,13 @@ cudaError_t launch_bin_trace(const BinParams &bp, const uint32_t *t_ms, const ui
     if (n_req > 0) {
         const uint64_t batches = (n_req + kBatch - 1) / kBatch;
         uint64_t grid = (batches + kWarps - 1) / kWarps;
-        const uint64_t max_grid = uint64_t(sm_count()) * 8;
+        // eight CTAs per SM for traces up to a few tens of millions of requests; beyond that more CTAs rather
+        // than longer slices (a slice of about 24 K requests streams best: measured 6.7 TB/s on 112 M requests
+        // against 5.5 TB/s with slices of 95 K)
+        uint64_t max_grid = uint64_t(sm_count()) * 8;
+        const uint64_t by_slice = (n_req + 24575) / 24576;
+        if (max_grid < by_slice) max_grid = by_slice;
+        if (max_grid > (uint64_t(1) << 30)) max_grid = uint64_t(1) << 30;
         if (grid > max_grid) grid = max_grid;
         const uint64_t chunk = ((batches + grid - 1) / grid) * kBatch;     // multiple of 128: keeps 16-byte alignment
         grid = (n_req + chunk - 1) / chunk;
