@@ -1,8 +1,12 @@
 // Hierarchical control [Sec. 4.2]: nodes per pool from the epoch's peak load (scale-out/in), sharding
 // at the highest frequency within those GPUs (shard-up/down), frequency per window (scale-up/down).
-// Same models and the same resolved tables as the joint sweep; each level is a small restricted search,
-// so these kernels are bound by reading the load matrix, not by arithmetic.
+// Same models and the same resolved tables as the joint sweep; each level is a small restricted search.
+// When every TBT row is monotone in load (the resolve step's flags) and the threshold tables fit in shared
+// memory, the sharding and frequency kernels evaluate candidates as the sweep's threshold path does (compare on
+// the per-instance load, 8-byte lookup of the energy line in shared memory); otherwise from the general-path
+// tables through L1.  Both variants are launched; each looks at the flags and only the selected one works.
 #include "dyn_internal.cuh"
+#include "eval_dev.cuh"
 
 #include <math_constants.h>
 
@@ -40,6 +44,9 @@ struct HierArgs {
     const float4 *rows;      // [C][P][M+1]
     const float2 *pairc;     // [C][P]
     const float *slo;        // [C]
+    const char *ws;          // scratch block (threshold tables at off_pair2 .. off_end)
+    int32_t off_pair2, off_rows2, off_end;
+    int32_t use_fast;        // the threshold tables fit in shared memory
     const double *ml;        // [C]
     const float *load;       // [S][W][C]
     int64_t S;
@@ -50,6 +57,68 @@ struct HierArgs {
     int32_t *nodes, *shard, *best_idx;
     float *best_E;
 };
+
+
+// true when every pair row has a load threshold (vlim is NaN for a row whose TBT decreases somewhere)
+__device__ __forceinline__ bool rows_monotone(const HierArgs &a) {
+    int bad = 0;
+    for (int i = threadIdx.x; i < a.C * a.T * a.F; i += blockDim.x) bad |= isnan(__ldg(a.pairc + i).y) ? 1 : 0;
+    return __syncthreads_or(bad) == 0;
+}
+
+// FAST kernels do the work iff the tables are monotone (and staged); the others iff not.  Returns false when
+// this kernel has nothing to do; for FAST it also stages pair2 | rows2 into shared memory.
+template <bool FAST>
+__device__ __forceinline__ bool hier_begin(const HierArgs &a) {
+    const bool mono = rows_monotone(a);
+    if (FAST) {
+        if (!mono) return false;
+        extern __shared__ float4 smem[];
+        const float4 *src = reinterpret_cast<const float4 *>(a.ws + a.off_pair2);
+        const int n16 = (a.off_end - a.off_pair2) / 16;
+        for (int i = threadIdx.x; i < n16; i += blockDim.x) smem[i] = src[i];
+        __syncthreads();
+        return true;
+    }
+    return !(a.use_fast && mono);
+}
+
+// pool energy of n instances of pair p (class c) at per-instance load ln; ok = within SLO and capacity
+template <bool FAST>
+__device__ __forceinline__ float hier_eval(const HierArgs &a, uint32_t origin, int c, int p, float ln, float nf, float slo,
+                                           bool &ok) {
+    const int P = a.T * a.F, RS = a.M + 1;
+    if (FAST) {
+        const float4 pc = load16<true>(a.ws, origin + uint32_t(c * P + p) * 16u);
+        float e;
+        fast_one<true>(a.ws, origin + uint32_t(a.off_rows2 - a.off_pair2) + uint32_t((c * P + p) * RS) * 8u, ln, pc.x, pc.z,
+                       e, ok);
+        return nf * e;
+    }
+    return eval_pair(a.rows + (size_t(c) * P + p) * RS, __ldg(&a.pairc[c * P + p]).x, float(a.M), ln, nf, slo, ok);
+}
+
+
+// Index of the (epoch or window, class) pair a thread serves among `n_items` epochs/windows.  The plain
+// variants take x = item*C + c in thread order (neighbouring threads read neighbouring loads).  The
+// staging variants give a warp ONE class and 32 consecutive items, so that the lanes of a lookup read the same
+// few table rows in shared memory instead of rows of nine classes (bank conflicts); the strided loads and
+// stores of the nine warps that share a block of items meet in L1 / L2.
+template <bool FAST>
+__device__ __forceinline__ bool hier_item(const HierArgs &a, uint32_t n_items, uint32_t &item, uint32_t &c) {
+    const uint32_t y = blockIdx.x * blockDim.x + threadIdx.x;
+    if (FAST) {
+        const uint32_t g = y >> 5;
+        const uint32_t blk = fastdiv(g, a.divC);
+        c = g - blk * a.C;
+        item = blk * 32u + (y & 31u);
+        return item < n_items;
+    }
+    if (y >= n_items * uint32_t(a.C)) return false;
+    item = fastdiv(y, a.divC);
+    c = y - item * a.C;
+    return true;
+}
 
 // grid: x over the (epoch or window, class) pairs of one scenario, y over scenarios (strided)
 
@@ -74,14 +143,17 @@ __global__ void __launch_bounds__(256) hier_nodes_kernel(const HierArgs a) {
 
 // one thread per (s, k2, c): neighbouring threads are neighbouring classes, so the loads coalesce; the
 // node budget cuts the (n, TP) space to a few dozen candidates, walked in index order
+template <bool FAST>
 __global__ void __launch_bounds__(256) hier_shard_kernel(const HierArgs a) {
-    const uint32_t x = blockIdx.x * blockDim.x + threadIdx.x;              // k2 * C + c
-    if (x >= uint32_t(a.K2 * a.C)) return;
-    const uint32_t k2 = fastdiv(x, a.divC), c = x - k2 * a.C;
+    if (!hier_begin<FAST>(a)) return;
+    uint32_t origin = table_origin<FAST>();
+    asm volatile("" : "+r"(origin) : : "memory");        // table loads stay behind the staging barrier
+    uint32_t k2, c;
+    if (!hier_item<FAST>(a, uint32_t(a.K2), k2, c)) return;
+    const uint32_t x = k2 * a.C + c;
     const int w0 = int(k2) * a.e2, w1 = min(w0 + a.e2, a.W);
     const uint32_t k1 = fastdiv(uint32_t(w0), a.divE1);
-    const int P = a.T * a.F, RS = a.M + 1;
-    const float Mf = float(a.M), slo = a.slo[c];
+    const float slo = a.slo[c];
     const int tpmax = a.tp[a.T - 1];
     const int cap_budget = a.Nmax * tpmax;            // a larger budget changes nothing
     for (int64_t s = blockIdx.y; s < a.S; s += gridDim.y) {
@@ -101,7 +173,7 @@ __global__ void __launch_bounds__(256) hier_shard_kernel(const HierArgs a) {
                 if (n * a.tp[t] > budget) break;      // TP ascending
                 const int p = t * a.F + a.F - 1;
                 bool ok;
-                const float E = eval_pair(a.rows + (size_t(c) * P + p) * RS, __ldg(&a.pairc[c * P + p]).x, Mf, ln, nf, slo, ok);
+                const float E = hier_eval<FAST>(a, origin, int(c), p, ln, nf, slo, ok);
                 if (ok && E < best) {                 // ascending (n, t): strict compare keeps the lowest index
                     best = E;
                     bnt = (n - 1) * a.T + t;
@@ -113,13 +185,16 @@ __global__ void __launch_bounds__(256) hier_shard_kernel(const HierArgs a) {
 }
 
 // one thread per (s, w, c): the frequency for the sharding of its shard epoch
+template <bool FAST>
 __global__ void __launch_bounds__(256) hier_freq_kernel(const HierArgs a) {
-    const uint32_t x = blockIdx.x * blockDim.x + threadIdx.x;              // w * C + c
-    if (x >= uint32_t(a.W * a.C)) return;
-    const uint32_t w = fastdiv(x, a.divC), c = x - w * a.C;
+    if (!hier_begin<FAST>(a)) return;
+    uint32_t origin = table_origin<FAST>();
+    asm volatile("" : "+r"(origin) : : "memory");        // table loads stay behind the staging barrier
+    uint32_t w, c;
+    if (!hier_item<FAST>(a, uint32_t(a.W), w, c)) return;
+    const uint32_t x = w * a.C + c;
     const uint32_t k2 = fastdiv(w, a.divE2);
-    const int P = a.T * a.F, RS = a.M + 1;
-    const float Mf = float(a.M), slo = a.slo[c];
+    const float slo = a.slo[c];
     for (int64_t s = blockIdx.y; s < a.S; s += gridDim.y) {
         const size_t i = size_t(s) * size_t(a.W) * a.C + x;
         const int nt = a.shard[size_t(s) * size_t(a.K2) * a.C + k2 * a.C + c];
@@ -129,11 +204,9 @@ __global__ void __launch_bounds__(256) hier_freq_kernel(const HierArgs a) {
             const int n1 = int(fastdiv(uint32_t(nt), a.divT)), t = nt - n1 * a.T;
             const float nf = float(n1 + 1);
             const float ln = fmaxf(a.load[i], 0.f) * (1.0f / nf);
-            const float4 *rows_t = a.rows + (size_t(c) * P + t * a.F) * RS;
-            const float2 *pc_t = a.pairc + c * P + t * a.F;
             for (int q = 0; q < a.F; ++q) {
                 bool ok;
-                const float E = eval_pair(rows_t + size_t(q) * RS, __ldg(pc_t + q).x, Mf, ln, nf, slo, ok);
+                const float E = hier_eval<FAST>(a, origin, int(c), t * a.F + q, ln, nf, slo, ok);
                 if (ok && E < best) {
                     best = E;
                     bj = nt * a.F + q;
@@ -170,13 +243,37 @@ cudaError_t launch_hier(const ResolveParams &rp, const ResolvedLayout &lay, void
     a.nodes = d_nodes; a.shard = d_shard; a.best_idx = best_idx; a.best_E = best_E;
     const unsigned gy = unsigned(S < 32768 ? S : 32768);
     const int64_t n1 = int64_t(a.K1) * lay.C, n2 = int64_t(a.K2) * lay.C, n3 = W * lay.C;
+    a.ws = ws;
+    a.off_pair2 = int32_t(lay.off_pair2); a.off_rows2 = int32_t(lay.off_rows2); a.off_end = int32_t(lay.off_tp);
+    const size_t fast_bytes = lay.off_tp - lay.off_pair2;
+    a.use_fast = fast_bytes <= 96 * 1024 ? 1 : 0;
+    // the staging variants run about eight CTAs per SM, each walking many scenarios, so that the tables are
+    // staged a few thousand times per call rather than once per 256 tiles
+    auto few = [&](int64_t blocks_x) {
+        int64_t g = (int64_t(sm_count()) * 8 + blocks_x - 1) / blocks_x;
+        return unsigned(g < 1 ? 1 : (g > int64_t(gy) ? int64_t(gy) : g));
+    };
+    if (a.use_fast) {
+        if ((e = cudaFuncSetAttribute(hier_shard_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(fast_bytes))) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(hier_freq_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(fast_bytes))) != cudaSuccess) return e;
+    }
     hier_nodes_kernel<<<dim3(unsigned((n1 + 255) / 256), gy), 256, 0, st>>>(a);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    hier_shard_kernel<<<dim3(unsigned((n2 + 255) / 256), gy), 256, 0, st>>>(a);
+    // staging variants: a warp per (32 items, class)
+    const int64_t f2 = ((int64_t(a.K2) + 31) / 32 * lay.C * 32 + 255) / 256, f3 = ((W + 31) / 32 * lay.C * 32 + 255) / 256;
+    if (a.use_fast) {
+        hier_shard_kernel<true><<<dim3(unsigned(f2), few(f2)), 256, fast_bytes, st>>>(a);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
+    hier_shard_kernel<false><<<dim3(unsigned((n2 + 255) / 256), a.use_fast ? few((n2 + 255) / 256) : gy), 256, 0, st>>>(a);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     e = record_start(st);
     if (e != cudaSuccess) return e;
-    hier_freq_kernel<<<dim3(unsigned((n3 + 255) / 256), gy), 256, 0, st>>>(a);
+    if (a.use_fast) {
+        hier_freq_kernel<true><<<dim3(unsigned(f3), few(f3)), 256, fast_bytes, st>>>(a);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
+    hier_freq_kernel<false><<<dim3(unsigned((n3 + 255) / 256), a.use_fast ? few((n3 + 255) / 256) : gy), 256, 0, st>>>(a);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     return record_stop(st);
 }

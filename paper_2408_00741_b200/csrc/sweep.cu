@@ -464,8 +464,7 @@ __device__ __forceinline__ void configs_body(const SweepArgs &a, const Tables tb
                 fast_one<SMEM>(ws, row, L * nn.x, ic, (!BUDGET || Nmax <= nlim) ? lim : -1.f, e, ok);
                 if (active) __stcs(out, ok ? e * nn.z : CUDART_INF_F);
             }
-            continue;
-        }
+        } else
         for (int n1 = 0; n1 < Nmax; n1 += 2, out += 2 * P) {
             const float4 nn = s_n4[n1 >> 1];                       // {1/n, 1/(n+1), n, n+1}
             const float lnA = L * nn.x, lnB = L * nn.y;
