@@ -252,3 +252,21 @@ def mixed_select(profile, space, load):
     if rc != 0:
         raise ValueError("orc_mixed_select: invalid argument (a GPU budget > 0 is required)")
     return out
+
+
+def reconf_select(profile, space, R, load):
+    """Selection with re-configuration costs: R float32 [NS][NS] (Wh, NS = n_max*T, state = (n-1)*T + t).
+    dict(best_idx[S][W][C], best_E[S][W][C], path_total[S][C])."""
+    lib = _load()
+    p, s, keep = _structs(profile, space)
+    load = _arr(load, np.float32)
+    S, W, Cn = load.shape
+    NS = int(space.n_max) * int(p.T)
+    R = _arr(R, np.float32)
+    assert R.shape == (NS, NS) and Cn == p.C
+    out = dict(best_idx=np.empty((S, W, Cn), np.int32), best_E=np.empty((S, W, Cn)), path_total=np.empty((S, Cn)))
+    rc = lib.orc_reconf_select(C.byref(p), C.byref(s), _p(R), _p(load), C.c_int64(S), C.c_int64(W),
+                               _p(out["best_idx"]), _p(out["best_E"]), _p(out["path_total"]))
+    if rc != 0:
+        raise ValueError("orc_reconf_select: invalid argument")
+    return out

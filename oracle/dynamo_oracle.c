@@ -26,6 +26,8 @@
  *                     of chosen configurations [Sec. 6 cluster-level energy, GPUs per sharding].
  *   orc_mixed_select  Eq. 1 in full: a pool that mixes tensor parallelisms (counts per TP under a GPU
  *                     budget, load split by capacity, one frequency per TP), by enumeration.
+ *   orc_reconf_select selection that counts the cost of re-configuring between windows (overhead table):
+ *                     a shortest path over the windows, states = shardings, frequency free per window.
  *   orc_hier_select   the controller hierarchy of Sec. 4.2 on the same models: nodes per pool from the
  *                     epoch's peak load and the per-node maximum load (ceil(PL/ML)), sharding at the
  *                     highest frequency within those GPUs, then the frequency per window.
@@ -533,6 +535,90 @@ int orc_mixed_select(const orc_profile *p, const orc_space *sp, const float *loa
         best_E[i] = eb;
         if (E2) E2[i] = e2nd;
         if (margin) margin[i] = mg;
+    }
+    free(row); free(wt);
+    return ORC_OK;
+}
+
+/* ---- selection that accounts for the cost of re-configuring (Sec. 4.2, "Accounting for the overheads") ---- */
+
+/*
+ * The controllers weigh the energy a new configuration saves against the cost of getting there, which they
+ * read from an Overhead Table [Sec. 4.2]; changing the sharding of an instance costs transfer time that depends
+ * on the source and destination parallelism [Sec. 4.3, table of re-sharding overheads], changing the frequency
+ * costs next to nothing [Sec. 4.3, "Scaling up/down the frequency"].  Here that trade-off is solved exactly for
+ * one (scenario, class) over the whole horizon.  Readings:
+ *   - a state is a sharding sigma = (n, TP index t), numbered sigma = (n-1)*T + t, NS = Nmax*T states;
+ *   - the frequency is free in every window: the cost of state sigma in window w is
+ *     cost_w(sigma) = min over q of E(w, n, t, q) (the evaluation of Eq. 1), lowest q on ties, +inf if none;
+ *   - moving from sigma' in window w-1 to sigma in window w costs R[sigma'][sigma] (Wh, the caller's overhead
+ *     table, NS x NS, used as given); the first window is free to start anywhere;
+ *   - the schedule minimises  sum_w cost_w(sigma_w) + sum_{w>=1} R[sigma_{w-1}][sigma_w]  (a shortest path
+ *     through the windows); forward recursion D_w(sigma) = cost_w(sigma) + min_{sigma'} (D_{w-1}(sigma') +
+ *     R[sigma'][sigma]) with the lowest sigma' on ties, last state the lowest sigma attaining the minimum;
+ *   - a (scenario, class) with a window in which no state is feasible has no schedule: indices -1, total +inf.
+ * Outputs: best_idx[S][W][C] = sigma_w*F + q_w (or -1), best_E[S][W][C] = cost_w(sigma_w) (+inf if none),
+ * path_total[S][C] = the minimised sum (window energies plus transition costs).
+ */
+int orc_reconf_select(const orc_profile *p, const orc_space *sp, const float *R, const float *load, int64_t S, int64_t W,
+                      int32_t *best_idx, double *best_E, double *path_total) {
+    const int32_t C = p->C, T = p->T, F = sp->F, Nmax = sp->Nmax;
+    const int64_t NS = (int64_t)Nmax * T;
+    int32_t *row = (int32_t *)malloc(sizeof(int32_t) * (size_t)F);
+    double *wt = (double *)malloc(sizeof(double) * (size_t)F);
+    int rc = orc_resolve(p->f_grid, p->R, sp->f_cand, F, row, wt);
+    if (rc != ORC_OK) { free(row); free(wt); return rc; }
+#pragma omp parallel for schedule(dynamic, 1) collapse(2)
+    for (int64_t s = 0; s < S; ++s) {
+        for (int32_t c = 0; c < C; ++c) {
+            double *cost = (double *)malloc(sizeof(double) * (size_t)(W * NS));
+            int32_t *qb = (int32_t *)malloc(sizeof(int32_t) * (size_t)(W * NS));
+            int32_t *from = (int32_t *)malloc(sizeof(int32_t) * (size_t)(W * NS));
+            double *D = (double *)malloc(sizeof(double) * (size_t)NS), *Dn = (double *)malloc(sizeof(double) * (size_t)NS);
+            /* window costs: the frequency of least energy for every sharding */
+            for (int64_t w = 0; w < W; ++w) {
+                const double L = (double)load[(s * W + w) * C + c];
+                for (int64_t g = 0; g < NS; ++g) {
+                    const int32_t n = (int32_t)(g / T) + 1, t = (int32_t)(g % T);
+                    double eb = INFINITY;
+                    int32_t bq = -1;
+                    for (int32_t q = 0; q < F; ++q) {
+                        const double e = eval_candidate(p, sp, row, wt, c, L, n, t, q, sp->gpu_budget, NULL);
+                        if (e < eb) { eb = e; bq = q; }
+                    }
+                    cost[w * NS + g] = eb;
+                    qb[w * NS + g] = bq;
+                }
+            }
+            /* shortest path through the windows */
+            for (int64_t g = 0; g < NS; ++g) { D[g] = W > 0 ? cost[g] : 0.0; from[g] = -1; }
+            for (int64_t w = 1; w < W; ++w) {
+                for (int64_t g = 0; g < NS; ++g) {
+                    double best = INFINITY;
+                    int32_t arg = -1;
+                    for (int64_t h = 0; h < NS; ++h) {
+                        const double v = D[h] + (double)R[h * NS + g];
+                        if (v < best) { best = v; arg = (int32_t)h; }
+                    }
+                    Dn[g] = cost[w * NS + g] + best;
+                    from[w * NS + g] = arg;
+                }
+                double *tmp = D; D = Dn; Dn = tmp;
+            }
+            double tot = INFINITY;
+            int64_t g = -1;
+            for (int64_t h = 0; h < NS; ++h)
+                if (D[h] < tot) { tot = D[h]; g = h; }
+            path_total[s * C + c] = W > 0 ? tot : 0.0;
+            for (int64_t w = W - 1; w >= 0; --w) {
+                const int64_t i = (s * W + w) * C + c;
+                if (g < 0) { best_idx[i] = -1; best_E[i] = INFINITY; continue; }
+                best_idx[i] = (int32_t)(g * F + qb[w * NS + g]);
+                best_E[i] = cost[w * NS + g];
+                g = from[w * NS + g];
+            }
+            free(cost); free(qb); free(from); free(D); free(Dn);
+        }
     }
     free(row); free(wt);
     return ORC_OK;
