@@ -238,6 +238,35 @@ int dyn_mixed_select(const dyn_profile *profile, const dyn_space *space, const f
                      const dyn_mixed_out *out, void *d_ws, size_t ws_bytes, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Selection that counts the cost of re-configuring.  [Sec. 4.2 "Accounting for the overheads": the transition
+ * overheads are kept in an Overhead Table, and a controller sets the energy a new configuration saves against the
+ * cost of getting there; Sec. 4.3: what a re-sharding costs depends on the source and destination parallelism
+ * (table of re-sharding overheads), a frequency change costs next to nothing.]
+ *
+ * Per scenario s and class c the call finds the schedule over all W windows of least total cost:
+ *   - a state is a sharding sigma = (n-1)*T + t (n instances of TP index t), NS = Nmax*T states (NS <= 1024);
+ *   - the cost of state sigma in window w is the least energy over the candidate frequencies q of candidate
+ *     (n, t, q) at the window's load (evaluation and constraints as for dyn_eval_configs, gpu_budget included),
+ *     lowest q on ties, +inf if none is feasible;
+ *   - moving from sigma' in window w-1 to sigma in window w costs d_R[sigma'][sigma] (Wh; the caller's overhead
+ *     table, device float [NS][NS], used as given, entries >= 0 expected); the first window starts anywhere;
+ *   - minimise  sum_w cost_w(sigma_w) + sum_{w>=1} d_R[sigma_{w-1}][sigma_w];  among schedules of equal cost the
+ *     forward recursion keeps the lowest predecessor and the lowest final state.
+ * Results: out->d_best_idx[s][w][c] = sigma_w*F + q_w and out->d_best_E = cost_w(sigma_w); if some window of
+ * (s, c) has no feasible state there is no schedule: -1 / +inf in all its windows.  Totals in `out` as in
+ * dyn_select (window energies only); d_path_total[s][c] (double, required) is the minimised sum including the
+ * transition costs (+inf without a schedule).  Arithmetic: fp32 window costs; the running path costs are held as
+ * fp32 differences to their minimum, the minimum itself in fp64.
+ * Workspace: dyn_reconf_workspace_bytes() (7 bytes per (s, c, w, sigma) plus the resolved tables).
+ * Errors: as dyn_eval_select, plus DYN_EINVAL for NULL d_R / d_path_total, DYN_EUNSUPPORTED for NS > 1024 or
+ * F > 256.
+ * ------------------------------------------------------------------------------------------- */
+size_t dyn_reconf_workspace_bytes(const dyn_profile *profile, const dyn_space *space, int64_t S, int64_t W);
+int dyn_reconf_select(const dyn_profile *profile, const dyn_space *space, const float *d_R, const float *d_load,
+                      int64_t S, int64_t W, const dyn_select_out *out, double *d_path_total, void *d_ws,
+                      size_t ws_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Whole path from HOST buffers: (a) -> (b) -> (c) in one call.  [Sec. 3 trace -> Sec. 3.2 loads ->
  * Sec. 4.1 / Eq. 1 evaluation -> Sec. 4.2 selection -> Sec. 6 totals]
  *

@@ -25,7 +25,7 @@ DYN_OK, DYN_EINVAL, DYN_ECUDA, DYN_EUNSUPPORTED, DYN_EWORKSPACE = 0, -1, -2, -3,
 EXPORTS = ("dyn_strerror", "dyn_last_cuda_error", "dyn_bin_trace", "dyn_workspace_bytes", "dyn_eval_configs",
            "dyn_select_workspace_bytes", "dyn_select", "dyn_eval_select", "dyn_pipeline_arena_bytes",
            "dyn_pipeline_host", "dyn_set_timing_events", "dyn_eval_select_static", "dyn_hier_workspace_bytes",
-           "dyn_hier_select", "dyn_mixed_workspace_bytes", "dyn_mixed_tuple_count", "dyn_mixed_select")
+           "dyn_hier_select", "dyn_mixed_workspace_bytes", "dyn_mixed_tuple_count", "dyn_mixed_select", "dyn_reconf_workspace_bytes", "dyn_reconf_select")
 
 
 class DynError(RuntimeError):
@@ -134,6 +134,11 @@ _lib.dyn_mixed_tuple_count.argtypes = [C.POINTER(_Profile), C.POINTER(_Space)]
 _lib.dyn_mixed_select.restype = C.c_int
 _lib.dyn_mixed_select.argtypes = [C.POINTER(_Profile), C.POINTER(_Space), C.c_void_p, C.c_int64, C.c_int64,
                                   C.POINTER(_MixedOut), C.c_void_p, C.c_size_t, C.c_void_p]
+_lib.dyn_reconf_workspace_bytes.restype = C.c_size_t
+_lib.dyn_reconf_workspace_bytes.argtypes = [C.POINTER(_Profile), C.POINTER(_Space), C.c_int64, C.c_int64]
+_lib.dyn_reconf_select.restype = C.c_int
+_lib.dyn_reconf_select.argtypes = [C.POINTER(_Profile), C.POINTER(_Space), C.c_void_p, C.c_void_p, C.c_int64, C.c_int64,
+                                   C.POINTER(_SelectOut), C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
 
 
 def _dev(t, dtype, what):
@@ -397,3 +402,19 @@ def dyn_mixed_select(profile: Profile, space: Space, d_load, out: MixedOut, d_ws
     rc = _lib.dyn_mixed_select(C.byref(p), C.byref(s), _dev(d_load, torch.float32, "d_load"), S, W, C.byref(o), ws, nb,
                                _stream())
     _check(rc, "dyn_mixed_select")
+
+
+def dyn_reconf_workspace_bytes(profile: Profile, space: Space, S, W) -> int:
+    p, s = profile._struct(), space._struct()
+    return int(_lib.dyn_reconf_workspace_bytes(C.byref(p), C.byref(s), int(S), int(W)))
+
+
+def dyn_reconf_select(profile: Profile, space: Space, d_R, d_load, out: SelectOut, d_path_total, d_ws):
+    """Selection with re-configuration costs: d_R float32 [NS][NS] (Wh), d_path_total float64 [S][C]."""
+    S, W, Cn = d_load.shape
+    p, s = profile._struct(), space._struct()
+    o = out._struct()
+    ws, nb = _ws(d_ws)
+    rc = _lib.dyn_reconf_select(C.byref(p), C.byref(s), _dev(d_R, torch.float32, "d_R"), _dev(d_load, torch.float32, "d_load"),
+                                S, W, C.byref(o), _dev(d_path_total, torch.float64, "d_path_total"), ws, nb, _stream())
+    _check(rc, "dyn_reconf_select")

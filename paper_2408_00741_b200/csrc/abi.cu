@@ -385,4 +385,41 @@ int dyn_mixed_select(const dyn_profile *profile, const dyn_space *space, const f
     return DYN_OK;
 }
 
+size_t dyn_reconf_workspace_bytes(const dyn_profile *profile, const dyn_space *space, int64_t S, int64_t W) {
+    const size_t base = dyn_workspace_bytes(profile, space, S, W);
+    if (!base) return 0;
+    const size_t n = size_t(S) * size_t(profile->C) * size_t(W) * size_t(space->Nmax) * size_t(profile->T);
+    return base + align256(n * sizeof(float)) + align256(n) + align256(n * sizeof(uint16_t));
+}
+
+int dyn_reconf_select(const dyn_profile *profile, const dyn_space *space, const float *d_R, const float *d_load,
+                      int64_t S, int64_t W, const dyn_select_out *out, double *d_path_total, void *d_ws,
+                      size_t ws_bytes, void *stream) {
+    ResolveParams rp;
+    int rc = check_problem(profile, space, S, W, &rp);
+    if (rc != DYN_OK) return rc;
+    const int64_t NS = int64_t(space->Nmax) * profile->T;
+    if (NS > 1024 || space->F > 256) return DYN_EUNSUPPORTED;
+    const int64_t tiles = S * W * profile->C;
+    rc = check_out(out, S, tiles);
+    if (rc != DYN_OK) return rc;
+    if (!d_R || (S > 0 && !d_path_total) || (tiles > 0 && !d_load)) return DYN_EINVAL;
+    const ResolvedLayout lay = resolved_layout(profile->C, profile->T, space->F, profile->M, space->Nmax, S, W);
+    const size_t n = size_t(S) * size_t(profile->C) * size_t(W) * size_t(NS);
+    const size_t off_cost = lay.total, off_q = off_cost + align256(n * sizeof(float)), off_from = off_q + align256(n);
+    rc = check_ws(d_ws, ws_bytes, off_from + align256(n * sizeof(uint16_t)));
+    if (rc != DYN_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char *ws = static_cast<char *>(d_ws);
+    DYN_CUDA_TRY(launch_resolve(rp, lay, d_ws, st));
+    DYN_CUDA_TRY(launch_reconf(lay, d_ws, off_cost, off_q, off_from, d_R, d_load, S, W, space->gpu_budget, out->d_best_idx,
+                               out->d_best_E, d_path_total, st));
+    const int64_t chunks = totals_chunks(W);
+    double *partial = reinterpret_cast<double *>(ws + lay.off_partial);
+    uint32_t *partial_bad = reinterpret_cast<uint32_t *>(ws + lay.off_partial + size_t(S) * size_t(chunks) * sizeof(double));
+    DYN_CUDA_TRY(launch_totals(to_out(out), S, W, profile->C, lay.J, nullptr, nullptr, profile->T, space->F,
+                               reinterpret_cast<const int32_t *>(ws + lay.off_tp), partial, partial_bad, st));
+    return DYN_OK;
+}
+
 }  // extern "C"
