@@ -391,6 +391,10 @@ def run_ours(args, rank, world, local_rank):
             result["mixed_pools"] = measure_mixed(dyn, gen, dev)
         except Exception as exc:
             result["mixed_pools"] = {"error": repr(exc)}
+        try:
+            result["reconfiguration"] = measure_reconf(dyn, gen, dev)
+        except Exception as exc:
+            result["reconfiguration"] = {"error": repr(exc)}
 
     if not args.no_cpu_baseline and world == 1:
         cb, _, _ = time_oracle(wl, trace, prof, sp, base_counts)
@@ -579,6 +583,57 @@ def measure_mixed(dyn, gen, dev, S=16, n_max=16, budget=16):
             "tiles_that_mix_parallelisms": mixed_frac}
 
 
+def measure_reconf(dyn, gen, dev, S=16):
+    """Selection with re-configuration costs on S day-long scenarios of the 1-day profile (256 shardings, 1440
+    windows): the path kernel alone; its work is W * NS^2 add-compare steps per (scenario, class)."""
+    import torch
+    wl = gen.workload("cfg2")
+    prof, sp = wl.profile(), wl.space()
+    W, Cn, J = wl.trace.n_windows, 9, wl.J
+    NS = sp.n_max * len(prof.tp)
+    load = torch.from_numpy(gen.random_loads((S, W, Cn), seed=13, mean=2.5)).to(dev)
+    R = np.random.default_rng(14).uniform(0.0, 5.0, (NS, NS)).astype(np.float32)
+    np.fill_diagonal(R, 0.0)
+    d_R = torch.from_numpy(R).to(dev)
+    P = dyn.Profile(prof.tp, prof.f_grid_mhz, prof.ttft, prof.cap, prof.tbt, prof.pow, device=dev)
+    SP = dyn.Space(sp.f_cand_mhz, sp.n_max, sp.slo_ttft_s, sp.slo_tbt_s, sp.window_s, sp.gpu_budget)
+    out = dyn.SelectOut(S, W, Cn, J, device=dev, windows=False, hist=False, gpus=False)
+    total = torch.empty((S, Cn), dtype=torch.float64, device=dev)
+    ws = torch.empty(dyn.dyn_reconf_workspace_bytes(P, SP, S, W), dtype=torch.uint8, device=dev)
+    call = lambda: dyn.dyn_reconf_select(P, SP, d_R, load, out, total, ws)
+    for _ in range(2):
+        call()
+    K = 5
+    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    for a, b in kev:
+        a.record(); b.record()
+    c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    c0.record()
+    for k in range(K):
+        dyn.dyn_set_timing_events(*kev[k])
+        call()
+    dyn.dyn_set_timing_events(None, None)
+    c1.record()
+    torch.cuda.synchronize()
+    ms = float(np.mean([a.elapsed_time(b) for a, b in kev]))
+    steps = S * Cn * (W - 1) * NS * NS                      # add + compare of the min-plus recursion
+    fp32_peak = SM_COUNT * FP32_LANES * 2 * SM_MAX_MHZ * 1e6 / 1e12
+    tfl = 2.0 * steps / (ms * 1e-3) / 1e12
+    # energy of the schedules against the per-window optimum that ignores transition costs
+    jout = dyn.SelectOut(S, W, Cn, J, device=dev, windows=False, hist=False, gpus=False)
+    jws = torch.empty(dyn.dyn_workspace_bytes(P, SP, S, W), dtype=torch.uint8, device=dev)
+    dyn.dyn_eval_select(P, SP, load, jout, jws)
+    torch.cuda.synchronize()
+    return {"workload": f"cfg2 profile x {S} scenarios, {NS} shardings, random overhead table 0..5 Wh", "problems": S * Cn,
+            "path_kernel_ms": ms, "call_ms": c0.elapsed_time(c1) / K, "minplus_steps": int(steps),
+            "steps_per_s": steps / (ms * 1e-3),
+            "roofline": {"bound": "alu", "achieved": tfl, "peak": fp32_peak, "unit": "TFLOP/s", "frac": tfl / fp32_peak,
+                         "traffic": None, "peak_source": "derived fp32 peak; 2 flop (add, compare) per step"},
+            "window_energy_over_free_optimum": float(out.E_total.sum().item() / jout.E_total.sum().item()),
+            "schedules": int(torch.isfinite(total).sum().item())}
+
+
 def main():
     args = parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -594,7 +649,8 @@ def main():
         dev = torch.device("cuda", local_rank)
         torch.cuda.set_device(dev)
         print(json.dumps({"bin_trace": measure_bin(dyn, gen, dev), "materialised": measure_materialised(dyn, gen, dev),
-                          "hierarchical": measure_hier(dyn, gen, dev), "mixed_pools": measure_mixed(dyn, gen, dev)}))
+                          "hierarchical": measure_hier(dyn, gen, dev), "mixed_pools": measure_mixed(dyn, gen, dev),
+                          "reconfiguration": measure_reconf(dyn, gen, dev)}))
         return
     run_ours(args, rank, world, local_rank)
 

@@ -257,7 +257,7 @@ int dyn_mixed_select(const dyn_profile *profile, const dyn_space *space, const f
  * dyn_select (window energies only); d_path_total[s][c] (double, required) is the minimised sum including the
  * transition costs (+inf without a schedule).  Arithmetic: fp32 window costs; the running path costs are held as
  * fp32 differences to their minimum, the minimum itself in fp64.
- * Workspace: dyn_reconf_workspace_bytes() (7 bytes per (s, c, w, sigma) plus the resolved tables).
+ * Workspace: dyn_reconf_workspace_bytes() (9 bytes per (s, c, w, sigma) plus the resolved tables).
  * Errors: as dyn_eval_select, plus DYN_EINVAL for NULL d_R / d_path_total, DYN_EUNSUPPORTED for NS > 1024 or
  * F > 256.
  * ------------------------------------------------------------------------------------------- */

@@ -114,7 +114,6 @@ cudaError_t launch_mixed(const ResolvedLayout &lay, void *d_ws, size_t off_tuple
                          float *d_best_E, cudaStream_t st);
 
 // selection with re-configuration costs (shortest path over the windows)
-size_t reconf_smem_bytes(int32_t NS);
 cudaError_t launch_reconf(const ResolvedLayout &lay, void *d_ws, size_t off_cost, size_t off_q, size_t off_from,
                           const float *d_R, const float *d_load, int64_t S, int64_t W, int32_t budget, int32_t *best_idx,
                           float *best_E, double *path_total, cudaStream_t st);

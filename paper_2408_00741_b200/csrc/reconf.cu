@@ -7,10 +7,10 @@
 // a move sigma' -> sigma between consecutive windows costs R[sigma'][sigma] (the caller's table, Wh).
 //   reconf_cost_kernel  cost[s][c][w][sigma] and the frequency that attains it: one thread per entry, a warp
 //                       covers 32 shardings of one tile (one load, the table rows of T degrees), F evaluations each
-//   reconf_path_kernel  one CTA per (scenario, class): forward recursion over the windows, a thread per target
-//                       state scanning all source states (min-plus product of the state vector with R, R read
-//                       through L1, the state vector in shared memory), back pointers to global memory; then the
-//                       walk back, 32 windows of pointers staged per step.  The running values are kept relative
+//   reconf_path_kernel  one CTA per (scenario, class): forward recursion over the windows (min-plus product of the
+//                       state vector with R: add + min per step; R in shared memory as far as it fits, the state
+//                       vector too), the vectors written to global memory; then the walk back by one warp, which
+//                       finds each predecessor again with the same addition.  The running values are kept relative
 //                       to their minimum, which is accumulated in fp64, so that fp32 holds only differences.
 #include "dyn_internal.cuh"
 
@@ -21,7 +21,6 @@ namespace dyn {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kBack = 32;                       // windows of back pointers staged per step of the walk back
 
 struct ReconfArgs {
     const float4 *rows;       // [C][P][M+1]
@@ -32,7 +31,7 @@ struct ReconfArgs {
     const float *load;        // [S][W][C]
     float *cost;              // [S][C][W][NS]
     uint8_t *qbest;           // [S][C][W][NS]
-    uint16_t *from;           // [S][C][W][NS]
+    float *hist;              // [S][C][W][NS] running values relative to their minimum, window by window
     int64_t S, W;
     int32_t C, T, F, M, Nmax, NS, budget;
     int32_t *best_idx;
@@ -74,7 +73,10 @@ __global__ void __launch_bounds__(kThreads) reconf_cost_kernel(const ReconfArgs 
     }
 }
 
-// block-wide minimum of v (all threads get it); `red` holds kThreads / 32 floats
+constexpr int kPathThreads = 512;
+constexpr int kRegRows = 6;                     // rows of R a thread keeps in registers (its four columns of them)
+
+// block-wide minimum of v (all threads get it); `red` holds kPathThreads / 32 floats
 __device__ __forceinline__ float block_min(float v, float *red) {
     float m;
     asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(m) : "f"(v));
@@ -83,111 +85,193 @@ __device__ __forceinline__ float block_min(float v, float *red) {
     __syncthreads();
     float r = red[0];
 #pragma unroll
-    for (int i = 1; i < kThreads / 32; ++i) r = fminf(r, red[i]);
+    for (int i = 1; i < kPathThreads / 32; ++i) r = fminf(r, red[i]);
     return r;
 }
 
-// dynamic shared memory: D[2][NS] floats | back[kBack][NS] uint16 | path[kBack] int32
-__global__ void __launch_bounds__(kThreads) reconf_path_kernel(const ReconfArgs a) {
+// R[h][g]: the first rows_s rows sit in shared memory with row stride NS4 + 4 floats (rows stay 16-byte aligned;
+// NS4 = NS rounded up to a multiple of 4), the rest is read through L1 / L2
+__device__ __forceinline__ float r_at(const float *Rs, const float *R, int rows_s, int NS, int NS4, int h, int g) {
+    return h < rows_s ? Rs[h * (NS4 + 4) + g] : __ldg(R + size_t(h) * NS + g);
+}
+
+// One CTA per (scenario, class).  Dynamic shared memory: Dp[NS4] | part[G][NS4] | Rs[rows_s][NS4 + 4].
+// Forward: D_w(g) = cost_w(g) + min_h (D_{w-1}(h) + R[h][g]).  Only the minimum is formed here (add + min per
+// step): a thread takes four neighbouring targets and a share of the sources, four sources per trip (one 16-byte
+// read of the state vector, four of R).  The values D_{w-1}, relative to their minimum, are written to `hist`,
+// and the walk back finds each predecessor again as the lowest h that attains the minimum, with the same addition.
+__global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfArgs a, const int rows_s) {
     extern __shared__ float4 smem4[];
-    __shared__ float red[kThreads / 32];
-    __shared__ int s_last;
-    const int NS = a.NS;
-    float *D0 = reinterpret_cast<float *>(smem4), *D1 = D0 + NS;
-    uint16_t *back = reinterpret_cast<uint16_t *>(D1 + NS);
-    int32_t *path = reinterpret_cast<int32_t *>(back + size_t(kBack) * NS);
+    __shared__ float red[kPathThreads / 32];
+    const int NS = a.NS, NS4 = (NS + 3) & ~3, RSd = NS4 + 4;
+    const int TG = NS4 / 4;                                  // groups of four targets
+    const int lanes_t = (TG + 31) / 32 * 32;                 // threads side by side over the target groups (<= 256)
+    const int G = kPathThreads / lanes_t;                    // thread groups that split the sources
+    float *Dp = reinterpret_cast<float *>(smem4);
+    float *part = Dp + NS4;
+    float *Rs = part + size_t(G) * NS4;
     const int64_t sc = blockIdx.x;                           // s * C + c
     const int c = int(sc % a.C);
     const int64_t s = sc / a.C;
     const int64_t W = a.W;
     const float *cost = a.cost + sc * W * NS;
-    uint16_t *from = a.from + sc * W * NS;
+    float *hist = a.hist + sc * W * NS;
     const int tid = threadIdx.x;
+    const int hg = tid / lanes_t, tg = tid - hg * lanes_t;
+    const bool worker = hg < G && tg < TG;
+    const int SQ = rows_s / 4;                               // quads of rows held in shared memory
+    const int q_lo = int(int64_t(hg) * SQ / G), q_hi = worker ? int(int64_t(hg + 1) * SQ / G) : q_lo;   // this group's share
 
-    // forward: D_w(g) = cost_w(g) + min_h (D_{w-1}(h) + R[h][g]), lowest h on ties; values relative to `base`
+    for (int i = tid; i < rows_s * RSd; i += kPathThreads) {
+        const int h = i / RSd, g = i - h * RSd;
+        Rs[i] = g < NS ? a.R[size_t(h) * NS + g] : 0.f;
+    }
+    // rows of R that do not fit in shared memory: the first G * kRegRows of them stay in registers, each source
+    // group holding kRegRows rows (its four columns of them); any further rows are read through L1 / L2
+    float4 rreg[kRegRows];
+    int hreg[kRegRows];
+#pragma unroll
+    for (int j = 0; j < kRegRows; ++j) {
+        const int h = rows_s + hg * kRegRows + j;
+        hreg[j] = (worker && h < NS) ? h : -1;
+        rreg[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (hreg[j] >= 0) {
+            const float *row = a.R + size_t(h) * NS + 4 * tg;
+            rreg[j].x = __ldg(row);
+            rreg[j].y = 4 * tg + 1 < NS ? __ldg(row + 1) : 0.f;
+            rreg[j].z = 4 * tg + 2 < NS ? __ldg(row + 2) : 0.f;
+            rreg[j].w = 4 * tg + 3 < NS ? __ldg(row + 3) : 0.f;
+        }
+    }
+    const int rows_sr = rows_s + G * kRegRows;               // rows below this are in shared memory or registers
+    // the rest, split evenly over the source groups
+    const int n_rest = NS > rows_sr ? NS - rows_sr : 0;
+    const int g_lo = rows_sr + int(int64_t(hg) * n_rest / G), g_hi = worker ? rows_sr + int(int64_t(hg + 1) * n_rest / G) : g_lo;
+    // window 0 (the padding entries past NS are sources that never win: +inf); a thread owns entries tid and
+    // tid + kPathThreads of the state vector in every pass below except the scan
     double base = 0.0;
-    float *Dp = D0, *Dn = D1;
     float lmin = CUDART_INF_F;
-    for (int g = tid; g < NS; g += kThreads) {
-        const float v = W > 0 ? cost[g] : 0.f;
+    for (int g = tid; g < NS4; g += kPathThreads) {
+        const float v = g < NS ? (W > 0 ? cost[g] : 0.f) : CUDART_INF_F;
         Dp[g] = v;
         lmin = fminf(lmin, v);
     }
-    float m = block_min(lmin, red);                          // also orders the writes of Dp before the reads below
+    float m = block_min(lmin, red);                          // its barriers also publish Rs
     for (int64_t w = 1; w < W; ++w) {
-        // renormalise: keep differences only (the minimum goes to the fp64 base); all +inf stays +inf
+        // keep differences only: the minimum goes to the fp64 base (all +inf stays +inf)
         const float shift = (m < CUDART_INF_F) ? m : 0.f;
         base += double(shift);
-        lmin = CUDART_INF_F;
-        for (int g = tid; g < NS; g += kThreads) {
-            float best = CUDART_INF_F;
-            int arg = 0;
-            const float *Rg = a.R + g;
-#pragma unroll 8
-            for (int h = 0; h < NS; ++h) {
-                const float v = (Dp[h] - shift) + __ldg(Rg + size_t(h) * NS);
-                if (v < best) {
-                    best = v;
-                    arg = h;
+        for (int g = tid; g < NS; g += kPathThreads) {
+            const float v = Dp[g] - shift;
+            Dp[g] = v;
+            hist[(w - 1) * NS + g] = v;
+        }
+        // the next window's costs, asked for before the barrier so that their latency hides behind the scan
+        const float cw0 = tid < NS ? cost[w * NS + tid] : 0.f;
+        const float cw1 = tid + kPathThreads < NS ? cost[w * NS + tid + kPathThreads] : 0.f;
+        __syncthreads();
+        if (worker) {
+            float b0 = CUDART_INF_F, b1 = CUDART_INF_F, b2 = CUDART_INF_F, b3 = CUDART_INF_F;
+#pragma unroll 2
+            for (int q = q_lo; q < q_hi; ++q) {
+                const float4 d4 = reinterpret_cast<const float4 *>(Dp)[q];
+                const float dv[4] = {d4.x, d4.y, d4.z, d4.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float4 r = *reinterpret_cast<const float4 *>(Rs + (4 * q + j) * RSd + 4 * tg);
+                    b0 = fminf(b0, dv[j] + r.x);
+                    b1 = fminf(b1, dv[j] + r.y);
+                    b2 = fminf(b2, dv[j] + r.z);
+                    b3 = fminf(b3, dv[j] + r.w);
                 }
             }
-            const float d = cost[w * NS + g] + best;
-            Dn[g] = d;
-            from[w * NS + g] = uint16_t(arg);
+#pragma unroll
+            for (int j = 0; j < kRegRows; ++j) {
+                const float d = hreg[j] >= 0 ? Dp[hreg[j]] : CUDART_INF_F;
+                b0 = fminf(b0, d + rreg[j].x);
+                b1 = fminf(b1, d + rreg[j].y);
+                b2 = fminf(b2, d + rreg[j].z);
+                b3 = fminf(b3, d + rreg[j].w);
+            }
+            for (int h = g_lo; h < g_hi; ++h) {
+                const float d = Dp[h];
+                const float *row = a.R + size_t(h) * NS + 4 * tg;
+                b0 = fminf(b0, d + __ldg(row));
+                if (4 * tg + 1 < NS) b1 = fminf(b1, d + __ldg(row + 1));
+                if (4 * tg + 2 < NS) b2 = fminf(b2, d + __ldg(row + 2));
+                if (4 * tg + 3 < NS) b3 = fminf(b3, d + __ldg(row + 3));
+            }
+            reinterpret_cast<float4 *>(part + size_t(hg) * NS4)[tg] = make_float4(b0, b1, b2, b3);
+        }
+        __syncthreads();
+        lmin = CUDART_INF_F;
+        for (int g = tid; g < NS; g += kPathThreads) {
+            float best = part[g];
+            for (int k = 1; k < G; ++k) best = fminf(best, part[k * NS4 + g]);
+            const float d = (g == tid ? cw0 : cw1) + best;
+            Dp[g] = d;                                       // every reader of Dp has passed the barrier above
             lmin = fminf(lmin, d);
         }
-        m = block_min(lmin, red);                            // its barriers separate this window's writes from the next reads
-        float *tmp = Dp; Dp = Dn; Dn = tmp;
+        m = block_min(lmin, red);
     }
-    // last state: lowest g attaining the minimum
-    if (tid == 0) {
-        int last = -1;
-        if (m < CUDART_INF_F && W > 0)
-            for (int g = 0; g < NS; ++g)
-                if (Dp[g] == m) { last = g; break; }
-        s_last = last;
-        a.path_total[sc] = W > 0 ? ((m < CUDART_INF_F) ? base + double(m) : double(CUDART_INF_F)) : 0.0;
+    if (W == 0) {
+        if (tid == 0) a.path_total[sc] = 0.0;
+        return;
     }
-    __syncthreads();
-    int cur = s_last;
-    // walk back, kBack windows per step: stage their back pointers, one thread follows them, all write results
-    for (int64_t hi = W; hi > 0; hi -= kBack) {
-        const int64_t lo = hi > kBack ? hi - kBack : 0;
-        const int nw = int(hi - lo);
-        if (cur >= 0) {
-            for (int i = tid; i < nw * NS; i += kThreads) back[i] = from[lo * NS + i];
-        }
-        __syncthreads();
-        if (tid == 0) {
-            int g = cur;
-            for (int k = nw - 1; k >= 0; --k) {
-                path[k] = g;
-                if (g >= 0 && lo + k > 0) g = back[k * NS + g];       // pointer of window lo+k leads to window lo+k-1
-            }
-            s_last = g;
-        }
-        __syncthreads();
-        for (int k = tid; k < nw; k += kThreads) {
-            const int g = path[k];
-            const int64_t w = lo + k;
+    const bool have = m < CUDART_INF_F;
+    if (tid == 0) a.path_total[sc] = have ? base + double(m) : double(CUDART_INF_F);
+    // the walk back, by the first warp: at window w in state g the predecessor is the lowest h that attains
+    // min_h hist[w-1][h] + R[h][g]
+    if (tid >= 32) return;
+    const int lane = tid;
+    int cur = -1;
+    if (have) {
+        uint32_t cand = 0xffffffffu;
+        for (int g = lane; g < NS; g += 32)
+            if (Dp[g] == m && uint32_t(g) < cand) cand = uint32_t(g);
+        cur = int(__reduce_min_sync(0xffffffffu, cand));
+    }
+    for (int64_t w = W - 1; w >= 0; --w) {
+        if (lane == 0) {
             const int64_t i = (s * W + w) * a.C + c;
-            if (g >= 0) {
-                a.best_idx[i] = g * a.F + int(a.qbest[sc * W * NS + w * NS + g]);
-                a.best_E[i] = cost[w * NS + g];
+            if (cur >= 0) {
+                a.best_idx[i] = cur * a.F + int(a.qbest[sc * W * NS + w * NS + cur]);
+                a.best_E[i] = cost[w * NS + cur];
             } else {
                 a.best_idx[i] = -1;
                 a.best_E[i] = CUDART_INF_F;
             }
         }
-        cur = s_last;
-        __syncthreads();
+        if (cur < 0 || w == 0) continue;
+        const float *hp = hist + (w - 1) * NS;
+        float best = CUDART_INF_F;
+        uint32_t arg = 0xffffffffu;
+        for (int h = lane; h < NS; h += 32) {
+            const float v = hp[h] + r_at(Rs, a.R, rows_s, NS, NS4, h, cur);
+            if (v < best) {                                  // ascending h per lane: strict compare keeps the lowest
+                best = v;
+                arg = uint32_t(h);
+            }
+        }
+        float mm;
+        asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(mm) : "f"(best));
+        cur = int(__reduce_min_sync(0xffffffffu, best == mm ? arg : 0xffffffffu));
     }
 }
 
 }  // namespace
 
-size_t reconf_smem_bytes(int32_t NS) {
-    return size_t(2) * NS * sizeof(float) + size_t(kBack) * NS * sizeof(uint16_t) + size_t(kBack) * sizeof(int32_t) + 16;
+// rows of R kept in shared memory for NS states, given the device's limit
+static size_t reconf_fixed_floats(int32_t NS) {
+    const int NS4 = (NS + 3) & ~3, TG = NS4 / 4, lanes_t = (TG + 31) / 32 * 32, G = kPathThreads / lanes_t;
+    return size_t(1 + G) * NS4;
+}
+static int reconf_rows_in_smem(int32_t NS, size_t limit) {
+    const int NS4 = (NS + 3) & ~3;
+    const size_t fixed = reconf_fixed_floats(NS) * sizeof(float) + 1024;
+    if (limit <= fixed) return 0;
+    const int64_t rows = int64_t((limit - fixed) / (size_t(NS4 + 4) * sizeof(float)));
+    return int(rows > NS ? NS : rows) & ~3;                  // whole quads of rows
 }
 
 cudaError_t launch_reconf(const ResolvedLayout &lay, void *d_ws, size_t off_cost, size_t off_q, size_t off_from,
@@ -202,7 +286,7 @@ cudaError_t launch_reconf(const ResolvedLayout &lay, void *d_ws, size_t off_cost
     a.R = d_R; a.load = d_load;
     a.cost = reinterpret_cast<float *>(ws + off_cost);
     a.qbest = reinterpret_cast<uint8_t *>(ws + off_q);
-    a.from = reinterpret_cast<uint16_t *>(ws + off_from);
+    a.hist = reinterpret_cast<float *>(ws + off_from);
     a.S = S; a.W = W;
     a.C = lay.C; a.T = lay.T; a.F = lay.F; a.M = lay.M; a.Nmax = lay.Nmax; a.NS = lay.Nmax * lay.T; a.budget = budget;
     a.best_idx = best_idx; a.best_E = best_E; a.path_total = path_total;
@@ -216,12 +300,18 @@ cudaError_t launch_reconf(const ResolvedLayout &lay, void *d_ws, size_t off_cost
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
-    const size_t smem = reconf_smem_bytes(a.NS);
-    cudaError_t e = cudaFuncSetAttribute(reconf_path_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+    int dev = 0, lim = 48 * 1024;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (cudaDeviceGetAttribute(&lim, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) lim = 48 * 1024;
+    const int rows_s = reconf_rows_in_smem(a.NS, size_t(lim));
+    const int NS4 = (a.NS + 3) & ~3;
+    const size_t smem = (reconf_fixed_floats(a.NS) + size_t(rows_s) * (NS4 + 4)) * sizeof(float) + 16;
+    e = cudaFuncSetAttribute(reconf_path_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
     if (e != cudaSuccess) return e;
     e = record_start(st);
     if (e != cudaSuccess) return e;
-    reconf_path_kernel<<<unsigned(S * lay.C), kThreads, smem, st>>>(a);
+    reconf_path_kernel<<<unsigned(S * lay.C), kPathThreads, smem, st>>>(a, rows_s);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     return record_stop(st);
