@@ -231,31 +231,72 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
             if (Dp[g] == m && uint32_t(g) < cand) cand = uint32_t(g);
         cur = int(__reduce_min_sync(0xffffffffu, cand));
     }
-    for (int64_t w = W - 1; w >= 0; --w) {
-        if (lane == 0) {
+    // The states of up to `chunk` windows are first noted in shared memory (the partial-minimum buffer is free
+    // now), then the lanes write the results of those windows side by side.  With at most 256 states a lane
+    // holds its eight entries of the next window's vector ahead of time (they do not depend on the state).
+    int *path = reinterpret_cast<int *>(part);
+    const int chunk = G * NS4;
+    const bool ahead = NS <= 256;
+    float hv[8];
+    if (ahead && W > 1) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) hv[j] = (lane + 32 * j < NS) ? hist[(W - 2) * NS + lane + 32 * j] : CUDART_INF_F;
+    }
+    for (int64_t hi = W; hi > 0; hi -= chunk) {
+        const int64_t lo = hi > chunk ? hi - chunk : 0;
+        for (int64_t w = hi - 1; w >= lo; --w) {
+            if (lane == 0) path[w - lo] = cur;
+            if (cur < 0 || w == 0) continue;
+            float best = CUDART_INF_F;
+            uint32_t arg = 0xffffffffu;
+            if (ahead) {
+                float nx[8];
+                if (w > 1) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) nx[j] = (lane + 32 * j < NS) ? hist[(w - 2) * NS + lane + 32 * j] : CUDART_INF_F;
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int h = lane + 32 * j;
+                    if (h < NS) {
+                        const float v = hv[j] + r_at(Rs, a.R, rows_s, NS, NS4, h, cur);
+                        if (v < best) {                      // ascending h per lane: strict compare keeps the lowest
+                            best = v;
+                            arg = uint32_t(h);
+                        }
+                    }
+                }
+                if (w > 1) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) hv[j] = nx[j];
+                }
+            } else {
+                const float *hp = hist + (w - 1) * NS;
+                for (int h = lane; h < NS; h += 32) {
+                    const float v = hp[h] + r_at(Rs, a.R, rows_s, NS, NS4, h, cur);
+                    if (v < best) {
+                        best = v;
+                        arg = uint32_t(h);
+                    }
+                }
+            }
+            float mm;
+            asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(mm) : "f"(best));
+            cur = int(__reduce_min_sync(0xffffffffu, best == mm ? arg : 0xffffffffu));
+        }
+        __syncwarp();
+        for (int64_t w = lo + lane; w < hi; w += 32) {
+            const int g = path[w - lo];
             const int64_t i = (s * W + w) * a.C + c;
-            if (cur >= 0) {
-                a.best_idx[i] = cur * a.F + int(a.qbest[sc * W * NS + w * NS + cur]);
-                a.best_E[i] = cost[w * NS + cur];
+            if (g >= 0) {
+                a.best_idx[i] = g * a.F + int(a.qbest[sc * W * NS + w * NS + g]);
+                a.best_E[i] = cost[w * NS + g];
             } else {
                 a.best_idx[i] = -1;
                 a.best_E[i] = CUDART_INF_F;
             }
         }
-        if (cur < 0 || w == 0) continue;
-        const float *hp = hist + (w - 1) * NS;
-        float best = CUDART_INF_F;
-        uint32_t arg = 0xffffffffu;
-        for (int h = lane; h < NS; h += 32) {
-            const float v = hp[h] + r_at(Rs, a.R, rows_s, NS, NS4, h, cur);
-            if (v < best) {                                  // ascending h per lane: strict compare keeps the lowest
-                best = v;
-                arg = uint32_t(h);
-            }
-        }
-        float mm;
-        asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(mm) : "f"(best));
-        cur = int(__reduce_min_sync(0xffffffffu, best == mm ? arg : 0xffffffffu));
+        __syncwarp();
     }
 }
 
