@@ -389,7 +389,8 @@ size_t dyn_reconf_workspace_bytes(const dyn_profile *profile, const dyn_space *s
     const size_t base = dyn_workspace_bytes(profile, space, S, W);
     if (!base) return 0;
     const size_t n = size_t(S) * size_t(profile->C) * size_t(W) * size_t(space->Nmax) * size_t(profile->T);
-    return base + align256(n * sizeof(float)) + align256(n) + align256(n * sizeof(float));
+    const size_t ns = size_t(space->Nmax) * size_t(profile->T);
+    return base + align256(n * sizeof(float)) + align256(n) + align256(n * sizeof(float)) + align256(ns * ns * sizeof(float));
 }
 
 int dyn_reconf_select(const dyn_profile *profile, const dyn_space *space, const float *d_R, const float *d_load,
@@ -407,12 +408,13 @@ int dyn_reconf_select(const dyn_profile *profile, const dyn_space *space, const 
     const ResolvedLayout lay = resolved_layout(profile->C, profile->T, space->F, profile->M, space->Nmax, S, W);
     const size_t n = size_t(S) * size_t(profile->C) * size_t(W) * size_t(NS);
     const size_t off_cost = lay.total, off_q = off_cost + align256(n * sizeof(float)), off_from = off_q + align256(n);
-    rc = check_ws(d_ws, ws_bytes, off_from + align256(n * sizeof(float)));
+    const size_t off_rt = off_from + align256(n * sizeof(float));
+    rc = check_ws(d_ws, ws_bytes, off_rt + align256(size_t(NS) * size_t(NS) * sizeof(float)));
     if (rc != DYN_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     char *ws = static_cast<char *>(d_ws);
     DYN_CUDA_TRY(launch_resolve(rp, lay, d_ws, st));
-    DYN_CUDA_TRY(launch_reconf(lay, d_ws, off_cost, off_q, off_from, d_R, d_load, S, W, space->gpu_budget, out->d_best_idx,
+    DYN_CUDA_TRY(launch_reconf(lay, d_ws, off_cost, off_q, off_from, off_rt, d_R, d_load, S, W, space->gpu_budget, out->d_best_idx,
                                out->d_best_E, d_path_total, st));
     const int64_t chunks = totals_chunks(W);
     double *partial = reinterpret_cast<double *>(ws + lay.off_partial);

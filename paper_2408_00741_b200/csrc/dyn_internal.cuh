@@ -114,7 +114,7 @@ cudaError_t launch_mixed(const ResolvedLayout &lay, void *d_ws, size_t off_tuple
                          float *d_best_E, cudaStream_t st);
 
 // selection with re-configuration costs (shortest path over the windows)
-cudaError_t launch_reconf(const ResolvedLayout &lay, void *d_ws, size_t off_cost, size_t off_q, size_t off_from,
+cudaError_t launch_reconf(const ResolvedLayout &lay, void *d_ws, size_t off_cost, size_t off_q, size_t off_from, size_t off_rt,
                           const float *d_R, const float *d_load, int64_t S, int64_t W, int32_t budget, int32_t *best_idx,
                           float *best_E, double *path_total, cudaStream_t st);
 

@@ -9,9 +9,10 @@
 //                       covers 32 shardings of one tile (one load, the table rows of T degrees), F evaluations each
 //   reconf_path_kernel  one CTA per (scenario, class): forward recursion over the windows (min-plus product of the
 //                       state vector with R: add + min per step; R in shared memory as far as it fits, the state
-//                       vector too), the vectors written to global memory; then the walk back by one warp, which
-//                       finds each predecessor again with the same addition.  The running values are kept relative
+//                       vector too), the vectors written to global memory.  The running values are kept relative
 //                       to their minimum, which is accumulated in fp64, so that fp32 holds only differences.
+//   reconf_back_kernel  the walk back, one warp per (scenario, class): it finds each predecessor again with the
+//                       same addition (lowest source on ties) and writes the chosen candidates.
 #include "dyn_internal.cuh"
 
 #include <math_constants.h>
@@ -28,6 +29,7 @@ struct ReconfArgs {
     const float *slo;         // [C]
     const int32_t *tp;        // [T]
     const float *R;           // [NS][NS]
+    float *Rt;                // [NS][NS] transposed copy: Rt[g][h] = R[h][g] (the walk back reads columns of R)
     const float *load;        // [S][W][C]
     float *cost;              // [S][C][W][NS]
     uint8_t *qbest;           // [S][C][W][NS]
@@ -90,11 +92,7 @@ __device__ __forceinline__ float block_min(float v, float *red) {
 }
 
 // R[h][g]: the first rows_s rows sit in shared memory with row stride NS4 + 4 floats (rows stay 16-byte aligned;
-// NS4 = NS rounded up to a multiple of 4), the rest is read through L1 / L2
-__device__ __forceinline__ float r_at(const float *Rs, const float *R, int rows_s, int NS, int NS4, int h, int g) {
-    return h < rows_s ? Rs[h * (NS4 + 4) + g] : __ldg(R + size_t(h) * NS + g);
-}
-
+// NS4 = NS rounded up to a multiple of 4)
 // One CTA per (scenario, class).  Dynamic shared memory: Dp[NS4] | part[G][NS4] | Rs[rows_s][NS4 + 4].
 // Forward: D_w(g) = cost_w(g) + min_h (D_{w-1}(h) + R[h][g]).  Only the minimum is formed here (add + min per
 // step): a thread takes four neighbouring targets and a share of the sources, four sources per trip (one 16-byte
@@ -111,8 +109,6 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
     float *part = Dp + NS4;
     float *Rs = part + size_t(G) * NS4;
     const int64_t sc = blockIdx.x;                           // s * C + c
-    const int c = int(sc % a.C);
-    const int64_t s = sc / a.C;
     const int64_t W = a.W;
     const float *cost = a.cost + sc * W * NS;
     float *hist = a.hist + sc * W * NS;
@@ -218,85 +214,129 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
         if (tid == 0) a.path_total[sc] = 0.0;
         return;
     }
-    const bool have = m < CUDART_INF_F;
-    if (tid == 0) a.path_total[sc] = have ? base + double(m) : double(CUDART_INF_F);
-    // the walk back, by the first warp: at window w in state g the predecessor is the lowest h that attains
-    // min_h hist[w-1][h] + R[h][g]
-    if (tid >= 32) return;
-    const int lane = tid;
+    // the last window's vector goes to the row of `hist` that the recursion leaves free; the walk back starts there
+    for (int g = tid; g < NS; g += kPathThreads) hist[(W - 1) * NS + g] = Dp[g];
+    if (tid == 0) a.path_total[sc] = (m < CUDART_INF_F) ? base + double(m) : double(CUDART_INF_F);
+}
+
+// The walk back: one warp per (scenario, class), four of them per CTA.  At window w in state g the predecessor is
+// the lowest h that attains min_h hist[w-1][h] + R[h][g] (the same addition as in the forward scan).  R is read
+// from a transposed copy (a column of R is then one contiguous row) through L1.  With at most 256 states
+// a lane keeps its eight entries of the vectors of the next eight windows in registers: they do not depend on the
+// state, and asking for them eight steps ahead hides the memory latency of the walk.  The states of a stretch of
+// windows are noted in shared memory, then the lanes write the results of those windows side by side.
+__global__ void reconf_transpose_kernel(const ReconfArgs a) {
+    const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= int64_t(a.NS) * a.NS) return;
+    const int g = int(i / a.NS), h = int(i - int64_t(g) * a.NS);
+    a.Rt[i] = a.R[size_t(h) * a.NS + g];
+}
+
+constexpr int kBackWarps = 1;
+constexpr int kBackChunk = 512;                 // windows per stretch (a multiple of the ring depth)
+
+__global__ void __launch_bounds__(kBackWarps * 32) reconf_back_kernel(const ReconfArgs a) {
+    __shared__ int path_all[kBackWarps][kBackChunk];
+    const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
+    const int64_t sc = int64_t(blockIdx.x) * kBackWarps + wi;
+    if (sc >= a.S * a.C) return;
+    int *path = path_all[wi];
+    const int NS = a.NS;
+    const int c = int(sc % a.C);
+    const int64_t s = sc / a.C;
+    const int64_t W = a.W;
+    if (W == 0) return;
+    const float *cost = a.cost + sc * W * NS;
+    const float *hist = a.hist + sc * W * NS;
+    const float *Rt = a.Rt;
+    // last state: the lowest g that attains the minimum of the final vector
     int cur = -1;
-    if (have) {
-        uint32_t cand = 0xffffffffu;
-        for (int g = lane; g < NS; g += 32)
-            if (Dp[g] == m && uint32_t(g) < cand) cand = uint32_t(g);
-        cur = int(__reduce_min_sync(0xffffffffu, cand));
+    {
+        float best = CUDART_INF_F;
+        uint32_t arg = 0xffffffffu;
+        for (int g = lane; g < NS; g += 32) {
+            const float v = hist[(W - 1) * NS + g];
+            if (v < best) {
+                best = v;
+                arg = uint32_t(g);
+            }
+        }
+        float mm;
+        asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(mm) : "f"(best));
+        if (mm < CUDART_INF_F) cur = int(__reduce_min_sync(0xffffffffu, best == mm ? arg : 0xffffffffu));
     }
-    // The states of up to `chunk` windows are first noted in shared memory (the partial-minimum buffer is free
-    // now), then the lanes write the results of those windows side by side.  With at most 256 states a lane
-    // holds its eight entries of the next window's vector ahead of time (they do not depend on the state).
-    int *path = reinterpret_cast<int *>(part);
-    const int chunk = G * NS4;
     const bool ahead = NS <= 256;
-    float hv[8];
-    if (ahead && W > 1) {
+    float ring[8][8];
+    if (ahead) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) hv[j] = (lane + 32 * j < NS) ? hist[(W - 2) * NS + lane + 32 * j] : CUDART_INF_F;
+        for (int k = 0; k < 8; ++k) {
+            const int64_t row = W - 2 - k;                   // the vector used at window W-1-k
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                ring[k][j] = (row >= 0 && lane + 32 * j < NS) ? hist[row * NS + lane + 32 * j] : CUDART_INF_F;
+        }
     }
-    for (int64_t hi = W; hi > 0; hi -= chunk) {
-        const int64_t lo = hi > chunk ? hi - chunk : 0;
-        for (int64_t w = hi - 1; w >= lo; --w) {
-            if (lane == 0) path[w - lo] = cur;
-            if (cur < 0 || w == 0) continue;
-            float best = CUDART_INF_F;
-            uint32_t arg = 0xffffffffu;
-            if (ahead) {
-                float nx[8];
-                if (w > 1) {
+    int64_t seg_hi = W;                                      // windows [w, seg_hi) are noted in path[seg_hi - 1 - w]
+    for (int64_t wb = W - 1; wb >= 0; wb -= 8) {
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) nx[j] = (lane + 32 * j < NS) ? hist[(w - 2) * NS + lane + 32 * j] : CUDART_INF_F;
-                }
+        for (int k = 0; k < 8; ++k) {
+            const int64_t w = wb - k;
+            if (w >= 0) {
+                if (lane == 0) path[seg_hi - 1 - w] = cur;
+                if (cur >= 0 && w > 0) {
+                    float best = CUDART_INF_F;
+                    uint32_t arg = 0xffffffffu;
+                    if (ahead) {
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const int h = lane + 32 * j;
-                    if (h < NS) {
-                        const float v = hv[j] + r_at(Rs, a.R, rows_s, NS, NS4, h, cur);
-                        if (v < best) {                      // ascending h per lane: strict compare keeps the lowest
-                            best = v;
-                            arg = uint32_t(h);
+                        for (int j = 0; j < 8; ++j) {
+                            const int h = lane + 32 * j;
+                            if (h < NS) {
+                                const float v = ring[k][j] + __ldg(Rt + size_t(cur) * NS + h);
+                                if (v < best) {              // ascending h per lane: strict compare keeps the lowest
+                                    best = v;
+                                    arg = uint32_t(h);
+                                }
+                            }
+                        }
+                    } else {
+                        const float *hp = hist + (w - 1) * NS;
+                        for (int h = lane; h < NS; h += 32) {
+                            const float v = hp[h] + __ldg(Rt + size_t(cur) * NS + h);
+                            if (v < best) {
+                                best = v;
+                                arg = uint32_t(h);
+                            }
                         }
                     }
+                    float mm;
+                    asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(mm) : "f"(best));
+                    cur = int(__reduce_min_sync(0xffffffffu, best == mm ? arg : 0xffffffffu));
                 }
-                if (w > 1) {
+                if (ahead) {                                 // the vector used eight windows further down
+                    const int64_t row = w - 9;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) hv[j] = nx[j];
-                }
-            } else {
-                const float *hp = hist + (w - 1) * NS;
-                for (int h = lane; h < NS; h += 32) {
-                    const float v = hp[h] + r_at(Rs, a.R, rows_s, NS, NS4, h, cur);
-                    if (v < best) {
-                        best = v;
-                        arg = uint32_t(h);
-                    }
+                    for (int j = 0; j < 8; ++j)
+                        ring[k][j] = (row >= 0 && lane + 32 * j < NS) ? hist[row * NS + lane + 32 * j] : CUDART_INF_F;
                 }
             }
-            float mm;
-            asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(mm) : "f"(best));
-            cur = int(__reduce_min_sync(0xffffffffu, best == mm ? arg : 0xffffffffu));
         }
-        __syncwarp();
-        for (int64_t w = lo + lane; w < hi; w += 32) {
-            const int g = path[w - lo];
-            const int64_t i = (s * W + w) * a.C + c;
-            if (g >= 0) {
-                a.best_idx[i] = g * a.F + int(a.qbest[sc * W * NS + w * NS + g]);
-                a.best_E[i] = cost[w * NS + g];
-            } else {
-                a.best_idx[i] = -1;
-                a.best_E[i] = CUDART_INF_F;
+        const int64_t lo = wb - 7 > 0 ? wb - 7 : 0;          // lowest window handled so far
+        if (seg_hi - lo >= kBackChunk || lo == 0) {
+            __syncwarp();
+            for (int64_t w = lo + lane; w < seg_hi; w += 32) {
+                const int g = path[seg_hi - 1 - w];
+                const int64_t i = (s * W + w) * a.C + c;
+                if (g >= 0) {
+                    a.best_idx[i] = g * a.F + int(a.qbest[sc * W * NS + w * NS + g]);
+                    a.best_E[i] = cost[w * NS + g];
+                } else {
+                    a.best_idx[i] = -1;
+                    a.best_E[i] = CUDART_INF_F;
+                }
             }
+            __syncwarp();
+            seg_hi = lo;
         }
-        __syncwarp();
     }
 }
 
@@ -315,7 +355,7 @@ static int reconf_rows_in_smem(int32_t NS, size_t limit) {
     return int(rows > NS ? NS : rows) & ~3;                  // whole quads of rows
 }
 
-cudaError_t launch_reconf(const ResolvedLayout &lay, void *d_ws, size_t off_cost, size_t off_q, size_t off_from,
+cudaError_t launch_reconf(const ResolvedLayout &lay, void *d_ws, size_t off_cost, size_t off_q, size_t off_from, size_t off_rt,
                           const float *d_R, const float *d_load, int64_t S, int64_t W, int32_t budget, int32_t *best_idx,
                           float *best_E, double *path_total, cudaStream_t st) {
     char *ws = static_cast<char *>(d_ws);
@@ -328,10 +368,12 @@ cudaError_t launch_reconf(const ResolvedLayout &lay, void *d_ws, size_t off_cost
     a.cost = reinterpret_cast<float *>(ws + off_cost);
     a.qbest = reinterpret_cast<uint8_t *>(ws + off_q);
     a.hist = reinterpret_cast<float *>(ws + off_from);
+    a.Rt = reinterpret_cast<float *>(ws + off_rt);
     a.S = S; a.W = W;
     a.C = lay.C; a.T = lay.T; a.F = lay.F; a.M = lay.M; a.Nmax = lay.Nmax; a.NS = lay.Nmax * lay.T; a.budget = budget;
     a.best_idx = best_idx; a.best_E = best_E; a.path_total = path_total;
     if (S == 0) return cudaSuccess;
+    reconf_transpose_kernel<<<unsigned((int64_t(a.NS) * a.NS + 255) / 256), 256, 0, st>>>(a);
     const int64_t total = S * lay.C * W * a.NS;
     if (total > 0) {
         int64_t grid = (total + kThreads - 1) / kThreads;
@@ -353,6 +395,8 @@ cudaError_t launch_reconf(const ResolvedLayout &lay, void *d_ws, size_t off_cost
     e = record_start(st);
     if (e != cudaSuccess) return e;
     reconf_path_kernel<<<unsigned(S * lay.C), kPathThreads, smem, st>>>(a, rows_s);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    reconf_back_kernel<<<unsigned((S * lay.C + kBackWarps - 1) / kBackWarps), kBackWarps * 32, 0, st>>>(a);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     return record_stop(st);
