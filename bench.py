@@ -312,14 +312,15 @@ def run_ours(args, rank, world, local_rank):
     arena = torch.empty(hp.arena_bytes(n_req, S), dtype=torch.uint8, device=dev)
     h2d = 3 * 4 * n_req + sum(x.nbytes for x in hp.tabs) + (h_extra.numel() * 4 if h_extra is not None else 0)
     d2h = sum(v.numel() * v.element_size() for v in h_out.values())
+    side = torch.cuda.Stream(device=dev)           # the scenario loads travel on it while earlier ones are evaluated
     for _ in range(2):
-        hp.run(h_t, h_i, h_o, h_extra, h_out, arena)
+        hp.run(h_t, h_i, h_o, h_extra, h_out, arena, copy_stream=side)
     barrier()
     KE = max(1, args.e2e_steps)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(KE):
-        hp.run(h_t, h_i, h_o, h_extra, h_out, arena)
+        hp.run(h_t, h_i, h_o, h_extra, h_out, arena, copy_stream=side)
     e1.record()
     barrier()
     e2e_ms = max_over_ranks(e0.elapsed_time(e1), dist, dev)

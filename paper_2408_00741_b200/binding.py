@@ -67,7 +67,7 @@ class _ProfileHost(C.Structure):
 
 class _HostIn(C.Structure):
     _fields_ = [("t_ms", C.c_void_p), ("in_tok", C.c_void_p), ("out_tok", C.c_void_p), ("n_req", C.c_uint64),
-                ("extra_load", C.c_void_p), ("S_extra", C.c_int64)]
+                ("extra_load", C.c_void_p), ("S_extra", C.c_int64), ("copy_stream", C.c_void_p)]
 
 
 class _HostOut(C.Structure):
@@ -320,13 +320,15 @@ class HostPipeline:
         assert x.flags["C_CONTIGUOUS"]
         return x.ctypes.data
 
-    def run(self, t_ms, in_tok, out_tok, extra_load, out: dict, d_arena):
+    def run(self, t_ms, in_tok, out_tok, extra_load, out: dict, d_arena, copy_stream=None):
         """out: dict with any of counts, dropped, best_idx, best_E, E_total, n_infeasible, E_window, hist,
         gpus -> host buffers of the right size.  Enqueues on torch's current stream; synchronise before
-        reading the results."""
+        reading the results.  copy_stream: an optional torch.cuda.Stream on which the scenario loads are copied
+        in pieces while earlier pieces are evaluated."""
         S_extra = 0 if extra_load is None else int(extra_load.shape[0])
         n = int(t_ms.shape[0])
-        hin = _HostIn(self._hptr(t_ms), self._hptr(in_tok), self._hptr(out_tok), n, self._hptr(extra_load), S_extra)
+        hin = _HostIn(self._hptr(t_ms), self._hptr(in_tok), self._hptr(out_tok), n, self._hptr(extra_load), S_extra,
+                      C.c_void_p(copy_stream.cuda_stream) if copy_stream is not None else None)
         hout = _HostOut(*[self._hptr(out.get(k)) for k in ("counts", "dropped", "best_idx", "best_E", "E_total",
                                                           "n_infeasible", "E_window", "hist", "gpus")])
         sp = self.space._struct()

@@ -37,6 +37,24 @@ bool plan(const dyn_bin_spec *spec, const dyn_profile_host *p, const dyn_space *
     return true;
 }
 
+constexpr int kPieces = 8;       // pieces the scenario loads are copied in when a copy stream is given
+
+// events that order the copy stream against the caller's stream: created on first use per thread and device,
+// kept for the life of the process (they hold no device memory)
+cudaEvent_t *overlap_events() {
+    constexpr int kMaxDev = 64;
+    static thread_local cudaEvent_t ev[kMaxDev][kPieces + 1];
+    static thread_local bool made[kMaxDev] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return nullptr;
+    if (!made[dev]) {
+        for (int i = 0; i <= kPieces; ++i)
+            if (cudaEventCreateWithFlags(&ev[dev][i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        made[dev] = true;
+    }
+    return ev[dev];
+}
+
 }  // namespace
 
 extern "C" {
@@ -79,9 +97,27 @@ int dyn_pipeline_host(const dyn_bin_spec *spec, const dyn_profile_host *p, const
     DYN_CUDA_TRY(cudaMemcpyAsync(dptr(ar.cap), p->cap, ctr * 4, H2D, st));
     DYN_CUDA_TRY(cudaMemcpyAsync(dptr(ar.tbt), p->tbt, ctr * size_t(p->M) * 4, H2D, st));
     DYN_CUDA_TRY(cudaMemcpyAsync(dptr(ar.pw), p->pow, ctr * size_t(p->M) * 4, H2D, st));
-    if (in->S_extra > 0)
+    // the caller's scenario loads: on `stream`, or in pieces on the copy stream so that a piece is evaluated while
+    // the next ones are still on their way
+    cudaStream_t cs = static_cast<cudaStream_t>(in->copy_stream);
+    const int pieces = (cs && cs != st && in->S_extra > 0) ? int(in->S_extra < kPieces ? in->S_extra : kPieces) : 0;
+    cudaEvent_t *ev = nullptr;
+    if (pieces > 0) {
+        ev = overlap_events();
+        if (!ev) return DYN_ECUDA;
+        // the arena may still be in use by work enqueued earlier on `stream`
+        DYN_CUDA_TRY(cudaEventRecord(ev[kPieces], st));
+        DYN_CUDA_TRY(cudaStreamWaitEvent(cs, ev[kPieces], 0));
+        for (int k = 0; k < pieces; ++k) {
+            const size_t e0 = size_t(in->S_extra) * k / pieces, e1 = size_t(in->S_extra) * (k + 1) / pieces;
+            DYN_CUDA_TRY(cudaMemcpyAsync(static_cast<char *>(dptr(ar.load)) + (1 + e0) * wc * 4, in->extra_load + e0 * wc,
+                                         (e1 - e0) * wc * 4, H2D, cs));
+            DYN_CUDA_TRY(cudaEventRecord(ev[k], cs));
+        }
+    } else if (in->S_extra > 0) {
         DYN_CUDA_TRY(cudaMemcpyAsync(static_cast<char *>(dptr(ar.load)) + wc * 4, in->extra_load,
                                      size_t(in->S_extra) * wc * 4, H2D, st));
+    }
 
     // (a): scenario 0 of the load tensor is the binned trace
     int rc = dyn_bin_trace(spec, static_cast<const uint32_t *>(dptr(ar.t)), static_cast<const uint32_t *>(dptr(ar.a)),
@@ -101,9 +137,26 @@ int dyn_pipeline_host(const dyn_bin_spec *spec, const dyn_profile_host *p, const
     so.d_E_window = out->E_window ? static_cast<double *>(dptr(ar.ewin)) : nullptr;
     so.d_hist = out->hist ? static_cast<uint32_t *>(dptr(ar.hist)) : nullptr;
     so.d_gpus = out->gpus ? static_cast<uint32_t *>(dptr(ar.gpus)) : nullptr;
-    rc = dyn_eval_select(&dp, sp, static_cast<const float *>(dptr(ar.load)), S, int64_t(W), &so, dptr(ar.ws),
-                         ar.ws_bytes, stream);
-    if (rc != DYN_OK) return rc;
+    if (pieces == 0) {
+        rc = dyn_eval_select(&dp, sp, static_cast<const float *>(dptr(ar.load)), S, int64_t(W), &so, dptr(ar.ws),
+                             ar.ws_bytes, stream);
+        if (rc != DYN_OK) return rc;
+    } else {
+        // piece k: scenarios [s0, s1) (piece 0 also holds scenario 0, the binned trace), evaluated once its loads are in
+        for (int k = 0; k < pieces; ++k) {
+            const size_t s0 = k == 0 ? 0 : 1 + size_t(in->S_extra) * k / pieces;
+            const size_t s1 = 1 + size_t(in->S_extra) * (k + 1) / pieces;
+            DYN_CUDA_TRY(cudaStreamWaitEvent(st, ev[k], 0));
+            dyn_select_out sk = so;
+            sk.d_best_idx += s0 * wc; sk.d_best_E += s0 * wc; sk.d_E_total += s0; sk.d_n_infeasible += s0;
+            if (sk.d_E_window) sk.d_E_window += s0 * W;
+            if (sk.d_hist) sk.d_hist += s0 * J;
+            if (sk.d_gpus) sk.d_gpus += s0 * W;
+            rc = dyn_eval_select(&dp, sp, static_cast<const float *>(dptr(ar.load)) + s0 * wc, int64_t(s1 - s0), int64_t(W), &sk,
+                                 dptr(ar.ws), ar.ws_bytes, stream);
+            if (rc != DYN_OK) return rc;
+        }
+    }
 
     if (out->counts) DYN_CUDA_TRY(cudaMemcpyAsync(out->counts, dptr(ar.counts), wc * 4, D2H, st));
     if (out->dropped) DYN_CUDA_TRY(cudaMemcpyAsync(out->dropped, dptr(ar.dropped), 8, D2H, st));

@@ -60,3 +60,37 @@ def test_pipeline_host_matches_oracle(dyn, name, S, pinned):
     with pytest.raises(dyn.DynError) as e:
         hp.run(t.view(np.int32), i.view(np.int32), o.view(np.int32), extra, out, arena[:nb - 256])
     assert e.value.status == dyn.DYN_EWORKSPACE
+
+
+@pytest.mark.parametrize("S", [2, 12])
+def test_copy_stream_gives_the_same_results(dyn, S):
+    """With a second stream the scenario loads arrive in pieces (here fewer and more scenarios than pieces) and
+    every piece is evaluated on its own: all outputs equal those of the single-stream call bit for bit."""
+    wl = gen.workload("cfg1")
+    t, i, o = gen.make_trace(wl.trace)
+    prof, sp = wl.profile(), wl.space()
+    W, Cn, J = wl.trace.n_windows, 9, wl.J
+    ref_c, _ = oracle.bin_trace(t, i, o, wl.trace.window_ms, W, gen.IN_EDGES, gen.OUT_EDGES)
+    extra = torch.from_numpy(oracle.load_from_counts(gen.resample_counts(ref_c, S - 1, seed=4, s_begin=1),
+                                                     wl.window_s)).pin_memory()
+    SP = dyn.Space(sp.f_cand_mhz, sp.n_max, sp.slo_ttft_s, sp.slo_tbt_s, sp.window_s, sp.gpu_budget)
+    hp = dyn.HostPipeline(wl.trace.window_ms, W, gen.IN_EDGES, gen.OUT_EDGES, prof.tp, prof.f_grid_mhz, prof.ttft,
+                          prof.cap, prof.tbt, prof.pow, SP)
+
+    def buffers():
+        mk = lambda *shape, dtype: torch.zeros(shape, dtype=dtype).pin_memory()
+        return {"counts": mk(W, Cn, dtype=torch.int32), "best_idx": mk(S, W, Cn, dtype=torch.int32),
+                "best_E": mk(S, W, Cn, dtype=torch.float32), "E_total": mk(S, dtype=torch.float64),
+                "n_infeasible": mk(S, dtype=torch.int32), "E_window": mk(S, W, dtype=torch.float64),
+                "hist": mk(S, J, dtype=torch.int32), "gpus": mk(S, W, dtype=torch.int32)}
+
+    arena = torch.empty(hp.arena_bytes(len(t), S), dtype=torch.uint8, device="cuda")
+    one, two = buffers(), buffers()
+    hp.run(t.view(np.int32), i.view(np.int32), o.view(np.int32), extra, one, arena)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    for _ in range(2):                                      # back to back: the second call waits for the first one's use of the arena
+        hp.run(t.view(np.int32), i.view(np.int32), o.view(np.int32), extra, two, arena, copy_stream=side)
+    torch.cuda.synchronize()
+    for k in one:
+        assert torch.equal(one[k], two[k]), k
