@@ -270,3 +270,35 @@ def reconf_select(profile, space, R, load):
     if rc != 0:
         raise ValueError("orc_reconf_select: invalid argument")
     return out
+
+
+def bin_tokens(t_ms, in_tok, out_tok, window_ms, n_windows, in_edges, out_edges):
+    """Sums of input and output tokens per (window, class): (tok_in, tok_out), uint64 [W][C]."""
+    t, a, b = _arr(t_ms, np.uint32), _arr(in_tok, np.uint32), _arr(out_tok, np.uint32)
+    ie, oe = _arr(in_edges, np.uint32), _arr(out_edges, np.uint32)
+    Cn = (len(ie) + 1) * (len(oe) + 1)
+    ti = np.empty((int(n_windows), Cn), np.uint64)
+    to = np.empty((int(n_windows), Cn), np.uint64)
+    rc = _load().orc_bin_tokens(_p(t), _p(a), _p(b), C.c_uint64(len(t)), C.c_uint32(int(window_ms)),
+                                C.c_uint32(int(n_windows)), _p(ie), C.c_int32(len(ie)), _p(oe), C.c_int32(len(oe)),
+                                _p(ti), _p(to))
+    if rc != 0:
+        raise ValueError("orc_bin_tokens: invalid argument")
+    return ti, to
+
+
+def load_tps(tok_in, tok_out, window_s):
+    ti, to = _arr(tok_in, np.uint64), _arr(tok_out, np.uint64)
+    out = np.empty(ti.shape, np.float32)
+    _load().orc_load_tps(_p(ti), _p(to), C.c_uint64(ti.size), C.c_float(float(window_s)), _p(out))
+    return out
+
+
+def carbon(E_window, intensity):
+    """gCO2 per scenario: sum over windows of E_window [Wh] * intensity [gCO2/kWh] / 1000."""
+    ew, it = _arr(E_window, np.float64), _arr(intensity, np.float32)
+    S, W = ew.shape
+    assert it.shape == (W,)
+    out = np.empty(S, np.float64)
+    _load().orc_carbon(_p(ew), _p(it), C.c_int64(S), C.c_int64(W), _p(out))
+    return out

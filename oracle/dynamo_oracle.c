@@ -28,6 +28,8 @@
  *                     budget, load split by capacity, one frequency per TP), by enumeration.
  *   orc_reconf_select selection that counts the cost of re-configuring between windows (overhead table):
  *                     a shortest path over the windows, states = shardings, frequency free per window.
+ *   orc_bin_tokens    token sums per (window, class): the load in tokens per second of Sec. 3.
+ *   orc_carbon        operational carbon: window energies times a carbon-intensity trace [Sec. 6.4].
  *   orc_hier_select   the controller hierarchy of Sec. 4.2 on the same models: nodes per pool from the
  *                     epoch's peak load and the per-node maximum load (ceil(PL/ML)), sharding at the
  *                     highest frequency within those GPUs, then the frequency per window.
@@ -622,4 +624,46 @@ int orc_reconf_select(const orc_profile *p, const orc_space *sp, const float *R,
     }
     free(row); free(wt);
     return ORC_OK;
+}
+
+/* ---- token-weighted loads and carbon (Sec. 3 load in tokens per second; Sec. 6.4 carbon) ------------ */
+
+/*
+ * The paper states loads in tokens per second (TPS) [Sec. 3, characterisation tables; Sec. 3.2].  Per (window,
+ * class) the sums of input tokens and of output tokens of the requests that fall there; window and class as in
+ * orc_bin_trace; requests past the last window add nothing.  Exact 64-bit integer sums.
+ */
+int orc_bin_tokens(const uint32_t *t_ms, const uint32_t *in_tok, const uint32_t *out_tok, uint64_t n_req,
+                   uint32_t window_ms, uint32_t n_windows, const uint32_t *in_edges, int32_t n_in_edges,
+                   const uint32_t *out_edges, int32_t n_out_edges, uint64_t *tok_in, uint64_t *tok_out) {
+    if (window_ms == 0 || n_in_edges < 0 || n_out_edges < 0) return ORC_EINVAL;
+    const int32_t KO = n_out_edges + 1, C = (n_in_edges + 1) * KO;
+    memset(tok_in, 0, sizeof(uint64_t) * (size_t)n_windows * (size_t)C);
+    memset(tok_out, 0, sizeof(uint64_t) * (size_t)n_windows * (size_t)C);
+    for (uint64_t i = 0; i < n_req; ++i) {
+        const uint32_t w = t_ms[i] / window_ms;
+        if (w >= n_windows) continue;
+        const int32_t c = edge_class(in_tok[i], in_edges, n_in_edges) * KO + edge_class(out_tok[i], out_edges, n_out_edges);
+        tok_in[(size_t)w * C + c] += in_tok[i];
+        tok_out[(size_t)w * C + c] += out_tok[i];
+    }
+    return ORC_OK;
+}
+
+/* tokens per second of a (window, class), computed and rounded in fp32 like orc_load */
+void orc_load_tps(const uint64_t *tok_in, const uint64_t *tok_out, uint64_t n_bins, float window_s, float *tps) {
+    for (uint64_t i = 0; i < n_bins; ++i) tps[i] = (float)(tok_in[i] + tok_out[i]) / window_s;
+}
+
+/*
+ * Operational carbon of a scenario: the energy of every window times the carbon intensity of the grid in that
+ * window, summed over the windows in order [Sec. 6.4: energy over time combined with an intensity trace].
+ * E_window[S][W] in Wh, intensity[W] in gCO2 per kWh; carbon[S] in gCO2.
+ */
+void orc_carbon(const double *E_window, const float *intensity, int64_t S, int64_t W, double *carbon) {
+    for (int64_t s = 0; s < S; ++s) {
+        double acc = 0.0;
+        for (int64_t w = 0; w < W; ++w) acc += E_window[s * W + w] * (double)intensity[w] / 1000.0;
+        carbon[s] = acc;
+    }
 }
