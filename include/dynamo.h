@@ -85,6 +85,19 @@ int dyn_bin_trace(const dyn_bin_spec *spec, const uint32_t *d_t_ms, const uint32
                   const uint32_t *d_out_tok, uint64_t n_req, uint32_t *d_counts, float *d_load,
                   uint64_t *d_dropped, void *stream);
 
+/*
+ * Token-weighted loads.  [Sec. 3 and Sec. 3.2 state loads in tokens per second (TPS); the characterisation
+ * tables quote a medium load as 2K TPS.]  Same windows and classes as dyn_bin_trace; per (window, class) the sum
+ * of the input tokens and the sum of the output tokens of its requests, exact in 64 bits for any values and any
+ * order of the trace; requests past the last window add nothing.
+ * d_tok_in, d_tok_out : device, uint64 [W][C], overwritten.
+ * d_load_tps          : device, float [W][C] = (float)(tok_in + tok_out) / (window_ms/1000 as float), or NULL.
+ * Errors: as dyn_bin_trace.
+ */
+int dyn_bin_tokens(const dyn_bin_spec *spec, const uint32_t *d_t_ms, const uint32_t *d_in_tok,
+                   const uint32_t *d_out_tok, uint64_t n_req, uint64_t *d_tok_in, uint64_t *d_tok_out,
+                   float *d_load_tps, void *stream);
+
 /* ---------------------------------------------------------------------------------------------
  * (b) Profiles and the candidate space.  [Sec. 4.1 "Generating LLM profiles": the profile maps
  *     (load, request class, TP, frequency) to energy/power and TTFT/TBT, measured at a few
@@ -170,6 +183,13 @@ int dyn_select(const float *d_E, int64_t S, int64_t W, int32_t C, int32_t J, con
 int dyn_eval_select(const dyn_profile *profile, const dyn_space *space, const float *d_load,
                     int64_t S, int64_t W, const dyn_select_out *out, void *d_ws, size_t ws_bytes,
                     void *stream);
+
+/*
+ * Operational carbon.  [Sec. 6.4: the energy over time is combined with the carbon intensity of the grid over
+ * time.]  d_carbon[s] = sum over windows, in a fixed order, of d_E_window[s][w] (Wh, e.g. dyn_select_out.d_E_window)
+ * x d_intensity[w] (gCO2 per kWh) / 1000, in fp64 (gCO2); bit-identical from run to run.
+ */
+int dyn_carbon(const double *d_E_window, const float *d_intensity, int64_t S, int64_t W, double *d_carbon, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Hierarchical control.  [Sec. 4.2: instead of the joint search, three controllers set one knob each

@@ -25,7 +25,7 @@ DYN_OK, DYN_EINVAL, DYN_ECUDA, DYN_EUNSUPPORTED, DYN_EWORKSPACE = 0, -1, -2, -3,
 EXPORTS = ("dyn_strerror", "dyn_last_cuda_error", "dyn_bin_trace", "dyn_workspace_bytes", "dyn_eval_configs",
            "dyn_select_workspace_bytes", "dyn_select", "dyn_eval_select", "dyn_pipeline_arena_bytes",
            "dyn_pipeline_host", "dyn_set_timing_events", "dyn_eval_select_static", "dyn_hier_workspace_bytes",
-           "dyn_hier_select", "dyn_mixed_workspace_bytes", "dyn_mixed_tuple_count", "dyn_mixed_select", "dyn_reconf_workspace_bytes", "dyn_reconf_select")
+           "dyn_hier_select", "dyn_mixed_workspace_bytes", "dyn_mixed_tuple_count", "dyn_mixed_select", "dyn_reconf_workspace_bytes", "dyn_reconf_select", "dyn_bin_tokens", "dyn_carbon")
 
 
 class DynError(RuntimeError):
@@ -139,6 +139,11 @@ _lib.dyn_reconf_workspace_bytes.argtypes = [C.POINTER(_Profile), C.POINTER(_Spac
 _lib.dyn_reconf_select.restype = C.c_int
 _lib.dyn_reconf_select.argtypes = [C.POINTER(_Profile), C.POINTER(_Space), C.c_void_p, C.c_void_p, C.c_int64, C.c_int64,
                                    C.POINTER(_SelectOut), C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+_lib.dyn_bin_tokens.restype = C.c_int
+_lib.dyn_bin_tokens.argtypes = [C.POINTER(_BinSpec), C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p,
+                                C.c_void_p, C.c_void_p]
+_lib.dyn_carbon.restype = C.c_int
+_lib.dyn_carbon.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p]
 
 
 def _dev(t, dtype, what):
@@ -420,3 +425,24 @@ def dyn_reconf_select(profile: Profile, space: Space, d_R, d_load, out: SelectOu
     rc = _lib.dyn_reconf_select(C.byref(p), C.byref(s), _dev(d_R, torch.float32, "d_R"), _dev(d_load, torch.float32, "d_load"),
                                 S, W, C.byref(o), _dev(d_path_total, torch.float64, "d_path_total"), ws, nb, _stream())
     _check(rc, "dyn_reconf_select")
+
+
+def dyn_bin_tokens(window_ms, n_windows, in_edges, out_edges, d_t_ms, d_in_tok, d_out_tok, d_tok_in, d_tok_out,
+                   d_load_tps=None, n_req=None):
+    """Token sums per (window, class): d_tok_in / d_tok_out int64 tensors [W][C] (uint64 bits), d_load_tps float32 or None."""
+    ie, oe = _host(in_edges, np.uint32), _host(out_edges, np.uint32)
+    spec = _BinSpec(int(window_ms), int(n_windows), len(ie), len(oe), ie.ctypes.data, oe.ctypes.data)
+    n = int(d_t_ms.numel() if n_req is None else n_req)
+    rc = _lib.dyn_bin_tokens(C.byref(spec), _dev(d_t_ms, torch.int32, "d_t_ms"), _dev(d_in_tok, torch.int32, "d_in_tok"),
+                             _dev(d_out_tok, torch.int32, "d_out_tok"), n, _dev(d_tok_in, torch.int64, "d_tok_in"),
+                             _dev(d_tok_out, torch.int64, "d_tok_out"), _dev(d_load_tps, torch.float32, "d_load_tps"),
+                             _stream())
+    _check(rc, "dyn_bin_tokens")
+
+
+def dyn_carbon(d_E_window, d_intensity, d_carbon):
+    """gCO2 per scenario from window energies (float64 [S][W], Wh) and an intensity trace (float32 [W], gCO2/kWh)."""
+    S, W = d_E_window.shape
+    rc = _lib.dyn_carbon(_dev(d_E_window, torch.float64, "d_E_window"), _dev(d_intensity, torch.float32, "d_intensity"), S, W,
+                         _dev(d_carbon, torch.float64, "d_carbon"), _stream())
+    _check(rc, "dyn_carbon")

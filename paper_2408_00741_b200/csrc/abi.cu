@@ -113,6 +113,34 @@ int check_ws(const void *d_ws, size_t ws_bytes, size_t need) {
 
 size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
+// validation of a binning request shared by dyn_bin_trace and dyn_bin_tokens; fills the kernel parameters
+int make_bin_params(const dyn_bin_spec *spec, const uint32_t *d_t_ms, const uint32_t *d_in_tok, const uint32_t *d_out_tok,
+                    uint64_t n_req, BinParams *out) {
+    if (!spec) return DYN_EINVAL;
+    if (n_req > 0 && (!d_t_ms || !d_in_tok || !d_out_tok)) return DYN_EINVAL;
+    if (spec->window_ms == 0 || spec->n_windows == 0) return DYN_EINVAL;
+    if (spec->n_in_edges < 0 || spec->n_out_edges < 0 || spec->n_in_edges > DYN_MAX_EDGES ||
+        spec->n_out_edges > DYN_MAX_EDGES)
+        return DYN_EINVAL;
+    if ((spec->n_in_edges > 0 && !spec->in_edges) || (spec->n_out_edges > 0 && !spec->out_edges)) return DYN_EINVAL;
+    if (!strictly_ascending_u32(spec->in_edges, spec->n_in_edges) ||
+        !strictly_ascending_u32(spec->out_edges, spec->n_out_edges))
+        return DYN_EINVAL;
+    BinParams bp;
+    std::memset(&bp, 0, sizeof(bp));
+    bp.win = make_fastdiv(spec->window_ms);
+    bp.n_windows = spec->n_windows;
+    bp.n_in = spec->n_in_edges;
+    bp.n_out = spec->n_out_edges;
+    bp.C = (bp.n_in + 1) * (bp.n_out + 1);
+    if (uint64_t(spec->n_windows) * uint64_t(bp.C) >= (uint64_t(1) << 31)) return DYN_EINVAL;
+    for (int e = 0; e < bp.n_in; ++e) bp.in_edges[e] = spec->in_edges[e];
+    for (int e = 0; e < bp.n_out; ++e) bp.out_edges[e] = spec->out_edges[e];
+    bp.window_s = float(spec->window_ms) / 1000.0f;
+    *out = bp;
+    return DYN_OK;
+}
+
 // count tuples within the GPU budget in odometer order (n_0 fastest): {counts, 8 bits per TP index; number};
 // with out == nullptr only counts.  Returns -1 when there are more than `limit` tuples.
 int64_t enumerate_tuples(const dyn_profile *p, const dyn_space *sp, int64_t limit, uint2 *out) {
@@ -176,27 +204,10 @@ void dyn_set_timing_events(void *start_event, void *stop_event) {
 int dyn_bin_trace(const dyn_bin_spec *spec, const uint32_t *d_t_ms, const uint32_t *d_in_tok,
                   const uint32_t *d_out_tok, uint64_t n_req, uint32_t *d_counts, float *d_load,
                   uint64_t *d_dropped, void *stream) {
-    if (!spec || !d_counts || !d_dropped) return DYN_EINVAL;
-    if (n_req > 0 && (!d_t_ms || !d_in_tok || !d_out_tok)) return DYN_EINVAL;
-    if (spec->window_ms == 0 || spec->n_windows == 0) return DYN_EINVAL;
-    if (spec->n_in_edges < 0 || spec->n_out_edges < 0 || spec->n_in_edges > DYN_MAX_EDGES ||
-        spec->n_out_edges > DYN_MAX_EDGES)
-        return DYN_EINVAL;
-    if ((spec->n_in_edges > 0 && !spec->in_edges) || (spec->n_out_edges > 0 && !spec->out_edges)) return DYN_EINVAL;
-    if (!strictly_ascending_u32(spec->in_edges, spec->n_in_edges) ||
-        !strictly_ascending_u32(spec->out_edges, spec->n_out_edges))
-        return DYN_EINVAL;
+    if (!d_counts || !d_dropped) return DYN_EINVAL;
     BinParams bp;
-    std::memset(&bp, 0, sizeof(bp));
-    bp.win = make_fastdiv(spec->window_ms);
-    bp.n_windows = spec->n_windows;
-    bp.n_in = spec->n_in_edges;
-    bp.n_out = spec->n_out_edges;
-    bp.C = (bp.n_in + 1) * (bp.n_out + 1);
-    if (uint64_t(spec->n_windows) * uint64_t(bp.C) >= (uint64_t(1) << 31)) return DYN_EINVAL;
-    for (int e = 0; e < bp.n_in; ++e) bp.in_edges[e] = spec->in_edges[e];
-    for (int e = 0; e < bp.n_out; ++e) bp.out_edges[e] = spec->out_edges[e];
-    bp.window_s = float(spec->window_ms) / 1000.0f;
+    const int rc = make_bin_params(spec, d_t_ms, d_in_tok, d_out_tok, n_req, &bp);
+    if (rc != DYN_OK) return rc;
     DYN_CUDA_TRY(launch_bin_trace(bp, d_t_ms, d_in_tok, d_out_tok, n_req, d_counts, d_load,
                                   reinterpret_cast<unsigned long long *>(d_dropped),
                                   static_cast<cudaStream_t>(stream)));
@@ -421,6 +432,25 @@ int dyn_reconf_select(const dyn_profile *profile, const dyn_space *space, const 
     uint32_t *partial_bad = reinterpret_cast<uint32_t *>(ws + lay.off_partial + size_t(S) * size_t(chunks) * sizeof(double));
     DYN_CUDA_TRY(launch_totals(to_out(out), S, W, profile->C, lay.J, nullptr, nullptr, profile->T, space->F,
                                reinterpret_cast<const int32_t *>(ws + lay.off_tp), partial, partial_bad, st));
+    return DYN_OK;
+}
+
+int dyn_bin_tokens(const dyn_bin_spec *spec, const uint32_t *d_t_ms, const uint32_t *d_in_tok, const uint32_t *d_out_tok,
+                   uint64_t n_req, uint64_t *d_tok_in, uint64_t *d_tok_out, float *d_load_tps, void *stream) {
+    if (!d_tok_in || !d_tok_out) return DYN_EINVAL;
+    BinParams bp;
+    const int rc = make_bin_params(spec, d_t_ms, d_in_tok, d_out_tok, n_req, &bp);
+    if (rc != DYN_OK) return rc;
+    DYN_CUDA_TRY(launch_bin_tokens(bp, d_t_ms, d_in_tok, d_out_tok, n_req, reinterpret_cast<unsigned long long *>(d_tok_in),
+                                   reinterpret_cast<unsigned long long *>(d_tok_out), d_load_tps,
+                                   static_cast<cudaStream_t>(stream)));
+    return DYN_OK;
+}
+
+int dyn_carbon(const double *d_E_window, const float *d_intensity, int64_t S, int64_t W, double *d_carbon, void *stream) {
+    if (S < 0 || W < 0) return DYN_EINVAL;
+    if (S > 0 && (!d_carbon || (W > 0 && (!d_E_window || !d_intensity)))) return DYN_EINVAL;
+    DYN_CUDA_TRY(launch_carbon(d_E_window, d_intensity, S, W, d_carbon, static_cast<cudaStream_t>(stream)));
     return DYN_OK;
 }
 

@@ -129,6 +129,11 @@ cudaError_t launch_bin_trace(const BinParams &bp, const uint32_t *t_ms, const ui
                              uint64_t n_req, uint32_t *counts, float *load, unsigned long long *dropped,
                              cudaStream_t st);
 
+cudaError_t launch_bin_tokens(const BinParams &bp, const uint32_t *t_ms, const uint32_t *in_tok, const uint32_t *out_tok,
+                              uint64_t n_req, unsigned long long *tok_in, unsigned long long *tok_out, float *tps,
+                              cudaStream_t st);
+cudaError_t launch_carbon(const double *E_window, const float *intensity, int64_t S, int64_t W, double *carbon, cudaStream_t st);
+
 int sm_count();
 
 #ifdef __CUDACC__
