@@ -443,6 +443,24 @@ def measure_bin(dyn, gen, dev):
             out = {"workload": "cfg3", "kernel": "bin_trace_kernel", **r}
         else:
             out["long_trace_x8"] = r
+        if rep == 1:
+            # the token-weighted variant (sums of input and output tokens per window and class) on the same trace
+            ti = torch.empty((W, 9), dtype=torch.int64, device=dev)
+            to = torch.empty((W, 9), dtype=torch.int64, device=dev)
+            runt = lambda: dyn.dyn_bin_tokens(wl.trace.window_ms, W, gen.IN_EDGES, gen.OUT_EDGES, d[0], d[1], d[2], ti, to, load)
+            for _ in range(3):
+                runt()
+            torch.cuda.synchronize()
+            for k in range(K):
+                dyn.dyn_set_timing_events(*kev[k])
+                runt()
+            dyn.dyn_set_timing_events(None, None)
+            torch.cuda.synchronize()
+            mst = float(np.mean([a.elapsed_time(b) for a, b in kev]))
+            gbt = BYTES_PER_REQUEST * n / (mst * 1e-3) / 1e9
+            out["token_sums"] = {"kernel": "bin_tokens_kernel", "kernel_ms": mst, "requests_per_s": n / (mst * 1e-3),
+                                 "roofline": {"bound": "hbm", "achieved": gbt, "peak": peak, "unit": "GB/s",
+                                              "frac": gbt / peak, "traffic": None, "peak_source": src}}
         del d
     return out
 
