@@ -78,19 +78,6 @@ __global__ void __launch_bounds__(kThreads) reconf_cost_kernel(const ReconfArgs 
 constexpr int kPathThreads = 512;
 constexpr int kRegRows = 6;                     // rows of R a thread keeps in registers (its four columns of them)
 
-// block-wide minimum of v (all threads get it); `red` holds kPathThreads / 32 floats
-__device__ __forceinline__ float block_min(float v, float *red) {
-    float m;
-    asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(m) : "f"(v));
-    __syncthreads();                                         // `red` may still be read from the previous call
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
-    __syncthreads();
-    float r = red[0];
-#pragma unroll
-    for (int i = 1; i < kPathThreads / 32; ++i) r = fminf(r, red[i]);
-    return r;
-}
-
 // R[h][g]: the first rows_s rows sit in shared memory with row stride NS4 + 4 floats (rows stay 16-byte aligned;
 // NS4 = NS rounded up to a multiple of 4)
 // One CTA per (scenario, class).  Dynamic shared memory: Dp[NS4] | part[G][NS4] | Rs[rows_s][NS4 + 4].
@@ -100,7 +87,6 @@ __device__ __forceinline__ float block_min(float v, float *red) {
 // and the walk back finds each predecessor again as the lowest h that attains the minimum, with the same addition.
 __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfArgs a, const int rows_s) {
     extern __shared__ float4 smem4[];
-    __shared__ float red[kPathThreads / 32];
     const int NS = a.NS, NS4 = (NS + 3) & ~3, RSd = NS4 + 4;
     const int TG = NS4 / 4;                                  // groups of four targets
     const int lanes_t = (TG + 31) / 32 * 32;                 // threads side by side over the target groups (<= 256)
@@ -143,35 +129,50 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
     // the rest, split evenly over the source groups
     const int n_rest = NS > rows_sr ? NS - rows_sr : 0;
     const int g_lo = rows_sr + int(int64_t(hg) * n_rest / G), g_hi = worker ? rows_sr + int(int64_t(hg + 1) * n_rest / G) : g_lo;
-    // window 0 (the padding entries past NS are sources that never win: +inf); a thread owns entries tid and
-    // tid + kPathThreads of the state vector in every pass below except the scan
+    // Two barriers per window.  Dp holds the vector of the previous window as computed (not yet relative to its
+    // minimum); the minimum is gathered with one shared atomic per warp on an order-preserving integer key, in
+    // one of two slots that alternate between windows.  A thread owns entries tid and tid + kPathThreads of the
+    // vector outside the scan.  Padding entries past NS are sources that never win: +inf.
+    __shared__ unsigned int s_min[2];
+    auto key_of = [](float v) {
+        const unsigned int b = __float_as_uint(v);
+        return b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
+    };
+    auto val_of = [](unsigned int k) { return __uint_as_float(k ^ ((k >> 31) ? 0x80000000u : 0xffffffffu)); };
+    auto publish_min = [&](float lmin, int slot) {
+        float wm;
+        asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(wm) : "f"(lmin));
+        if ((tid & 31) == 0) atomicMin(&s_min[slot], key_of(wm));
+    };
+    if (tid == 0) s_min[0] = s_min[1] = 0xffffffffu;
+    __syncthreads();
     double base = 0.0;
-    float lmin = CUDART_INF_F;
-    for (int g = tid; g < NS4; g += kPathThreads) {
-        const float v = g < NS ? (W > 0 ? cost[g] : 0.f) : CUDART_INF_F;
-        Dp[g] = v;
-        lmin = fminf(lmin, v);
-    }
-    float m = block_min(lmin, red);                          // its barriers also publish Rs
-    for (int64_t w = 1; w < W; ++w) {
-        // keep differences only: the minimum goes to the fp64 base (all +inf stays +inf)
-        const float shift = (m < CUDART_INF_F) ? m : 0.f;
-        base += double(shift);
-        for (int g = tid; g < NS; g += kPathThreads) {
-            const float v = Dp[g] - shift;
+    {
+        float lmin = CUDART_INF_F;
+        for (int g = tid; g < NS4; g += kPathThreads) {
+            const float v = g < NS ? (W > 0 ? cost[g] : 0.f) : CUDART_INF_F;
             Dp[g] = v;
-            hist[(w - 1) * NS + g] = v;
+            lmin = fminf(lmin, v);
         }
-        // the next window's costs, asked for before the barrier so that their latency hides behind the scan
+        publish_min(lmin, 0);
+    }
+    __syncthreads();                                         // publishes Dp, the minimum and Rs
+    for (int64_t w = 1; w < W; ++w) {
+        // keep differences only: the previous minimum goes to the fp64 base (all +inf stays +inf)
+        const float mprev = val_of(s_min[(w - 1) & 1]);
+        const float shift = (mprev < CUDART_INF_F) ? mprev : 0.f;
+        base += double(shift);
+        if (tid == 0) s_min[w & 1] = 0xffffffffu;            // this window's slot; last read before the previous barrier
+        for (int g = tid; g < NS; g += kPathThreads) hist[(w - 1) * NS + g] = Dp[g] - shift;
+        // this window's costs, asked for now so that their latency hides behind the scan
         const float cw0 = tid < NS ? cost[w * NS + tid] : 0.f;
         const float cw1 = tid + kPathThreads < NS ? cost[w * NS + tid + kPathThreads] : 0.f;
-        __syncthreads();
         if (worker) {
             float b0 = CUDART_INF_F, b1 = CUDART_INF_F, b2 = CUDART_INF_F, b3 = CUDART_INF_F;
 #pragma unroll 2
             for (int q = q_lo; q < q_hi; ++q) {
                 const float4 d4 = reinterpret_cast<const float4 *>(Dp)[q];
-                const float dv[4] = {d4.x, d4.y, d4.z, d4.w};
+                const float dv[4] = {d4.x - shift, d4.y - shift, d4.z - shift, d4.w - shift};
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const float4 r = *reinterpret_cast<const float4 *>(Rs + (4 * q + j) * RSd + 4 * tg);
@@ -183,14 +184,14 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
             }
 #pragma unroll
             for (int j = 0; j < kRegRows; ++j) {
-                const float d = hreg[j] >= 0 ? Dp[hreg[j]] : CUDART_INF_F;
+                const float d = hreg[j] >= 0 ? Dp[hreg[j]] - shift : CUDART_INF_F;
                 b0 = fminf(b0, d + rreg[j].x);
                 b1 = fminf(b1, d + rreg[j].y);
                 b2 = fminf(b2, d + rreg[j].z);
                 b3 = fminf(b3, d + rreg[j].w);
             }
             for (int h = g_lo; h < g_hi; ++h) {
-                const float d = Dp[h];
+                const float d = Dp[h] - shift;
                 const float *row = a.R + size_t(h) * NS + 4 * tg;
                 b0 = fminf(b0, d + __ldg(row));
                 if (4 * tg + 1 < NS) b1 = fminf(b1, d + __ldg(row + 1));
@@ -199,17 +200,19 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
             }
             reinterpret_cast<float4 *>(part + size_t(hg) * NS4)[tg] = make_float4(b0, b1, b2, b3);
         }
-        __syncthreads();
-        lmin = CUDART_INF_F;
+        __syncthreads();                                     // every reader of Dp is done; the partial minima are in
+        float lmin = CUDART_INF_F;
         for (int g = tid; g < NS; g += kPathThreads) {
             float best = part[g];
             for (int k = 1; k < G; ++k) best = fminf(best, part[k * NS4 + g]);
             const float d = (g == tid ? cw0 : cw1) + best;
-            Dp[g] = d;                                       // every reader of Dp has passed the barrier above
+            Dp[g] = d;
             lmin = fminf(lmin, d);
         }
-        m = block_min(lmin, red);
+        publish_min(lmin, int(w & 1));
+        __syncthreads();                                     // publishes Dp and the minimum
     }
+    const float m = W > 0 ? val_of(s_min[(W - 1) & 1]) : 0.f;
     if (W == 0) {
         if (tid == 0) a.path_total[sc] = 0.0;
         return;
