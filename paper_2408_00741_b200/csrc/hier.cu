@@ -167,6 +167,37 @@ __global__ void __launch_bounds__(256) hier_shard_kernel(const HierArgs a) {
         if (nmax > a.Nmax) nmax = a.Nmax;
         float best = CUDART_INF_F;
         int bnt = -1;
+        if (FAST && a.T <= 4) {
+            // the constants of the (at most four) highest-frequency pairs stay in registers for the whole walk
+            float icm[4], llim[4];
+            uint32_t row[4];
+            int nlim[4];
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const int tt = t < a.T ? t : 0;
+                const int p = tt * a.F + a.F - 1;
+                const float4 pc = load16<true>(a.ws, origin + uint32_t(int(c) * a.T * a.F + p) * 16u);
+                icm[t] = pc.x;
+                llim[t] = t < a.T ? pc.z : -1.f;
+                row[t] = origin + uint32_t(a.off_rows2 - a.off_pair2) + uint32_t((int(c) * a.T * a.F + p) * (a.M + 1)) * 8u;
+                nlim[t] = t < a.T ? budget / a.tp[tt] : 0;  // TP ascending: the limits descend
+            }
+            for (int n = 1; n <= nmax; ++n) {
+                const float nf = float(n), ln = PL * (1.0f / nf);
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    if (n > nlim[t]) break;
+                    float e;
+                    bool ok;
+                    fast_one<true>(a.ws, row[t], ln, icm[t], llim[t], e, ok);
+                    const float E = nf * e;
+                    if (ok && E < best) {             // ascending (n, t): strict compare keeps the lowest index
+                        best = E;
+                        bnt = (n - 1) * a.T + t;
+                    }
+                }
+            }
+        } else
         for (int n = 1; n <= nmax; ++n) {
             const float nf = float(n), ln = PL * (1.0f / nf);
             for (int t = 0; t < a.T; ++t) {
