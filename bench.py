@@ -389,7 +389,9 @@ def run_ours(args, rank, world, local_rank):
         except Exception as exc:
             result["hierarchical"] = {"error": repr(exc)}
         try:
-            result["mixed_pools"] = measure_mixed(dyn, gen, dev)
+            # 32 GPUs per pool (1624 count tuples) and a small pool of 16 (200 tuples, passes half empty)
+            result["mixed_pools"] = measure_mixed(dyn, gen, dev, n_max=32, budget=32)
+            result["mixed_pools"]["small_pool"] = measure_mixed(dyn, gen, dev, n_max=16, budget=16)
         except Exception as exc:
             result["mixed_pools"] = {"error": repr(exc)}
         try:
@@ -668,7 +670,8 @@ def main():
         dev = torch.device("cuda", local_rank)
         torch.cuda.set_device(dev)
         print(json.dumps({"bin_trace": measure_bin(dyn, gen, dev), "materialised": measure_materialised(dyn, gen, dev),
-                          "hierarchical": measure_hier(dyn, gen, dev), "mixed_pools": measure_mixed(dyn, gen, dev),
+                          "hierarchical": measure_hier(dyn, gen, dev), "mixed_pools": measure_mixed(dyn, gen, dev, n_max=32, budget=32),
+                          "mixed_pools_small": measure_mixed(dyn, gen, dev),
                           "reconfiguration": measure_reconf(dyn, gen, dev)}))
         return
     run_ours(args, rank, world, local_rank)
