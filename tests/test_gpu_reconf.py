@@ -75,8 +75,8 @@ def test_hour_trace_shape(dyn):
 
 
 def test_many_states_with_budget_and_ragged_sizes(dyn):
-    """NS = 37 * 4 states (more than one per thread of a warp, not a multiple of 32), 45 windows (a partial block
-    of back pointers), a GPU budget that rules out part of the states."""
+    """NS = 37 * 4 states (not a multiple of 32), 45 windows (not a multiple of the eight windows the walk back
+    looks ahead), a GPU budget that rules out part of the states."""
     wl = gen.workload("cfg2")
     prof = wl.profile()
     sp = gen.make_space(wl.f_cand_mhz, 37, wl.window_s, gpu_budget=48)
@@ -117,3 +117,22 @@ def test_single_window_and_errors(dyn):
         dyn.dyn_reconf_select(p, s, torch.zeros((NS, NS), device="cuda"), torch.zeros((1, 1, 9), device="cuda"), out, tot,
                               ws[:256])
     assert e.value.status == dyn.DYN_EWORKSPACE
+
+
+@pytest.mark.parametrize("n_max,W", [(5, 19), (7, 9)])
+def test_state_counts_that_are_not_multiples_of_four(dyn, n_max, W):
+    """TP 2/4/8 with 5 or 7 instance counts: 15 and 21 states (padded vector entries, ragged rows of the table)."""
+    wl = gen.workload("cfg1")
+    prof, sp = wl.profile(), gen.make_space(wl.f_cand_mhz, n_max, wl.window_s)
+    load = gen.random_loads((2, W, 9), seed=55 + n_max, mean=0.8, zero_frac=0.0)
+    _check(dyn, prof, sp, _table(n_max * prof.T, 4, 2.0), load)
+
+
+def test_more_states_than_fit_on_chip(dyn):
+    """400 states: the overhead table (640 KB) only partly fits in shared memory and registers, the rest is read
+    from global memory; the walk back takes its plain path (more than 256 states)."""
+    wl = gen.workload("cfg2")
+    prof = wl.profile()
+    sp = gen.make_space(wl.f_cand_mhz, 100, wl.window_s)
+    load = gen.random_loads((1, 12, 9), seed=56, mean=6.0, zero_frac=0.0)
+    _check(dyn, prof, sp, _table(400, 5, 8.0), load)
