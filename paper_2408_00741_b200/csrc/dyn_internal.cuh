@@ -56,7 +56,7 @@ __device__ __forceinline__ uint32_t fastdiv(uint32_t n, const FastDiv &f) {
 //                   vlim = largest v with TBT <= slo_tbt[c] and u <= 1 when TBT does not decrease
 //                   along the row (-1 for a never-feasible pair), NaN when it does decrease somewhere.
 //   slo[c]          slo_tbt[c]
-//   pair2[c][p]     float4 {icm, icm, llim, 0} for the threshold path: icm = (M-1)/cap, the table position per
+//   pair2[c][p]     float4 {icm, icm, llim, cap} for the threshold path (cap: the pair's interpolated capacity): icm = (M-1)/cap, the table position per
 //                   unit of per-instance load l (x = l*icm); llim = largest l with TBT <= slo_tbt[c] and
 //                   u <= 1 (-1 for a never-feasible pair)
 //   rows2[c][p][m]  m = 0..M, float2 {a, b}: the energy line of segment m in l, e = a + l*b (a = e_a - m*e_d,

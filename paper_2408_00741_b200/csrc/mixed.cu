@@ -46,13 +46,14 @@ struct MixedArgs {
     float *best_E;
 };
 
-// capacity at the highest candidate frequency, from the resolved pair constant ic = (M-1)/(M*cap)
+// capacity at the highest candidate frequency, as interpolated from the profile (whether or not that pair meets its
+// TTFT SLO: the split of the load does not depend on feasibility)
 __global__ void mixed_caph_kernel(const MixedArgs a) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= a.C * a.T) return;
     const int c = i / a.T, t = i - c * a.T;
-    const float ic = a.pairc[c * (a.T * a.F) + t * a.F + a.F - 1].x;
-    a.caph[i] = ic > 0.f ? float(double(a.M - 1) / (double(a.M) * double(ic))) : 0.f;
+    const float4 *pair2 = reinterpret_cast<const float4 *>(a.ws + a.off_pair2);
+    a.caph[i] = pair2[c * (a.T * a.F) + t * a.F + a.F - 1].w;
 }
 
 // true when every pair row has a load threshold (vlim is NaN for a row whose TBT decreases somewhere)
@@ -316,6 +317,8 @@ cudaError_t launch_mixed(const ResolvedLayout &lay, void *d_ws, size_t off_tuple
     a.tiles = tiles; a.K = K;
     a.C = lay.C; a.T = lay.T; a.F = lay.F; a.M = lay.M;
     a.counts = d_counts; a.freq = d_freq; a.tuple = d_tuple; a.best_E = d_best_E;
+    a.ws = ws;
+    a.off_pair2 = int32_t(lay.off_pair2); a.off_rows2 = int32_t(lay.off_rows2); a.off_end = int32_t(lay.off_tp);
     mixed_caph_kernel<<<(lay.C * lay.T + 127) / 128, 128, 0, st>>>(a);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess || tiles == 0) return e;

@@ -121,7 +121,7 @@ __global__ void resolve_kernel(const ResolveParams rp, float4 *__restrict__ rows
             // packed pair) and the largest per-instance load within the SLO and the capacity
             const float icm = pair_ok ? float(double(M - 1) / cap) : 0.f;
             const float llim = (pair_ok && xlim >= 0.0) ? float(xlim / double(M - 1) * cap) : -1.f;
-            pair2[size_t(c) * P + p] = make_float4(icm, icm, llim, 0.f);
+            pair2[size_t(c) * P + p] = make_float4(icm, icm, llim, float(cap));   // cap as interpolated, feasible or not
             if (p == 0) slo[c] = rp.slo_tbt[c];
             if (c == 0 && p < rp.T) tp[p] = rp.tp[p];
         }

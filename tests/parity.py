@@ -5,6 +5,7 @@ from __future__ import annotations
 import numpy as np
 import torch
 
+import gen
 import oracle
 
 REL_TOL = 1e-5          # energies, totals; also the near-tie / near-bound exemption width
@@ -85,3 +86,25 @@ def check_selection(prof, sp, load, got_idx, got_E, ref, max_exempt_frac=0.01):
             f"tile {(s, w, c)}: oracle j={jo} E={E[jo] if jo >= 0 else None}, gpu j={jg} E={got_E[s, w, c]}"
         fixed[s, w, c] = jo
     return fixed, len(bad)
+
+
+def random_tables(seed, monotone_tbt, large=False):
+    """Free-form tables (not the closed forms): TBT rises and falls with load unless monotone_tbt.
+    large: 48 load knots and 40 candidate frequencies, too big to stage for all classes at once."""
+    rng = np.random.default_rng(seed)
+    Cn, T, R, M = 9, 3, 5, (48 if large else 6)
+    tp = np.array([1, 2, 8], np.int32)
+    fg = np.array([800, 1000, 1300, 1700, 1980], np.float32)
+    ttft = (0.2 + 0.9 * rng.random((Cn, T, R))).astype(np.float32)
+    cap = (1.0 + 6.0 * rng.random((Cn, T, R))).astype(np.float32)
+    tbt = (0.04 + 0.1 * rng.random((Cn, T, R, M)))
+    if monotone_tbt:
+        tbt = np.sort(tbt, axis=-1)
+        tbt[:, :, :, 3] = tbt[:, :, :, 2]                 # a flat segment is still "never decreases"
+    pw = (150 + 600 * rng.random((Cn, T, R, M)))
+    prof = gen.Profile(tp, fg, ttft, cap, tbt.astype(np.float32), pw.astype(np.float32))
+    cand = np.array([800, 850, 1000, 1111, 1500, 1700, 1979, 1980], np.float32)
+    if large:
+        cand = np.linspace(800, 1980, 40).astype(np.float32)
+    sp = gen.make_space(cand, 40, 60.0, slo_ttft=0.8, slo_tbt=0.1)
+    return prof, sp

@@ -132,3 +132,15 @@ def test_limits_and_errors(dyn):
     with pytest.raises(dyn.DynError) as e:
         dyn.dyn_mixed_select(p, s1, torch.zeros((1, 1, 9), device="cuda"), out, ws[:256])
     assert e.value.status == dyn.DYN_EWORKSPACE
+
+
+@pytest.mark.parametrize("large", [False, True], ids=["tables-in-shared-memory", "tables-through-L1"])
+@pytest.mark.parametrize("monotone", [False, True], ids=["tbt-rises-and-falls", "tbt-never-decreases"])
+def test_free_form_tables(dyn, monotone, large):
+    """Both variants of the kernel: the threshold variant needs every TBT row monotone and tables that fit in
+    shared memory; a row that decreases somewhere, or larger tables, go to the plain variant."""
+    from parity import random_tables
+    prof, sp0 = random_tables(23, monotone, large)
+    sp = gen.make_space(sp0.f_cand_mhz[::5] if large else sp0.f_cand_mhz, 6, 60.0, slo_ttft=0.8, slo_tbt=0.1, gpu_budget=14)
+    load = gen.random_loads((2, 9, 9), seed=35, mean=6.0)
+    _check(dyn, prof, sp, load, max_exempt=0.03)

@@ -6,7 +6,7 @@ import torch
 
 import gen
 import oracle
-from parity import REL_TOL, check_selection, gpu_eval_select, gpu_profile_space, out_to_host
+from parity import REL_TOL, check_selection, gpu_eval_select, gpu_profile_space, out_to_host, random_tables
 
 pytestmark = pytest.mark.gpu
 
@@ -126,35 +126,13 @@ def test_eval_configs_then_select_small(dyn, case):
     assert np.array_equal(o["gpus"].astype(np.int64), tot["gpus"].astype(np.int64))
 
 
-def _random_tables(seed, monotone_tbt, large=False):
-    """Free-form tables (not the closed forms): TBT rises and falls with load unless monotone_tbt.
-    large: 48 load knots and 40 candidate frequencies, too big to stage for all classes at once."""
-    rng = np.random.default_rng(seed)
-    Cn, T, R, M = 9, 3, 5, (48 if large else 6)
-    tp = np.array([1, 2, 8], np.int32)
-    fg = np.array([800, 1000, 1300, 1700, 1980], np.float32)
-    ttft = (0.2 + 0.9 * rng.random((Cn, T, R))).astype(np.float32)
-    cap = (1.0 + 6.0 * rng.random((Cn, T, R))).astype(np.float32)
-    tbt = (0.04 + 0.1 * rng.random((Cn, T, R, M)))
-    if monotone_tbt:
-        tbt = np.sort(tbt, axis=-1)
-        tbt[:, :, :, 3] = tbt[:, :, :, 2]                 # a flat segment is still "never decreases"
-    pw = (150 + 600 * rng.random((Cn, T, R, M)))
-    prof = gen.Profile(tp, fg, ttft, cap, tbt.astype(np.float32), pw.astype(np.float32))
-    cand = np.array([800, 850, 1000, 1111, 1500, 1700, 1979, 1980], np.float32)
-    if large:
-        cand = np.linspace(800, 1980, 40).astype(np.float32)
-    sp = gen.make_space(cand, 40, 60.0, slo_ttft=0.8, slo_tbt=0.1)
-    return prof, sp
-
-
 @pytest.mark.parametrize("large", [False, True], ids=["tables-in-shared-memory", "tables-per-class"])
 @pytest.mark.parametrize("monotone", [False, True], ids=["tbt-rises-and-falls", "tbt-never-decreases"])
 def test_eval_select_free_form_tables(dyn, monotone, large):
     """Both evaluation paths of the fused kernel: per-candidate TBT interpolation when some table row
     decreases with load, the load-threshold path when none does; with all classes' tables staged at
     once, and with the per-class kernel that larger tables need."""
-    prof, sp = _random_tables(17, monotone, large)
+    prof, sp = random_tables(17, monotone, large)
     load = gen.random_loads((2, 37 if not large else 11, 9), seed=5, mean=6.0)
     J = sp.n_max * prof.T * sp.F
     ref = oracle.eval_select(prof, sp, load)
