@@ -136,3 +136,13 @@ def test_more_states_than_fit_on_chip(dyn):
     sp = gen.make_space(wl.f_cand_mhz, 100, wl.window_s)
     load = gen.random_loads((1, 12, 9), seed=56, mean=6.0, zero_frac=0.0)
     _check(dyn, prof, sp, _table(400, 5, 8.0), load)
+
+
+@pytest.mark.parametrize("monotone", [False, True], ids=["tbt-rises-and-falls", "tbt-never-decreases"])
+def test_free_form_tables(dyn, monotone):
+    """Profiles that are not the closed forms (per-pair TTFT misses, TBT that rises and falls with load)."""
+    from parity import random_tables
+    prof, sp0 = random_tables(31, monotone)
+    sp = gen.make_space(sp0.f_cand_mhz, 12, 60.0, slo_ttft=0.8, slo_tbt=0.1)
+    load = gen.random_loads((1, 14, 9), seed=57, mean=6.0, zero_frac=0.0)
+    _check(dyn, prof, sp, _table(sp.n_max * prof.T, 6, 4.0), load)
