@@ -80,7 +80,11 @@ def test_eval_select_small(dyn, case):
     assert (ref["best_idx"] >= 0).sum() > 0.3 * ref["best_idx"].size
 
 
-@pytest.mark.parametrize("case", CASES[:5] + CASES[7:], ids=lambda c: "-".join(f"{k}{v}" for k, v in c.items()))
+ODD = [dict(name="cfg2", W=9, S=1, n_max=7, budget=20, seed=8),       # odd instance count under a GPU budget
+       dict(name="cfg3", W=9, S=1, n_max=33, seed=9)]                 # odd, more than a warp of counts
+
+
+@pytest.mark.parametrize("case", CASES + ODD, ids=lambda c: "-".join(f"{k}{v}" for k, v in c.items()))
 def test_eval_configs_then_select_small(dyn, case):
     wl, prof, sp, load = _small(**case)
     if case["name"] == "cfg5":
