@@ -54,10 +54,11 @@ def test_unsorted_trace_and_few_windows(dyn):
     _check(dyn, t, i, o, 86_400_000, 1)                                     # one window
 
 
-@pytest.mark.parametrize("n,per_window", [(3_000_000, 0.7), (20_000_000, 12.0)])
+@pytest.mark.parametrize("n,per_window", [(3_000_000, 0.7), (20_000_000, 12.0), (45_000_000, 40.0)])
 def test_long_sparse_trace(dyn, n, per_window):
     """Many windows per request slice: a CTA's slice no longer fits its shared-memory bins and is taken in
-    pieces (long slices, 12 requests per window) or spills to global atomics (fewer than one per window)."""
+    pieces (long slices, 12 requests per window) or spills to global atomics (fewer than one per window); with
+    45 M requests the grid grows so that a slice stays at about 24 K requests."""
     rng = np.random.default_rng(7)
     W = int(n / per_window)
     wm = 3
