@@ -20,6 +20,13 @@ __device__ __forceinline__ float warp_min(float v) {
     return r;
 }
 
+// smallest value over the lanes of `mask` (the caller's group; all its lanes call with the same mask)
+__device__ __forceinline__ float group_min(float v, unsigned mask) {
+    float r;
+    asm volatile("redux.sync.min.f32 %0, %1, %2;" : "=f"(r) : "f"(v), "r"(mask));
+    return r;
+}
+
 // ---- table access -----------------------------------------------------------------------------
 // General path: `base` is the byte address of the pair's row minus 16 * bits(2^23): the entry address is
 // one multiply-add away from the bit pattern of y = 2^23 + floor(x).  Shared memory is addressed in 32 bits.

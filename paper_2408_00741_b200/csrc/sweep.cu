@@ -113,12 +113,16 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
     const int64_t r_begin = (CLS ? unit : unit / a.C) * a.rows_per_warp;
     const int64_t r_end = r_begin + a.rows_per_warp < a.rows_total ? r_begin + a.rows_per_warp : a.rows_total;
 
-    // FULL: lanes are 32 instance counts and every lane walks all pairs (compile-time stride 1);
-    // otherwise (Nmax < 32) the warp splits into G groups that take every G-th pair
+    // FULL: the 32 lanes are 32 instance counts of the same tiles.  Otherwise (Nmax <= 16) the warp splits
+    // into TG groups of LN lanes; the lanes of a group are the instance counts, and every group takes its own
+    // TT tiles of a pass, so the per-tile reductions and the pair recovery of all groups share their instructions
     const int LN = FULL ? 32 : 1 << a.ln_log2;
-    const int G = FULL ? 1 : 32 >> a.ln_log2;
+    const int TG = FULL ? 1 : 32 >> a.ln_log2;
     const int nl = lane & (LN - 1);
     const int g = FULL ? 0 : lane >> a.ln_log2;
+    const int gsh = g * LN;                          // first lane of the group
+    const unsigned lowmask = FULL ? kFull : (1u << LN) - 1u;
+    const unsigned gmask = lowmask << gsh;           // the lanes of this group
     const int P = a.P, RS = a.M + 1, C = a.C;
     const float Mf = float(a.M);
     const char *ws = a.ws;
@@ -172,19 +176,19 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
     // threshold path with staged tables: row offsets as subnormal floats (see fast_two)
     const uint64_t two23_2 = pack2(kTwo23, kTwo23);
     const uint64_t eight2 = pack2(units(8u), units(8u));
-    const float off0 = row_offset_units(crow + uint32_t(g) * pstep);
-    const float offs = float(int(uint32_t(G) * pstep)) * units(1u);
+    const float off0 = row_offset_units(crow);
+    const float offs = float(int(pstep)) * units(1u);
     const uint64_t off2_first = pack2(off0, off0), off2_step = pack2(offs, offs);
     constexpr int NCH = TT * NPL;                    // candidates per lane and pair, an even number
     static_assert(NCH % 2 == 0, "candidates are evaluated two at a time");
 
     // per-lane constants of the pair recovery: lane p re-evaluates pair p0 + p.  With at most 32 pairs and
     // no GPU budget there is one round, and the lane's pair constants stay in registers for all tiles
-    const uint32_t cpair_lane = cpair + uint32_t(lane) * (FAST ? 16u : 8u);
-    const uint32_t crow_lane = crow + uint32_t(lane) * pstep;
-    const bool one_round = !BUDGET && P <= 32;
+    const uint32_t cpair_lane = cpair + uint32_t(nl) * (FAST ? 16u : 8u);
+    const uint32_t crow_lane = crow + uint32_t(nl) * pstep;
+    const bool one_round = !BUDGET && P <= LN;
     float rc_ic = 0.f, rc_lim = FAST ? -1.f : -CUDART_INF_F;          // a lane without a pair never hits
-    if (one_round && lane < P) {
+    if (one_round && nl < P) {
         if (FAST) {
             const float4 pc = load16<SMEM>(ws, cpair_lane);
             rc_ic = pc.x;
@@ -194,13 +198,15 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
             rc_lim = slo_c;
         }
     }
-    const uint32_t rc_row = (one_round && lane < P) ? crow_lane : crow;
+    const uint32_t rc_row = (one_round && nl < P) ? crow_lane : crow;
     const int sh_n = FULL ? 5 : a.ln_log2;           // n - 1 = (chain number << sh_n) + lane number
-    const float *lp = a.load + (r_begin * C + c);    // load of the pass's first tile; tiles are C floats apart
-    int64_t oi = r_begin * C + c;                    // its index in the outputs
+    const int tpp = TT * TG;                         // tiles of a pass
+    const float *lp = a.load + ((r_begin + g * TT) * C + c);          // load of the group's first tile; tiles are C floats apart
+    int64_t oi = (r_begin + g * TT) * C + c;         // its index in the outputs
 
-    for (int64_t r = r_begin; r < r_end; r += TT, lp += TT * C, oi += int64_t(TT) * C) {
-        const int nt = r_end - r < TT ? int(r_end - r) : TT;          // tiles of this pass (warp-uniform)
+    for (int64_t r = r_begin; r < r_end; r += tpp, lp += tpp * C, oi += int64_t(tpp) * C) {
+        const int64_t left = r_end - (r + g * TT);
+        const int nt = left < TT ? (left > 0 ? int(left) : 0) : TT;   // tiles of this group in this pass
         // chain q = t*NPL + k: tile t of this pass, k-th instance count of the lane; `best` is the least
         // energy of ONE instance over the feasible pairs of the chain
         float best[NCH];
@@ -223,7 +229,7 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
         if (FAST && SMEM) {
             uint64_t off2 = off2_first;
 #pragma unroll kPairUnroll
-            for (int p = g; p < P; p += G) {
+            for (int p = 0; p < P; ++p) {
                 uint64_t icm2, lim2;
                 asm("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(icm2), "=l"(lim2) : "r"(cpair + uint32_t(p) * 16u));
                 const float lim = __uint_as_float(uint32_t(lim2));
@@ -236,7 +242,7 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
             }
         } else if (FAST) {
 #pragma unroll 4
-            for (int p = g; p < P; p += G) {
+            for (int p = 0; p < P; ++p) {
                 const float4 pc = load16<SMEM>(ws, cpair + uint32_t(p) * 16u);
                 const uint32_t row = crow + uint32_t(p) * pstep;
 #pragma unroll
@@ -249,7 +255,7 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
             }
         } else {
 #pragma unroll 8
-            for (int p = g; p < P; p += G) {
+            for (int p = 0; p < P; ++p) {
                 const float2 pc = load8<SMEM>(ws, cpair + uint32_t(p) * 8u);
                 const uint32_t base = crow + uint32_t(p) * pstep - kTwo23Bits * 16u;
 #pragma unroll
@@ -263,7 +269,7 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
         float my_E = CUDART_INF_F;
 #pragma unroll
         for (int t = 0; t < TT; ++t) {
-            if (t >= nt) break;                      // warp-uniform
+            if (FULL && t >= nt) break;              // one group: uniform (several groups: the idle ones run along)
             // the lane's chains in ascending n: strict compare keeps the lower n on ties.  Pool energy =
             // n * (energy of one instance); the zero addend turns -0 into +0, so equal energies have equal bits
             float E = keep[0] ? fmaf(best[t * NPL], nf[0], 0.f) : CUDART_INF_F;
@@ -279,9 +285,9 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
             // smallest energy of the tile, then the fewest instances that attain it (lowest index: n is the
             // slowest digit of j); lanes of different pair groups may hold the same n.  A tile without a
             // feasible candidate (minimum +inf) runs through the same steps and finds no pair: -1 / +inf
-            const float Emin = warp_min(E);
+            const float Emin = group_min(E, gmask);
             const uint32_t n1 = uint32_t(kk << sh_n) + uint32_t(nl);              // n - 1
-            const uint32_t n1min = __reduce_min_sync(kFull, E == Emin ? n1 : 0xffffffffu);
+            const uint32_t n1min = __reduce_min_sync(gmask, E == Emin ? n1 : 0xffffffffu);
             const float nfm = float(n1min + 1u);
             // L/n of the winning instance count, from the lane that holds it (bit-identical by construction)
             float lnk = DYN_LN(t * NPL);
@@ -290,7 +296,7 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
 #pragma unroll
                 for (int k = 1; k < NPL; ++k) lnk = (k == kstar) ? DYN_LN(t * NPL + k) : lnk;
             }
-            const float lnm = __shfl_sync(kFull, lnk, int(n1min) & (LN - 1));
+            const float lnm = __shfl_sync(kFull, lnk, gsh + (int(n1min) & (LN - 1)));
             // recover the pair: lanes re-evaluate (nmin, p) for 32 pairs at a time, same arithmetic, and the
             // first pair that reproduces the minimum bit for bit is the lowest-index one
             int pstar = -1;
@@ -299,7 +305,7 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
                 bool ok;
                 if (FAST) fast_one<SMEM>(ws, rc_row, lnm, rc_ic, rc_lim, e, ok);
                 else general_one<SMEM>(ws, rc_row - kTwo23Bits * 16u, lnm, rc_ic, rc_lim, Mf, e, ok);
-                pstar = __ffs(__ballot_sync(kFull, ok && (fmaf(e, nfm, 0.f) == Emin))) - 1;
+                pstar = __ffs((__ballot_sync(kFull, ok && (fmaf(e, nfm, 0.f) == Emin)) >> gsh) & lowmask) - 1;
             } else {
                 int pm = P;
                 if (BUDGET) {
@@ -307,9 +313,10 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
                     for (int tt = 0; tt < a.T; ++tt) ntp += (int64_t(n1min + 1u) * a.tp[tt] <= int64_t(a.budget)) ? 1 : 0;
                     pm = ntp * a.F;
                 }
-                for (int p0 = 0; p0 < pm; p0 += 32) {
+                // one group stops at its first hit; several groups walk all rounds together (their bounds differ)
+                for (int p0 = 0; p0 < (FULL ? pm : P); p0 += LN) {
                     bool hit = false;
-                    if (p0 + lane < pm) {
+                    if (pstar < 0 && p0 + nl < pm) {
                         float e;
                         bool ok;
                         if (FAST) {
@@ -321,21 +328,19 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
                         }
                         hit = ok && (fmaf(e, nfm, 0.f) == Emin);
                     }
-                    const unsigned m = __ballot_sync(kFull, hit);
-                    if (m) {
-                        pstar = p0 + __ffs(m) - 1;
-                        break;
-                    }
+                    const unsigned m = (__ballot_sync(kFull, hit) >> gsh) & lowmask;
+                    if (m && pstar < 0) pstar = p0 + __ffs(m) - 1;
+                    if (FULL && m) break;
                 }
             }
-            if (lane == t) {
+            if (nl == t) {
                 my_idx = pstar >= 0 ? int32_t(n1min * uint32_t(P) + uint32_t(pstar)) : -1;
                 my_E = Emin;
             }
         }
-        if (lane < nt) {
-            best_idx[oi + lane * C] = my_idx;
-            best_E[oi + lane * C] = my_E;
+        if (nl < nt) {
+            best_idx[oi + nl * C] = my_idx;
+            best_E[oi + nl * C] = my_E;
         }
     }
 }
@@ -563,7 +568,8 @@ cudaError_t launch_es_variant(SweepArgs &a, int32_t *best_idx, float *best_E, cu
     // about four work units per resident warp: all units cost the same, so the tail is short
     const int64_t want_units = int64_t(sm_count()) * resident * kWarps * 4;
     int64_t rpw = (a.tiles + want_units - 1) / want_units;          // rows of one class per unit
-    rpw = (rpw + TT - 1) / TT * TT;
+    const int tpp = TT * (FULL ? 1 : 32 >> a.ln_log2);               // tiles of a pass
+    rpw = (rpw + tpp - 1) / tpp * tpp;
     a.rows_per_warp = rpw;
     a.blocks = (a.rows_total + rpw - 1) / rpw;
     const int64_t units = a.blocks * a.C;
@@ -623,6 +629,7 @@ cudaError_t launch_eval_select(const ResolvedLayout &lay, const void *d_ws, cons
     // lanes per n-group: smallest power of two covering Nmax, at most 32
     int ln = 0;
     while ((1 << ln) < lay.Nmax && ln < 5) ++ln;
+    if (ln < 3) ln = 3;                             // a group of lanes also holds the results of its 8 tiles
     a.ln_log2 = ln;
     const int npl = (lay.Nmax + 31) / 32;           // instance counts per lane
     // four candidates per lane share each pair's constants
