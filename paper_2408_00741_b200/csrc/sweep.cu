@@ -206,7 +206,7 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
 
     for (int64_t r = r_begin; r < r_end; r += tpp, lp += tpp * C, oi += int64_t(tpp) * C) {
         const int64_t left = r_end - (r + g * TT);
-        const int nt = left < TT ? (left > 0 ? int(left) : 0) : TT;   // tiles of this group in this pass
+        const int nt = left < TT ? (FULL || left > 0 ? int(left) : 0) : TT;          // tiles of this group in this pass
         // chain q = t*NPL + k: tile t of this pass, k-th instance count of the lane; `best` is the least
         // energy of ONE instance over the feasible pairs of the chain
         float best[NCH];
@@ -285,9 +285,9 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
             // smallest energy of the tile, then the fewest instances that attain it (lowest index: n is the
             // slowest digit of j); lanes of different pair groups may hold the same n.  A tile without a
             // feasible candidate (minimum +inf) runs through the same steps and finds no pair: -1 / +inf
-            const float Emin = group_min(E, gmask);
+            const float Emin = FULL ? warp_min(E) : group_min(E, gmask);
             const uint32_t n1 = uint32_t(kk << sh_n) + uint32_t(nl);              // n - 1
-            const uint32_t n1min = __reduce_min_sync(gmask, E == Emin ? n1 : 0xffffffffu);
+            const uint32_t n1min = __reduce_min_sync(FULL ? kFull : gmask, E == Emin ? n1 : 0xffffffffu);
             const float nfm = float(n1min + 1u);
             // L/n of the winning instance count, from the lane that holds it (bit-identical by construction)
             float lnk = DYN_LN(t * NPL);

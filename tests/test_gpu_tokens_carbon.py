@@ -52,6 +52,31 @@ def test_unsorted_sparse_huge_tokens_and_dropped_requests(dyn):
     assert int(ri.max()) > 2 ** 32
 
 
+@pytest.mark.parametrize("offset", [0, 1], ids=["aligned", "4-byte-aligned"])
+@pytest.mark.parametrize("grid", ["3x3", "5x2"])
+def test_sorted_trace_with_token_counts_beyond_16_bits(dyn, offset, grid):
+    """A time-sorted dense trace (the path without per-request range tests) whose token counts mix values below and
+    above 65536; arrays that start 4 bytes off a 16-byte boundary take the scalar loads."""
+    rng = np.random.default_rng(10 + offset)
+    n = 150_003
+    t = np.sort(rng.integers(0, 90_000, n)).astype(np.uint32)
+    a = np.where(rng.random(n) < 0.1, rng.integers(0, 2 ** 32, n, dtype=np.uint64), rng.integers(1, 8193, n)).astype(np.uint32)
+    b = np.where(rng.random(n) < 0.1, rng.integers(0, 2 ** 32, n, dtype=np.uint64), rng.integers(1, 2049, n)).astype(np.uint32)
+    if grid == "3x3":
+        ie, oe = gen.IN_EDGES, gen.OUT_EDGES
+    else:
+        ie, oe = np.array([64, 256, 1024, 1 << 20], np.uint32), np.array([300], np.uint32)
+    Cn, W = (len(ie) + 1) * (len(oe) + 1), 80               # windows 80..89 are dropped
+    dt, da, db = (dev_u32(np.concatenate([np.zeros(offset, np.uint32), x]))[offset:] for x in (t, a, b))
+    ti = torch.full((W, Cn), -1, dtype=torch.int64, device="cuda")
+    to = torch.full((W, Cn), -1, dtype=torch.int64, device="cuda")
+    dyn.dyn_bin_tokens(1000, W, ie, oe, dt, da, db, ti, to, None)
+    torch.cuda.synchronize()
+    ri, ro = oracle.bin_tokens(t, a, b, 1000, W, ie, oe)
+    assert np.array_equal(ti.cpu().numpy().view(np.uint64), ri) and np.array_equal(to.cpu().numpy().view(np.uint64), ro)
+    assert int(ri.max()) > 2 ** 32
+
+
 def test_empty_trace_and_errors(dyn):
     z = torch.zeros(0, dtype=torch.int32, device="cuda")
     ti = torch.full((3, 9), 5, dtype=torch.int64, device="cuda")
