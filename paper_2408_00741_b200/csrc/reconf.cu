@@ -15,6 +15,7 @@
 //                       same addition (lowest source on ties) and writes the chosen candidates.
 #include "dyn_internal.cuh"
 
+#include <cuda_pipeline.h>
 #include <math_constants.h>
 
 namespace dyn {
@@ -75,12 +76,34 @@ __global__ void __launch_bounds__(kThreads) reconf_cost_kernel(const ReconfArgs 
     }
 }
 
-constexpr int kPathThreads = 512;
-constexpr int kRegRows = 6;                     // rows of R a thread keeps in registers (its four columns of them)
+// smallest of three (one instruction on this architecture; exact, so equal to two nested minima)
+__device__ __forceinline__ float min3f(float a, float b, float c) {
+    float r;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
+// two sources (values dA, dB; their rows of R for four neighbouring targets) against the running minima of the
+// four targets: four packed additions (each the same round-to-nearest sum as a single one) and four minima
+__device__ __forceinline__ void relax2(float &b0, float &b1, float &b2, float &b3, float dA, float dB, const float4 rA,
+                                       const float4 rB) {
+    const float2 dA2 = make_float2(dA, dA), dB2 = make_float2(dB, dB);
+    const float2 a01 = __fadd2_rn(dA2, make_float2(rA.x, rA.y)), a23 = __fadd2_rn(dA2, make_float2(rA.z, rA.w));
+    const float2 c01 = __fadd2_rn(dB2, make_float2(rB.x, rB.y)), c23 = __fadd2_rn(dB2, make_float2(rB.z, rB.w));
+    b0 = min3f(b0, a01.x, c01.x);
+    b1 = min3f(b1, a01.y, c01.y);
+    b2 = min3f(b2, a23.x, c23.x);
+    b3 = min3f(b3, a23.y, c23.y);
+}
+
+constexpr int kPathThreads = 256;
+constexpr int kRegRows = 40;                    // rows of R a thread keeps in registers (its four columns of them); whole quads
+constexpr int kRing = 4;                        // windows whose costs are on their way into shared memory
+constexpr int kOwn = 4;                         // entries of the state vector a thread owns outside the scan (NS <= 1024)
 
 // R[h][g]: the first rows_s rows sit in shared memory with row stride NS4 + 4 floats (rows stay 16-byte aligned;
 // NS4 = NS rounded up to a multiple of 4)
-// One CTA per (scenario, class).  Dynamic shared memory: Dp[NS4] | part[G][NS4] | Rs[rows_s][NS4 + 4].
+// One CTA per (scenario, class).  Dynamic shared memory: Dp[NS4] | part[G][NS4] | cring[kRing][NS4] | Rs[rows_s][NS4 + 4].
 // Forward: D_w(g) = cost_w(g) + min_h (D_{w-1}(h) + R[h][g]).  Only the minimum is formed here (add + min per
 // step): a thread takes four neighbouring targets and a share of the sources, four sources per trip (one 16-byte
 // read of the state vector, four of R).  The values D_{w-1}, relative to their minimum, are written to `hist`,
@@ -93,7 +116,8 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
     const int G = kPathThreads / lanes_t;                    // thread groups that split the sources
     float *Dp = reinterpret_cast<float *>(smem4);
     float *part = Dp + NS4;
-    float *Rs = part + size_t(G) * NS4;
+    float *cring = part + size_t(G) * NS4;                   // [kRing][NS4]: costs of the next windows
+    float *Rs = cring + size_t(kRing) * NS4;
     const int64_t sc = blockIdx.x;                           // s * C + c
     const int64_t W = a.W;
     const float *cost = a.cost + sc * W * NS;
@@ -111,13 +135,12 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
     // rows of R that do not fit in shared memory: the first G * kRegRows of them stay in registers, each source
     // group holding kRegRows rows (its four columns of them); any further rows are read through L1 / L2
     float4 rreg[kRegRows];
-    int hreg[kRegRows];
+    const int h_reg = rows_s + hg * kRegRows;                // this group's first register row (a multiple of 4)
 #pragma unroll
     for (int j = 0; j < kRegRows; ++j) {
-        const int h = rows_s + hg * kRegRows + j;
-        hreg[j] = (worker && h < NS) ? h : -1;
-        rreg[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (hreg[j] >= 0) {
+        const int h = h_reg + j;
+        rreg[j] = make_float4(CUDART_INF_F, CUDART_INF_F, CUDART_INF_F, CUDART_INF_F);      // no such row: never wins
+        if (worker && h < NS) {
             const float *row = a.R + size_t(h) * NS + 4 * tg;
             rreg[j].x = __ldg(row);
             rreg[j].y = 4 * tg + 1 < NS ? __ldg(row + 1) : 0.f;
@@ -131,8 +154,8 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
     const int g_lo = rows_sr + int(int64_t(hg) * n_rest / G), g_hi = worker ? rows_sr + int(int64_t(hg + 1) * n_rest / G) : g_lo;
     // Two barriers per window.  Dp holds the vector of the previous window as computed (not yet relative to its
     // minimum); the minimum is gathered with one shared atomic per warp on an order-preserving integer key, in
-    // one of two slots that alternate between windows.  A thread owns entries tid and tid + kPathThreads of the
-    // vector outside the scan.  Padding entries past NS are sources that never win: +inf.
+    // one of two slots that alternate between windows.  A thread owns entries tid, tid + kPathThreads, ... (kOwn of
+    // them) of the vector outside the scan.  Padding entries past NS are sources that never win: +inf.
     __shared__ unsigned int s_min[2];
     auto key_of = [](float v) {
         const unsigned int b = __float_as_uint(v);
@@ -156,6 +179,15 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
         }
         publish_min(lmin, 0);
     }
+    // The window costs come from DRAM; a thread asks for its own entries of the next kRing windows ahead of time
+    // (asynchronous copies into a ring in shared memory, one group per window), so the recursion never waits
+    // for memory.  A thread reads only what it copied itself: no barrier is needed for the ring.
+#pragma unroll
+    for (int r = 1; r <= kRing; ++r) {
+        if (r < W)
+            for (int g = tid; g < NS; g += kPathThreads) __pipeline_memcpy_async(cring + size_t(r % kRing) * NS4 + g, cost + r * NS + g, 4);
+        __pipeline_commit();
+    }
     __syncthreads();                                         // publishes Dp, the minimum and Rs
     for (int64_t w = 1; w < W; ++w) {
         // keep differences only: the previous minimum goes to the fp64 base (all +inf stays +inf)
@@ -164,31 +196,25 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
         base += double(shift);
         if (tid == 0) s_min[w & 1] = 0xffffffffu;            // this window's slot; last read before the previous barrier
         for (int g = tid; g < NS; g += kPathThreads) hist[(w - 1) * NS + g] = Dp[g] - shift;
-        // this window's costs, asked for now so that their latency hides behind the scan
-        const float cw0 = tid < NS ? cost[w * NS + tid] : 0.f;
-        const float cw1 = tid + kPathThreads < NS ? cost[w * NS + tid + kPathThreads] : 0.f;
         if (worker) {
             float b0 = CUDART_INF_F, b1 = CUDART_INF_F, b2 = CUDART_INF_F, b3 = CUDART_INF_F;
-#pragma unroll 2
+#pragma unroll 1
             for (int q = q_lo; q < q_hi; ++q) {
                 const float4 d4 = reinterpret_cast<const float4 *>(Dp)[q];
                 const float dv[4] = {d4.x - shift, d4.y - shift, d4.z - shift, d4.w - shift};
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const float4 r = *reinterpret_cast<const float4 *>(Rs + (4 * q + j) * RSd + 4 * tg);
-                    b0 = fminf(b0, dv[j] + r.x);
-                    b1 = fminf(b1, dv[j] + r.y);
-                    b2 = fminf(b2, dv[j] + r.z);
-                    b3 = fminf(b3, dv[j] + r.w);
-                }
+                for (int j = 0; j < 4; j += 2)
+                    relax2(b0, b1, b2, b3, dv[j], dv[j + 1], *reinterpret_cast<const float4 *>(Rs + (4 * q + j) * RSd + 4 * tg),
+                           *reinterpret_cast<const float4 *>(Rs + (4 * q + j + 1) * RSd + 4 * tg));
             }
 #pragma unroll
-            for (int j = 0; j < kRegRows; ++j) {
-                const float d = hreg[j] >= 0 ? Dp[hreg[j]] - shift : CUDART_INF_F;
-                b0 = fminf(b0, d + rreg[j].x);
-                b1 = fminf(b1, d + rreg[j].y);
-                b2 = fminf(b2, d + rreg[j].z);
-                b3 = fminf(b3, d + rreg[j].w);
+            for (int j4 = 0; j4 < kRegRows / 4; ++j4) {
+                // past the last quad of the vector the rows hold +inf, so any entries of the vector will do
+                const int hq = h_reg / 4 + j4 < TG ? h_reg / 4 + j4 : TG - 1;
+                const float4 d4 = reinterpret_cast<const float4 *>(Dp)[hq];
+                const float dv[4] = {d4.x - shift, d4.y - shift, d4.z - shift, d4.w - shift};
+#pragma unroll
+                for (int j = 0; j < 4; j += 2) relax2(b0, b1, b2, b3, dv[j], dv[j + 1], rreg[4 * j4 + j], rreg[4 * j4 + j + 1]);
             }
             for (int h = g_lo; h < g_hi; ++h) {
                 const float d = Dp[h] - shift;
@@ -202,14 +228,24 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
         }
         __syncthreads();                                     // every reader of Dp is done; the partial minima are in
         float lmin = CUDART_INF_F;
-        for (int g = tid; g < NS; g += kPathThreads) {
-            float best = part[g];
-            for (int k = 1; k < G; ++k) best = fminf(best, part[k * NS4 + g]);
-            const float d = (g == tid ? cw0 : cw1) + best;
-            Dp[g] = d;
-            lmin = fminf(lmin, d);
+        __pipeline_wait_prior(kRing - 1);                    // this window's costs have arrived (the thread's own entries)
+        float *cslot = cring + size_t(w % kRing) * NS4;
+#pragma unroll
+        for (int o = 0; o < kOwn; ++o) {
+            const int g = tid + o * kPathThreads;
+            if (g < NS) {
+                float best = part[g];
+                for (int k = 1; k < G; ++k) best = fminf(best, part[k * NS4 + g]);
+                const float d = cslot[g] + best;
+                Dp[g] = d;
+                lmin = fminf(lmin, d);
+            }
         }
         publish_min(lmin, int(w & 1));
+        // the slot is free (its values went into the minimum just published): ask for the costs kRing windows on
+        if (w + kRing < W)
+            for (int g = tid; g < NS; g += kPathThreads) __pipeline_memcpy_async(cslot + g, cost + (w + kRing) * NS + g, 4);
+        __pipeline_commit();
         __syncthreads();                                     // publishes Dp and the minimum
     }
     const float m = W > 0 ? val_of(s_min[(W - 1) & 1]) : 0.f;
@@ -348,14 +384,18 @@ __global__ void __launch_bounds__(kBackWarps * 32) reconf_back_kernel(const Reco
 // rows of R kept in shared memory for NS states, given the device's limit
 static size_t reconf_fixed_floats(int32_t NS) {
     const int NS4 = (NS + 3) & ~3, TG = NS4 / 4, lanes_t = (TG + 31) / 32 * 32, G = kPathThreads / lanes_t;
-    return size_t(1 + G) * NS4;
+    return size_t(1 + G + kRing) * NS4;
 }
 static int reconf_rows_in_smem(int32_t NS, size_t limit) {
     const int NS4 = (NS + 3) & ~3;
     const size_t fixed = reconf_fixed_floats(NS) * sizeof(float) + 1024;
     if (limit <= fixed) return 0;
-    const int64_t rows = int64_t((limit - fixed) / (size_t(NS4 + 4) * sizeof(float)));
-    return int(rows > NS ? NS : rows) & ~3;                  // whole quads of rows
+    int64_t rows = int64_t((limit - fixed) / (size_t(NS4 + 4) * sizeof(float)));
+    // the registers come first (no shared-memory traffic): shared memory holds what they leave
+    const int TG = NS4 / 4, lanes_t = (TG + 31) / 32 * 32, G = kPathThreads / lanes_t;
+    const int64_t left = NS4 > G * kRegRows ? NS4 - G * kRegRows : 0;
+    if (rows > left) rows = left;
+    return int(rows) & ~3;                                   // whole quads of rows
 }
 
 cudaError_t launch_reconf(const ResolvedLayout &lay, void *d_ws, size_t off_cost, size_t off_q, size_t off_from, size_t off_rt,
