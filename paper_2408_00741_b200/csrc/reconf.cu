@@ -83,17 +83,17 @@ __device__ __forceinline__ float min3f(float a, float b, float c) {
     return r;
 }
 
-// two sources (values dA, dB; their rows of R for four neighbouring targets) against the running minima of the
-// four targets: four packed additions (each the same round-to-nearest sum as a single one) and four minima
-__device__ __forceinline__ void relax2(float &b0, float &b1, float &b2, float &b3, float dA, float dB, const float4 rA,
-                                       const float4 rB) {
-    const float2 dA2 = make_float2(dA, dA), dB2 = make_float2(dB, dB);
-    const float2 a01 = __fadd2_rn(dA2, make_float2(rA.x, rA.y)), a23 = __fadd2_rn(dA2, make_float2(rA.z, rA.w));
-    const float2 c01 = __fadd2_rn(dB2, make_float2(rB.x, rB.y)), c23 = __fadd2_rn(dB2, make_float2(rB.z, rB.w));
-    b0 = min3f(b0, a01.x, c01.x);
-    b1 = min3f(b1, a01.y, c01.y);
-    b2 = min3f(b2, a23.x, c23.x);
-    b3 = min3f(b3, a23.y, c23.y);
+// Two sources A, B (their values, relative to the minimum, in d) against the running minima of four neighbouring
+// targets.  v0 = {R[A][t0], R[B][t0], R[A][t1], R[B][t1]}, v1 the same for t2, t3: a packed addition forms both
+// sums of a target (each the same round-to-nearest sum as a single addition), one three-input minimum takes them in
+__device__ __forceinline__ void relax_pair(float &b0, float &b1, float &b2, float &b3, const float2 d, const float4 v0,
+                                           const float4 v1) {
+    const float2 s0 = __fadd2_rn(d, make_float2(v0.x, v0.y)), s1 = __fadd2_rn(d, make_float2(v0.z, v0.w));
+    const float2 s2 = __fadd2_rn(d, make_float2(v1.x, v1.y)), s3 = __fadd2_rn(d, make_float2(v1.z, v1.w));
+    b0 = min3f(b0, s0.x, s0.y);
+    b1 = min3f(b1, s1.x, s1.y);
+    b2 = min3f(b2, s2.x, s2.y);
+    b3 = min3f(b3, s3.x, s3.y);
 }
 
 constexpr int kPathThreads = 256;
@@ -101,10 +101,10 @@ constexpr int kRegRows = 40;                    // rows of R a thread keeps in r
 constexpr int kRing = 4;                        // windows whose costs are on their way into shared memory
 constexpr int kOwn = 4;                         // entries of the state vector a thread owns outside the scan (NS <= 1024)
 
-// R[h][g]: the first rows_s rows sit in shared memory with row stride NS4 + 4 floats (rows stay 16-byte aligned;
-// NS4 = NS rounded up to a multiple of 4)
-// One CTA per (scenario, class).  Dynamic shared memory: Dp[NS4] | part[G][NS4] | cring[kRing][NS4] | Rs[rows_s][NS4 + 4].
-// Forward: D_w(g) = cost_w(g) + min_h (D_{w-1}(h) + R[h][g]).  Only the minimum is formed here (add + min per
+// R[h][g]: rows_s rows sit in shared memory, NS4 + 4 floats per row (NS4 = NS rounded up to a multiple of 4; the
+// pieces stay 16-byte aligned), pairs of rows interleaved as described at the copy loop
+// One CTA per (scenario, class).  Dynamic shared memory: Dp[NS4] | part[G][NS4] | cring[kRing][NS4] | Rs[rows_s / 2][2][NS4 + 4].
+// Forward: D_w(g) = cost_w(g) + min_h (D_{w-1}(h) + R[h][g]).  Only the minimum is formed here (half a packed add and half a three-input min per
 // step): a thread takes four neighbouring targets and a share of the sources, four sources per trip (one 16-byte
 // read of the state vector, four of R).  The values D_{w-1}, relative to their minimum, are written to `hist`,
 // and the walk back finds each predecessor again as the lowest h that attains the minimum, with the same addition.
@@ -128,25 +128,30 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
     const int SQ = rows_s / 4;                               // quads of rows held in shared memory
     const int q_lo = int(int64_t(hg) * SQ / G), q_hi = worker ? int(int64_t(hg + 1) * SQ / G) : q_lo;   // this group's share
 
+    // rows A = 2k and B = 2k + 1 are interleaved (a packed addition takes {R[A][g], R[B][g]}): per pair of rows two
+    // planes of RSd floats, plane 0 holding {R[A][t0], R[B][t0], R[A][t1], R[B][t1]} of every group of four targets
+    // t0..t3 and plane 1 the same for t2, t3, so that the lanes of a warp read neighbouring 16-byte pieces
     for (int i = tid; i < rows_s * RSd; i += kPathThreads) {
-        const int h = i / RSd, g = i - h * RSd;
-        Rs[i] = g < NS ? a.R[size_t(h) * NS + g] : 0.f;
+        const int h = i / RSd, g = i - h * RSd, j = g & 3;
+        Rs[size_t(h >> 1) * (2 * RSd) + (j >> 1) * RSd + (g & ~3) + (j & 1) * 2 + (h & 1)] = g < NS ? a.R[size_t(h) * NS + g] : 0.f;
     }
     // rows of R that do not fit in shared memory: the first G * kRegRows of them stay in registers, each source
     // group holding kRegRows rows (its four columns of them); any further rows are read through L1 / L2
-    float4 rreg[kRegRows];
+    float4 rp0[kRegRows / 2], rp1[kRegRows / 2];             // per pair of rows, interleaved like the shared-memory copy
     const int h_reg = rows_s + hg * kRegRows;                // this group's first register row (a multiple of 4)
 #pragma unroll
-    for (int j = 0; j < kRegRows; ++j) {
-        const int h = h_reg + j;
-        rreg[j] = make_float4(CUDART_INF_F, CUDART_INF_F, CUDART_INF_F, CUDART_INF_F);      // no such row: never wins
-        if (worker && h < NS) {
+    for (int k = 0; k < kRegRows / 2; ++k) {
+        float v[2][4];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int h = h_reg + 2 * k + i;
+            const bool have = worker && h < NS;              // no such row: +inf never wins
             const float *row = a.R + size_t(h) * NS + 4 * tg;
-            rreg[j].x = __ldg(row);
-            rreg[j].y = 4 * tg + 1 < NS ? __ldg(row + 1) : 0.f;
-            rreg[j].z = 4 * tg + 2 < NS ? __ldg(row + 2) : 0.f;
-            rreg[j].w = 4 * tg + 3 < NS ? __ldg(row + 3) : 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) v[i][j] = have ? (4 * tg + j < NS ? __ldg(row + j) : 0.f) : CUDART_INF_F;
         }
+        rp0[k] = make_float4(v[0][0], v[1][0], v[0][1], v[1][1]);
+        rp1[k] = make_float4(v[0][2], v[1][2], v[0][3], v[1][3]);
     }
     const int rows_sr = rows_s + G * kRegRows;               // rows below this are in shared memory or registers
     // the rest, split evenly over the source groups
@@ -198,23 +203,23 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
         for (int g = tid; g < NS; g += kPathThreads) hist[(w - 1) * NS + g] = Dp[g] - shift;
         if (worker) {
             float b0 = CUDART_INF_F, b1 = CUDART_INF_F, b2 = CUDART_INF_F, b3 = CUDART_INF_F;
+            const float2 nshift = make_float2(-shift, -shift);                  // d + (-shift) is d - shift bit for bit
 #pragma unroll 1
             for (int q = q_lo; q < q_hi; ++q) {
                 const float4 d4 = reinterpret_cast<const float4 *>(Dp)[q];
-                const float dv[4] = {d4.x - shift, d4.y - shift, d4.z - shift, d4.w - shift};
-#pragma unroll
-                for (int j = 0; j < 4; j += 2)
-                    relax2(b0, b1, b2, b3, dv[j], dv[j + 1], *reinterpret_cast<const float4 *>(Rs + (4 * q + j) * RSd + 4 * tg),
-                           *reinterpret_cast<const float4 *>(Rs + (4 * q + j + 1) * RSd + 4 * tg));
+                const float *rq = Rs + size_t(2 * q) * (2 * RSd) + 4 * tg;
+                relax_pair(b0, b1, b2, b3, __fadd2_rn(make_float2(d4.x, d4.y), nshift), *reinterpret_cast<const float4 *>(rq),
+                           *reinterpret_cast<const float4 *>(rq + RSd));
+                relax_pair(b0, b1, b2, b3, __fadd2_rn(make_float2(d4.z, d4.w), nshift), *reinterpret_cast<const float4 *>(rq + 2 * RSd),
+                           *reinterpret_cast<const float4 *>(rq + 3 * RSd));
             }
 #pragma unroll
             for (int j4 = 0; j4 < kRegRows / 4; ++j4) {
                 // past the last quad of the vector the rows hold +inf, so any entries of the vector will do
                 const int hq = h_reg / 4 + j4 < TG ? h_reg / 4 + j4 : TG - 1;
                 const float4 d4 = reinterpret_cast<const float4 *>(Dp)[hq];
-                const float dv[4] = {d4.x - shift, d4.y - shift, d4.z - shift, d4.w - shift};
-#pragma unroll
-                for (int j = 0; j < 4; j += 2) relax2(b0, b1, b2, b3, dv[j], dv[j + 1], rreg[4 * j4 + j], rreg[4 * j4 + j + 1]);
+                relax_pair(b0, b1, b2, b3, __fadd2_rn(make_float2(d4.x, d4.y), nshift), rp0[2 * j4], rp1[2 * j4]);
+                relax_pair(b0, b1, b2, b3, __fadd2_rn(make_float2(d4.z, d4.w), nshift), rp0[2 * j4 + 1], rp1[2 * j4 + 1]);
             }
             for (int h = g_lo; h < g_hi; ++h) {
                 const float d = Dp[h] - shift;
