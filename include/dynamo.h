@@ -311,9 +311,11 @@ typedef struct {
     const float *extra_load;                   /* host [S_extra][W][C] requests/s, or NULL */
     int64_t S_extra;                           /* scenarios after scenario 0 (the binned trace); S = 1 + S_extra */
     void *copy_stream;                         /* optional second cudaStream_t (NULL = none): extra_load is then copied on
-                                                  it in up to 8 pieces, each evaluated on `stream` as soon as it has
-                                                  arrived, so that copying and evaluation overlap; the two streams are
-                                                  ordered by events the library creates once per thread and device */
+                                                  it in up to 16 pieces, each evaluated on `stream` as soon as it has
+                                                  arrived, and each piece's results are copied back on it while the
+                                                  next piece is evaluated; `stream` waits for the last of these copies,
+                                                  so synchronising `stream` is still all the caller does; the two streams
+                                                  are ordered by events the library creates once per thread and device */
 } dyn_host_in;
 
 typedef struct {                 /* host result buffers; any of them may be NULL to skip that copy */

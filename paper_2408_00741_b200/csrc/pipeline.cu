@@ -37,18 +37,20 @@ bool plan(const dyn_bin_spec *spec, const dyn_profile_host *p, const dyn_space *
     return true;
 }
 
-constexpr int kPieces = 8;       // pieces the scenario loads are copied in when a copy stream is given
+constexpr int kPieces = 16;      // pieces the scenario loads are copied in when a copy stream is given
+constexpr int kEvents = 2 * kPieces + 2;         // [k]: loads of piece k are in; [kPieces]: arena free;
+                                                 // [kPieces + 1 + k]: piece k is evaluated
 
 // events that order the copy stream against the caller's stream: created on first use per thread and device,
 // kept for the life of the process (they hold no device memory)
 cudaEvent_t *overlap_events() {
     constexpr int kMaxDev = 64;
-    static thread_local cudaEvent_t ev[kMaxDev][kPieces + 1];
+    static thread_local cudaEvent_t ev[kMaxDev][kEvents];
     static thread_local bool made[kMaxDev] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return nullptr;
     if (!made[dev]) {
-        for (int i = 0; i <= kPieces; ++i)
+        for (int i = 0; i < kEvents; ++i)
             if (cudaEventCreateWithFlags(&ev[dev][i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
         made[dev] = true;
     }
@@ -155,18 +157,35 @@ int dyn_pipeline_host(const dyn_bin_spec *spec, const dyn_profile_host *p, const
             rc = dyn_eval_select(&dp, sp, static_cast<const float *>(dptr(ar.load)) + s0 * wc, int64_t(s1 - s0), int64_t(W), &sk,
                                  dptr(ar.ws), ar.ws_bytes, stream);
             if (rc != DYN_OK) return rc;
+            // the piece's results go back on the copy stream (behind the loads, which are long in by then) while
+            // the next piece is evaluated
+            DYN_CUDA_TRY(cudaEventRecord(ev[kPieces + 1 + k], st));
+            DYN_CUDA_TRY(cudaStreamWaitEvent(cs, ev[kPieces + 1 + k], 0));
+            const size_t ns = s1 - s0;
+            if (out->best_idx) DYN_CUDA_TRY(cudaMemcpyAsync(out->best_idx + s0 * wc, sk.d_best_idx, ns * wc * 4, D2H, cs));
+            if (out->best_E) DYN_CUDA_TRY(cudaMemcpyAsync(out->best_E + s0 * wc, sk.d_best_E, ns * wc * 4, D2H, cs));
+            if (out->E_total) DYN_CUDA_TRY(cudaMemcpyAsync(out->E_total + s0, sk.d_E_total, ns * 8, D2H, cs));
+            if (out->n_infeasible) DYN_CUDA_TRY(cudaMemcpyAsync(out->n_infeasible + s0, sk.d_n_infeasible, ns * 4, D2H, cs));
+            if (out->E_window) DYN_CUDA_TRY(cudaMemcpyAsync(out->E_window + s0 * W, sk.d_E_window, ns * W * 8, D2H, cs));
+            if (out->hist) DYN_CUDA_TRY(cudaMemcpyAsync(out->hist + s0 * J, sk.d_hist, ns * J * 4, D2H, cs));
+            if (out->gpus) DYN_CUDA_TRY(cudaMemcpyAsync(out->gpus + s0 * W, sk.d_gpus, ns * W * 4, D2H, cs));
         }
+        // the caller's stream is done when the last results have left
+        DYN_CUDA_TRY(cudaEventRecord(ev[kPieces], cs));
+        DYN_CUDA_TRY(cudaStreamWaitEvent(st, ev[kPieces], 0));
     }
 
     if (out->counts) DYN_CUDA_TRY(cudaMemcpyAsync(out->counts, dptr(ar.counts), wc * 4, D2H, st));
     if (out->dropped) DYN_CUDA_TRY(cudaMemcpyAsync(out->dropped, dptr(ar.dropped), 8, D2H, st));
-    if (out->best_idx) DYN_CUDA_TRY(cudaMemcpyAsync(out->best_idx, dptr(ar.idx), tiles * 4, D2H, st));
-    if (out->best_E) DYN_CUDA_TRY(cudaMemcpyAsync(out->best_E, dptr(ar.be), tiles * 4, D2H, st));
-    if (out->E_total) DYN_CUDA_TRY(cudaMemcpyAsync(out->E_total, dptr(ar.etot), size_t(S) * 8, D2H, st));
-    if (out->n_infeasible) DYN_CUDA_TRY(cudaMemcpyAsync(out->n_infeasible, dptr(ar.ninf), size_t(S) * 4, D2H, st));
-    if (out->E_window) DYN_CUDA_TRY(cudaMemcpyAsync(out->E_window, dptr(ar.ewin), size_t(S) * W * 8, D2H, st));
-    if (out->hist) DYN_CUDA_TRY(cudaMemcpyAsync(out->hist, dptr(ar.hist), size_t(S) * J * 4, D2H, st));
-    if (out->gpus) DYN_CUDA_TRY(cudaMemcpyAsync(out->gpus, dptr(ar.gpus), size_t(S) * W * 4, D2H, st));
+    if (pieces == 0) {
+        if (out->best_idx) DYN_CUDA_TRY(cudaMemcpyAsync(out->best_idx, dptr(ar.idx), tiles * 4, D2H, st));
+        if (out->best_E) DYN_CUDA_TRY(cudaMemcpyAsync(out->best_E, dptr(ar.be), tiles * 4, D2H, st));
+        if (out->E_total) DYN_CUDA_TRY(cudaMemcpyAsync(out->E_total, dptr(ar.etot), size_t(S) * 8, D2H, st));
+        if (out->n_infeasible) DYN_CUDA_TRY(cudaMemcpyAsync(out->n_infeasible, dptr(ar.ninf), size_t(S) * 4, D2H, st));
+        if (out->E_window) DYN_CUDA_TRY(cudaMemcpyAsync(out->E_window, dptr(ar.ewin), size_t(S) * W * 8, D2H, st));
+        if (out->hist) DYN_CUDA_TRY(cudaMemcpyAsync(out->hist, dptr(ar.hist), size_t(S) * J * 4, D2H, st));
+        if (out->gpus) DYN_CUDA_TRY(cudaMemcpyAsync(out->gpus, dptr(ar.gpus), size_t(S) * W * 4, D2H, st));
+    }
     return DYN_OK;
 }
 
