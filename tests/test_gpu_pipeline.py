@@ -62,10 +62,11 @@ def test_pipeline_host_matches_oracle(dyn, name, S, pinned):
     assert e.value.status == dyn.DYN_EWORKSPACE
 
 
-@pytest.mark.parametrize("S", [2, 12])
+@pytest.mark.parametrize("S", [2, 12, 40])
 def test_copy_stream_gives_the_same_results(dyn, S):
-    """With a second stream the scenario loads arrive in pieces (here fewer and more scenarios than pieces) and
-    every piece is evaluated on its own: all outputs equal those of the single-stream call bit for bit."""
+    """With a second stream the scenario loads arrive in pieces (here fewer and more scenarios than pieces), every
+    piece is evaluated on its own and its results are copied back on the second stream: all outputs equal those of
+    the single-stream call bit for bit, and waiting for the caller's stream alone is enough to read them."""
     wl = gen.workload("cfg1")
     t, i, o = gen.make_trace(wl.trace)
     prof, sp = wl.profile(), wl.space()
@@ -91,6 +92,6 @@ def test_copy_stream_gives_the_same_results(dyn, S):
     side = torch.cuda.Stream()
     for _ in range(2):                                      # back to back: the second call waits for the first one's use of the arena
         hp.run(t.view(np.int32), i.view(np.int32), o.view(np.int32), extra, two, arena, copy_stream=side)
-    torch.cuda.synchronize()
+    torch.cuda.current_stream().synchronize()               # not the copy stream: the call orders it before this one
     for k in one:
         assert torch.equal(one[k], two[k]), k
