@@ -313,7 +313,8 @@ typedef struct {
     void *copy_stream;                         /* optional second cudaStream_t (NULL = none): extra_load is then copied on
                                                   it in up to 16 pieces, each evaluated on `stream` as soon as it has
                                                   arrived, and each piece's results are copied back on it while the
-                                                  next piece is evaluated; `stream` waits for the last of these copies,
+                                                  next piece is evaluated (the trace is copied on it too, behind
+                                                  the first piece, and scenario 0 is evaluated last); `stream` waits for the last of these copies,
                                                   so synchronising `stream` is still all the caller does; the two streams
                                                   are ordered by events the library creates once per thread and device */
 } dyn_host_in;

@@ -38,8 +38,9 @@ bool plan(const dyn_bin_spec *spec, const dyn_profile_host *p, const dyn_space *
 }
 
 constexpr int kPieces = 16;      // pieces the scenario loads are copied in when a copy stream is given
-constexpr int kEvents = 2 * kPieces + 2;         // [k]: loads of piece k are in; [kPieces]: arena free;
-                                                 // [kPieces + 1 + k]: piece k is evaluated
+constexpr int kEvents = 2 * kPieces + 3;         // [k]: loads of piece k are in; [kPieces]: arena free / results out;
+                                                 // [kPieces + 1 + k]: piece k is evaluated; [2 kPieces + 2]: trace is in
+constexpr int kTraceEvent = 2 * kPieces + 2;
 
 // events that order the copy stream against the caller's stream: created on first use per thread and device,
 // kept for the life of the process (they hold no device memory)
@@ -90,19 +91,28 @@ int dyn_pipeline_host(const dyn_bin_spec *spec, const dyn_profile_host *p, const
     const size_t ctr = C * size_t(p->T) * size_t(p->R);
     const cudaMemcpyKind H2D = cudaMemcpyHostToDevice, D2H = cudaMemcpyDeviceToHost;
 
-    if (in->n_req > 0) {
-        DYN_CUDA_TRY(cudaMemcpyAsync(dptr(ar.t), in->t_ms, in->n_req * 4, H2D, st));
-        DYN_CUDA_TRY(cudaMemcpyAsync(dptr(ar.a), in->in_tok, in->n_req * 4, H2D, st));
-        DYN_CUDA_TRY(cudaMemcpyAsync(dptr(ar.b), in->out_tok, in->n_req * 4, H2D, st));
+    // the caller's scenario loads: on `stream`, or in pieces on the copy stream so that a piece is evaluated while
+    // the next ones are still on their way
+    cudaStream_t cs = static_cast<cudaStream_t>(in->copy_stream);
+    const int pieces = (cs && cs != st && in->S_extra > 0) ? int(in->S_extra < kPieces ? in->S_extra : kPieces) : 0;
+    // the trace travels on `stream`, or, with a copy stream, behind the first piece of loads: scenario 0 (the binned
+    // trace) is then evaluated last, and the first piece does not wait for the trace
+    auto copy_trace = [&](cudaStream_t on) -> int {
+        if (in->n_req > 0) {
+            DYN_CUDA_TRY(cudaMemcpyAsync(dptr(ar.t), in->t_ms, in->n_req * 4, H2D, on));
+            DYN_CUDA_TRY(cudaMemcpyAsync(dptr(ar.a), in->in_tok, in->n_req * 4, H2D, on));
+            DYN_CUDA_TRY(cudaMemcpyAsync(dptr(ar.b), in->out_tok, in->n_req * 4, H2D, on));
+        }
+        return DYN_OK;
+    };
+    if (pieces == 0) {
+        const int rt = copy_trace(st);
+        if (rt != DYN_OK) return rt;
     }
     DYN_CUDA_TRY(cudaMemcpyAsync(dptr(ar.ttft), p->ttft, ctr * 4, H2D, st));
     DYN_CUDA_TRY(cudaMemcpyAsync(dptr(ar.cap), p->cap, ctr * 4, H2D, st));
     DYN_CUDA_TRY(cudaMemcpyAsync(dptr(ar.tbt), p->tbt, ctr * size_t(p->M) * 4, H2D, st));
     DYN_CUDA_TRY(cudaMemcpyAsync(dptr(ar.pw), p->pow, ctr * size_t(p->M) * 4, H2D, st));
-    // the caller's scenario loads: on `stream`, or in pieces on the copy stream so that a piece is evaluated while
-    // the next ones are still on their way
-    cudaStream_t cs = static_cast<cudaStream_t>(in->copy_stream);
-    const int pieces = (cs && cs != st && in->S_extra > 0) ? int(in->S_extra < kPieces ? in->S_extra : kPieces) : 0;
     cudaEvent_t *ev = nullptr;
     if (pieces > 0) {
         ev = overlap_events();
@@ -115,6 +125,11 @@ int dyn_pipeline_host(const dyn_bin_spec *spec, const dyn_profile_host *p, const
             DYN_CUDA_TRY(cudaMemcpyAsync(static_cast<char *>(dptr(ar.load)) + (1 + e0) * wc * 4, in->extra_load + e0 * wc,
                                          (e1 - e0) * wc * 4, H2D, cs));
             DYN_CUDA_TRY(cudaEventRecord(ev[k], cs));
+            if (k == 0) {
+                const int rt = copy_trace(cs);
+                if (rt != DYN_OK) return rt;
+                DYN_CUDA_TRY(cudaEventRecord(ev[kTraceEvent], cs));
+            }
         }
     } else if (in->S_extra > 0) {
         DYN_CUDA_TRY(cudaMemcpyAsync(static_cast<char *>(dptr(ar.load)) + wc * 4, in->extra_load,
@@ -122,10 +137,12 @@ int dyn_pipeline_host(const dyn_bin_spec *spec, const dyn_profile_host *p, const
     }
 
     // (a): scenario 0 of the load tensor is the binned trace
-    int rc = dyn_bin_trace(spec, static_cast<const uint32_t *>(dptr(ar.t)), static_cast<const uint32_t *>(dptr(ar.a)),
-                           static_cast<const uint32_t *>(dptr(ar.b)), in->n_req, static_cast<uint32_t *>(dptr(ar.counts)),
-                           static_cast<float *>(dptr(ar.load)), static_cast<uint64_t *>(dptr(ar.dropped)), stream);
-    if (rc != DYN_OK) return rc;
+    auto bin = [&]() {
+        return dyn_bin_trace(spec, static_cast<const uint32_t *>(dptr(ar.t)), static_cast<const uint32_t *>(dptr(ar.a)),
+                             static_cast<const uint32_t *>(dptr(ar.b)), in->n_req, static_cast<uint32_t *>(dptr(ar.counts)),
+                             static_cast<float *>(dptr(ar.load)), static_cast<uint64_t *>(dptr(ar.dropped)), stream);
+    };
+    int rc = DYN_OK;
 
     // (b)+(c)
     dyn_profile dp{p->C, p->T, p->R, p->M, p->tp, p->f_grid_mhz, static_cast<const float *>(dptr(ar.ttft)),
@@ -140,15 +157,18 @@ int dyn_pipeline_host(const dyn_bin_spec *spec, const dyn_profile_host *p, const
     so.d_hist = out->hist ? static_cast<uint32_t *>(dptr(ar.hist)) : nullptr;
     so.d_gpus = out->gpus ? static_cast<uint32_t *>(dptr(ar.gpus)) : nullptr;
     if (pieces == 0) {
+        if ((rc = bin()) != DYN_OK) return rc;
         rc = dyn_eval_select(&dp, sp, static_cast<const float *>(dptr(ar.load)), S, int64_t(W), &so, dptr(ar.ws),
                              ar.ws_bytes, stream);
         if (rc != DYN_OK) return rc;
     } else {
-        // piece k: scenarios [s0, s1) (piece 0 also holds scenario 0, the binned trace), evaluated once its loads are in
-        for (int k = 0; k < pieces; ++k) {
-            const size_t s0 = k == 0 ? 0 : 1 + size_t(in->S_extra) * k / pieces;
-            const size_t s1 = 1 + size_t(in->S_extra) * (k + 1) / pieces;
-            DYN_CUDA_TRY(cudaStreamWaitEvent(st, ev[k], 0));
+        // piece k: scenarios [s0, s1) of the caller's loads, evaluated once they are in; piece `pieces` is scenario 0,
+        // binned and evaluated once the trace is in
+        for (int k = 0; k <= pieces; ++k) {
+            const size_t s0 = k == pieces ? 0 : 1 + size_t(in->S_extra) * k / pieces;
+            const size_t s1 = k == pieces ? 1 : 1 + size_t(in->S_extra) * (k + 1) / pieces;
+            DYN_CUDA_TRY(cudaStreamWaitEvent(st, ev[k == pieces ? kTraceEvent : k], 0));
+            if (k == pieces && (rc = bin()) != DYN_OK) return rc;
             dyn_select_out sk = so;
             sk.d_best_idx += s0 * wc; sk.d_best_E += s0 * wc; sk.d_E_total += s0; sk.d_n_infeasible += s0;
             if (sk.d_E_window) sk.d_E_window += s0 * W;
