@@ -16,8 +16,10 @@ With N > 1 every rank runs an independent replica of the workload (the path has 
 from __future__ import annotations
 
 import argparse
+import datetime
 import json
 import os
+import socket
 import subprocess
 import sys
 import tempfile
@@ -30,9 +32,10 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 FLOP_PER_EVAL = 20.0            # algorithmic fp32 operations per candidate, counted from the definition
-SM_COUNT, FP32_LANES, SM_MAX_MHZ = 148, 128, 1965.0
+SM_COUNT, FP32_LANES, SM_MAX_MHZ = 148, 128, 1965.0     # nominal figures, reported beside the measured peak
 BYTES_PER_REQUEST = 12.0
-INST_PER_WARP_EVAL_CFG4 = 6.81    # warp instructions per 32 candidates of the sweep on the cfg4 shape (ncu)
+SIDE = ("cfg1", "cfg1_x4096", "cfg2", "cfg3", "cfg3code", "cfg5", "cfg2_x256_general", "bin_trace", "materialised",
+        "hierarchical", "mixed_pools", "mixed_pools_small", "reconfiguration")
 
 
 def parse_args():
@@ -48,6 +51,9 @@ def parse_args():
     ap.add_argument("--no-secondary", action="store_true", help="skip the side measurements of the other kernels")
     ap.add_argument("--secondary-only", action="store_true",
                     help="run only the side measurements (trace binning, unfused stages) and print them")
+    ap.add_argument("--only", default="", help="comma-separated side measurements to run alone: " + ", ".join(SIDE))
+    ap.add_argument("--quick", action="store_true",
+                    help="one round of few launches per measurement (for profiler captures; clock records stay thin)")
     return ap.parse_args()
 
 
@@ -65,9 +71,12 @@ def max_over_ranks(x: float, dist, device) -> float:
 # clocks
 # ----------------------------------------------------------------------------------------------
 class ClockSampler:
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
-              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
+    """nvidia-smi sampling SM clock and throttle reasons every 100 ms for the whole run; `window(t0, t1)`
+    summarises the samples taken between two host times (time.time())."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, gpu_index: int):
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
@@ -77,16 +86,40 @@ class ClockSampler:
                                        "-lms", "100", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
         except OSError:
             self.p = None
-        self.marks = []
 
-    def mark(self):
-        """remember how many samples exist now (start / end of the timed region)"""
+    @staticmethod
+    def parse_row(line: str):
+        """(host time, sm MHz, max sm MHz, [reasons]) of one CSV row, or None."""
+        r = [x.strip() for x in line.split(",")]
+        try:
+            ts = datetime.datetime.strptime(r[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+            sm, mx = float(r[1]), float(r[2])
+        except (ValueError, IndexError):
+            return None
+        reasons = [n for k, n in enumerate(ClockSampler.NAMES) if len(r) > 5 + k and r[5 + k].lower().startswith("active")]
+        return ts, sm, mx, reasons
+
+    def rows(self):
         self.f.flush()
         try:
             with open(self.f.name) as fh:
-                self.marks.append(sum(1 for _ in fh))
+                return [x for x in (self.parse_row(line) for line in fh if line.strip()) if x is not None]
         except OSError:
-            self.marks.append(0)
+            return []
+
+    @staticmethod
+    def summarise(rows):
+        sm = [r[1] for r in rows]
+        reasons = sorted({n for r in rows for n in r[3]})
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(r[2] for r in rows) if rows else None,
+                "reasons": reasons, "samples": len(sm)}
+
+    def window(self, t0: float, t1: float):
+        """Samples between the host times t0 and t1 (one sampling period of slack on either side)."""
+        time.sleep(0.12)                        # let the sample that covers t1 arrive
+        rows = self.rows()
+        sel = [r for r in rows if t0 - 0.1 <= r[0] <= t1 + 0.1]
+        return self.summarise(sel)
 
     def stop(self):
         if self.p is not None:
@@ -95,27 +128,12 @@ class ClockSampler:
                 self.p.wait(timeout=5)
             except subprocess.TimeoutExpired:
                 self.p.kill()
-        rows = []
+        rows = self.rows()
         try:
-            with open(self.f.name) as fh:
-                rows = [[x.strip() for x in line.split(",")] for line in fh if line.strip()]
             os.unlink(self.f.name)
         except OSError:
             pass
-        lo, hi = (self.marks + [0, len(rows)])[:2] if len(self.marks) >= 2 else (0, len(rows))
-        sel = rows[max(0, lo - 1):hi + 1] or rows
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in sel:
-            try:
-                sm.append(float(r[0])); mx.append(float(r[1]))
-            except (ValueError, IndexError):
-                continue
-            for k, name in enumerate(names):
-                if len(r) > 4 + k and r[4 + k].lower().startswith("active"):
-                    reasons.add(name)
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+        return self.summarise(rows)
 
 
 # ----------------------------------------------------------------------------------------------
@@ -218,6 +236,153 @@ def run_reference(args, rank):
     }))
 
 
+QUICK = False
+
+
+def timed_kernel(dyn, call, flush=None, min_s=0.5, per_round=25, max_rounds=400):
+    """Duration of the main kernel of `call` from the events the library records around it (see
+    dyn_set_timing_events): rounds of `per_round` instrumented calls until `min_s` seconds have passed, so
+    that the clock sampler sees the region.  `flush` (a buffer larger than L2) is rewritten before every
+    call when given.  Returns mean ms, min ms, calls, host times of the first and last call."""
+    import torch
+    if QUICK:
+        min_s, per_round = 0.0, 3
+    for _ in range(3):
+        call()
+    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(per_round)]
+    for a, b in kev:
+        a.record(); b.record()
+    torch.cuda.synchronize()
+    ms = []
+    t0 = time.time()
+    for _ in range(max_rounds):
+        for k, (a, b) in enumerate(kev):
+            if flush is not None:
+                flush.fill_(k & 0xff)
+            dyn.dyn_set_timing_events(a, b)
+            call()
+        dyn.dyn_set_timing_events(None, None)
+        torch.cuda.synchronize()
+        ms += [a.elapsed_time(b) for a, b in kev]
+        if time.time() - t0 >= min_s:
+            break
+    t1 = time.time()
+    return float(np.mean(ms)), float(np.min(ms)), len(ms), t0, t1
+
+
+def measure_peaks(dyn, dev, sampler):
+    """The fp32 peak of this GPU, measured now by the library's multiply-add probe, and the HBM figure."""
+    import torch
+    sink = torch.zeros(1, dtype=torch.float32, device=dev)
+    work = []
+    ms, ms_min, n, t0, t1 = timed_kernel(dyn, lambda: work.append(dyn.dyn_probe_fma(2000, sink)))
+    tflops = work[0] / (ms * 1e-3) / 1e12
+    hbm, hbm_src = _hbm_peak()
+    return {"fp32_tflops": tflops, "fp32_probe_ms": ms, "fp32_probe_launches": n,
+            "fp32_nominal_tflops": SM_COUNT * FP32_LANES * 2 * SM_MAX_MHZ * 1e6 / 1e12,
+            "issue_warp_inst_per_s": tflops * 1e12 / 64.0,
+            "clocks": sampler.window(t0, t1) if sampler else None,
+            "hbm_gbs": hbm, "hbm_source": hbm_src, "sink": sink}
+
+
+def feasible_share(dyn, P, SP, d_load_sample):
+    """Share of the candidates of these tiles that are feasible (from a materialised energy tensor)."""
+    import torch
+    S, W, Cn = d_load_sample.shape
+    J = SP.n_max * P.T * SP.F
+    E = torch.empty((S, W, Cn, J), dtype=torch.float32, device=d_load_sample.device)
+    ws = torch.empty(dyn.dyn_workspace_bytes(P, SP, S, W), dtype=torch.uint8, device=d_load_sample.device)
+    dyn.dyn_eval_configs(P, SP, d_load_sample, E, ws)
+    torch.cuda.synchronize()
+    return float(torch.isfinite(E).sum().item()) / float(E.numel())
+
+
+def executed_work(dyn, peaks, sampler, wl_name, kernel_rate, share):
+    """Hardware-side figures of the sweep: its instruction rate against the measured issue ceiling (instruction
+    count from recorded profiler counters, null once the kernel's sources have changed), and its rate against
+    the library's probe of the sweep's inner loop at the workload's share of feasible candidates."""
+    from paper_2408_00741_b200 import counters
+    out = {"issue": None, "inner_loop_probe": None}
+    rec = counters.lookup("eval_select_kernel", wl_name)
+    if rec is not None and rec.get("warp_inst_per_32_evals") is not None:
+        if rec["stale"]:
+            out["issue"] = {"warp_inst_per_32_evals": None, "frac": None, "counters": "stale: the kernel's sources "
+                            "changed after the counters were taken"}
+        else:
+            ipe = rec["warp_inst_per_32_evals"]
+            rate = ipe * kernel_rate / 32.0
+            out["issue"] = {"warp_inst_per_32_evals": ipe, "achieved_warp_inst_per_s": rate,
+                            "peak_warp_inst_per_s": peaks["issue_warp_inst_per_s"],
+                            "frac": rate / peaks["issue_warp_inst_per_s"],
+                            "counters": "smsp__inst_executed.sum of one launch, recorded for the current sources; "
+                                        "ceiling = measured multiply-add rate / 64"}
+    if share is not None:
+        work = []
+        ms, _, _, t0, t1 = timed_kernel(dyn, lambda: work.append(dyn.dyn_probe_sweep_inner(400, share, peaks["sink"])),
+                                        min_s=0.3)
+        probe_rate = work[0] / (ms * 1e-3)
+        out["inner_loop_probe"] = {"feasible_share": share, "probe_evals_per_s": probe_rate,
+                                   "kernel_over_probe": kernel_rate / probe_rate,
+                                   "clocks": sampler.window(t0, t1) if sampler else None,
+                                   "note": "the sweep's (TP, f) loop alone on a synthetic table (8 candidates per lane and "
+                                           "pair, no per-tile work) at this share of feasible candidates, spread evenly over "
+                                           "the lanes: every lookup keeps both half-warps busy, so the probe is bound by the "
+                                           "shared-memory data path (two cycles per 8-byte lookup and SM); the sweep skips "
+                                           "whole-warp lookups where no lane is feasible and can run above it"}
+    return out
+
+
+def measure_config(dyn, gen, dev, sampler, peaks, flush, name, S=1, general=False, trace=None, with_bin=True):
+    """One benchmark configuration: the histogram kernel on its trace and the fused sweep on its loads (S > 1:
+    Poisson-resampled scenarios of the binned trace; general: one TBT row made non-monotone, which puts that
+    class on the path that interpolates TBT per candidate)."""
+    import torch
+    wl = gen.workload(name)
+    t, i, o = trace if trace is not None else gen.make_trace(wl.trace)
+    prof, sp = wl.profile(), wl.space()
+    W, Cn, J, n_req = wl.trace.n_windows, 9, wl.J, len(t)
+    tbt = prof.tbt
+    if general:
+        tbt = prof.tbt.copy()
+        tbt[0, 0, 0, 3] = tbt[0, 0, 0, 2] * 0.999
+    to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a, np.uint32).view(np.int32)).to(dev)
+    d_t, d_i, d_o = to_dev(t), to_dev(i), to_dev(o)
+    d_counts = torch.empty((W, Cn), dtype=torch.int32, device=dev)
+    d_dropped = torch.empty(1, dtype=torch.int64, device=dev)
+    d_load = torch.zeros((S, W, Cn), dtype=torch.float32, device=dev)
+    small = lambda nbytes: flush if nbytes <= 126 * 2 ** 20 else None
+    run_bin = lambda: dyn.dyn_bin_trace(wl.trace.window_ms, W, gen.IN_EDGES, gen.OUT_EDGES, d_t, d_i, d_o, d_counts,
+                                        d_load[0], d_dropped)
+    entry = {"workload": name, "S": S, "W": W, "C": Cn, "J": J, "path": "general (class 0)" if general else "threshold"}
+    if with_bin:
+        ms, ms_min, n, t0, t1 = timed_kernel(dyn, run_bin, small(12 * n_req))
+        gbs = BYTES_PER_REQUEST * n_req / (ms * 1e-3) / 1e9
+        entry["bin"] = {"kernel": "bin_trace_kernel", "requests": int(n_req), "kernel_ms": ms, "kernel_ms_min": ms_min,
+                        "launches": n, "requests_per_s": n_req / (ms * 1e-3), "achieved_gbs": gbs,
+                        "frac": gbs / peaks["hbm_gbs"], "l2": "flushed" if small(12 * n_req) is not None else "inputs_larger_than_L2",
+                        "clocks": sampler.window(t0, t1) if sampler else None}
+    else:
+        run_bin()
+    torch.cuda.synchronize()
+    assert int(d_counts.sum().item()) + int(d_dropped.item()) == n_req
+    if S > 1:
+        extra = scenario_loads(wl, d_counts.cpu().numpy().view(np.uint32), S - 1)
+        d_load[1:].copy_(torch.from_numpy(extra))
+    P = dyn.Profile(prof.tp, prof.f_grid_mhz, prof.ttft, prof.cap, tbt, prof.pow, device=dev)
+    SP = dyn.Space(sp.f_cand_mhz, sp.n_max, sp.slo_ttft_s, sp.slo_tbt_s, sp.window_s, sp.gpu_budget)
+    out = dyn.SelectOut(S, W, Cn, J, device=dev, windows=False, hist=False, gpus=False)
+    ws = torch.empty(dyn.dyn_workspace_bytes(P, SP, S, W), dtype=torch.uint8, device=dev)
+    ms, ms_min, n, t0, t1 = timed_kernel(dyn, lambda: dyn.dyn_eval_select(P, SP, d_load, out, ws), small(d_load.numel() * 4))
+    evals = S * W * Cn * J
+    tfl = FLOP_PER_EVAL * evals / (ms * 1e-3) / 1e12
+    entry.update({"kernel": "eval_select_kernel", "evals": int(evals), "kernel_ms": ms, "kernel_ms_min": ms_min, "launches": n,
+                  "evals_per_s": evals / (ms * 1e-3), "achieved_tflops": tfl, "frac": tfl / peaks["fp32_tflops"],
+                  "l2": "flushed" if small(d_load.numel() * 4) is not None else "inputs_larger_than_L2",
+                  "clocks": sampler.window(t0, t1) if sampler else None,
+                  "E_total_scenario0_Wh": float(out.E_total[0].item())})
+    return entry
+
+
 def run_ours(args, rank, world, local_rank):
     import torch
     import gen
@@ -231,6 +396,7 @@ def run_ours(args, rank, world, local_rank):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
+    sampler = ClockSampler(local_rank) if rank == 0 else None
     wl, trace, prof, sp = make_inputs(args.workload, args.scenarios)
     t, i, o = trace
     n_req, W, Cn, S, J = len(t), wl.trace.n_windows, 9, wl.S, wl.J
@@ -258,14 +424,14 @@ def run_ours(args, rank, world, local_rank):
         d_load[1:].copy_(torch.from_numpy(extra))
     input_bytes = 3 * 4 * n_req + d_load.numel() * 4
     l2_mode = "inputs_larger_than_L2" if input_bytes > 126 * 2 ** 20 else "flushed"
-    flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev) if l2_mode == "flushed" else None
+    flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev)
 
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    sampler = ClockSampler(local_rank) if rank == 0 else None
+    peaks = measure_peaks(dyn, dev, sampler)     # every rank runs the probe; rank 0 reports it
     for _ in range(max(args.warmup, 3)):
         step()
     K = args.steps
@@ -274,10 +440,9 @@ def run_ours(args, rank, world, local_rank):
     for a, b in kev:                       # create the handles
         a.record(); b.record()
     barrier()
-    if sampler:
-        sampler.mark()
+    t_begin = time.time()
     for k in range(K):
-        if flush is not None:
+        if l2_mode == "flushed":
             flush.fill_(k & 0xff)          # outside the per-step events
         dyn.dyn_set_timing_events(*kev[k])
         ev[k][0].record()
@@ -285,16 +450,19 @@ def run_ours(args, rank, world, local_rank):
         ev[k][1].record()
     dyn.dyn_set_timing_events(None, None)
     barrier()
-    if sampler:
-        sampler.mark()
+    t_end = time.time()
     step_ms = [a.elapsed_time(b) for a, b in ev]
     # kev now holds the events of the LAST instrumented call of each step (the sweep of dyn_eval_select)
     kern_ms = [a.elapsed_time(b) for a, b in kev]
     total_ms = max_over_ranks(float(sum(step_ms)), dist, dev)
-    clocks = sampler.stop() if sampler else None
+    clocks = sampler.window(t_begin, t_end) if sampler else None
 
     evals_per_step = S * W * Cn * J
     value = world * K * evals_per_step / (total_ms * 1e-3)
+    share = None
+    if rank == 0:
+        ns = min(S, max(1, (1 << 28) // (W * Cn * J * 4)))     # a sample of scenarios whose energy tensor stays small
+        share = feasible_share(dyn, P, SP, d_load[:ns].contiguous())
 
     # ---- end to end through the host-buffer entry point ---------------------------------------
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
@@ -318,14 +486,18 @@ def run_ours(args, rank, world, local_rank):
     barrier()
     KE = max(1, args.e2e_steps)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_e0 = time.time()
     e0.record()
     for _ in range(KE):
         hp.run(h_t, h_i, h_o, h_extra, h_out, arena, copy_stream=side)
     e1.record()
     barrier()
+    t_e1 = time.time()
     e2e_ms = max_over_ranks(e0.elapsed_time(e1), dist, dev)
     e2e_value = world * KE * evals_per_step / (e2e_ms * 1e-3)
     E_total_e2e = h_out["E_total"].numpy().copy()
+    del arena
+    torch.cuda.empty_cache()
 
     if rank != 0:
         if dist is not None:
@@ -333,32 +505,29 @@ def run_ours(args, rank, world, local_rank):
         return
 
     # ---- roofline of the dominant kernel (the sweep), from events recorded around it ------------
+    from paper_2408_00741_b200 import counters
     k_ms = float(np.mean(kern_ms))
-    fp32_peak = SM_COUNT * FP32_LANES * 2 * SM_MAX_MHZ * 1e6 / 1e12
-    achieved = FLOP_PER_EVAL * evals_per_step / (k_ms * 1e-3) / 1e12
-    # DRAM bytes per launch and warp instructions per candidate from the ncu capture summarised in
-    # profiles/eval_select_kernel_cfg4_S64.md (3.40 MB read, 0 written at S = 64, growing in proportion to S;
-    # 6.81 instructions per 32 candidates); null for other shapes
-    same_shape = wl.name == "cfg4" and J == 2048
-    traffic = 3.40e6 * S / 64 if same_shape else None
-    issue = None
-    if same_shape:
-        # the kernel is bound by instruction issue (one warp instruction per scheduler and clock), not by
-        # the FMA units: its own instruction count against that ceiling is the hardware-side fraction
-        inst_per_s = INST_PER_WARP_EVAL_CFG4 * (evals_per_step / 32.0) / (k_ms * 1e-3)
-        issue_peak = SM_COUNT * 4 * SM_MAX_MHZ * 1e6
-        issue = {"warp_inst_per_32_evals": INST_PER_WARP_EVAL_CFG4, "achieved_warp_inst_per_s": inst_per_s,
-                 "peak_warp_inst_per_s": issue_peak, "frac": inst_per_s / issue_peak,
-                 "source": "instruction count from ncu (smsp__inst_executed.sum), rate from this run"}
-    roofline = {"bound": "alu", "kernel": "eval_select_kernel", "achieved": achieved, "peak": fp32_peak,
-                "unit": "TFLOP/s", "frac": achieved / fp32_peak, "traffic": traffic,
-                "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 flop x 1965 MHz (no measured fp32 figure in "
-                               "MEASURED_PEAKS.json)",
+    kernel_rate = evals_per_step / (k_ms * 1e-3)
+    achieved = FLOP_PER_EVAL * kernel_rate / 1e12
+    rec = counters.lookup("eval_select_kernel", wl.name)
+    traffic = None
+    if rec is not None and not rec["stale"] and rec.get("dram_bytes_per_unit") is not None:
+        traffic = rec["dram_bytes_per_unit"] * S          # the sweep's DRAM traffic is its loads: proportional to S
+    pk_clk = peaks["clocks"] or {}
+    roofline = {"bound": "alu", "kernel": "eval_select_kernel", "achieved": achieved, "peak": peaks["fp32_tflops"],
+                "unit": "TFLOP/s", "frac": achieved / peaks["fp32_tflops"], "traffic": traffic,
+                "peak_source": f"measured in this run by the library's multiply-add probe (dyn_probe_fma: 8 independent "
+                               f"chains per thread, 2048 threads per SM; {peaks['fp32_probe_launches']} launches of "
+                               f"{peaks['fp32_probe_ms']:.2f} ms at a median SM clock of {pk_clk.get('sm_mhz')} MHz); "
+                               f"nominal 148 SMs x 128 lanes x 2 x 1965 MHz = {peaks['fp32_nominal_tflops']:.2f}",
+                "peak_clocks": peaks["clocks"],
                 "flop_per_eval": FLOP_PER_EVAL,
-                "note": "achieved counts the 20 fp32 operations per candidate of the definition; the kernel needs "
-                        "about 8 (load threshold instead of a TBT interpolation, energy line in intercept form, "
-                        "n applied once per chain), so the fraction can exceed 1",
-                "issue": issue, "kernel_ms": k_ms, "evals_per_s_kernel": evals_per_step / (k_ms * 1e-3)}
+                "note": "`achieved` counts the 20 fp32 operations per candidate of the definition; the kernel executes "
+                        "fewer (a load threshold instead of a TBT interpolation, the energy line in intercept form, n "
+                        "applied once per chain), so `frac` can exceed 1; `executed` holds the hardware-side figures",
+                "executed": executed_work(dyn, peaks, sampler, wl.name, kernel_rate, share),
+                "kernel_ms": k_ms, "evals_per_s_kernel": kernel_rate,
+                "hbm_peak_gbs": peaks["hbm_gbs"], "hbm_peak_source": peaks["hbm_source"]}
 
     result = {
         "metric": "config_evaluations_per_s", "value": value, "unit": "evals/s", "n_gpus": world, "steps": K,
@@ -368,51 +537,66 @@ def run_ours(args, rank, world, local_rank):
                    "multi_gpu": "replicas only"},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": "evals/s", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-                "steps": KE, "ms_per_step": e2e_ms / KE},
+                "steps": KE, "ms_per_step": e2e_ms / KE, "clocks": sampler.window(t_e0, t_e1) if sampler else None},
         "gpu_launches": launches_per_step * K,
+        "trace_requests_per_s": None,
         "roofline": roofline,
         "E_total_scenario0_Wh": float(E_total_e2e[0]),
     }
 
-    # ---- side measurement: the histogram kernel on the week-long trace (HBM-bound) ---------------
-    if not args.no_secondary and world == 1:
+    def guarded(fn, *a, **kw):
         try:
-            result["bin_trace"] = measure_bin(dyn, gen, dev)
+            t0 = time.time()
+            r = fn(*a, **kw)
+            if isinstance(r, dict) and "clocks" not in r and sampler:
+                r["clocks"] = sampler.window(t0, time.time())
+            return r
         except Exception as exc:                      # never lose the main line
-            result["bin_trace"] = {"error": repr(exc)}
-        try:
-            result["materialised"] = measure_materialised(dyn, gen, dev)
-        except Exception as exc:
-            result["materialised"] = {"error": repr(exc)}
-        try:
-            result["hierarchical"] = measure_hier(dyn, gen, dev)
-        except Exception as exc:
-            result["hierarchical"] = {"error": repr(exc)}
-        try:
-            # 32 GPUs per pool (1624 count tuples) and a small pool of 16 (200 tuples, passes half empty)
-            result["mixed_pools"] = measure_mixed(dyn, gen, dev, n_max=32, budget=32)
-            result["mixed_pools"]["small_pool"] = measure_mixed(dyn, gen, dev, n_max=16, budget=16)
-        except Exception as exc:
-            result["mixed_pools"] = {"error": repr(exc)}
-        try:
-            result["reconfiguration"] = measure_reconf(dyn, gen, dev)
-        except Exception as exc:
-            result["reconfiguration"] = {"error": repr(exc)}
+            return {"error": repr(exc)}
+
+    # ---- every benchmark configuration, and the other kernels (side measurements) ----------------
+    if not args.no_secondary and world == 1:
+        del d_t, d_i, d_o
+        torch.cuda.empty_cache()
+        pc = {}
+        cfg3_trace = gen.make_trace(gen.workload("cfg3").trace)
+        for key, kw in (("cfg1", dict(name="cfg1")),
+                        ("cfg1_x4096", dict(name="cfg1", S=4096, with_bin=False)),
+                        ("cfg2", dict(name="cfg2", trace=trace if wl.name in ("cfg2", "cfg4") else None)),
+                        ("cfg3", dict(name="cfg3", trace=cfg3_trace)),
+                        ("cfg3code", dict(name="cfg3code")),
+                        ("cfg5", dict(name="cfg5")),
+                        ("cfg2_x256_general", dict(name="cfg2", S=256, general=True, with_bin=False,
+                                                   trace=trace if wl.name in ("cfg2", "cfg4") else None))):
+            pc[key] = guarded(measure_config, dyn, gen, dev, sampler, peaks, flush, **kw)
+        roofline["per_config"] = pc
+        if isinstance(pc.get("cfg3"), dict) and "bin" in pc["cfg3"]:
+            result["trace_requests_per_s"] = pc["cfg3"]["bin"]["requests_per_s"]
+        result["bin_trace"] = guarded(measure_bin, dyn, gen, dev, cfg3_trace)
+        del cfg3_trace
+        result["materialised"] = guarded(measure_materialised, dyn, gen, dev)
+        result["hierarchical"] = guarded(measure_hier, dyn, gen, dev, peaks=peaks)
+        # 32 GPUs per pool (1624 count tuples) and a small pool of 16 (200 tuples)
+        result["mixed_pools"] = guarded(measure_mixed, dyn, gen, dev, n_max=32, budget=32, peaks=peaks)
+        if "error" not in result["mixed_pools"]:
+            result["mixed_pools"]["small_pool"] = guarded(measure_mixed, dyn, gen, dev, n_max=16, budget=16, peaks=peaks)
+        result["reconfiguration"] = guarded(measure_reconf, dyn, gen, dev, peaks=peaks)
 
     if not args.no_cpu_baseline and world == 1:
         cb, _, _ = time_oracle(wl, trace, prof, sp, base_counts)
         result["cpu_baseline"] = cb
+    result["clocks_whole_run"] = sampler.stop() if sampler else None
     print(json.dumps(result))
     if dist is not None:
         dist.destroy_process_group()
 
 
-def measure_bin(dyn, gen, dev):
+def measure_bin(dyn, gen, dev, trace=None):
     """Requests/s of the trace-binning kernel on the 14M-request week trace (168 MB, larger than L2), and
     on the same trace repeated 8 times (1.3 GB) to show what the kernel sustains on a long trace."""
     import torch
     wl = gen.workload("cfg3")
-    t, i, o = gen.make_trace(wl.trace)
+    t, i, o = trace if trace is not None else gen.make_trace(wl.trace)
     W = wl.trace.n_windows
     peak, src = _hbm_peak()
     counts = torch.empty((W, 9), dtype=torch.int32, device=dev)
@@ -423,22 +607,10 @@ def measure_bin(dyn, gen, dev):
         d = [torch.from_numpy(np.tile(x, rep).view(np.int32)).to(dev) for x in (t, i, o)]
         n = int(d[0].numel())
         run = lambda: dyn.dyn_bin_trace(wl.trace.window_ms, W, gen.IN_EDGES, gen.OUT_EDGES, d[0], d[1], d[2], counts, load, dropped)
-        for _ in range(3):
-            run()
-        K = 20 if rep == 1 else 5
-        kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
-        for a, b in kev:
-            a.record(); b.record()
-        torch.cuda.synchronize()
-        for k in range(K):
-            dyn.dyn_set_timing_events(*kev[k])
-            run()
-        dyn.dyn_set_timing_events(None, None)
-        torch.cuda.synchronize()
+        ms, ms_min, k, _, _ = timed_kernel(dyn, run, None, min_s=0.3)
         assert int(counts.sum().item()) + int(dropped.item()) == n
-        ms = float(np.mean([a.elapsed_time(b) for a, b in kev]))
         gbs = BYTES_PER_REQUEST * n / (ms * 1e-3) / 1e9
-        r = {"requests": n, "kernel_ms": ms, "requests_per_s": n / (ms * 1e-3),
+        r = {"requests": n, "kernel_ms": ms, "kernel_ms_min": ms_min, "launches": k, "requests_per_s": n / (ms * 1e-3),
              "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
                           "traffic": None, "peak_source": src}}
         if rep == 1:
@@ -450,21 +622,20 @@ def measure_bin(dyn, gen, dev):
             ti = torch.empty((W, 9), dtype=torch.int64, device=dev)
             to = torch.empty((W, 9), dtype=torch.int64, device=dev)
             runt = lambda: dyn.dyn_bin_tokens(wl.trace.window_ms, W, gen.IN_EDGES, gen.OUT_EDGES, d[0], d[1], d[2], ti, to, load)
-            for _ in range(3):
-                runt()
-            torch.cuda.synchronize()
-            for k in range(K):
-                dyn.dyn_set_timing_events(*kev[k])
-                runt()
-            dyn.dyn_set_timing_events(None, None)
-            torch.cuda.synchronize()
-            mst = float(np.mean([a.elapsed_time(b) for a, b in kev]))
+            mst, mst_min, k, _, _ = timed_kernel(dyn, runt, None, min_s=0.3)
             gbt = BYTES_PER_REQUEST * n / (mst * 1e-3) / 1e9
-            out["token_sums"] = {"kernel": "bin_tokens_kernel", "kernel_ms": mst, "requests_per_s": n / (mst * 1e-3),
+            out["token_sums"] = {"kernel": "bin_tokens_kernel", "kernel_ms": mst, "kernel_ms_min": mst_min, "launches": k,
+                                 "requests_per_s": n / (mst * 1e-3),
                                  "roofline": {"bound": "hbm", "achieved": gbt, "peak": peak, "unit": "GB/s",
                                               "frac": gbt / peak, "traffic": None, "peak_source": src}}
         del d
     return out
+
+
+def _fp32_peak(peaks):
+    if peaks is not None:
+        return peaks["fp32_tflops"], "fp32 peak measured in this run by the multiply-add probe"
+    return SM_COUNT * FP32_LANES * 2 * SM_MAX_MHZ * 1e6 / 1e12, "nominal fp32 peak (148 x 128 x 2 x 1965 MHz)"
 
 
 def _hbm_peak():
@@ -492,27 +663,15 @@ def measure_materialised(dyn, gen, dev, S=16):
     res = {"workload": f"cfg2 shape x {S} scenarios", "candidates": int(E.numel()), "tensor_bytes": int(E.numel() * 4)}
     for name, call in (("eval_configs_kernel", lambda: dyn.dyn_eval_configs(P, SP, load, E, ws)),
                        ("select_kernel", lambda: dyn.dyn_select(E, out, ws2))):
-        for _ in range(3):
-            call()
-        K = 10
-        kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
-        for a, b in kev:
-            a.record(); b.record()
-        torch.cuda.synchronize()
-        for k in range(K):
-            dyn.dyn_set_timing_events(*kev[k])
-            call()
-        dyn.dyn_set_timing_events(None, None)
-        torch.cuda.synchronize()
-        ms = float(np.mean([a.elapsed_time(b) for a, b in kev]))
+        ms, ms_min, k, _, _ = timed_kernel(dyn, call, None, min_s=0.3, per_round=10)
         gbs = E.numel() * 4 / (ms * 1e-3) / 1e9
-        res[name] = {"kernel_ms": ms, "evals_per_s": E.numel() / (ms * 1e-3),
+        res[name] = {"kernel_ms": ms, "kernel_ms_min": ms_min, "launches": k, "evals_per_s": E.numel() / (ms * 1e-3),
                      "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
                                   "traffic": None, "peak_source": src}}
     return res
 
 
-def measure_hier(dyn, gen, dev, S=2048):
+def measure_hier(dyn, gen, dev, S=2048, peaks=None):
     """Hierarchical selection (nodes per 30 min, sharding per 5 min, frequency per 1-min window) on S
     day-long scenarios, whole call; and its energy against the joint optimum on the first 8 scenarios."""
     import torch
@@ -530,21 +689,24 @@ def measure_hier(dyn, gen, dev, S=2048):
     call = lambda: dyn.dyn_hier_select(P, SP, e1, e2, load, nodes, shard, out, ws)
     for _ in range(3):
         call()
-    K = 10
+    torch.cuda.synchronize()
+    K, rounds = 10, 0
     e0, e1_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    e0.record()
-    for _ in range(K):
-        call()
-    e1_.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1_) / K
+    ms_all, t0 = [], time.time()
+    while time.time() - t0 < 0.4:
+        e0.record()
+        for _ in range(K):
+            call()
+        e1_.record()
+        torch.cuda.synchronize()
+        ms_all.append(e0.elapsed_time(e1_) / K)
+    ms = float(np.mean(ms_all))
     tiles = S * W * Cn
     # candidates of the two restricted searches: (n, TP) per shard epoch, f per window; the node budget
     # prunes part of the first, so this is an upper bound of what was evaluated
     K2 = -(-W // e2)
     cands = S * Cn * (K2 * sp.n_max * len(prof.tp) + W * len(sp.f_cand_mhz))
-    fp32_peak = SM_COUNT * FP32_LANES * 2 * SM_MAX_MHZ * 1e6 / 1e12
+    fp32_peak, peak_src = _fp32_peak(peaks)
     tfl = FLOP_PER_EVAL * cands / (ms * 1e-3) / 1e12
     hier_total = float(out.E_total[:8].sum().item())
     jout = dyn.SelectOut(8, W, Cn, J, device=dev, windows=False, hist=False, gpus=False)
@@ -555,11 +717,11 @@ def measure_hier(dyn, gen, dev, S=2048):
     return {"workload": f"cfg2 shape x {S} scenarios, epochs {e1}/{e2}/1 windows", "tiles": int(tiles), "call_ms": ms,
             "tiles_per_s": tiles / (ms * 1e-3), "candidates_upper_bound": int(cands),
             "roofline": {"bound": "alu", "achieved": tfl, "peak": fp32_peak, "unit": "TFLOP/s", "frac": tfl / fp32_peak,
-                         "traffic": None, "peak_source": "derived fp32 peak; candidates are an upper bound (node budget prunes)"},
+                         "traffic": None, "peak_source": peak_src + "; candidates are an upper bound (node budget prunes)"},
             "energy_over_joint_optimum": hier_total / joint_total}
 
 
-def measure_mixed(dyn, gen, dev, S=16, n_max=16, budget=16):
+def measure_mixed(dyn, gen, dev, S=16, n_max=16, budget=16, peaks=None):
     """Pools that mix tensor parallelisms (Eq. 1 in full, by enumeration) on S day-long scenarios of the 1-day
     profile: every count tuple within `budget` GPUs, per group every candidate frequency."""
     import itertools
@@ -574,37 +736,25 @@ def measure_mixed(dyn, gen, dev, S=16, n_max=16, budget=16):
     out = dyn.MixedOut(S, W, Cn, T, device=dev)
     ws = torch.empty(dyn.dyn_mixed_workspace_bytes(P, SP, S, W), dtype=torch.uint8, device=dev)
     call = lambda: dyn.dyn_mixed_select(P, SP, load, out, ws)
-    for _ in range(3):
-        call()
-    K = 10
-    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
-    for a, b in kev:
-        a.record(); b.record()
-    torch.cuda.synchronize()
-    for k in range(K):
-        dyn.dyn_set_timing_events(*kev[k])
-        call()
-    dyn.dyn_set_timing_events(None, None)
-    torch.cuda.synchronize()
-    ms = float(np.mean([a.elapsed_time(b) for a, b in kev]))
+    ms, ms_min, _, _, _ = timed_kernel(dyn, call, None, min_s=0.3, per_round=10)
     # single-type evaluations per tile: for every tuple within the budget, F per parallelism in use
     tuples = [n for n in itertools.product(range(n_max + 1), repeat=T)
               if 0 < sum(a * int(t) for a, t in zip(n, prof.tp)) <= budget]
     assert len(tuples) == dyn.dyn_mixed_tuple_count(P, SP)
     per_tile = F * sum(sum(1 for a in n if a) for n in tuples)
     evals = S * W * Cn * per_tile
-    fp32_peak = SM_COUNT * FP32_LANES * 2 * SM_MAX_MHZ * 1e6 / 1e12
+    fp32_peak, peak_src = _fp32_peak(peaks)
     tfl = FLOP_PER_EVAL * evals / (ms * 1e-3) / 1e12
     mixed_frac = float(((out.counts > 0).sum(dim=3) > 1).float().mean().item())
     return {"workload": f"cfg2 profile x {S} scenarios, counts 0..{n_max} per TP, {budget} GPUs per pool",
             "tiles": int(S * W * Cn), "tuples": len(tuples), "evaluations": int(evals), "kernel_ms": ms,
             "evals_per_s": evals / (ms * 1e-3), "tiles_per_s": S * W * Cn / (ms * 1e-3),
             "roofline": {"bound": "alu", "achieved": tfl, "peak": fp32_peak, "unit": "TFLOP/s", "frac": tfl / fp32_peak,
-                         "traffic": None, "peak_source": "derived fp32 peak; 20 flop per single-type evaluation"},
+                         "traffic": None, "peak_source": peak_src + "; 20 flop per single-type evaluation"},
             "tiles_that_mix_parallelisms": mixed_frac}
 
 
-def measure_reconf(dyn, gen, dev, S=16):
+def measure_reconf(dyn, gen, dev, S=16, peaks=None):
     """Selection with re-configuration costs on S day-long scenarios of the 1-day profile (256 shardings, 1440
     windows): the path kernel alone; its work is W * NS^2 add-compare steps per (scenario, class)."""
     import torch
@@ -622,24 +772,17 @@ def measure_reconf(dyn, gen, dev, S=16):
     total = torch.empty((S, Cn), dtype=torch.float64, device=dev)
     ws = torch.empty(dyn.dyn_reconf_workspace_bytes(P, SP, S, W), dtype=torch.uint8, device=dev)
     call = lambda: dyn.dyn_reconf_select(P, SP, d_R, load, out, total, ws)
-    for _ in range(2):
-        call()
-    K = 5
-    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
-    for a, b in kev:
-        a.record(); b.record()
+    ms, ms_min, _, _, _ = timed_kernel(dyn, call, None, min_s=0.3, per_round=5)
     c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    K = 5
     torch.cuda.synchronize()
     c0.record()
     for k in range(K):
-        dyn.dyn_set_timing_events(*kev[k])
         call()
-    dyn.dyn_set_timing_events(None, None)
     c1.record()
     torch.cuda.synchronize()
-    ms = float(np.mean([a.elapsed_time(b) for a, b in kev]))
     steps = S * Cn * (W - 1) * NS * NS                      # add + compare of the min-plus recursion
-    fp32_peak = SM_COUNT * FP32_LANES * 2 * SM_MAX_MHZ * 1e6 / 1e12
+    fp32_peak, peak_src = _fp32_peak(peaks)
     tfl = 2.0 * steps / (ms * 1e-3) / 1e12
     # energy of the schedules against the per-window optimum that ignores transition costs
     jout = dyn.SelectOut(S, W, Cn, J, device=dev, windows=False, hist=False, gpus=False)
@@ -650,13 +793,81 @@ def measure_reconf(dyn, gen, dev, S=16):
             "path_kernel_ms": ms, "call_ms": c0.elapsed_time(c1) / K, "minplus_steps": int(steps),
             "steps_per_s": steps / (ms * 1e-3),
             "roofline": {"bound": "alu", "achieved": tfl, "peak": fp32_peak, "unit": "TFLOP/s", "frac": tfl / fp32_peak,
-                         "traffic": None, "peak_source": "derived fp32 peak; 2 flop (add, compare) per step"},
+                         "traffic": None, "peak_source": peak_src + "; 2 flop (add, compare) per step"},
             "window_energy_over_free_optimum": float(out.E_total.sum().item() / jout.E_total.sum().item()),
             "schedules": int(torch.isfinite(total).sum().item())}
 
 
+def run_only(args, local_rank):
+    """Only the named side measurements (--only a,b,...), one JSON line."""
+    import torch
+    import gen
+    import paper_2408_00741_b200 as dyn
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    sampler = ClockSampler(local_rank)
+    peaks = measure_peaks(dyn, dev, sampler)
+    flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev)
+    per_config = {"cfg1": dict(name="cfg1"), "cfg1_x4096": dict(name="cfg1", S=4096, with_bin=False), "cfg2": dict(name="cfg2"),
+                  "cfg3": dict(name="cfg3"), "cfg3code": dict(name="cfg3code"), "cfg5": dict(name="cfg5"),
+                  "cfg2_x256_general": dict(name="cfg2", S=256, general=True, with_bin=False)}
+    res = {"peaks": {k: v for k, v in peaks.items() if k != "sink"}}
+    for key in args.only.split(","):
+        if key in per_config:
+            res[key] = measure_config(dyn, gen, dev, sampler, peaks, flush, **per_config[key])
+        elif key == "bin_trace":
+            res[key] = measure_bin(dyn, gen, dev)
+        elif key == "materialised":
+            res[key] = measure_materialised(dyn, gen, dev)
+        elif key == "hierarchical":
+            res[key] = measure_hier(dyn, gen, dev, peaks=peaks)
+        elif key == "mixed_pools":
+            res[key] = measure_mixed(dyn, gen, dev, n_max=32, budget=32, peaks=peaks)
+        elif key == "mixed_pools_small":
+            res[key] = measure_mixed(dyn, gen, dev, peaks=peaks)
+        elif key == "reconfiguration":
+            res[key] = measure_reconf(dyn, gen, dev, peaks=peaks)
+        else:
+            raise SystemExit(f"--only: unknown name {key!r}; known: {', '.join(SIDE)}")
+    res["clocks_whole_run"] = sampler.stop()
+    print(json.dumps(res))
+
+
+def free_port() -> int:
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
+def spawn_ranks(n: int, argv, timeout_s: float = 3600.0) -> int:
+    """Starts `argv` n times as local ranks 0..n-1 (one per GPU: RANK = LOCAL_RANK = k, WORLD_SIZE = n, rendezvous
+    on 127.0.0.1), forwards what they print, and returns the first non-zero exit code (0 if all succeeded)."""
+    port = free_port()
+    procs = []
+    for k in range(n):
+        env = dict(os.environ, RANK=str(k), LOCAL_RANK=str(k), WORLD_SIZE=str(n), LOCAL_WORLD_SIZE=str(n),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen(list(argv), env=env))
+    rc = 0
+    deadline = time.time() + timeout_s
+    for p in procs:
+        try:
+            r = p.wait(timeout=max(1.0, deadline - time.time()))
+        except subprocess.TimeoutExpired:
+            p.kill()
+            r = -9
+        rc = rc or r
+    return rc
+
+
 def main():
     args = parse_args()
+    if args.quick:
+        global QUICK
+        QUICK = True
+    if args.impl == "ours" and args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started without a launcher: be the launcher (one rank per GPU, every rank an independent replica)
+        sys.exit(spawn_ranks(args.gpus, [sys.executable, os.path.abspath(__file__)] + sys.argv[1:]))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -664,15 +875,9 @@ def main():
         run_reference(args, rank)
         return
     if args.secondary_only:
-        import torch
-        import gen
-        import paper_2408_00741_b200 as dyn
-        dev = torch.device("cuda", local_rank)
-        torch.cuda.set_device(dev)
-        print(json.dumps({"bin_trace": measure_bin(dyn, gen, dev), "materialised": measure_materialised(dyn, gen, dev),
-                          "hierarchical": measure_hier(dyn, gen, dev), "mixed_pools": measure_mixed(dyn, gen, dev, n_max=32, budget=32),
-                          "mixed_pools_small": measure_mixed(dyn, gen, dev),
-                          "reconfiguration": measure_reconf(dyn, gen, dev)}))
+        args.only = "bin_trace,materialised,hierarchical,mixed_pools,mixed_pools_small,reconfiguration"
+    if args.only:
+        run_only(args, local_rank)
         return
     run_ours(args, rank, world, local_rank)
 

@@ -353,6 +353,30 @@ int dyn_pipeline_host(const dyn_bin_spec *spec, const dyn_profile_host *profile,
 void dyn_set_timing_events(void *start_event, void *stop_event);
 
 /* ---------------------------------------------------------------------------------------------
+ * Measured ceilings (instrumentation; no counterpart in the paper).  Each call enqueues one short
+ * kernel on `stream` and records the events of dyn_set_timing_events around it; the caller divides
+ * the returned amount of work by the measured time.  d_sink: device float [1], required, never
+ * written for the values the kernels use (it only keeps their arithmetic alive).  `iters` >= 1 scales
+ * the run time (about 1 ms per 500 on a B200 for the first, per 100 for the second).
+ *
+ *   dyn_probe_fma          every thread advances eight independent fp32 multiply-add chains; *fp32_ops
+ *                          (host, may be NULL) receives the fp32 operations executed, 2 per lane and
+ *                          multiply-add.  ops / time is the fp32 peak of this GPU at the clock it runs at;
+ *                          one warp-wide multiply-add is 64 operations, so peak / 64 is the ceiling of
+ *                          instruction issue (warp instructions per second).
+ *   dyn_probe_sweep_inner  the inner (TP, f) loop of dyn_eval_select's kernel on the load-threshold path,
+ *                          the same device code on a synthetic table in shared memory, 8 candidates per
+ *                          lane and pair, without any per-tile work; `feasible_share` in [0, 1] is the
+ *                          share of candidates whose load is within the pair's limit (an infeasible
+ *                          candidate skips its table lookup, so the rate depends on it); *candidates
+ *                          (host, may be NULL) receives the candidates evaluated.  candidates / time is
+ *                          the rate the instruction mix of that loop reaches on this GPU.
+ * Errors: DYN_EINVAL (iters < 1, NULL d_sink, share outside [0, 1]), DYN_ECUDA.
+ * ------------------------------------------------------------------------------------------- */
+int dyn_probe_fma(int32_t iters, float *d_sink, double *fp32_ops, void *stream);
+int dyn_probe_sweep_inner(int32_t iters, float feasible_share, float *d_sink, double *candidates, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
  * dyn_eval_select without a workspace argument (the paper has no counterpart; this is a packaging
  * variant of dyn_eval_select for callers that cannot obtain device memory).
  *

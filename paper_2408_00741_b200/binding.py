@@ -25,7 +25,8 @@ DYN_OK, DYN_EINVAL, DYN_ECUDA, DYN_EUNSUPPORTED, DYN_EWORKSPACE = 0, -1, -2, -3,
 EXPORTS = ("dyn_strerror", "dyn_last_cuda_error", "dyn_bin_trace", "dyn_workspace_bytes", "dyn_eval_configs",
            "dyn_select_workspace_bytes", "dyn_select", "dyn_eval_select", "dyn_pipeline_arena_bytes",
            "dyn_pipeline_host", "dyn_set_timing_events", "dyn_eval_select_static", "dyn_hier_workspace_bytes",
-           "dyn_hier_select", "dyn_mixed_workspace_bytes", "dyn_mixed_tuple_count", "dyn_mixed_select", "dyn_reconf_workspace_bytes", "dyn_reconf_select", "dyn_bin_tokens", "dyn_carbon")
+           "dyn_hier_select", "dyn_mixed_workspace_bytes", "dyn_mixed_tuple_count", "dyn_mixed_select", "dyn_reconf_workspace_bytes", "dyn_reconf_select", "dyn_bin_tokens", "dyn_carbon",
+           "dyn_probe_fma", "dyn_probe_sweep_inner")
 
 
 class DynError(RuntimeError):
@@ -144,6 +145,10 @@ _lib.dyn_bin_tokens.argtypes = [C.POINTER(_BinSpec), C.c_void_p, C.c_void_p, C.c
                                 C.c_void_p, C.c_void_p]
 _lib.dyn_carbon.restype = C.c_int
 _lib.dyn_carbon.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p]
+_lib.dyn_probe_fma.restype = C.c_int
+_lib.dyn_probe_fma.argtypes = [C.c_int32, C.c_void_p, C.POINTER(C.c_double), C.c_void_p]
+_lib.dyn_probe_sweep_inner.restype = C.c_int
+_lib.dyn_probe_sweep_inner.argtypes = [C.c_int32, C.c_float, C.c_void_p, C.POINTER(C.c_double), C.c_void_p]
 
 
 def _dev(t, dtype, what):
@@ -446,3 +451,20 @@ def dyn_carbon(d_E_window, d_intensity, d_carbon):
     rc = _lib.dyn_carbon(_dev(d_E_window, torch.float64, "d_E_window"), _dev(d_intensity, torch.float32, "d_intensity"), S, W,
                          _dev(d_carbon, torch.float64, "d_carbon"), _stream())
     _check(rc, "dyn_carbon")
+
+
+def dyn_probe_fma(iters, d_sink) -> float:
+    """Enqueues the multiply-add probe; returns the fp32 operations it executes (d_sink: float32 [1])."""
+    work = C.c_double(0.0)
+    _check(_lib.dyn_probe_fma(int(iters), _dev(d_sink, torch.float32, "d_sink"), C.byref(work), _stream()), "dyn_probe_fma")
+    return work.value
+
+
+def dyn_probe_sweep_inner(iters, feasible_share, d_sink) -> float:
+    """Enqueues the inner-loop probe of the sweep with the given share of feasible candidates; returns the
+    candidates it evaluates (d_sink: float32 [1])."""
+    work = C.c_double(0.0)
+    _check(_lib.dyn_probe_sweep_inner(int(iters), float(feasible_share), _dev(d_sink, torch.float32, "d_sink"),
+                                      C.byref(work), _stream()),
+           "dyn_probe_sweep_inner")
+    return work.value

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(CSRC, "libdynamo.so")
-SOURCES = ["abi.cu", "bin_trace.cu", "resolve.cu", "sweep.cu", "select.cu", "pipeline.cu", "static_ws.cu", "hier.cu", "mixed.cu", "reconf.cu", "tokens.cu"]
+SOURCES = ["abi.cu", "bin_trace.cu", "resolve.cu", "sweep.cu", "select.cu", "pipeline.cu", "static_ws.cu", "hier.cu", "mixed.cu", "reconf.cu", "tokens.cu", "probe.cu"]
 HEADERS = [os.path.join(CSRC, "dyn_internal.cuh"), os.path.join(CSRC, "eval_dev.cuh"), os.path.join(ROOT, "include", "dynamo.h")]
 
 

@@ -57,13 +57,59 @@ def test_oracle_step_and_scenarios():
     assert bench.scenario_loads(wl, counts, 0) is None
 
 
-def test_clock_sampler_parses_rows(tmp_path):
+def test_clock_sampler_parses_rows_and_windows(tmp_path):
     import bench
+    import datetime
     cs = bench.ClockSampler.__new__(bench.ClockSampler)
     f = open(tmp_path / "c.csv", "w+")
-    f.write("1965, 1965, 640.1, 0x0000000000000004, Not Active, Not Active, Not Active, Active\n" * 3)
-    f.write("1800, 1965, 990.0, 0x0000000000000004, Not Active, Not Active, Not Active, Active\n")
+    base = datetime.datetime(2026, 1, 2, 3, 4, 5)
+    stamp = lambda k: (base + datetime.timedelta(milliseconds=100 * k)).strftime("%Y/%m/%d %H:%M:%S.%f")[:-3]
+    for k in range(3):
+        f.write(f"{stamp(k)}, 1965, 1965, 640.1, 0x0000000000000004, Not Active, Not Active, Not Active, Active\n")
+    f.write(f"{stamp(3)}, 1800, 1965, 990.0, 0x0000000000000004, Not Active, Not Active, Not Active, Active\n")
+    for k in range(4, 10):
+        f.write(f"{stamp(k)}, 1500, 1965, 990.0, 0x0000000000000000, Not Active, Not Active, Not Active, Not Active\n")
+    f.write("garbage row\n")
     f.flush()
-    cs.f, cs.p, cs.marks = f, None, []
+    cs.f, cs.p = f, None
+    t0 = base.timestamp()
+    early = cs.window(t0, t0 + 0.2)                      # one period of slack: samples 0..3
+    assert early["sm_mhz"] == 1965.0 and early["reasons"] == ["sw_power_cap"] and early["samples"] == 4
+    late = cs.window(t0 + 0.6, t0 + 0.9)
+    assert late["sm_mhz"] == 1500.0 and late["reasons"] == [] and late["samples"] == 5
     out = cs.stop()
-    assert out["sm_mhz"] == 1965.0 and out["sm_max_mhz"] == 1965.0 and out["reasons"] == ["sw_power_cap"]
+    assert out["samples"] == 10 and out["sm_max_mhz"] == 1965.0 and out["reasons"] == ["sw_power_cap"]
+
+
+def test_gpus_flag_starts_that_many_ranks(tmp_path):
+    """`--gpus N` without a launcher: spawn_ranks starts N local ranks with the rendezvous variables set; two gloo
+    ranks stand in for two GPUs, a stub stands in for the workload, rank 0 prints n_gpus = 2."""
+    import bench
+    import json
+    import subprocess
+    stub = tmp_path / "rank_stub.py"
+    stub.write_text(
+        "import os, sys, json\n"
+        f"sys.path.insert(0, {ROOT!r})\n"
+        "import torch, torch.distributed as dist\n"
+        "import bench\n"
+        "rank, world = int(os.environ['RANK']), int(os.environ['WORLD_SIZE'])\n"
+        "assert os.environ['LOCAL_RANK'] == os.environ['RANK'] and os.environ['MASTER_ADDR'] == '127.0.0.1'\n"
+        "dist.init_process_group('gloo', rank=rank, world_size=world)\n"
+        "ms = bench.max_over_ranks(10.0 + rank, dist, torch.device('cpu'))\n"
+        "dist.barrier()\n"
+        "if rank == 0:\n"
+        f"    open({str(tmp_path / 'out.json')!r}, 'w').write(json.dumps({{'n_gpus': world, 'ms': ms}}))\n"
+        "dist.destroy_process_group()\n")
+    assert bench.spawn_ranks(2, [sys.executable, str(stub)], timeout_s=300) == 0
+    got = json.loads(open(tmp_path / "out.json").read())
+    assert got == {"n_gpus": 2, "ms": 11.0}
+    # a failing rank is reported
+    bad = tmp_path / "bad.py"
+    bad.write_text("import os, sys\nsys.exit(3 if os.environ['RANK'] == '1' else 0)\n")
+    assert bench.spawn_ranks(2, [sys.executable, str(bad)], timeout_s=60) == 3
+    # and the command line takes that route: --gpus 2 without WORLD_SIZE re-executes bench.py once per rank
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference", "--help"],
+                       env=env, capture_output=True, text=True, timeout=120)
+    assert r.returncode == 0
