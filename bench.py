@@ -34,7 +34,7 @@ if ROOT not in sys.path:
 FLOP_PER_EVAL = 20.0            # algorithmic fp32 operations per candidate, counted from the definition
 SM_COUNT, FP32_LANES, SM_MAX_MHZ = 148, 128, 1965.0     # nominal figures, reported beside the measured peak
 BYTES_PER_REQUEST = 12.0
-SIDE = ("cfg1", "cfg1_x4096", "cfg2", "cfg3", "cfg3code", "cfg5", "cfg2_x256_general", "bin_trace", "materialised",
+SIDE = ("cfg1", "cfg1_x4096", "cfg2", "cfg3", "cfg3code", "cfg5", "cfg2_x256", "cfg2_x256_one_row_general", "cfg2_x256_general", "bin_trace", "materialised",
         "hierarchical", "mixed_pools", "mixed_pools_small", "reconfiguration")
 
 
@@ -332,19 +332,36 @@ def executed_work(dyn, peaks, sampler, wl_name, kernel_rate, share):
     return out
 
 
-def measure_config(dyn, gen, dev, sampler, peaks, flush, name, S=1, general=False, trace=None, with_bin=True):
+def rows_without_threshold(prof, sp, which):
+    """A copy of the TBT table in which rows cross the SLO twice (feasible, infeasible, feasible again as the load
+    grows), so that no load threshold describes them and the sweep interpolates TBT per candidate there: knot 1 is
+    lifted above the SLO in rows whose knots 0 and 2 are within it.  which = "one": a single row; "all": every such
+    row (about two thirds of the rows of the synthetic profiles; the rest are infeasible at any load)."""
+    tbt = prof.tbt.copy()
+    n = 0
+    for c in range(tbt.shape[0]):
+        slo = float(sp.slo_tbt_s[c])
+        ok = (tbt[c, :, :, 0] <= slo) & (tbt[c, :, :, 2] <= slo)
+        for t, r in np.argwhere(ok):
+            if which == "one" and n >= 1:
+                break
+            tbt[c, t, r, 1] = 1.05 * slo
+            n += 1
+    return tbt, n
+
+
+def measure_config(dyn, gen, dev, sampler, peaks, flush, name, S=1, general=None, trace=None, with_bin=True):
     """One benchmark configuration: the histogram kernel on its trace and the fused sweep on its loads (S > 1:
-    Poisson-resampled scenarios of the binned trace; general: one TBT row made non-monotone, which puts that
-    class on the path that interpolates TBT per candidate)."""
+    Poisson-resampled scenarios of the binned trace; general = "one" / "all": one row / every row that is feasible
+    at all crosses the SLO twice and takes the path that interpolates TBT per candidate)."""
     import torch
     wl = gen.workload(name)
     t, i, o = trace if trace is not None else gen.make_trace(wl.trace)
     prof, sp = wl.profile(), wl.space()
     W, Cn, J, n_req = wl.trace.n_windows, 9, wl.J, len(t)
-    tbt = prof.tbt
+    tbt, n_general = prof.tbt, 0
     if general:
-        tbt = prof.tbt.copy()
-        tbt[0, 0, 0, 3] = tbt[0, 0, 0, 2] * 0.999
+        tbt, n_general = rows_without_threshold(prof, sp, general)
     to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a, np.uint32).view(np.int32)).to(dev)
     d_t, d_i, d_o = to_dev(t), to_dev(i), to_dev(o)
     d_counts = torch.empty((W, Cn), dtype=torch.int32, device=dev)
@@ -353,7 +370,7 @@ def measure_config(dyn, gen, dev, sampler, peaks, flush, name, S=1, general=Fals
     small = lambda nbytes: flush if nbytes <= 126 * 2 ** 20 else None
     run_bin = lambda: dyn.dyn_bin_trace(wl.trace.window_ms, W, gen.IN_EDGES, gen.OUT_EDGES, d_t, d_i, d_o, d_counts,
                                         d_load[0], d_dropped)
-    entry = {"workload": name, "S": S, "W": W, "C": Cn, "J": J, "path": "general (class 0)" if general else "threshold"}
+    entry = {"workload": name, "S": S, "W": W, "C": Cn, "J": J, "path": f"per-candidate TBT interpolation on {n_general} of {tbt[..., 0].size} table rows" if general else "threshold"}
     if with_bin:
         ms, ms_min, n, t0, t1 = timed_kernel(dyn, run_bin, small(12 * n_req))
         gbs = BYTES_PER_REQUEST * n_req / (ms * 1e-3) / 1e9
@@ -566,7 +583,11 @@ def run_ours(args, rank, world, local_rank):
                         ("cfg3", dict(name="cfg3", trace=cfg3_trace)),
                         ("cfg3code", dict(name="cfg3code")),
                         ("cfg5", dict(name="cfg5")),
-                        ("cfg2_x256_general", dict(name="cfg2", S=256, general=True, with_bin=False,
+                        ("cfg2_x256", dict(name="cfg2", S=256, with_bin=False,
+                                           trace=trace if wl.name in ("cfg2", "cfg4") else None)),
+                        ("cfg2_x256_one_row_general", dict(name="cfg2", S=256, general="one", with_bin=False,
+                                                           trace=trace if wl.name in ("cfg2", "cfg4") else None)),
+                        ("cfg2_x256_general", dict(name="cfg2", S=256, general="all", with_bin=False,
                                                    trace=trace if wl.name in ("cfg2", "cfg4") else None))):
             pc[key] = guarded(measure_config, dyn, gen, dev, sampler, peaks, flush, **kw)
         roofline["per_config"] = pc
@@ -810,7 +831,9 @@ def run_only(args, local_rank):
     flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev)
     per_config = {"cfg1": dict(name="cfg1"), "cfg1_x4096": dict(name="cfg1", S=4096, with_bin=False), "cfg2": dict(name="cfg2"),
                   "cfg3": dict(name="cfg3"), "cfg3code": dict(name="cfg3code"), "cfg5": dict(name="cfg5"),
-                  "cfg2_x256_general": dict(name="cfg2", S=256, general=True, with_bin=False)}
+                  "cfg2_x256": dict(name="cfg2", S=256, with_bin=False),
+                  "cfg2_x256_one_row_general": dict(name="cfg2", S=256, general="one", with_bin=False),
+                  "cfg2_x256_general": dict(name="cfg2", S=256, general="all", with_bin=False)}
     res = {"peaks": {k: v for k, v in peaks.items() if k != "sink"}}
     for key in args.only.split(","):
         if key in per_config:

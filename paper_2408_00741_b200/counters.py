@@ -7,7 +7,7 @@ once any of those sources has changed, so that a report never shows counters of 
 exists.
 
 Recording (after a profiler run that wrote a CSV with the metrics smsp__inst_executed.sum,
-dram__bytes_read.sum and dram__bytes_write.sum of one launch):
+l1tex__data_pipe_lsu_wavefronts_mem_shared.sum, dram__bytes_read.sum and dram__bytes_write.sum of one launch):
 
     python -m paper_2408_00741_b200.counters record --kernel eval_select_kernel --workload cfg4 \
         --csv capture.csv --units 64 --evals 1698693120 --command "<the profiler command>"
@@ -86,12 +86,15 @@ def record(kernel: str, workload: str, csv_path: str, units: float, evals: float
         "sources_sha256_16": source_hash(kernel),
         "units": units, "evals": evals,
         "warp_instructions": m.get("smsp__inst_executed.sum"),
+        "shared_wavefronts": m.get("l1tex__data_pipe_lsu_wavefronts_mem_shared.sum"),
         "dram_bytes_read": m.get("dram__bytes_read.sum"),
         "dram_bytes_written": m.get("dram__bytes_write.sum"),
         "command": command,
     }
     if rec["warp_instructions"] is not None:
         rec["warp_inst_per_32_evals"] = rec["warp_instructions"] * 32.0 / evals
+    if rec["shared_wavefronts"] is not None:
+        rec["shared_wavefronts_per_32_evals"] = rec["shared_wavefronts"] * 32.0 / evals
     if rec["dram_bytes_read"] is not None and rec["dram_bytes_written"] is not None:
         rec["dram_bytes_per_unit"] = (rec["dram_bytes_read"] + rec["dram_bytes_written"]) / units
     allrec = _load()

@@ -99,24 +99,39 @@ __global__ void resolve_kernel(const ResolveParams rp, float4 *__restrict__ rows
         }
         rows2[(size_t(c) * P + p) * RS + m] = line;
         if (m == 0) {
-            // Load threshold of the pair: if TBT never decreases along the row, "TBT <= slo and u <= 1"
-            // holds exactly for x in [0, xlim].  NaN marks a row without that property.
+            // Load threshold of the pair.  TBT is piecewise linear along the row, so {x : TBT(x) <= slo} is a
+            // union of intervals; when it is empty or one interval that starts at x = 0, "TBT <= slo and
+            // u <= 1" holds exactly for x in [0, xlim] and the sweep tests the load against a threshold.
+            // That is the case whenever TBT, walking up the row, never comes back to or below the SLO after
+            // having exceeded it (a row that rises with load always qualifies; so does a row with dips that
+            // do not reach the SLO again).  NaN marks a row without that property: its candidates interpolate
+            // TBT one by one.
             const double slo_c = double(rp.slo_tbt[c]);
             double vlim = -1.0;
-            bool monotone = true;
+            bool single = true;                  // the feasible set is empty or [0, xlim]
+            bool closed = false;                 // an infeasible position has been passed
             double prev = lerp64(tb0[0], tb1[0], w);
-            double xlim = prev <= slo_c ? 0.0 : -1.0;
+            double xlim = -1.0;
+            if (prev <= slo_c) xlim = 0.0;
+            else closed = true;
             for (int k = 1; k < M; ++k) {
                 const double cur = lerp64(tb0[k], tb1[k], w);
-                if (!(cur >= prev)) monotone = false;
-                if (cur <= slo_c) xlim = double(k);
-                else if (prev <= slo_c) xlim = double(k - 1) + (slo_c - prev) / (cur - prev);
+                if (cur <= slo_c) {
+                    if (closed || !(prev <= slo_c)) single = false;      // feasible again after an infeasible stretch
+                    xlim = double(k);
+                } else {
+                    if (prev <= slo_c && !closed) xlim = double(k - 1) + (slo_c - prev) / (cur - prev);
+                    closed = true;
+                    if (!(cur > slo_c)) single = false;                  // NaN entry: no threshold
+                }
                 prev = cur;
             }
+            if (!pair_ok) single = true;         // never feasible: the empty set
+            if (!single) xlim = -1.0;            // the threshold path skips this row; the general path serves it
             if (pair_ok && xlim >= 0.0) vlim = xlim / double(M);
             // x = u*(M-1) is formed as sat(L/n * ic) * M, so that saturation at 1 means x = M
             pairc[size_t(c) * P + p] = make_float2(pair_ok ? float(double(M - 1) / (double(M) * cap)) : 0.f,
-                                                   monotone ? float(vlim) : __int_as_float(0x7fc00000));
+                                                   single ? float(vlim) : __int_as_float(0x7fc00000));
             // threshold path: table position per unit of per-instance load (twice: the sweep uses it as a
             // packed pair) and the largest per-instance load within the SLO and the capacity
             const float icm = pair_ok ? float(double(M - 1) / cap) : 0.f;

@@ -10,9 +10,10 @@
 //   * within one (tile, n) chain the instance count is fixed, so the running minimum is kept on the
 //     energy of ONE instance and multiplied by n once per chain after the pair loop (rounding is
 //     monotone, so the minimum of the products is the product of the minimum, bit for bit);
-//   * when TBT never decreases with load in any table row (the resolve step checks), "TBT <= SLO and
-//     u <= 1" is a threshold on the per-instance load l = L/n (the largest load an instance sustains
-//     within the SLO, cf. ML in Sec. 4.2): one compare, no TBT interpolation.  The energy of the
+//   * for a table row whose TBT, once above the SLO, never returns to it as the load grows (the resolve
+//     step checks each row; every row that rises with load qualifies), "TBT <= SLO and u <= 1" is a
+//     threshold on the per-instance load l = L/n (the largest load an instance sustains within the SLO,
+//     cf. ML in Sec. 4.2): one compare, no TBT interpolation.  The energy of the
 //     segment is stored as a line in l (intercept, slope), so one FMA on l gives it and no fraction is
 //     formed.  The segment number is floor(l*icm), taken from a fused multiply-add with 2^23 rounded
 //     toward zero (the low mantissa bits are the integer; no float-to-int conversion); a second fused
@@ -22,8 +23,13 @@
 //     two-wide fp32 instructions of sm_100.  Per candidate that leaves: compare, 2 x half a packed
 //     FMA, lookup, FMA, predicated min.  Infeasible candidates skip the lookup (same predicate), so
 //     no clamp of the table position is needed;
-//   * otherwise the general path interpolates TBT and energy from the segment's left knot for every
-//     candidate (16-byte lookups, saturating multiply as clamp, sentinel entries for u > 1);
+//   * a row without that property (a measured profile with a dip at the SLO) takes the general path: TBT
+//     and energy are interpolated from the segment's left knot for every candidate (16-byte lookups,
+//     saturating multiply as clamp, sentinel entries for u > 1).  The choice is made per ROW: with few
+//     such rows the threshold loop runs over all pairs (a row without a threshold has the limit -1 there
+//     and accepts nothing) and a second loop serves only those rows, from the tables in global memory;
+//     when more than a quarter of the rows lack a threshold, all rows take the general path on staged
+//     tables;
 //   * only the running minimum is kept; the pair that attained it is recovered once per tile by
 //     re-evaluating that instance count for 32 pairs at a time with bit-identical arithmetic.
 // The resolved tables of all classes are staged in shared memory once per CTA when they fit; larger
@@ -89,12 +95,47 @@ __device__ __forceinline__ void stage(const SweepArgs &a, int from, int to) {
     __syncthreads();
 }
 
-// true when every pair row has a load threshold (vlim is NaN for a row whose TBT decreases somewhere)
-__device__ __forceinline__ bool all_rows_monotone(const SweepArgs &a) {
-    const float2 *pc = reinterpret_cast<const float2 *>(a.ws + a.off_pairc);
+// number of pair rows among [first, first + n) without a load threshold (the resolve step stores NaN as
+// their vlim); the same value in every thread of the CTA
+__device__ __forceinline__ int rows_without_threshold(const SweepArgs &a, int first, int n) {
+    __shared__ int s_bad;
+    if (threadIdx.x == 0) s_bad = 0;
+    __syncthreads();
+    const float2 *pc = reinterpret_cast<const float2 *>(a.ws + a.off_pairc) + first;
     int bad = 0;
-    for (int i = threadIdx.x; i < a.C * a.P; i += blockDim.x) bad |= isnan(__ldg(pc + i).y) ? 1 : 0;
-    return __syncthreads_or(bad) == 0;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) bad += isnan(__ldg(pc + i).y) ? 1 : 0;
+    if (bad) atomicAdd(&s_bad, bad);
+    __syncthreads();
+    return s_bad;
+}
+
+// what the general-path evaluation of one class's rows needs, formed at the point of use from values the
+// compiler cannot trace (so that none of it is kept in registers across the threshold loop)
+struct MixedRows {
+    const float2 *flags;     // pairc of the class: {ic, vlim}; vlim is NaN for a row without a load threshold
+    uint32_t rows;           // byte offset of the class's general-path rows in the scratch block
+    int P, RS;
+    float Mf, slo;
+    Consts2 k2;
+};
+__device__ __forceinline__ int opaque(int v) {
+    asm volatile("mov.b32 %0, %0;" : "+r"(v));
+    return v;
+}
+__device__ __forceinline__ MixedRows mixed_rows(const SweepArgs &a, int c) {
+    MixedRows g;
+    const int co = opaque(c), M = opaque(a.M);
+    g.P = opaque(a.P);
+    g.RS = M + 1;
+    g.Mf = float(M);
+    g.flags = reinterpret_cast<const float2 *>(a.ws + opaque(a.off_pairc)) + co * g.P;
+    g.rows = uint32_t(opaque(a.off_rows)) + uint32_t(co * g.P * g.RS) * 16u;
+    g.slo = __ldg(reinterpret_cast<const float *>(a.ws + opaque(a.off_slo)) + co);
+    g.k2.M = make_float2(g.Mf, g.Mf);
+    g.k2.negM = make_float2(-g.Mf, -g.Mf);
+    g.k2.two23 = make_float2(kTwo23, kTwo23);
+    g.k2.neg23 = make_float2(-kTwo23, -kTwo23);
+    return g;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -102,8 +143,10 @@ __device__ __forceinline__ bool all_rows_monotone(const SweepArgs &a) {
 //   NPL  instance counts per lane (Nmax <= 32*NPL)
 //   TT   tiles (rows of the same class) a warp evaluates per pass over the pairs
 //   CLS  the CTA serves one class (blockIdx.y) and `tb` points at that class's tables alone
+//   MIXED (threshold path only) some rows have no load threshold: a second loop and the pair recovery
+//        evaluate those rows on the general path from the tables in global memory
 // ---------------------------------------------------------------------------------------------
-template <int NPL, int TT, bool BUDGET, bool SMEM, bool FAST, bool FULL, bool CLS = false>
+template <int NPL, int TT, bool BUDGET, bool SMEM, bool FAST, bool FULL, bool CLS = false, bool MIXED = false>
 __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, int32_t *__restrict__ best_idx,
                                            float *__restrict__ best_E) {
     const int lane = threadIdx.x & 31;
@@ -137,7 +180,7 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
     for (int k = 0; k < NPL; ++k) {
         const int n = nl + 1 + LN * k;
         const bool valid = n <= a.Nmax;
-        keep[k] = FAST || valid;
+        keep[k] = (FAST && !MIXED) || valid;
         nf[k] = float(n);
         rn[k] = valid ? 1.0f / float(n) : (FAST ? CUDART_INF_F : 0.f);
         pmax[k] = P;
@@ -199,6 +242,15 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
         }
     }
     const uint32_t rc_row = (one_round && nl < P) ? crow_lane : crow;
+    // Rows of this class without a load threshold: their general-path tables are read from global memory.
+    // Only this flag (and the class number) stays live across the pair loop; whatever else those rows need
+    // is formed where it is used, behind opaque moves, so that the threshold loop keeps its registers.
+    bool class_mixed = false;
+    if (MIXED) {
+        const float2 *flags = reinterpret_cast<const float2 *>(ws + a.off_pairc) + c * P;
+        for (int p0 = 0; p0 < P; p0 += 32)
+            class_mixed |= __any_sync(kFull, p0 + lane < P && isnan(__ldg(flags + p0 + lane).y));
+    }
     const int sh_n = FULL ? 5 : a.ln_log2;           // n - 1 = (chain number << sh_n) + lane number
     const int tpp = TT * TG;                         // tiles of a pass
     const float *lp = a.load + ((r_begin + g * TT) * C + c);          // load of the group's first tile; tiles are C floats apart
@@ -264,6 +316,24 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
                                       !BUDGET || p < pmax[(q + 1) % NPL], best[q], best[q + 1]);
             }
         }
+        if (MIXED && class_mixed) {
+            // the rows without a threshold, one by one (warp-uniform), on the general path
+            const MixedRows g = mixed_rows(a, c);
+            for (int p0 = 0; p0 < g.P; p0 += 32) {
+                unsigned todo = __ballot_sync(kFull, p0 + lane < g.P && isnan(__ldg(g.flags + p0 + lane).y));
+                while (todo) {
+                    const int p = p0 + __ffs(todo) - 1;
+                    todo &= todo - 1;
+                    const float ic = __ldg(g.flags + p).x;
+                    const uint32_t base = g.rows + uint32_t(p * g.RS) * 16u - kTwo23Bits * 16u;
+#pragma unroll
+                    for (int q = 0; q < NCH; q += 2)
+                        general_two<false>(ws, base, DYN_LN(q), DYN_LN(q + 1), ic, g.slo, g.k2,
+                                           !BUDGET || p < pmax[q % NPL], !BUDGET || p < pmax[(q + 1) % NPL],
+                                           best[q], best[q + 1]);
+                }
+            }
+        }
         // per tile: warp argmin on (pool energy, n), then the pair; lane t keeps the result of tile t
         int32_t my_idx = -1;
         float my_E = CUDART_INF_F;
@@ -305,6 +375,13 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
                 bool ok;
                 if (FAST) fast_one<SMEM>(ws, rc_row, lnm, rc_ic, rc_lim, e, ok);
                 else general_one<SMEM>(ws, rc_row - kTwo23Bits * 16u, lnm, rc_ic, rc_lim, Mf, e, ok);
+                if (MIXED && class_mixed && nl < P) {                // a lane whose row has no threshold: general path
+                    const MixedRows g = mixed_rows(a, c);
+                    const float2 gp = __ldg(g.flags + nl);
+                    if (isnan(gp.y))
+                        general_one<false>(ws, g.rows + uint32_t(nl * g.RS) * 16u - kTwo23Bits * 16u, lnm, gp.x, g.slo,
+                                           g.Mf, e, ok);
+                }
                 pstar = __ffs((__ballot_sync(kFull, ok && (fmaf(e, nfm, 0.f) == Emin)) >> gsh) & lowmask) - 1;
             } else {
                 int pm = P;
@@ -319,7 +396,16 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
                     if (pstar < 0 && p0 + nl < pm) {
                         float e;
                         bool ok;
-                        if (FAST) {
+                        float2 gp = make_float2(0.f, 0.f);
+                        MixedRows g;
+                        if (MIXED && class_mixed) {
+                            g = mixed_rows(a, c);
+                            gp = __ldg(g.flags + p0 + nl);
+                        }
+                        if (MIXED && class_mixed && isnan(gp.y)) {
+                            general_one<false>(ws, g.rows + uint32_t((p0 + nl) * g.RS) * 16u - kTwo23Bits * 16u, lnm, gp.x,
+                                               g.slo, g.Mf, e, ok);
+                        } else if (FAST) {
                             const float4 pc = load16<SMEM>(ws, cpair_lane + uint32_t(p0) * 16u);
                             fast_one<SMEM>(ws, crow_lane + uint32_t(p0) * pstep, lnm, pc.x, pc.z, e, ok);
                         } else {
@@ -352,12 +438,14 @@ __global__ void __launch_bounds__(kThreads, (NPL * TT <= 4 ? DYN_SW_MINB4 : (NPL
 eval_select_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__restrict__ best_E) {
     Tables tb;
     tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.pair2 = a.off_pair2; tb.rows2 = a.off_rows2;
-    if (all_rows_monotone(a)) {                      // uniform over the grid: every CTA reads the same flags
+    const int bad = rows_without_threshold(a, 0, a.C * a.P);     // uniform over the grid: every CTA reads the same flags
+    if (bad * 4 <= a.C * a.P) {
         if (SMEM) {
             stage(a, a.off_pair2, a.off_end);        // pair2 | rows2
             tb.pair2 = 0; tb.rows2 = a.off_rows2 - a.off_pair2;
         }
-        sweep_body<NPL, TT, BUDGET, SMEM, true, FULL>(a, tb, best_idx, best_E);
+        if (bad == 0) sweep_body<NPL, TT, BUDGET, SMEM, true, FULL>(a, tb, best_idx, best_E);
+        else sweep_body<NPL, TT, BUDGET, SMEM, true, FULL, false, true>(a, tb, best_idx, best_E);
     } else {
         if (SMEM) {
             stage(a, a.off_rows, a.off_pair2);       // rows | pairc | slo
@@ -369,13 +457,15 @@ eval_select_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__r
 
 // Tables too large to stage for all classes at once (fine frequency grids): a CTA serves ONE class
 // (blockIdx.y) and stages that class's threshold tables, pair2_c | rows2_c, in shared memory; one CTA
-// of 16 warps per SM.  When some row is not monotone the general path reads the full tables through L1.
+// of 16 warps per SM.  The rows of the class that have no load threshold are served from the tables in global
+// memory; when they are more than a quarter of the class's rows the general path serves all of them.
 template <int NPL, int TT, bool BUDGET>
 __global__ void __launch_bounds__(512, 1)
 eval_select_class_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__restrict__ best_E) {
     Tables tb;
     tb.rows = tb.pairc = tb.slo = tb.pair2 = tb.rows2 = 0;
-    if (all_rows_monotone(a)) {
+    const int bad = rows_without_threshold(a, int(blockIdx.y) * a.P, a.P);
+    if (bad * 4 <= a.P) {
         extern __shared__ float4 smem[];
         const int c = blockIdx.y;
         const int pair_bytes = a.P * 16, rows2_bytes = a.P * (a.M + 1) * 8;
@@ -386,7 +476,8 @@ eval_select_class_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, floa
         for (int i = threadIdx.x; i < nr16; i += blockDim.x) smem[np16 + i] = src_r[i];
         __syncthreads();
         tb.pair2 = 0; tb.rows2 = uint32_t(pair_bytes);
-        sweep_body<NPL, TT, BUDGET, true, true, true, true>(a, tb, best_idx, best_E);
+        if (bad == 0) sweep_body<NPL, TT, BUDGET, true, true, true, true>(a, tb, best_idx, best_E);
+        else sweep_body<NPL, TT, BUDGET, true, true, true, true, true>(a, tb, best_idx, best_E);
     } else {
         const int c = blockIdx.y;
         tb.rows = a.off_rows + uint32_t(c) * uint32_t(a.P * (a.M + 1)) * 16u;
@@ -400,9 +491,10 @@ eval_select_class_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, floa
 // evaluate only: E[tile][j], j = (n-1)*P + p.  A warp takes one tile and 32 consecutive pairs: lanes
 // are pairs (their constants stay in registers), the loop runs over n two at a time, and each pass
 // writes two coalesced runs of 32 energies.  Threshold or general path as in the fused kernel, with
-// the same arithmetic per candidate.
+// the same arithmetic per candidate; MIXED: a lane whose row has no load threshold evaluates it on the
+// general path from the tables in global memory.
 // ---------------------------------------------------------------------------------------------
-template <bool BUDGET, bool SMEM, bool FAST>
+template <bool BUDGET, bool SMEM, bool FAST, bool MIXED = false>
 __device__ __forceinline__ void configs_body(const SweepArgs &a, const Tables tb, const float2 *s_n, const int64_t units_total,
                                              float *__restrict__ E_out) {
     const int lane = threadIdx.x & 31;
@@ -435,6 +527,14 @@ __device__ __forceinline__ void configs_body(const SweepArgs &a, const Tables tb
             ic = load8<SMEM>(ws, origin + tb.pairc + uint32_t(c * P + pp) * 8u).x;
             lim = slo_c;
         }
+        bool lane_general = false;
+        float gic = 0.f;
+        if (MIXED) {
+            const float2 gp = __ldg(reinterpret_cast<const float2 *>(ws + a.off_pairc) + (c * P + pp));
+            lane_general = isnan(gp.y);
+            gic = gp.x;
+        }
+        const uint32_t grow = uint32_t(a.off_rows) + uint32_t((c * P + pp) * RS) * 16u - kTwo23Bits * 16u;
         int nlim = Nmax;                              // Eq. 1 GPU budget: n * TP <= budget
         if (BUDGET) {
             const int64_t q = int64_t(a.budget) / a.tp[pp / a.F];
@@ -457,6 +557,14 @@ __device__ __forceinline__ void configs_body(const SweepArgs &a, const Tables tb
                 float EA, EB;
                 fast_two_energy(mul2(L2, rn2), icm2, off2, two23_2, eight2, limA, limB, half_of(nf2, 0), half_of(nf2, 1),
                                 EA, EB);
+                if (MIXED && lane_general) {
+                    float eA, eB;
+                    bool okA, okB;
+                    general_one<false>(ws, grow, L * half_of(rn2, 0), gic, slo_c, Mf, eA, okA);
+                    general_one<false>(ws, grow, L * half_of(rn2, 1), gic, slo_c, Mf, eB, okB);
+                    EA = (okA && (!BUDGET || 2 * h + 1 <= nlim)) ? eA * half_of(nf2, 0) : CUDART_INF_F;
+                    EB = (okB && (!BUDGET || 2 * h + 2 <= nlim)) ? eB * half_of(nf2, 1) : CUDART_INF_F;
+                }
                 if (active) {
                     __stcs(out, EA);
                     __stcs(out + P, EB);
@@ -467,6 +575,10 @@ __device__ __forceinline__ void configs_body(const SweepArgs &a, const Tables tb
                 float e;
                 bool ok;
                 fast_one<SMEM>(ws, row, L * nn.x, ic, (!BUDGET || Nmax <= nlim) ? lim : -1.f, e, ok);
+                if (MIXED && lane_general) {
+                    general_one<false>(ws, grow, L * nn.x, gic, slo_c, Mf, e, ok);
+                    ok = ok && (!BUDGET || Nmax <= nlim);
+                }
                 if (active) __stcs(out, ok ? e * nn.z : CUDART_INF_F);
             }
         } else
@@ -475,7 +587,10 @@ __device__ __forceinline__ void configs_body(const SweepArgs &a, const Tables tb
             const float lnA = L * nn.x, lnB = L * nn.y;
             float eA, eB;
             bool okA, okB;
-            if (FAST) {
+            if (MIXED && lane_general) {
+                general_one<false>(ws, grow, lnA, gic, slo_c, Mf, eA, okA);
+                general_one<false>(ws, grow, lnB, gic, slo_c, Mf, eB, okB);
+            } else if (FAST) {
                 fast_one<SMEM>(ws, row, lnA, ic, lim, eA, okA);
                 fast_one<SMEM>(ws, row, lnB, ic, lim, eB, okB);
             } else {
@@ -506,12 +621,14 @@ eval_configs_kernel(const SweepArgs a, const int64_t units_total, float *__restr
     }
     Tables tb;
     tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.pair2 = a.off_pair2; tb.rows2 = a.off_rows2;
-    if (all_rows_monotone(a)) {                      // load-threshold path: 8-byte lookups (also a barrier for s_n)
+    const int bad = rows_without_threshold(a, 0, a.C * a.P);     // (also a barrier for s_n)
+    if (bad * 4 <= a.C * a.P) {                      // load-threshold path: 8-byte lookups
         if (SMEM) {
             stage(a, a.off_pair2, a.off_end);
             tb.pair2 = 0; tb.rows2 = a.off_rows2 - a.off_pair2;
         }
-        configs_body<BUDGET, SMEM, true>(a, tb, s_n, units_total, E_out);
+        if (bad == 0) configs_body<BUDGET, SMEM, true>(a, tb, s_n, units_total, E_out);
+        else configs_body<BUDGET, SMEM, true, true>(a, tb, s_n, units_total, E_out);
     } else {
         if (SMEM) {
             stage(a, a.off_rows, a.off_pair2);

@@ -108,3 +108,38 @@ def random_tables(seed, monotone_tbt, large=False):
         cand = np.linspace(800, 1980, 40).astype(np.float32)
     sp = gen.make_space(cand, 40, 60.0, slo_ttft=0.8, slo_tbt=0.1)
     return prof, sp
+
+
+def tables_with_few_rows_without_threshold(seed, large=False, n_bad=5):
+    """Free-form tables whose TBT rises with load, except: (i) every third row dips once but stays on its side
+    of the SLO (the feasible loads are still one interval from zero: such a row keeps its load threshold), and
+    (ii) `n_bad` rows, all in classes 0, 4 and 8, leave the SLO and come back below it at a higher load (two feasible
+    intervals: only per-candidate interpolation of TBT decides these).  Returns profile, space and the (c, t, r)
+    triples of the rows of kind (ii)."""
+    rng = np.random.default_rng(seed)
+    prof, sp = random_tables(seed, True, large)
+    tbt = prof.tbt.astype(np.float64).copy()
+    Cn, T, R, M = tbt.shape
+    slo = 0.1
+    flat = tbt.reshape(-1, M)
+    for i in range(0, flat.shape[0], 3):                 # (i) a dip that does not cross the SLO
+        row = flat[i]
+        k = int(rng.integers(1, M - 1))
+        lo = row[k - 1]
+        side = (row[k] <= slo) == (lo <= slo)
+        if side:                                          # knots k-1 and k on the same side: dip below k-1, same side
+            row[k] = lo - 0.3 * (lo - (0.0 if lo <= slo else slo)) * rng.random() - 1e-4 if lo <= slo else \
+                max(slo + 1e-4, lo - 0.5 * (lo - slo) * rng.random())
+    bad = []
+    for c in (0, 4, 8):
+        for _ in range((n_bad + 2) // 3):
+            t, r = int(rng.integers(T)), int(rng.integers(R))
+            row = tbt[c, t, r]
+            ks = sorted(rng.choice(np.arange(1, M), size=2, replace=False).tolist())
+            row[:] = 0.05 + 0.04 * np.sort(rng.random(M))        # all below the SLO ...
+            row[ks[0]] = slo + 0.01 + 0.02 * rng.random()        # ... except one knot above it
+            if ks[1] - ks[0] > 1:
+                row[ks[0] + 1:ks[1]] = slo + 0.03                # or a stretch of them
+            bad.append((c, t, r))
+    prof = gen.Profile(prof.tp, prof.f_grid_mhz, prof.ttft, prof.cap, tbt.astype(np.float32), prof.pow)
+    return prof, sp, bad

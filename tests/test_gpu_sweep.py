@@ -6,7 +6,8 @@ import torch
 
 import gen
 import oracle
-from parity import REL_TOL, check_selection, gpu_eval_select, gpu_profile_space, out_to_host, random_tables
+from parity import (REL_TOL, check_selection, gpu_eval_select, gpu_profile_space, out_to_host, random_tables,
+                    tables_with_few_rows_without_threshold)
 
 pytestmark = pytest.mark.gpu
 
@@ -145,6 +146,48 @@ def test_eval_select_free_form_tables(dyn, monotone, large):
     _check_totals(sp, prof, out, ref, fixed, J)
     feas = (ref["best_idx"] >= 0).mean()
     assert 0.2 < feas <= 1.0
+
+
+@pytest.mark.parametrize("budget", [0, 60], ids=["no-budget", "gpu-budget"])
+@pytest.mark.parametrize("large", [False, True], ids=["tables-in-shared-memory", "tables-per-class"])
+def test_few_rows_without_a_load_threshold(dyn, large, budget):
+    """The evaluation path is chosen per table row: a profile whose TBT rows rise with load except for a few that
+    cross the SLO twice keeps the load-threshold path for all other rows (dips that stay on one side of the SLO
+    included) and interpolates TBT per candidate only for those few.  Fused kernel and evaluate-only kernel."""
+    prof, sp, bad = tables_with_few_rows_without_threshold(23, large)
+    assert len(bad) >= 3
+    sp = gen.make_space(sp.f_cand_mhz, sp.n_max, sp.window_s, slo_ttft=0.8, slo_tbt=0.1, gpu_budget=budget)
+    load = gen.random_loads((2, 29 if not large else 7, 9), seed=6, mean=6.0)
+    J = sp.n_max * prof.T * sp.F
+    ref = oracle.eval_select(prof, sp, load)
+    out = out_to_host(gpu_eval_select(dyn, prof, sp, load))
+    fixed, n_ex = check_selection(prof, sp, load, out["best_idx"], out["best_E"], ref)
+    _check_totals(sp, prof, out, ref, fixed, J)
+    # the rows that need the general path do get chosen somewhere (otherwise the case tests nothing)
+    jbest = ref["best_idx"]
+    tq = (jbest % (prof.T * sp.F))[jbest >= 0]
+    cls = np.broadcast_to(np.arange(9), jbest.shape)[jbest >= 0]
+    chosen_t = set(zip(cls.tolist(), (tq // sp.F).tolist()))
+    assert any((c, t) in chosen_t for c, t, _ in bad)
+    # evaluate-only kernel on the same tables
+    S, W, Cn = load.shape
+    W2 = min(W, 3)
+    p, s = gpu_profile_space(dyn, prof, sp)
+    d_load = torch.from_numpy(load[:, :W2].copy()).cuda()
+    d_E = torch.empty((S, W2, Cn, J), dtype=torch.float32, device="cuda")
+    ws = torch.empty(dyn.dyn_workspace_bytes(p, s, S, W2), dtype=torch.uint8, device="cuda")
+    dyn.dyn_eval_configs(p, s, d_load, d_E, ws)
+    torch.cuda.synchronize()
+    E = d_E.cpu().numpy()
+    refE = oracle.eval_configs(prof, sp, load[:, :W2])
+    fin_r, fin_g = np.isfinite(refE), np.isfinite(E)
+    both = fin_r & fin_g
+    assert (np.abs(E[both] - refE[both]) / np.abs(refE[both])).max() <= REL_TOL
+    diff = np.argwhere(fin_r != fin_g)
+    assert len(diff) <= 1e-4 * E.size + 2
+    for s_, w_, c_, j_ in diff:
+        _, tb, _, u, _ = oracle.eval_tile(prof, sp, int(c_), float(load[s_, w_, c_]), details=True)
+        assert min(abs(tb[j_] - 0.1) / 0.1, abs(u[j_] - 1.0)) < REL_TOL
 
 
 def test_limits_of_the_candidate_space(dyn):
