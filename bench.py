@@ -267,7 +267,11 @@ def timed_kernel(dyn, call, flush=None, min_s=0.5, per_round=25, max_rounds=400)
         if time.time() - t0 >= min_s:
             break
     t1 = time.time()
+    timed_kernel.last_median_ms = float(np.median(ms))
     return float(np.mean(ms)), float(np.min(ms)), len(ms), t0, t1
+
+
+timed_kernel.last_median_ms = None
 
 
 def measure_peaks(dyn, dev, sampler):
@@ -277,10 +281,16 @@ def measure_peaks(dyn, dev, sampler):
     work = []
     ms, ms_min, n, t0, t1 = timed_kernel(dyn, lambda: work.append(dyn.dyn_probe_fma(2000, sink)))
     tflops = work[0] / (ms * 1e-3) / 1e12
+    # what a pair of events shows around a kernel that does next to nothing (the same probe, one round of 64
+    # multiply-adds per thread): the part of every event-timed duration that is not the kernel's work
+    fl_ms, fl_min, _, _, _ = timed_kernel(dyn, lambda: dyn.dyn_probe_fma(1, sink), None, min_s=0.2)
+    floor_med = timed_kernel.last_median_ms
     hbm, hbm_src = _hbm_peak()
     return {"fp32_tflops": tflops, "fp32_probe_ms": ms, "fp32_probe_launches": n,
             "fp32_nominal_tflops": SM_COUNT * FP32_LANES * 2 * SM_MAX_MHZ * 1e6 / 1e12,
             "issue_warp_inst_per_s": tflops * 1e12 / 64.0,
+            "event_floor_us": {"mean": fl_ms * 1e3, "median": floor_med * 1e3, "min": fl_min * 1e3,
+                               "what": "duration the events report around an (almost) empty kernel of 1184 CTAs"},
             "clocks": sampler.window(t0, t1) if sampler else None,
             "hbm_gbs": hbm, "hbm_source": hbm_src, "sink": sink}
 
@@ -373,8 +383,13 @@ def measure_config(dyn, gen, dev, sampler, peaks, flush, name, S=1, general=None
     entry = {"workload": name, "S": S, "W": W, "C": Cn, "J": J, "path": f"per-candidate TBT interpolation on {n_general} of {tbt[..., 0].size} table rows" if general else "threshold"}
     if with_bin:
         ms, ms_min, n, t0, t1 = timed_kernel(dyn, run_bin, small(12 * n_req))
+        ms_med = timed_kernel.last_median_ms
         gbs = BYTES_PER_REQUEST * n_req / (ms * 1e-3) / 1e9
+        floor_ms = peaks["event_floor_us"]["median"] * 1e-3
         entry["bin"] = {"kernel": "bin_trace_kernel", "requests": int(n_req), "kernel_ms": ms, "kernel_ms_min": ms_min,
+                        "kernel_ms_median": ms_med,
+                        "frac_median_minus_event_floor": (BYTES_PER_REQUEST * n_req / (max(ms_med - floor_ms, 1e-9) * 1e-3) / 1e9
+                                                          / peaks["hbm_gbs"]),
                         "launches": n, "requests_per_s": n_req / (ms * 1e-3), "achieved_gbs": gbs,
                         "frac": gbs / peaks["hbm_gbs"], "l2": "flushed" if small(12 * n_req) is not None else "inputs_larger_than_L2",
                         "clocks": sampler.window(t0, t1) if sampler else None}
@@ -593,7 +608,7 @@ def run_ours(args, rank, world, local_rank):
         roofline["per_config"] = pc
         if isinstance(pc.get("cfg3"), dict) and "bin" in pc["cfg3"]:
             result["trace_requests_per_s"] = pc["cfg3"]["bin"]["requests_per_s"]
-        result["bin_trace"] = guarded(measure_bin, dyn, gen, dev, cfg3_trace)
+        result["bin_trace"] = guarded(measure_bin, dyn, gen, dev, cfg3_trace, peaks=peaks)
         del cfg3_trace
         result["materialised"] = guarded(measure_materialised, dyn, gen, dev)
         result["hierarchical"] = guarded(measure_hier, dyn, gen, dev, peaks=peaks)
@@ -612,7 +627,7 @@ def run_ours(args, rank, world, local_rank):
         dist.destroy_process_group()
 
 
-def measure_bin(dyn, gen, dev, trace=None):
+def measure_bin(dyn, gen, dev, trace=None, peaks=None):
     """Requests/s of the trace-binning kernel on the 14M-request week trace (168 MB, larger than L2), and
     on the same trace repeated 8 times (1.3 GB) to show what the kernel sustains on a long trace."""
     import torch
@@ -629,9 +644,13 @@ def measure_bin(dyn, gen, dev, trace=None):
         n = int(d[0].numel())
         run = lambda: dyn.dyn_bin_trace(wl.trace.window_ms, W, gen.IN_EDGES, gen.OUT_EDGES, d[0], d[1], d[2], counts, load, dropped)
         ms, ms_min, k, _, _ = timed_kernel(dyn, run, None, min_s=0.3)
+        ms_med = timed_kernel.last_median_ms
         assert int(counts.sum().item()) + int(dropped.item()) == n
         gbs = BYTES_PER_REQUEST * n / (ms * 1e-3) / 1e9
-        r = {"requests": n, "kernel_ms": ms, "kernel_ms_min": ms_min, "launches": k, "requests_per_s": n / (ms * 1e-3),
+        floor_ms = peaks["event_floor_us"]["median"] * 1e-3 if peaks else 0.0
+        less_floor = lambda med: BYTES_PER_REQUEST * n / (max(med - floor_ms, 1e-9) * 1e-3) / 1e9 / peak
+        r = {"requests": n, "kernel_ms": ms, "kernel_ms_min": ms_min, "kernel_ms_median": ms_med, "launches": k,
+             "requests_per_s": n / (ms * 1e-3), "frac_median_minus_event_floor": less_floor(ms_med),
              "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
                           "traffic": None, "peak_source": src}}
         if rep == 1:
@@ -645,7 +664,9 @@ def measure_bin(dyn, gen, dev, trace=None):
             runt = lambda: dyn.dyn_bin_tokens(wl.trace.window_ms, W, gen.IN_EDGES, gen.OUT_EDGES, d[0], d[1], d[2], ti, to, load)
             mst, mst_min, k, _, _ = timed_kernel(dyn, runt, None, min_s=0.3)
             gbt = BYTES_PER_REQUEST * n / (mst * 1e-3) / 1e9
-            out["token_sums"] = {"kernel": "bin_tokens_kernel", "kernel_ms": mst, "kernel_ms_min": mst_min, "launches": k,
+            out["token_sums"] = {"kernel": "bin_tokens_kernel", "kernel_ms": mst, "kernel_ms_min": mst_min,
+                                 "kernel_ms_median": timed_kernel.last_median_ms,
+                                 "frac_median_minus_event_floor": less_floor(timed_kernel.last_median_ms), "launches": k,
                                  "requests_per_s": n / (mst * 1e-3),
                                  "roofline": {"bound": "hbm", "achieved": gbt, "peak": peak, "unit": "GB/s",
                                               "frac": gbt / peak, "traffic": None, "peak_source": src}}
@@ -839,7 +860,7 @@ def run_only(args, local_rank):
         if key in per_config:
             res[key] = measure_config(dyn, gen, dev, sampler, peaks, flush, **per_config[key])
         elif key == "bin_trace":
-            res[key] = measure_bin(dyn, gen, dev)
+            res[key] = measure_bin(dyn, gen, dev, peaks=peaks)
         elif key == "materialised":
             res[key] = measure_materialised(dyn, gen, dev)
         elif key == "hierarchical":

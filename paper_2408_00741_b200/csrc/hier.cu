@@ -1,10 +1,11 @@
 // Hierarchical control [Sec. 4.2]: nodes per pool from the epoch's peak load (scale-out/in), sharding
 // at the highest frequency within those GPUs (shard-up/down), frequency per window (scale-up/down).
 // Same models and the same resolved tables as the joint sweep; each level is a small restricted search.
-// When every TBT row is monotone in load (the resolve step's flags) and the threshold tables fit in shared
-// memory, the sharding and frequency kernels evaluate candidates as the sweep's threshold path does (compare on
-// the per-instance load, 8-byte lookup of the energy line in shared memory); otherwise from the general-path
-// tables through L1.  Both variants are launched; each looks at the flags and only the selected one works.
+// When the threshold tables fit in shared memory, the sharding and frequency kernels stage them and evaluate
+// candidates as the sweep's threshold path does (compare on the per-instance load, 8-byte lookup of the energy
+// line in shared memory); a warp serves one class there, and a class with a table row that has no load
+// threshold (the resolve step's flags) is evaluated from the general-path tables through L1 instead, as is
+// everything when the tables do not fit.
 #include "dyn_internal.cuh"
 #include "eval_dev.cuh"
 
@@ -59,36 +60,33 @@ struct HierArgs {
 };
 
 
-// true when every pair row has a load threshold (vlim is NaN for a row whose TBT decreases somewhere)
-__device__ __forceinline__ bool rows_monotone(const HierArgs &a) {
-    int bad = 0;
-    for (int i = threadIdx.x; i < a.C * a.T * a.F; i += blockDim.x) bad |= isnan(__ldg(a.pairc + i).y) ? 1 : 0;
-    return __syncthreads_or(bad) == 0;
+// true when some pair row of class c has no load threshold (vlim is NaN there); warp-uniform
+__device__ __forceinline__ bool class_without_threshold(const HierArgs &a, int c) {
+    const int P = a.T * a.F, lane = threadIdx.x & 31;
+    bool bad = false;
+    for (int p0 = 0; p0 < P; p0 += 32)
+        bad |= __any_sync(kFull, p0 + lane < P && isnan(__ldg(a.pairc + c * P + p0 + lane).y));
+    return bad;
 }
 
-// FAST kernels do the work iff the tables are monotone (and staged); the others iff not.  Returns false when
-// this kernel has nothing to do; for FAST it also stages pair2 | rows2 into shared memory.
+// FAST kernels stage pair2 | rows2 into shared memory
 template <bool FAST>
-__device__ __forceinline__ bool hier_begin(const HierArgs &a) {
-    const bool mono = rows_monotone(a);
+__device__ __forceinline__ void hier_begin(const HierArgs &a) {
     if (FAST) {
-        if (!mono) return false;
         extern __shared__ float4 smem[];
         const float4 *src = reinterpret_cast<const float4 *>(a.ws + a.off_pair2);
         const int n16 = (a.off_end - a.off_pair2) / 16;
         for (int i = threadIdx.x; i < n16; i += blockDim.x) smem[i] = src[i];
         __syncthreads();
-        return true;
     }
-    return !(a.use_fast && mono);
 }
 
 // pool energy of n instances of pair p (class c) at per-instance load ln; ok = within SLO and capacity
 template <bool FAST>
 __device__ __forceinline__ float hier_eval(const HierArgs &a, uint32_t origin, int c, int p, float ln, float nf, float slo,
-                                           bool &ok) {
+                                           bool general, bool &ok) {
     const int P = a.T * a.F, RS = a.M + 1;
-    if (FAST) {
+    if (FAST && !general) {
         const float4 pc = load16<true>(a.ws, origin + uint32_t(c * P + p) * 16u);
         float e;
         fast_one<true>(a.ws, origin + uint32_t(a.off_rows2 - a.off_pair2) + uint32_t((c * P + p) * RS) * 8u, ln, pc.x, pc.z,
@@ -141,21 +139,68 @@ __global__ void __launch_bounds__(256) hier_nodes_kernel(const HierArgs a) {
     }
 }
 
-// one thread per (s, k2, c): neighbouring threads are neighbouring classes, so the loads coalesce; the
-// node budget cuts the (n, TP) space to a few dozen candidates, walked in index order
+// one thread per (s, k2, c).  Staging variant: lanes are 32 consecutive shard epochs of one class.  With at most
+// four TP degrees the constants of the highest-frequency pairs stay in registers; instance counts are walked two
+// at a time with the sweep's packed evaluation (the two counts are the two chains, the TP degrees the pairs),
+// the running minimum is kept on the energy of one instance and multiplied by n once per count; counts below
+// the smallest one that can carry the load at any degree are skipped; the TP degree of the winning count is found
+// again afterwards with bit-identical arithmetic (lowest degree first).
 template <bool FAST>
-__global__ void __launch_bounds__(256) hier_shard_kernel(const HierArgs a) {
-    if (!hier_begin<FAST>(a)) return;
+__global__ void __launch_bounds__(256, FAST ? 4 : 1) hier_shard_kernel(const HierArgs a) {
+    __shared__ float s_rn[257];                          // 1/n
+    for (int n = threadIdx.x; n <= 256; n += blockDim.x) s_rn[n] = n ? 1.0f / float(n) : 0.f;
+    hier_begin<FAST>(a);
+    if (!FAST) __syncthreads();
     uint32_t origin = table_origin<FAST>();
     asm volatile("" : "+r"(origin) : : "memory");        // table loads stay behind the staging barrier
     uint32_t k2, c;
-    if (!hier_item<FAST>(a, uint32_t(a.K2), k2, c)) return;
+    const bool have = hier_item<FAST>(a, uint32_t(a.K2), k2, c);
+    const bool general = FAST ? class_without_threshold(a, int(c)) : true;   // (c is warp-uniform in the staging variant)
+    if (!have) return;
     const uint32_t x = k2 * a.C + c;
     const int w0 = int(k2) * a.e2, w1 = min(w0 + a.e2, a.W);
     const uint32_t k1 = fastdiv(uint32_t(w0), a.divE1);
     const float slo = a.slo[c];
     const int tpmax = a.tp[a.T - 1];
     const int cap_budget = a.Nmax * tpmax;            // a larger budget changes nothing
+    const bool packed = FAST && !general && a.T <= 4;
+    // constants of the (at most four) highest-frequency pairs
+    uint64_t icm2[4], off2[4];
+    float llim[4], icm[4], inv_llim[4];
+    uint32_t row[4];
+    if (packed) {
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const int tt = t < a.T ? t : 0;
+            const int p = tt * a.F + a.F - 1;
+            const float4 pc = load16<true>(a.ws, origin + uint32_t(int(c) * a.T * a.F + p) * 16u);
+            icm[t] = pc.x;
+            icm2[t] = pack2(pc.x, pc.x);
+            llim[t] = t < a.T ? pc.z : -1.f;
+            inv_llim[t] = llim[t] > 0.f ? 1.0f / llim[t] : (llim[t] == 0.f ? 0.f : CUDART_INF_F);   // limit 0: no pruning
+            row[t] = origin + uint32_t(a.off_rows2 - a.off_pair2) + uint32_t((int(c) * a.T * a.F + p) * (a.M + 1)) * 8u;
+            const float off = row_offset_units(row[t]);
+            off2[t] = pack2(off, off);
+        }
+    }
+    // The energy of one instance never falls below the least knot energy of its row (the rows are piecewise
+    // linear), so a pool of n instances costs at least n * e_floor whatever the load: once that reaches the best
+    // energy found, no larger count can improve on it and the walk over n stops.  (Taken a little low, so that
+    // rounding cannot cut off a candidate.)
+    float e_floor = CUDART_INF_F;
+    if (packed) {
+        for (int t = 0; t < a.T; ++t) {
+            if (!(llim[t] >= 0.f)) continue;
+            for (int m = 0; m < a.M; ++m) {
+                const float2 en = load8<true>(a.ws, row[t] + uint32_t(m) * 8u);
+                const float l0 = float(m) / icm[t], l1 = float(m + 1) / icm[t];
+                e_floor = fminf(e_floor, fminf(fmaf(l0, en.y, en.x), m + 1 < a.M ? fmaf(l1, en.y, en.x) : en.x));
+            }
+        }
+        e_floor *= 0.99999f;
+        if (!(e_floor > 0.f)) e_floor = 0.f;          // no positive floor: no pruning
+    }
+    const uint64_t two23_2 = pack2(kTwo23, kTwo23), eight2 = pack2(units(8u), units(8u));
     for (int64_t s = blockIdx.y; s < a.S; s += gridDim.y) {
         const float *ld = a.load + size_t(s) * size_t(a.W) * a.C + c;
         float PL = 0.f;
@@ -167,44 +212,48 @@ __global__ void __launch_bounds__(256) hier_shard_kernel(const HierArgs a) {
         if (nmax > a.Nmax) nmax = a.Nmax;
         float best = CUDART_INF_F;
         int bnt = -1;
-        if (FAST && a.T <= 4) {
-            // the constants of the (at most four) highest-frequency pairs stay in registers for the whole walk
-            float icm[4], llim[4];
-            uint32_t row[4];
+        if (packed) {
             int nlim[4];
+            float xmin = CUDART_INF_F;                // least n (as a real number) that carries PL at some degree
 #pragma unroll
             for (int t = 0; t < 4; ++t) {
-                const int tt = t < a.T ? t : 0;
-                const int p = tt * a.F + a.F - 1;
-                const float4 pc = load16<true>(a.ws, origin + uint32_t(int(c) * a.T * a.F + p) * 16u);
-                icm[t] = pc.x;
-                llim[t] = t < a.T ? pc.z : -1.f;
-                row[t] = origin + uint32_t(a.off_rows2 - a.off_pair2) + uint32_t((int(c) * a.T * a.F + p) * (a.M + 1)) * 8u;
-                nlim[t] = t < a.T ? budget / a.tp[tt] : 0;  // TP ascending: the limits descend
+                nlim[t] = t < a.T ? budget / a.tp[t < a.T ? t : 0] : 0;     // TP ascending: the limits descend
+                xmin = fminf(xmin, PL * inv_llim[t]);
             }
-            for (int n = 1; n <= nmax; ++n) {
-                const float nf = float(n), ln = PL * (1.0f / nf);
+            // every n below xmin - 1 is infeasible at every degree by a margin of 1/n, far above rounding
+            int n = xmin < 300.f ? max(1, int(xmin) - 1) : nmax + 1;
+            int bn = 0;
+            for (; n <= nmax; n += 2) {
+                if (float(n) * e_floor >= best) break;       // n and every larger count cost at least `best`
+                const float lnA = PL * s_rn[n], lnB = n + 1 <= nmax ? PL * s_rn[n + 1] : CUDART_INF_F;
+                const uint64_t ln2 = pack2(lnA, lnB);
+                float eA = CUDART_INF_F, eB = CUDART_INF_F;
 #pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                    if (n > nlim[t]) break;
+                for (int t = 0; t < 4; ++t)
+                    fast_two(ln2, icm2[t], off2[t], two23_2, eight2, n <= nlim[t] ? llim[t] : -1.f,
+                             n + 1 <= nlim[t] ? llim[t] : -1.f, eA, eB);
+                const float EA = float(n) * eA, EB = float(n + 1) * eB;
+                if (EA < best) { best = EA; bn = n; }         // ascending n: strict compare keeps the lowest
+                if (EB < best) { best = EB; bn = n + 1; }
+            }
+            if (bn > 0) {
+                const float nf = float(bn), ln = PL * s_rn[bn];
+#pragma unroll
+                for (int t = 3; t >= 0; --t) {               // descending, so the lowest matching degree stays
                     float e;
                     bool ok;
-                    fast_one<true>(a.ws, row[t], ln, icm[t], llim[t], e, ok);
-                    const float E = nf * e;
-                    if (ok && E < best) {             // ascending (n, t): strict compare keeps the lowest index
-                        best = E;
-                        bnt = (n - 1) * a.T + t;
-                    }
+                    fast_one<true>(a.ws, row[t], ln, icm[t], bn <= nlim[t] ? llim[t] : -1.f, e, ok);
+                    if (ok && nf * e == best) bnt = (bn - 1) * a.T + t;
                 }
             }
         } else
         for (int n = 1; n <= nmax; ++n) {
-            const float nf = float(n), ln = PL * (1.0f / nf);
+            const float nf = float(n), ln = PL * s_rn[n];
             for (int t = 0; t < a.T; ++t) {
                 if (n * a.tp[t] > budget) break;      // TP ascending
                 const int p = t * a.F + a.F - 1;
                 bool ok;
-                const float E = hier_eval<FAST>(a, origin, int(c), p, ln, nf, slo, ok);
+                const float E = hier_eval<FAST>(a, origin, int(c), p, ln, nf, slo, general, ok);
                 if (ok && E < best) {                 // ascending (n, t): strict compare keeps the lowest index
                     best = E;
                     bnt = (n - 1) * a.T + t;
@@ -215,37 +264,73 @@ __global__ void __launch_bounds__(256) hier_shard_kernel(const HierArgs a) {
     }
 }
 
-// one thread per (s, w, c): the frequency for the sharding of its shard epoch
+// one thread per (s, w, c): the frequency for the sharding of its shard epoch.  Staging variant: lanes are 32
+// consecutive windows of one class; whatever depends on (window, class) only is formed once per thread, the
+// walk over the scenarios keeps the F pairs of (class, TP) as running addresses (16 bytes of constants and one
+// table row apart) and the minimum on the energy of one instance.
 template <bool FAST>
 __global__ void __launch_bounds__(256) hier_freq_kernel(const HierArgs a) {
-    if (!hier_begin<FAST>(a)) return;
+    __shared__ float s_rn[257];                          // 1/n
+    for (int n = threadIdx.x; n <= 256; n += blockDim.x) s_rn[n] = n ? 1.0f / float(n) : 0.f;
+    hier_begin<FAST>(a);
+    if (!FAST) __syncthreads();
     uint32_t origin = table_origin<FAST>();
     asm volatile("" : "+r"(origin) : : "memory");        // table loads stay behind the staging barrier
     uint32_t w, c;
-    if (!hier_item<FAST>(a, uint32_t(a.W), w, c)) return;
+    const bool have = hier_item<FAST>(a, uint32_t(a.W), w, c);
+    const bool general = FAST ? class_without_threshold(a, int(c)) : true;   // (c is warp-uniform in the staging variant)
+    if (!have) return;
     const uint32_t x = w * a.C + c;
     const uint32_t k2 = fastdiv(w, a.divE2);
     const float slo = a.slo[c];
+    const size_t tile_stride = size_t(a.W) * a.C, shard_stride = size_t(a.K2) * a.C;
+    const uint32_t pair_c = origin + uint32_t(int(c) * a.T * a.F) * 16u;
+    const uint32_t rows_c = origin + uint32_t(a.off_rows2 - a.off_pair2) + uint32_t(int(c) * a.T * a.F * (a.M + 1)) * 8u;
+    const uint32_t row_step = uint32_t(a.M + 1) * 8u;
+    const float *ld = a.load + x;
+    const int32_t *sh = a.shard + (k2 * a.C + c);
+    int32_t *out_idx = a.best_idx + x;
+    float *out_E = a.best_E + x;
     for (int64_t s = blockIdx.y; s < a.S; s += gridDim.y) {
-        const size_t i = size_t(s) * size_t(a.W) * a.C + x;
-        const int nt = a.shard[size_t(s) * size_t(a.K2) * a.C + k2 * a.C + c];
+        const int nt = sh[size_t(s) * shard_stride];
         int32_t bj = -1;
         float best = CUDART_INF_F;
         if (nt >= 0) {
             const int n1 = int(fastdiv(uint32_t(nt), a.divT)), t = nt - n1 * a.T;
             const float nf = float(n1 + 1);
-            const float ln = fmaxf(a.load[i], 0.f) * (1.0f / nf);
+            const float ln = fmaxf(ld[size_t(s) * tile_stride], 0.f) * (n1 < 256 ? s_rn[n1 + 1] : 1.0f / nf);
+            if (FAST && !general) {
+                uint32_t pc_addr = pair_c + uint32_t(t * a.F) * 16u;
+                uint32_t row = rows_c + uint32_t(t * a.F) * row_step;
+                float emin = CUDART_INF_F;
+                int bq = -1;
+#pragma unroll 4
+                for (int q = 0; q < a.F; ++q, pc_addr += 16u, row += row_step) {
+                    const float4 pc = load16<true>(a.ws, pc_addr);
+                    float e;
+                    bool ok;
+                    fast_one<true>(a.ws, row, ln, pc.x, pc.z, e, ok);
+                    if (ok && e < emin) {            // ascending q: strict compare keeps the lowest
+                        emin = e;
+                        bq = q;
+                    }
+                }
+                if (bq >= 0) {
+                    best = nf * emin;
+                    bj = nt * a.F + bq;
+                }
+            } else
             for (int q = 0; q < a.F; ++q) {
                 bool ok;
-                const float E = hier_eval<FAST>(a, origin, int(c), t * a.F + q, ln, nf, slo, ok);
+                const float E = hier_eval<FAST>(a, origin, int(c), t * a.F + q, ln, nf, slo, general, ok);
                 if (ok && E < best) {
                     best = E;
                     bj = nt * a.F + q;
                 }
             }
         }
-        a.best_idx[i] = bj;
-        a.best_E[i] = best;
+        out_idx[size_t(s) * tile_stride] = bj;
+        out_E[size_t(s) * tile_stride] = best;
     }
 }
 
@@ -273,7 +358,7 @@ cudaError_t launch_hier(const ResolveParams &rp, const ResolvedLayout &lay, void
     for (int t = 0; t < lay.T; ++t) a.tp[t] = rp.tp[t];
     a.nodes = d_nodes; a.shard = d_shard; a.best_idx = best_idx; a.best_E = best_E;
     const unsigned gy = unsigned(S < 32768 ? S : 32768);
-    const int64_t n1 = int64_t(a.K1) * lay.C, n2 = int64_t(a.K2) * lay.C, n3 = W * lay.C;
+    const int64_t n1 = int64_t(a.K1) * lay.C, n2 = int64_t(a.K2) * lay.C;
     a.ws = ws;
     a.off_pair2 = int32_t(lay.off_pair2); a.off_rows2 = int32_t(lay.off_rows2); a.off_end = int32_t(lay.off_tp);
     const size_t fast_bytes = lay.off_tp - lay.off_pair2;
@@ -286,25 +371,23 @@ cudaError_t launch_hier(const ResolveParams &rp, const ResolvedLayout &lay, void
     };
     if (a.use_fast) {
         if ((e = cudaFuncSetAttribute(hier_shard_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(fast_bytes))) != cudaSuccess) return e;
-        if ((e = cudaFuncSetAttribute(hier_freq_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(fast_bytes))) != cudaSuccess) return e;
     }
     hier_nodes_kernel<<<dim3(unsigned((n1 + 255) / 256), gy), 256, 0, st>>>(a);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     // staging variants: a warp per (32 items, class)
-    const int64_t f2 = ((int64_t(a.K2) + 31) / 32 * lay.C * 32 + 255) / 256, f3 = ((W + 31) / 32 * lay.C * 32 + 255) / 256;
-    if (a.use_fast) {
-        hier_shard_kernel<true><<<dim3(unsigned(f2), few(f2)), 256, fast_bytes, st>>>(a);
-        if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    }
-    hier_shard_kernel<false><<<dim3(unsigned((n2 + 255) / 256), a.use_fast ? few((n2 + 255) / 256) : gy), 256, 0, st>>>(a);
+    const int64_t f2 = ((int64_t(a.K2) + 31) / 32 * lay.C * 32 + 255) / 256;
+    if (a.use_fast) hier_shard_kernel<true><<<dim3(unsigned(f2), few(f2)), 256, fast_bytes, st>>>(a);
+    else hier_shard_kernel<false><<<dim3(unsigned((n2 + 255) / 256), gy), 256, 0, st>>>(a);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     e = record_start(st);
     if (e != cudaSuccess) return e;
+    const int64_t f3 = ((W + 31) / 32 * lay.C * 32 + 255) / 256, n3 = W * lay.C;
     if (a.use_fast) {
+        if ((e = cudaFuncSetAttribute(hier_freq_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(fast_bytes))) != cudaSuccess) return e;
         hier_freq_kernel<true><<<dim3(unsigned(f3), few(f3)), 256, fast_bytes, st>>>(a);
-        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    } else {
+        hier_freq_kernel<false><<<dim3(unsigned((n3 + 255) / 256), gy), 256, 0, st>>>(a);
     }
-    hier_freq_kernel<false><<<dim3(unsigned((n3 + 255) / 256), a.use_fast ? few((n3 + 255) / 256) : gy), 256, 0, st>>>(a);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     return record_stop(st);
 }
