@@ -170,7 +170,9 @@ typedef struct {
 /*
  * Argmin over a materialised energy tensor d_E [S][W][C][J] (+inf = infeasible).
  * n_of_j, tp_of_j : host int32 [J], instance count and TP degree of candidate j; needed only when
- * out->d_gpus is set (else may be NULL).  Sums are fp64, accumulated in a fixed order: results are
+ * out->d_gpus is set (else may be NULL).  They are copied with cudaMemcpyAsync on `stream`: pageable arrays are
+ * staged before the call returns (which makes the call wait for earlier work on the stream), pinned arrays
+ * are read when the stream reaches the copy and must stay valid until then.  dyn_eval_select needs neither.  Sums are fp64, accumulated in a fixed order: results are
  * bit-identical from run to run.  Workspace: dyn_select_workspace_bytes(S, W, J).
  */
 size_t dyn_select_workspace_bytes(int64_t S, int64_t W, int64_t J);
@@ -353,6 +355,16 @@ int dyn_pipeline_host(const dyn_bin_spec *spec, const dyn_profile_host *profile,
 void dyn_set_timing_events(void *start_event, void *stop_event);
 
 /* ---------------------------------------------------------------------------------------------
+ * Start-up self-check (no counterpart in the paper).  The sweep forms table addresses as subnormal
+ * floating-point numbers; a library built with flush-to-zero arithmetic (-ftz=true, --use_fast_math) would
+ * read entry 0 for every candidate and return plausible but wrong results.  This call runs one tiny kernel on
+ * `stream`, WAITS for it (the only call here that synchronises) and returns DYN_OK when the device computes
+ * such an address exactly, DYN_EUNSUPPORTED when it does not (rebuild without those flags), DYN_ECUDA on a
+ * runtime error.  Call it once per process at start-up; the stage calls do not call it.
+ * ------------------------------------------------------------------------------------------- */
+int dyn_self_check(void *stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Measured ceilings (instrumentation; no counterpart in the paper).  Each call enqueues one short
  * kernel on `stream` and records the events of dyn_set_timing_events around it; the caller divides
  * the returned amount of work by the measured time.  d_sink: device float [1], required, never
@@ -393,9 +405,12 @@ int dyn_probe_sweep_inner(int32_t iters, float feasible_share, float *d_sink, do
  *   - Limit: the call serves a problem only if dyn_workspace_bytes(profile, space, S, W) is at most
  *     DYN_STATIC_WS_BYTES; a larger problem is refused with DYN_EUNSUPPORTED and nothing is enqueued
  *     (use dyn_eval_select with your own workspace instead).
- *   - The first call on each device looks up the array's device address (once per device, with that
- *     device current) and keeps it; make that first call before any stream capture begins.
- *   - The call itself performs no allocation of any kind and frees nothing.
+ *   - The first call on each device is a warm-up: it looks up the array's device address (once per device,
+ *     with that device current) and keeps it.  With lazy module loading that look-up is also the moment the
+ *     CUDA runtime loads this library's device code onto the device, array included, which can take device
+ *     memory and synchronise the device once.  Make that first call at start-up, before any stream capture
+ *     begins.  A cudaDeviceReset invalidates the kept address: do not reset a device this call has been used on.
+ *   - Every later call performs no allocation of any kind, frees nothing and does not synchronise.
  *   - All calls on a device share the one array, and it keeps whatever the previous call left there.
  *     That is harmless for back-to-back calls on one stream, because every word the kernels read from
  *     the scratch is written earlier in the same call (nothing relies on zero-initialised scratch).

@@ -26,7 +26,7 @@ EXPORTS = ("dyn_strerror", "dyn_last_cuda_error", "dyn_bin_trace", "dyn_workspac
            "dyn_select_workspace_bytes", "dyn_select", "dyn_eval_select", "dyn_pipeline_arena_bytes",
            "dyn_pipeline_host", "dyn_set_timing_events", "dyn_eval_select_static", "dyn_hier_workspace_bytes",
            "dyn_hier_select", "dyn_mixed_workspace_bytes", "dyn_mixed_tuple_count", "dyn_mixed_select", "dyn_reconf_workspace_bytes", "dyn_reconf_select", "dyn_bin_tokens", "dyn_carbon",
-           "dyn_probe_fma", "dyn_probe_sweep_inner")
+           "dyn_probe_fma", "dyn_probe_sweep_inner", "dyn_self_check")
 
 
 class DynError(RuntimeError):
@@ -145,6 +145,8 @@ _lib.dyn_bin_tokens.argtypes = [C.POINTER(_BinSpec), C.c_void_p, C.c_void_p, C.c
                                 C.c_void_p, C.c_void_p]
 _lib.dyn_carbon.restype = C.c_int
 _lib.dyn_carbon.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p]
+_lib.dyn_self_check.restype = C.c_int
+_lib.dyn_self_check.argtypes = [C.c_void_p]
 _lib.dyn_probe_fma.restype = C.c_int
 _lib.dyn_probe_fma.argtypes = [C.c_int32, C.c_void_p, C.POINTER(C.c_double), C.c_void_p]
 _lib.dyn_probe_sweep_inner.restype = C.c_int
@@ -468,3 +470,9 @@ def dyn_probe_sweep_inner(iters, feasible_share, d_sink) -> float:
                                       C.byref(work), _stream()),
            "dyn_probe_sweep_inner")
     return work.value
+
+
+def dyn_self_check():
+    """Start-up self-check of the subnormal address arithmetic (synchronises); raises DynError with
+    DYN_EUNSUPPORTED when the library was built with flush-to-zero arithmetic."""
+    _check(_lib.dyn_self_check(_stream()), "dyn_self_check")

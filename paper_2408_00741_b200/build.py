@@ -19,6 +19,8 @@ def nvcc_command(verbose_ptxas: bool = False):
     if verbose_ptxas:
         cmd += ["-Xptxas", "-v"]
     cmd += [os.path.join(CSRC, s) for s in SOURCES] + ["-o", LIB]
+    # the sweep's table addresses are subnormal floats: flush-to-zero arithmetic would break them silently
+    assert not any(f.startswith("-ftz") or f in ("--use_fast_math", "-use_fast_math") for f in cmd)
     return cmd
 
 

@@ -29,6 +29,12 @@ int sm_count() {
     return cached;
 }
 
+int device_slot() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) return 0;
+    return dev < kMaxDevices ? dev : kMaxDevices - 1;
+}
+
 namespace {
 
 bool strictly_ascending_u32(const uint32_t *v, int n) {
@@ -177,6 +183,34 @@ int check_mixed(const dyn_profile *p, const dyn_space *sp, int64_t S, int64_t W,
 }
 
 }  // namespace
+
+// dyn_eval_select; with resolve == false the tables in d_ws are taken as resolved by an earlier call for the same
+// profile, space and W (the host pipeline evaluates its pieces that way)
+int eval_select_impl(const dyn_profile *profile, const dyn_space *space, const float *d_load, int64_t S, int64_t W,
+                     const dyn_select_out *out, void *d_ws, size_t ws_bytes, cudaStream_t st, bool resolve) {
+    ResolveParams rp;
+    int rc = check_problem(profile, space, S, W, &rp);
+    if (rc != DYN_OK) return rc;
+    const int64_t tiles = S * W * profile->C;
+    rc = check_out(out, S, tiles);
+    if (rc != DYN_OK) return rc;
+    if (tiles > 0 && !d_load) return DYN_EINVAL;
+    const ResolvedLayout lay = resolved_layout(profile->C, profile->T, space->F, profile->M, space->Nmax, S, W);
+    rc = check_ws(d_ws, ws_bytes, lay.total);
+    if (rc != DYN_OK) return rc;
+    char *ws = static_cast<char *>(d_ws);
+    if (resolve) DYN_CUDA_TRY(launch_resolve(rp, lay, d_ws, st));
+    DYN_CUDA_TRY(record_start(st));
+    DYN_CUDA_TRY(launch_eval_select(lay, d_ws, d_load, tiles, space->gpu_budget, out->d_best_idx, out->d_best_E, st));
+    DYN_CUDA_TRY(record_stop(st));
+    const int64_t chunks = totals_chunks(W);
+    double *partial = reinterpret_cast<double *>(ws + lay.off_partial);
+    uint32_t *partial_bad = reinterpret_cast<uint32_t *>(ws + lay.off_partial + size_t(S) * size_t(chunks) * sizeof(double));
+    DYN_CUDA_TRY(launch_totals(to_out(out), S, W, profile->C, lay.J, nullptr, nullptr, profile->T, space->F,
+                               reinterpret_cast<const int32_t *>(ws + lay.off_tp), partial, partial_bad, st));
+    return DYN_OK;
+}
+
 }  // namespace dyn
 
 using namespace dyn;
@@ -266,7 +300,8 @@ int dyn_select(const float *d_E, int64_t S, int64_t W, int32_t C, int32_t J, con
     if (out->d_gpus) {
         d_nj = reinterpret_cast<int32_t *>(ws + off_nj);
         d_tj = reinterpret_cast<int32_t *>(ws + off_nj + align256(size_t(J) * sizeof(int32_t)));
-        // pageable host memory: the copy is staged before the call returns, the arrays may be reused
+        // pageable host arrays are staged before cudaMemcpyAsync returns (the call then waits for earlier work
+        // on the stream); pinned arrays are read when the stream gets here and must stay valid until then
         DYN_CUDA_TRY(cudaMemcpyAsync(d_nj, n_of_j, size_t(J) * sizeof(int32_t), cudaMemcpyHostToDevice, st));
         DYN_CUDA_TRY(cudaMemcpyAsync(d_tj, tp_of_j, size_t(J) * sizeof(int32_t), cudaMemcpyHostToDevice, st));
     }
@@ -279,28 +314,7 @@ int dyn_select(const float *d_E, int64_t S, int64_t W, int32_t C, int32_t J, con
 
 int dyn_eval_select(const dyn_profile *profile, const dyn_space *space, const float *d_load, int64_t S, int64_t W,
                     const dyn_select_out *out, void *d_ws, size_t ws_bytes, void *stream) {
-    ResolveParams rp;
-    int rc = check_problem(profile, space, S, W, &rp);
-    if (rc != DYN_OK) return rc;
-    const int64_t tiles = S * W * profile->C;
-    rc = check_out(out, S, tiles);
-    if (rc != DYN_OK) return rc;
-    if (tiles > 0 && !d_load) return DYN_EINVAL;
-    const ResolvedLayout lay = resolved_layout(profile->C, profile->T, space->F, profile->M, space->Nmax, S, W);
-    rc = check_ws(d_ws, ws_bytes, lay.total);
-    if (rc != DYN_OK) return rc;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    char *ws = static_cast<char *>(d_ws);
-    DYN_CUDA_TRY(launch_resolve(rp, lay, d_ws, st));
-    DYN_CUDA_TRY(record_start(st));
-    DYN_CUDA_TRY(launch_eval_select(lay, d_ws, d_load, tiles, space->gpu_budget, out->d_best_idx, out->d_best_E, st));
-    DYN_CUDA_TRY(record_stop(st));
-    const int64_t chunks = totals_chunks(W);
-    double *partial = reinterpret_cast<double *>(ws + lay.off_partial);
-    uint32_t *partial_bad = reinterpret_cast<uint32_t *>(ws + lay.off_partial + size_t(S) * size_t(chunks) * sizeof(double));
-    DYN_CUDA_TRY(launch_totals(to_out(out), S, W, profile->C, lay.J, nullptr, nullptr, profile->T, space->F,
-                               reinterpret_cast<const int32_t *>(ws + lay.off_tp), partial, partial_bad, st));
-    return DYN_OK;
+    return eval_select_impl(profile, space, d_load, S, W, out, d_ws, ws_bytes, static_cast<cudaStream_t>(stream), true);
 }
 
 size_t dyn_hier_workspace_bytes(const dyn_profile *profile, const dyn_space *space, int64_t S, int64_t W) {

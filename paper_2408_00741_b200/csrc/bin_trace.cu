@@ -222,7 +222,8 @@ cudaError_t launch_bin_trace(const BinParams &bp, const uint32_t *t_ms, const ui
         // two whole waves of resident CTAs (a whole number of waves keeps every SM slot busy to the end; worth a
         // few percent on 14 M requests) for traces up to a few tens of millions of requests; beyond that more CTAs rather than longer slices (a slice of about 24 K requests streams best:
         // measured 6.7 TB/s on 112 M requests against 5.5 TB/s with slices of 95 K)
-        static thread_local int resident = 0;
+        static thread_local int resident_of[kMaxDevices] = {};      // per device
+        int &resident = resident_of[device_slot()];
         if (resident == 0) {
             int r = 0;
             if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&r, bin_trace_kernel<2, 2, true, false>, kThreads, 0) !=

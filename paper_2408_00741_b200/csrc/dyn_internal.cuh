@@ -135,6 +135,12 @@ cudaError_t launch_bin_tokens(const BinParams &bp, const uint32_t *t_ms, const u
 cudaError_t launch_carbon(const double *E_window, const float *intensity, int64_t S, int64_t W, double *carbon, cudaStream_t st);
 
 int sm_count();
+// device ordinal of the calling thread's current device, clamped to [0, kMaxDevices): index of per-device caches
+constexpr int kMaxDevices = 64;
+int device_slot();
+
+int eval_select_impl(const dyn_profile *profile, const dyn_space *space, const float *d_load, int64_t S, int64_t W,
+                     const dyn_select_out *out, void *d_ws, size_t ws_bytes, cudaStream_t st, bool resolve);
 
 #ifdef __CUDACC__
 // general-path evaluation of one candidate from the resolved rows (used by the small restricted searches)

@@ -5,6 +5,11 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+// The table addresses of the threshold path are formed as subnormal floats (see units() below): a build that
+// flushes subnormals to zero (-ftz=true, --use_fast_math) would turn every address into zero.  The compiler
+// defines nothing a source file could test for this, so the build script refuses such flags and
+// dyn_self_check() tests the arithmetic on the device.
+
 namespace dyn {
 
 namespace {

@@ -51,8 +51,14 @@ cudaEvent_t *overlap_events() {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return nullptr;
     if (!made[dev]) {
-        for (int i = 0; i < kEvents; ++i)
-            if (cudaEventCreateWithFlags(&ev[dev][i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        for (int i = 0; i < kEvents; ++i) {
+            const cudaError_t e = cudaEventCreateWithFlags(&ev[dev][i], cudaEventDisableTiming);
+            if (e != cudaSuccess) {                      // give back what was created and report why
+                for (int k = 0; k < i; ++k) cudaEventDestroy(ev[dev][k]);
+                dyn::set_last_cuda_error(e);
+                return nullptr;
+            }
+        }
         made[dev] = true;
     }
     return ev[dev];
@@ -174,8 +180,9 @@ int dyn_pipeline_host(const dyn_bin_spec *spec, const dyn_profile_host *p, const
             if (sk.d_E_window) sk.d_E_window += s0 * W;
             if (sk.d_hist) sk.d_hist += s0 * J;
             if (sk.d_gpus) sk.d_gpus += s0 * W;
-            rc = dyn_eval_select(&dp, sp, static_cast<const float *>(dptr(ar.load)) + s0 * wc, int64_t(s1 - s0), int64_t(W), &sk,
-                                 dptr(ar.ws), ar.ws_bytes, stream);
+            // the tables are resolved once, by the first piece; the others run the sweep and the totals on them
+            rc = dyn::eval_select_impl(&dp, sp, static_cast<const float *>(dptr(ar.load)) + s0 * wc, int64_t(s1 - s0), int64_t(W),
+                                       &sk, dptr(ar.ws), ar.ws_bytes, st, k == 0);
             if (rc != DYN_OK) return rc;
             // the piece's results go back on the copy stream (behind the loads, which are long in by then) while
             // the next piece is evaluated

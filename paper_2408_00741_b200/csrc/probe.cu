@@ -109,6 +109,18 @@ sweep_inner_probe_kernel(const int iters, const float scale, const float feasibl
     if (s == -1.2345e30f) *sink = s;
 }
 
+// 0 until the check has run; 1 = subnormal arithmetic is exact, 2 = it is not (flushed to zero)
+__device__ int g_self_check;
+
+// forms the shared-memory byte address of entry m of a row at byte offset `bytes` the way fast_two does, from
+// values the compiler cannot fold, and compares with the integer arithmetic
+__global__ void self_check_kernel(const float m_plus_two23, const uint32_t bytes, const uint32_t want) {
+    const float off = row_offset_units(bytes);
+    float z;
+    asm volatile("fma.rn.f32 %0, %1, %2, %3;" : "=f"(z) : "f"(m_plus_two23), "f"(units(8u)), "f"(off));
+    g_self_check = (__float_as_uint(z) == want) ? 1 : 2;
+}
+
 }  // namespace
 
 }  // namespace dyn
@@ -116,6 +128,17 @@ sweep_inner_probe_kernel(const int iters, const float scale, const float feasibl
 using namespace dyn;
 
 extern "C" {
+
+int dyn_self_check(void *stream) {
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const uint32_t m = 5u, bytes = 4096u + 72u;
+    self_check_kernel<<<1, 1, 0, st>>>(kTwo23 + float(m), bytes, bytes + 8u * m);
+    DYN_CUDA_TRY(cudaGetLastError());
+    DYN_CUDA_TRY(cudaStreamSynchronize(st));
+    int got = 0;
+    DYN_CUDA_TRY(cudaMemcpyFromSymbol(&got, g_self_check, sizeof(int)));
+    return got == 1 ? DYN_OK : DYN_EUNSUPPORTED;
+}
 
 int dyn_probe_fma(int32_t iters, float *d_sink, double *fp32_ops, void *stream) {
     if (iters < 1 || !d_sink) return DYN_EINVAL;

@@ -639,14 +639,17 @@ eval_configs_kernel(const SweepArgs a, const int64_t units_total, float *__restr
 }
 
 size_t smem_limit() {
-    static size_t lim = [] {
+    // opt-in shared memory per block of the current device (cached per device)
+    static thread_local size_t lim[kMaxDevices] = {};
+    const int slot = device_slot();
+    if (lim[slot] == 0) {
         int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return size_t(48 * 1024);
-        if (cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
-            return size_t(48 * 1024);
-        return size_t(v);
-    }();
-    return lim;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess || v <= 0)
+            v = 48 * 1024;
+        lim[slot] = size_t(v);
+    }
+    return lim[slot];
 }
 
 SweepArgs make_args(const ResolvedLayout &lay, const void *d_ws, const float *d_load, int64_t tiles, int32_t budget) {

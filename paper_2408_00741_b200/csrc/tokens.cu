@@ -199,7 +199,8 @@ cudaError_t launch_bin_tokens(const BinParams &bp, const uint32_t *t_ms, const u
     if (e != cudaSuccess) return e;
     if (n_req > 0) {
         // slices sized for whole waves of resident CTAs, as few waves as the slice limit allows
-        static thread_local int resident = 0;
+        static thread_local int resident_of[kMaxDevices] = {};      // per device
+        int &resident = resident_of[device_slot()];
         if (resident == 0) {
             int r = 0;
             e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&r, bin_tokens_kernel<2, 2, true>, kThreads, 0);

@@ -40,3 +40,11 @@ def test_host_side_contract_without_a_gpu():
     lib.dyn_eval_select.restype = ctypes.c_int
     assert lib.dyn_eval_select(None, None, None, ctypes.c_int64(1), ctypes.c_int64(1), None, None,
                                ctypes.c_size_t(0), None) == dyn.DYN_EINVAL
+
+
+def test_build_keeps_subnormal_arithmetic():
+    """The sweep forms table addresses as subnormal floats: the build must not ask for flush-to-zero arithmetic."""
+    from paper_2408_00741_b200 import build
+    cmd = build.nvcc_command()
+    assert not any(f.startswith("-ftz") or "fast_math" in f for f in cmd)
+    assert "arch=compute_100a,code=sm_100a" in cmd

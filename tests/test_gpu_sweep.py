@@ -190,6 +190,10 @@ def test_few_rows_without_a_load_threshold(dyn, large, budget):
         assert min(abs(tb[j_] - 0.1) / 0.1, abs(u[j_] - 1.0)) < REL_TOL
 
 
+def test_self_check_passes_on_this_build(dyn):
+    dyn.dyn_self_check()                      # raises when subnormal arithmetic is flushed to zero
+
+
 def test_limits_of_the_candidate_space(dyn):
     """Largest built shape per axis (256 instance counts, 16 TP degrees) and the smallest tables
     (two frequency rows, two load knots); the GPU budget cuts the space unevenly."""

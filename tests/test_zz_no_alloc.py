@@ -7,7 +7,8 @@ import pytest
 import torch
 
 import gen
-from parity import gpu_profile_space
+import oracle
+from parity import check_selection, gpu_profile_space
 
 pytestmark = pytest.mark.gpu
 
@@ -34,6 +35,9 @@ def _both(dyn, wl, S, W, seed):
         t.fill_(-12345)
     dyn.dyn_eval_select_static(p, s, d_load, got)          # new entry point, no workspace
     torch.cuda.synchronize()
+    # and against the CPU oracle directly, under the rule of the other parity tests
+    o = oracle.eval_select(prof, sp, load)
+    check_selection(prof, sp, load, got.best_idx.cpu().numpy(), got.best_E.cpu().numpy(), o)
     return ref, got
 
 
@@ -79,3 +83,45 @@ def test_problem_larger_than_the_static_scratch_is_refused(dyn):
     dyn.dyn_eval_select(p, s, torch.zeros((1, 2, 9), dtype=torch.float32, device="cuda"), out, ws)
     torch.cuda.synchronize()
     assert int((out.best_idx == 7).sum()) < 18
+
+
+def test_largest_problem_that_fits_and_no_allocation(dyn):
+    """A problem whose scratch need is within 256 bytes of the static array is served, the next larger one is
+    refused; and a call changes nothing in the device's free memory (it allocates nothing)."""
+    wl = gen.workload("cfg1")
+    prof, sp = wl.profile(), wl.space()
+    p, s = gpu_profile_space(dyn, prof, sp)
+    W = 1
+    lo, hi = 1, 1 << 22
+    while lo < hi:                                          # largest S whose workspace fits
+        mid = (lo + hi + 1) // 2
+        if dyn.dyn_workspace_bytes(p, s, mid, W) <= dyn.DYN_STATIC_WS_BYTES:
+            lo = mid
+        else:
+            hi = mid - 1
+    S = lo
+    need = dyn.dyn_workspace_bytes(p, s, S, W)
+    assert dyn.DYN_STATIC_WS_BYTES - 256 <= need <= dyn.DYN_STATIC_WS_BYTES
+    load = gen.random_loads((S, W, 9), seed=31, mean=2.5)
+    d_load = torch.from_numpy(load).cuda()
+    got = dyn.SelectOut(S, W, 9, wl.J, windows=False, hist=False, gpus=False)
+    ref = dyn.SelectOut(S, W, 9, wl.J, windows=False, hist=False, gpus=False)
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    dyn.dyn_eval_select_static(p, s, d_load, got)           # (also the warm-up call of this device, if none came before)
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    dyn.dyn_eval_select_static(p, s, d_load, got)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    dyn.dyn_eval_select(p, s, d_load, ref, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(ref.best_idx, got.best_idx) and torch.equal(ref.n_infeasible, got.n_infeasible)
+    assert np.allclose(got.E_total.cpu().numpy(), ref.E_total.cpu().numpy(), rtol=1e-5)
+    # one scenario block more no longer fits
+    S2 = S + 64
+    assert dyn.dyn_workspace_bytes(p, s, S2, W) > dyn.DYN_STATIC_WS_BYTES
+    with pytest.raises(dyn.DynError) as e:
+        dyn.dyn_eval_select_static(p, s, torch.zeros((S2, W, 9), dtype=torch.float32, device="cuda"),
+                                   dyn.SelectOut(S2, W, 9, wl.J, windows=False, hist=False, gpus=False))
+    assert e.value.status == dyn.DYN_EUNSUPPORTED
