@@ -277,15 +277,29 @@ __global__ void reconf_transpose_kernel(const ReconfArgs a) {
 }
 
 constexpr int kBackWarps = 1;
-constexpr int kBackChunk = 512;                 // windows per stretch (a multiple of the ring depth)
+constexpr int kBackThreads = 256;               // threads of a CTA: all copy the table, one warp walks
+constexpr int kBackChunk = 512;                 // windows per stretch
+constexpr int kBackRing = 12;                   // windows whose vectors are on their way into shared memory
 
-__global__ void __launch_bounds__(kBackWarps * 32) reconf_back_kernel(const ReconfArgs a) {
+__global__ void __launch_bounds__(kBackThreads) reconf_back_kernel(const ReconfArgs a, const int rows_b) {
     __shared__ int path_all[kBackWarps][kBackChunk];
+    extern __shared__ float4 smem4[];
+    const int NS = a.NS;
+    // the first rows_b rows of the transposed table (columns of R) in shared memory: the walk reads one of them per
+    // window, and which one is known only when the previous window is done
+    float *Rts = reinterpret_cast<float *>(smem4);
+    if ((NS & 3) == 0) {
+        const float4 *src = reinterpret_cast<const float4 *>(a.Rt);
+        for (int i = threadIdx.x; i < rows_b * (NS / 4); i += kBackThreads) smem4[i] = __ldg(src + i);
+    } else {
+        for (int i = threadIdx.x; i < rows_b * NS; i += kBackThreads) Rts[i] = __ldg(a.Rt + i);
+    }
+    __syncthreads();
+    if (threadIdx.x >= kBackWarps * 32) return;
     const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
     const int64_t sc = int64_t(blockIdx.x) * kBackWarps + wi;
     if (sc >= a.S * a.C) return;
     int *path = path_all[wi];
-    const int NS = a.NS;
     const int c = int(sc % a.C);
     const int64_t s = sc / a.C;
     const int64_t W = a.W;
@@ -309,58 +323,71 @@ __global__ void __launch_bounds__(kBackWarps * 32) reconf_back_kernel(const Reco
         asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(mm) : "f"(best));
         if (mm < CUDART_INF_F) cur = int(__reduce_min_sync(0xffffffffu, best == mm ? arg : 0xffffffffu));
     }
+    // With at most 256 states a lane owns eight entries h = lane + 32 j of every vector.  The vectors of the next
+    // kBackRing windows do not depend on the state: a lane asks for its own entries that many windows ahead with
+    // asynchronous copies into a ring in shared memory and later reads only what it copied itself, so no barrier
+    // is needed and the walk does not wait for DRAM.  (Loads into registers that far ahead do not work: a warp
+    // can wait only for all of its outstanding loads at once.)
     const bool ahead = NS <= 256;
-    float ring[8][8];
-    if (ahead) {
+    float *ring = Rts + size_t(rows_b) * NS;                 // [kBackRing][256]
+    auto ask = [&](int64_t row, int slot) {                  // entries of vector `row` (clamped; rows < 0 are never used)
+        const float *src = hist + (row > 0 ? row : 0) * NS;
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const int64_t row = W - 2 - k;                   // the vector used at window W-1-k
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-                ring[k][j] = (row >= 0 && lane + 32 * j < NS) ? hist[row * NS + lane + 32 * j] : CUDART_INF_F;
-        }
-    }
+        for (int j = 0; j < 8; ++j)
+            if (lane + 32 * j < NS) __pipeline_memcpy_async(ring + slot * 256 + lane + 32 * j, src + lane + 32 * j, 4);
+        __pipeline_commit();
+    };
+    if (ahead)
+        for (int k = 0; k < kBackRing; ++k) ask(W - 2 - k, k);         // slot k: the vector used at window W-1-k
+    // the column of R that leads into the current state (a row of the transposed copy), a lane's eight entries of
+    // it: it is read again only when the state changes
+    float rcol[8];
+    int rcol_of = -1;
     int64_t seg_hi = W;                                      // windows [w, seg_hi) are noted in path[seg_hi - 1 - w]
+    int slot = 0;
     for (int64_t wb = W - 1; wb >= 0; wb -= 8) {
-#pragma unroll
+#pragma unroll 1
         for (int k = 0; k < 8; ++k) {
             const int64_t w = wb - k;
             if (w >= 0) {
                 if (lane == 0) path[seg_hi - 1 - w] = cur;
+                if (ahead) __pipeline_wait_prior(kBackRing - 1);        // this window's vector has arrived
                 if (cur >= 0 && w > 0) {
-                    float best = CUDART_INF_F;
+                    float mm;
                     uint32_t arg = 0xffffffffu;
                     if (ahead) {
+                        if (rcol_of != cur) {                // warp-uniform
+                            const float *col = cur < rows_b ? Rts + size_t(cur) * NS : Rt + size_t(cur) * NS;
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            const int h = lane + 32 * j;
-                            if (h < NS) {
-                                const float v = ring[k][j] + __ldg(Rt + size_t(cur) * NS + h);
-                                if (v < best) {              // ascending h per lane: strict compare keeps the lowest
-                                    best = v;
-                                    arg = uint32_t(h);
-                                }
-                            }
+                            for (int j = 0; j < 8; ++j) rcol[j] = lane + 32 * j < NS ? col[lane + 32 * j] : CUDART_INF_F;
+                            rcol_of = cur;
                         }
+                        float v[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) v[j] = lane + 32 * j < NS ? ring[slot * 256 + lane + 32 * j] + rcol[j] : CUDART_INF_F;
+                        const float best = fminf(min3f(min3f(v[0], v[1], v[2]), v[3], v[4]), min3f(v[5], v[6], v[7]));
+                        asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(mm) : "f"(best));
+                        // lowest h that attains the minimum: descending j, so the lowest matching entry stays
+#pragma unroll
+                        for (int j = 7; j >= 0; --j) arg = (v[j] == mm) ? uint32_t(lane + 32 * j) : arg;
                     } else {
+                        float best = CUDART_INF_F;
                         const float *hp = hist + (w - 1) * NS;
                         for (int h = lane; h < NS; h += 32) {
-                            const float v = hp[h] + __ldg(Rt + size_t(cur) * NS + h);
-                            if (v < best) {
-                                best = v;
+                            const float x = hp[h] + __ldg(Rt + size_t(cur) * NS + h);
+                            if (x < best) {              // ascending h per lane: strict compare keeps the lowest
+                                best = x;
                                 arg = uint32_t(h);
                             }
                         }
+                        asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(mm) : "f"(best));
+                        if (best != mm) arg = 0xffffffffu;
                     }
-                    float mm;
-                    asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(mm) : "f"(best));
-                    cur = int(__reduce_min_sync(0xffffffffu, best == mm ? arg : 0xffffffffu));
+                    cur = int(__reduce_min_sync(0xffffffffu, arg));
                 }
-                if (ahead) {                                 // the vector used eight windows further down
-                    const int64_t row = w - 9;
-#pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        ring[k][j] = (row >= 0 && lane + 32 * j < NS) ? hist[row * NS + lane + 32 * j] : CUDART_INF_F;
+                if (ahead) {                                 // the slot is free: the vector used kBackRing windows further down
+                    ask(w - 1 - kBackRing, slot);
+                    slot = slot + 1 == kBackRing ? 0 : slot + 1;
                 }
             }
         }
@@ -444,7 +471,17 @@ cudaError_t launch_reconf(const ResolvedLayout &lay, void *d_ws, size_t off_cost
     if (e != cudaSuccess) return e;
     reconf_path_kernel<<<unsigned(S * lay.C), kPathThreads, smem, st>>>(a, rows_s);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    reconf_back_kernel<<<unsigned((S * lay.C + kBackWarps - 1) / kBackWarps), kBackWarps * 32, 0, st>>>(a);
+    {
+        // as many columns of R as fit beside the kernel's static shared memory
+        const size_t ring_b = size_t(kBackRing) * 256 * sizeof(float);
+        const size_t room = size_t(lim) > 8192 + ring_b ? size_t(lim) - 8192 - ring_b : 0;
+        int rows_b = int(room / (size_t(a.NS) * sizeof(float)));
+        if (rows_b > a.NS) rows_b = a.NS;
+        const size_t smem_b = size_t(rows_b) * a.NS * sizeof(float) + ring_b;
+        e = cudaFuncSetAttribute(reconf_back_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_b));
+        if (e != cudaSuccess) return e;
+        reconf_back_kernel<<<unsigned((S * lay.C + kBackWarps - 1) / kBackWarps), kBackThreads, smem_b, st>>>(a, rows_b);
+    }
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     return record_stop(st);
