@@ -355,6 +355,24 @@ int dyn_pipeline_host(const dyn_bin_spec *spec, const dyn_profile_host *profile,
 void dyn_set_timing_events(void *start_event, void *stop_event);
 
 /* ---------------------------------------------------------------------------------------------
+ * Checking build (no counterpart in the paper).  The library can be built a second time with index checks
+ * (libdynamo_check.so): every computed index into a global array, a shared-memory bin or a table is tested
+ * against its extent before use, and every table address that the sweep forms arithmetically against the
+ * range it staged; an index out of range is recorded and replaced by 0, so that the access stays in bounds and
+ * the kernel runs to its end -- nothing traps, nothing waits.  This call WAITS for the device, then reports
+ * and clears what the kernels of this process recorded since the last call: the number of violations and, of
+ * the first one, the site (translation unit number * 65536 + source line), the offending index and the extent
+ * it was tested against (both saturate at 2^32 - 1).  Any of the four pointers may be NULL.
+ * Returns DYN_OK in a checking build, DYN_EUNSUPPORTED (and zeros) in the ordinary build, which has no checks.
+ * ------------------------------------------------------------------------------------------- */
+int dyn_debug_status(uint32_t *violations, uint32_t *site, uint32_t *index, uint32_t *extent);
+/* Checking build only (DYN_EUNSUPPORTED otherwise): enqueues a one-thread kernel that indexes a three-element
+ * local array with 5 through the check, which must record {site in probe.cu, index 5, extent 3} and read
+ * element 0 instead (d_out, device int32 [1], receives 7).  It shows that the reporting path works; no access
+ * leaves its array. */
+int dyn_debug_selftest(int32_t *d_out, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Start-up self-check (no counterpart in the paper).  The sweep forms table addresses as subnormal
  * floating-point numbers; a library built with flush-to-zero arithmetic (-ftz=true, --use_fast_math) would
  * read entry 0 for every candidate and return plausible but wrong results.  This call runs one tiny kernel on

@@ -12,7 +12,7 @@ _BINDING_NAMES = ("DYN_ECUDA", "DYN_EINVAL", "DYN_EUNSUPPORTED", "DYN_EWORKSPACE
                   "dyn_workspace_bytes", "dyn_eval_select_static", "DYN_STATIC_WS_BYTES", "dyn_hier_workspace_bytes", "dyn_hier_select",
                   "MixedOut", "dyn_mixed_workspace_bytes", "dyn_mixed_tuple_count", "dyn_mixed_select",
                   "dyn_reconf_workspace_bytes", "dyn_reconf_select", "dyn_bin_tokens", "dyn_carbon",
-                  "dyn_probe_fma", "dyn_probe_sweep_inner", "dyn_self_check")
+                  "dyn_probe_fma", "dyn_probe_sweep_inner", "dyn_self_check", "dyn_debug_status", "dyn_debug_selftest", "CHECKED")
 __all__ = list(_BINDING_NAMES)
 
 

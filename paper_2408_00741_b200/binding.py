@@ -14,7 +14,9 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "csrc", "libdynamo.so")
+# DYN_CHECKED=1 in the environment selects the checking build of the library (index checks in every kernel)
+CHECKED = os.environ.get("DYN_CHECKED", "") not in ("", "0")
+LIB_PATH = os.path.join(_HERE, "csrc", "libdynamo_check.so" if CHECKED else "libdynamo.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2408_00741_b200.build` "
@@ -26,7 +28,7 @@ EXPORTS = ("dyn_strerror", "dyn_last_cuda_error", "dyn_bin_trace", "dyn_workspac
            "dyn_select_workspace_bytes", "dyn_select", "dyn_eval_select", "dyn_pipeline_arena_bytes",
            "dyn_pipeline_host", "dyn_set_timing_events", "dyn_eval_select_static", "dyn_hier_workspace_bytes",
            "dyn_hier_select", "dyn_mixed_workspace_bytes", "dyn_mixed_tuple_count", "dyn_mixed_select", "dyn_reconf_workspace_bytes", "dyn_reconf_select", "dyn_bin_tokens", "dyn_carbon",
-           "dyn_probe_fma", "dyn_probe_sweep_inner", "dyn_self_check")
+           "dyn_probe_fma", "dyn_probe_sweep_inner", "dyn_self_check", "dyn_debug_status", "dyn_debug_selftest")
 
 
 class DynError(RuntimeError):
@@ -145,6 +147,10 @@ _lib.dyn_bin_tokens.argtypes = [C.POINTER(_BinSpec), C.c_void_p, C.c_void_p, C.c
                                 C.c_void_p, C.c_void_p]
 _lib.dyn_carbon.restype = C.c_int
 _lib.dyn_carbon.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p]
+_lib.dyn_debug_status.restype = C.c_int
+_lib.dyn_debug_status.argtypes = [C.POINTER(C.c_uint32)] * 4
+_lib.dyn_debug_selftest.restype = C.c_int
+_lib.dyn_debug_selftest.argtypes = [C.c_void_p, C.c_void_p]
 _lib.dyn_self_check.restype = C.c_int
 _lib.dyn_self_check.argtypes = [C.c_void_p]
 _lib.dyn_probe_fma.restype = C.c_int
@@ -476,3 +482,19 @@ def dyn_self_check():
     """Start-up self-check of the subnormal address arithmetic (synchronises); raises DynError with
     DYN_EUNSUPPORTED when the library was built with flush-to-zero arithmetic."""
     _check(_lib.dyn_self_check(_stream()), "dyn_self_check")
+
+
+def dyn_debug_status():
+    """(violations, site, index, extent) recorded by the checking build since the last call (synchronises the
+    device and clears the record); None in the ordinary build, which has no checks."""
+    v = [C.c_uint32(0) for _ in range(4)]
+    rc = _lib.dyn_debug_status(*[C.byref(x) for x in v])
+    if rc == DYN_EUNSUPPORTED:
+        return None
+    _check(rc, "dyn_debug_status")
+    return tuple(int(x.value) for x in v)
+
+
+def dyn_debug_selftest(d_out):
+    """Checking build only: plants one out-of-range index behind the check (d_out: int32 [1], receives 7)."""
+    _check(_lib.dyn_debug_selftest(_dev(d_out, torch.int32, "d_out"), _stream()), "dyn_debug_selftest")

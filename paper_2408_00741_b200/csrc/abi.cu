@@ -1,5 +1,6 @@
 // Host side of the C ABI declared in include/dynamo.h: argument validation and launch sequencing.
 // Every step of the path runs in the kernels of this library; nothing here computes results.
+#define DYN_TU_ID 1
 #include "dyn_internal.cuh"
 
 #include <cmath>
@@ -28,6 +29,19 @@ int sm_count() {
     }
     return cached;
 }
+
+#ifdef DYN_CHECK
+namespace check {
+namespace {
+constexpr int kMaxReaders = 32;
+Reader g_readers[kMaxReaders];
+int g_n_readers = 0;
+}  // namespace
+void register_reader(Reader r) {
+    if (g_n_readers < kMaxReaders) g_readers[g_n_readers++] = r;
+}
+}  // namespace check
+#endif
 
 int device_slot() {
     int dev = 0;
@@ -229,6 +243,30 @@ const char *dyn_strerror(int status) {
 }
 
 int dyn_last_cuda_error(void) { return tls_cuda_error; }
+
+int dyn_debug_status(uint32_t *violations, uint32_t *site, uint32_t *index, uint32_t *extent) {
+#ifdef DYN_CHECK
+    DYN_CUDA_TRY(cudaDeviceSynchronize());
+    uint32_t total = 0, s0 = 0, i0 = 0, n0 = 0;
+    for (int k = 0; k < check::g_n_readers; ++k) {
+        check::Record r = {0u, 0u, 0u, 0u};
+        DYN_CUDA_TRY(check::g_readers[k](&r));
+        if (r.count && !total) { s0 = r.site; i0 = r.index; n0 = r.extent; }
+        total += r.count;
+    }
+    if (violations) *violations = total;
+    if (site) *site = s0;
+    if (index) *index = i0;
+    if (extent) *extent = n0;
+    return DYN_OK;
+#else
+    if (violations) *violations = 0;
+    if (site) *site = 0;
+    if (index) *index = 0;
+    if (extent) *extent = 0;
+    return DYN_EUNSUPPORTED;
+#endif
+}
 
 void dyn_set_timing_events(void *start_event, void *stop_event) {
     tls_events.start = static_cast<cudaEvent_t>(start_event);

@@ -14,6 +14,7 @@
 // tested per request, and two divisions serve all four unless a window boundary falls among them; the
 // window is a multiply-shift division by the invariant window length.  Requests outside the CTA's
 // window range (unsorted input) go to global atomics, so the counts are exact for any order.
+#define DYN_TU_ID 2
 #include "dyn_internal.cuh"
 
 namespace dyn {
@@ -91,7 +92,7 @@ bin_trace_kernel(const BinParams bp, const uint32_t *__restrict__ t_ms, const ui
         if (nwin > W - w_lo) nwin = W - w_lo;
     }
     const uint32_t nbins = nwin * C;                         // distinct bins held here
-    for (uint32_t i = threadIdx.x; i < nbins * kCopies; i += kThreads) sbins[i] = 0u;
+    for (uint32_t i = threadIdx.x; i < nbins * kCopies; i += kThreads) sbins[DYN_IDX(i, kSmemBins)] = 0u;
     __syncthreads();
 
     // any request, any order: window by division, dropped / shared / global by range
@@ -103,8 +104,8 @@ bin_trace_kernel(const BinParams bp, const uint32_t *__restrict__ t_ms, const ui
         }
         const uint32_t c = classify<NI, NO>(bp, a, b);
         const uint32_t rel = w - w_lo;                       // wraps for w < w_lo: then rel >= nwin
-        if (rel < nwin) atomicAdd(&sbins[(rel * C + c) * kCopies + copy], 1u);
-        else atomicAdd(&counts[size_t(w) * C + c], 1u);
+        if (rel < nwin) atomicAdd(&sbins[DYN_IDX((rel * C + c) * kCopies + copy, kSmemBins)], 1u);
+        else atomicAdd(&counts[DYN_IDX(size_t(w) * C + c, size_t(W) * C)], 1u);
     };
 
     // four consecutive requests of one lane
@@ -123,10 +124,10 @@ bin_trace_kernel(const BinParams bp, const uint32_t *__restrict__ t_ms, const ui
             }
             uint32_t *row = sbins + copy;
             const uint32_t stride = C * kCopies;
-            atomicAdd(row + r0 * stride + classify<NI, NO>(bp, va.x, vb.x) * kCopies, 1u);
-            atomicAdd(row + r1 * stride + classify<NI, NO>(bp, va.y, vb.y) * kCopies, 1u);
-            atomicAdd(row + r2 * stride + classify<NI, NO>(bp, va.z, vb.z) * kCopies, 1u);
-            atomicAdd(row + r3 * stride + classify<NI, NO>(bp, va.w, vb.w) * kCopies, 1u);
+            atomicAdd(row + DYN_IDX((r0 * stride + classify<NI, NO>(bp, va.x, vb.x) * kCopies), uint32_t(kSmemBins) - copy), 1u);
+            atomicAdd(row + DYN_IDX((r1 * stride + classify<NI, NO>(bp, va.y, vb.y) * kCopies), uint32_t(kSmemBins) - copy), 1u);
+            atomicAdd(row + DYN_IDX((r2 * stride + classify<NI, NO>(bp, va.z, vb.z) * kCopies), uint32_t(kSmemBins) - copy), 1u);
+            atomicAdd(row + DYN_IDX((r3 * stride + classify<NI, NO>(bp, va.w, vb.w) * kCopies), uint32_t(kSmemBins) - copy), 1u);
         } else {
             count_one(vt.x, va.x, vb.x, ndrop);
             count_one(vt.y, va.y, vb.y, ndrop);
@@ -139,7 +140,7 @@ bin_trace_kernel(const BinParams bp, const uint32_t *__restrict__ t_ms, const ui
     if (VEC) {
         // two full batches per pass: six 16-byte loads in flight per lane before any of them is used
         for (; base + step + kBatch <= end; base += 2 * step) {
-            const uint64_t i0 = base + uint64_t(lane) * 4, i1 = i0 + step;
+            const uint64_t i0 = DYN_IDX(base + uint64_t(lane) * 4, n_req - 3), i1 = DYN_IDX(i0 + step, n_req - 3);
             const uint4 t0 = __ldcs(reinterpret_cast<const uint4 *>(t_ms + i0));
             const uint4 a0 = __ldcs(reinterpret_cast<const uint4 *>(in_tok + i0));
             const uint4 b0 = __ldcs(reinterpret_cast<const uint4 *>(out_tok + i0));
@@ -150,7 +151,7 @@ bin_trace_kernel(const BinParams bp, const uint32_t *__restrict__ t_ms, const ui
             count_four(t1, a1, b1, my_dropped);
         }
         for (; base + kBatch <= end; base += step) {
-            const uint64_t i0 = base + uint64_t(lane) * 4;
+            const uint64_t i0 = DYN_IDX(base + uint64_t(lane) * 4, n_req - 3);
             count_four(__ldcs(reinterpret_cast<const uint4 *>(t_ms + i0)),
                        __ldcs(reinterpret_cast<const uint4 *>(in_tok + i0)),
                        __ldcs(reinterpret_cast<const uint4 *>(out_tok + i0)), my_dropped);
@@ -161,14 +162,17 @@ bin_trace_kernel(const BinParams bp, const uint32_t *__restrict__ t_ms, const ui
         const uint64_t i0 = base + uint64_t(lane) * 4;
 #pragma unroll
         for (int r = 0; r < 4; ++r)
-            if (i0 + r < end) count_one(t_ms[i0 + r], in_tok[i0 + r], out_tok[i0 + r], my_dropped);
+            if (i0 + r < end) {
+                const uint64_t ir = DYN_IDX(i0 + r, n_req);
+                count_one(t_ms[ir], in_tok[ir], out_tok[ir], my_dropped);
+            }
     }
 
     __syncthreads();
     for (uint32_t i = threadIdx.x; i < nbins; i += kThreads) {
-        const uint4 v = *reinterpret_cast<const uint4 *>(&sbins[i * kCopies]);
+        const uint4 v = *reinterpret_cast<const uint4 *>(&sbins[DYN_IDX(i * kCopies, kSmemBins - 3)]);
         const uint32_t sum = v.x + v.y + v.z + v.w;
-        if (sum) atomicAdd(&counts[size_t(w_lo) * C + i], sum);
+        if (sum) atomicAdd(&counts[DYN_IDX(size_t(w_lo) * C + i, size_t(W) * C)], sum);
     }
     };   // run_piece
 
@@ -189,7 +193,7 @@ bin_trace_kernel(const BinParams bp, const uint32_t *__restrict__ t_ms, const ui
 __global__ void counts_to_load_kernel(const uint32_t *__restrict__ counts, float *__restrict__ load, uint64_t n,
                                       float window_s) {
     for (uint64_t i = uint64_t(blockIdx.x) * blockDim.x + threadIdx.x; i < n; i += uint64_t(gridDim.x) * blockDim.x)
-        load[i] = __fdiv_rn(float(counts[i]), window_s);
+        load[DYN_IDX(i, n)] = __fdiv_rn(float(counts[DYN_IDX(i, n)]), window_s);
 }
 
 template <int NI, int NO>

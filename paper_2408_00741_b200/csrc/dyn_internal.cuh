@@ -5,6 +5,7 @@
 #include <stdint.h>
 
 #include "dynamo.h"
+#include "check.cuh"
 
 namespace dyn {
 
@@ -151,7 +152,7 @@ __device__ __forceinline__ float eval_pair(const float4 *__restrict__ row, float
     const float x = __saturatef(ln * ic) * Mf;
     const int m = int(x);
     const float nu = x - float(m);
-    const float4 e = __ldg(row + m);
+    const float4 e = __ldg(row + DYN_IDX(m, int(Mf) + 1));
     ok = fmaf(-nu, e.y, e.x) <= slo;
     return nf * fmaf(-nu, e.w, e.z);
 }

@@ -37,17 +37,19 @@ __device__ __forceinline__ float group_min(float v, unsigned mask) {
 // one multiply-add away from the bit pattern of y = 2^23 + floor(x).  Shared memory is addressed in 32 bits.
 template <bool SMEM>
 __device__ __forceinline__ float4 entry16(const char *__restrict__ ws, uint32_t base, float y) {
-    const uint32_t addr = __float_as_uint(y) * 16u + base;
+    uint32_t addr = __float_as_uint(y) * 16u + base;
     if (SMEM) {
+        addr = DYN_SMEM_ADDR(addr, 16u);
         float4 r;
         asm("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "r"(addr));
         return r;
     }
-    return __ldg(reinterpret_cast<const float4 *>(ws + addr));
+    return __ldg(reinterpret_cast<const float4 *>(ws + DYN_GLOBAL_OFF(addr, 16u)));
 }
 // 8-byte entry / 16-byte pair constants at byte address (shared) or byte offset (scratch block) `addr`
 template <bool SMEM>
 __device__ __forceinline__ float2 load8(const char *__restrict__ ws, uint32_t addr) {
+    addr = SMEM ? DYN_SMEM_ADDR(addr, 8u) : DYN_GLOBAL_OFF(addr, 8u);
     if (SMEM) {
         float2 r;
         asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(r.x), "=f"(r.y) : "r"(addr));
@@ -57,6 +59,7 @@ __device__ __forceinline__ float2 load8(const char *__restrict__ ws, uint32_t ad
 }
 template <bool SMEM>
 __device__ __forceinline__ float4 load16(const char *__restrict__ ws, uint32_t addr) {
+    addr = SMEM ? DYN_SMEM_ADDR(addr, 16u) : DYN_GLOBAL_OFF(addr, 16u);
     if (SMEM) {
         float4 r;
         asm("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "r"(addr));
@@ -111,8 +114,44 @@ __device__ __forceinline__ float row_offset_units(uint32_t bytes) {
 // load limit of the pair (or -1 where the GPU budget excludes the candidate).  Per candidate:
 //   feasible = l <= lim;  y = rz(l*icm + 2^23);  z = y*2^-146 + off  (bits(z) = address of the entry);
 //   if feasible: {a, b} = entry;  best = min(best, a + l*b).
+#ifdef DYN_CHECK
+// the checking build forms the two addresses with scalar instructions of the same rounding (bit-identical
+// results) and tests them against the staged range before the lookups
+__device__ __forceinline__ void fast_two_checked(uint64_t ln2, uint64_t icm2, uint64_t off2, float limA, float limB, float &eA,
+                                                 float &eB, bool &okA, bool &okB) {
+    float l[2], icm[2], off[2], e[2];
+    bool ok[2];
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(l[0]), "=f"(l[1]) : "l"(ln2));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(icm[0]), "=f"(icm[1]) : "l"(icm2));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(off[0]), "=f"(off[1]) : "l"(off2));
+    const float lim[2] = {limA, limB};
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        ok[k] = l[k] <= lim[k];
+        e[k] = 0.f;
+        if (ok[k]) {
+            const float y = __fmaf_rz(l[k], icm[k], 8388608.0f);
+            const float z = __fmaf_rn(y, __uint_as_float(8u), off[k]);
+            const uint32_t addr = DYN_SMEM_ADDR(__float_as_uint(z), 8u);
+            float2 en;
+            asm("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(en.x), "=f"(en.y) : "r"(addr));
+            e[k] = fmaf(l[k], en.y, en.x);
+        }
+    }
+    eA = e[0]; eB = e[1]; okA = ok[0]; okB = ok[1];
+}
+#endif
+
 __device__ __forceinline__ void fast_two(uint64_t ln2, uint64_t icm2, uint64_t off2, uint64_t two23_2, uint64_t eight2,
                                          float limA, float limB, float &bestA, float &bestB) {
+#ifdef DYN_CHECK
+    float eA, eB;
+    bool okA, okB;
+    fast_two_checked(ln2, icm2, off2, limA, limB, eA, eB, okA, okB);
+    if (okA) bestA = fminf(bestA, eA);
+    if (okB) bestB = fminf(bestB, eB);
+    return;
+#endif
     // The lookups are predicated and land in the registers that held y and z: those are defined on every
     // path, so nothing stays live around the pair loop for the sake of a skipped load (an infeasible
     // candidate forms a meaningless energy from them, which its predicated min ignores).
@@ -144,6 +183,14 @@ __device__ __forceinline__ void fast_two(uint64_t ln2, uint64_t icm2, uint64_t o
 __device__ __forceinline__ void fast_two_energy(uint64_t ln2, uint64_t icm2, uint64_t off2, uint64_t two23_2,
                                                 uint64_t eight2, float limA, float limB, float nfA, float nfB,
                                                 float &EA, float &EB) {
+#ifdef DYN_CHECK
+    float eA, eB;
+    bool okA, okB;
+    fast_two_checked(ln2, icm2, off2, limA, limB, eA, eB, okA, okB);
+    EA = okA ? eA * nfA : __int_as_float(0x7f800000);
+    EB = okB ? eB * nfB : __int_as_float(0x7f800000);
+    return;
+#endif
     asm("{\n\t"
         ".reg .pred pA, pB;\n\t"
         ".reg .f32 lA, lB, a0, b0, a1, b1, eA, eB;\n\t"

@@ -6,6 +6,7 @@
 // line in shared memory); a warp serves one class there, and a class with a table row that has no load
 // threshold (the resolve step's flags) is evaluated from the general-path tables through L1 instead, as is
 // everything when the tables do not fit.
+#define DYN_TU_ID 8
 #include "dyn_internal.cuh"
 #include "eval_dev.cuh"
 
@@ -78,6 +79,10 @@ __device__ __forceinline__ void hier_begin(const HierArgs &a) {
         const int n16 = (a.off_end - a.off_pair2) / 16;
         for (int i = threadIdx.x; i < n16; i += blockDim.x) smem[i] = src[i];
         __syncthreads();
+        DYN_SET_RANGES(uint32_t(__cvta_generic_to_shared(smem)), uint32_t(__cvta_generic_to_shared(smem)) + uint32_t(n16) * 16u,
+                       uint32_t(a.off_end));
+    } else {
+        DYN_SET_RANGES(0u, 0u, uint32_t(a.off_end));
     }
 }
 
@@ -93,7 +98,8 @@ __device__ __forceinline__ float hier_eval(const HierArgs &a, uint32_t origin, i
                        e, ok);
         return nf * e;
     }
-    return eval_pair(a.rows + (size_t(c) * P + p) * RS, __ldg(&a.pairc[c * P + p]).x, float(a.M), ln, nf, slo, ok);
+    return eval_pair(a.rows + size_t(DYN_IDX(c * P + p, a.C * P)) * RS, __ldg(&a.pairc[DYN_IDX(c * P + p, a.C * P)]).x, float(a.M), ln,
+                     nf, slo, ok);
 }
 
 
@@ -129,13 +135,13 @@ __global__ void __launch_bounds__(256) hier_nodes_kernel(const HierArgs a) {
     for (int64_t s = blockIdx.y; s < a.S; s += gridDim.y) {
         const float *ld = a.load + size_t(s) * size_t(a.W) * a.C + c;
         float PL = 0.f;
-        for (int w = w0; w < w1; ++w) PL = fmaxf(PL, ld[size_t(w) * a.C]);
+        for (int w = w0; w < w1; ++w) PL = fmaxf(PL, *DYN_PTR(ld + size_t(w) * a.C, a.load, a.S * a.W * a.C));
         int nn = -1;
         if (ml > 0.0) {
             const double q = ceil(double(PL) / ml);
             nn = q < 1.0 ? 1 : (q > 1e9 ? 1000000000 : int(q));
         }
-        a.nodes[size_t(s) * size_t(a.K1) * a.C + x] = nn;
+        a.nodes[DYN_IDX(size_t(s) * size_t(a.K1) * a.C + x, size_t(a.S) * a.K1 * a.C)] = nn;
     }
 }
 
@@ -204,8 +210,8 @@ __global__ void __launch_bounds__(256, FAST ? 4 : 1) hier_shard_kernel(const Hie
     for (int64_t s = blockIdx.y; s < a.S; s += gridDim.y) {
         const float *ld = a.load + size_t(s) * size_t(a.W) * a.C + c;
         float PL = 0.f;
-        for (int w = w0; w < w1; ++w) PL = fmaxf(PL, ld[size_t(w) * a.C]);
-        const int nn = a.nodes[size_t(s) * size_t(a.K1) * a.C + k1 * a.C + c];
+        for (int w = w0; w < w1; ++w) PL = fmaxf(PL, *DYN_PTR(ld + size_t(w) * a.C, a.load, a.S * a.W * a.C));
+        const int nn = a.nodes[DYN_IDX(size_t(s) * size_t(a.K1) * a.C + k1 * a.C + c, size_t(a.S) * a.K1 * a.C)];
         int budget = nn > 0 ? (nn > a.Nmax ? cap_budget : nn * tpmax) : 0;
         if (a.space_budget > 0 && budget > a.space_budget) budget = a.space_budget;
         int nmax = budget / a.tp[0];                  // no n above this fits even the smallest TP
@@ -225,7 +231,7 @@ __global__ void __launch_bounds__(256, FAST ? 4 : 1) hier_shard_kernel(const Hie
             int bn = 0;
             for (; n <= nmax; n += 2) {
                 if (float(n) * e_floor >= best) break;       // n and every larger count cost at least `best`
-                const float lnA = PL * s_rn[n], lnB = n + 1 <= nmax ? PL * s_rn[n + 1] : CUDART_INF_F;
+                const float lnA = PL * s_rn[DYN_IDX(n, 257)], lnB = n + 1 <= nmax ? PL * s_rn[DYN_IDX(n + 1, 257)] : CUDART_INF_F;
                 const uint64_t ln2 = pack2(lnA, lnB);
                 float eA = CUDART_INF_F, eB = CUDART_INF_F;
 #pragma unroll
@@ -260,7 +266,7 @@ __global__ void __launch_bounds__(256, FAST ? 4 : 1) hier_shard_kernel(const Hie
                 }
             }
         }
-        a.shard[size_t(s) * size_t(a.K2) * a.C + x] = bnt;
+        a.shard[DYN_IDX(size_t(s) * size_t(a.K2) * a.C + x, size_t(a.S) * a.K2 * a.C)] = bnt;
     }
 }
 
@@ -292,13 +298,14 @@ __global__ void __launch_bounds__(256) hier_freq_kernel(const HierArgs a) {
     int32_t *out_idx = a.best_idx + x;
     float *out_E = a.best_E + x;
     for (int64_t s = blockIdx.y; s < a.S; s += gridDim.y) {
-        const int nt = sh[size_t(s) * shard_stride];
+        const int nt = *DYN_PTR(sh + size_t(s) * shard_stride, a.shard, a.S * int64_t(shard_stride));
         int32_t bj = -1;
         float best = CUDART_INF_F;
         if (nt >= 0) {
             const int n1 = int(fastdiv(uint32_t(nt), a.divT)), t = nt - n1 * a.T;
             const float nf = float(n1 + 1);
-            const float ln = fmaxf(ld[size_t(s) * tile_stride], 0.f) * (n1 < 256 ? s_rn[n1 + 1] : 1.0f / nf);
+            const float ln = fmaxf(*DYN_PTR(ld + size_t(s) * tile_stride, a.load, a.S * int64_t(tile_stride)), 0.f) *
+                             (n1 < 256 ? s_rn[DYN_IDX(n1 + 1, 257)] : 1.0f / nf);
             if (FAST && !general) {
                 uint32_t pc_addr = pair_c + uint32_t(t * a.F) * 16u;
                 uint32_t row = rows_c + uint32_t(t * a.F) * row_step;
@@ -329,8 +336,8 @@ __global__ void __launch_bounds__(256) hier_freq_kernel(const HierArgs a) {
                 }
             }
         }
-        out_idx[size_t(s) * tile_stride] = bj;
-        out_E[size_t(s) * tile_stride] = best;
+        out_idx[DYN_IDX(size_t(s) * tile_stride, size_t(a.S) * tile_stride - x)] = bj;
+        out_E[DYN_IDX(size_t(s) * tile_stride, size_t(a.S) * tile_stride - x)] = best;
     }
 }
 

@@ -17,6 +17,7 @@
 // recovers the frequencies of the winning tuple afterwards with the same arithmetic; otherwise a plain
 // variant evaluates from the general-path tables through L1.  Both are launched; each looks at the flags
 // and only the one they select does the work.
+#define DYN_TU_ID 9
 #include "dyn_internal.cuh"
 #include "eval_dev.cuh"
 
@@ -53,7 +54,7 @@ __global__ void mixed_caph_kernel(const MixedArgs a) {
     if (i >= a.C * a.T) return;
     const int c = i / a.T, t = i - c * a.T;
     const float4 *pair2 = reinterpret_cast<const float4 *>(a.ws + a.off_pair2);
-    a.caph[i] = pair2[c * (a.T * a.F) + t * a.F + a.F - 1].w;
+    a.caph[i] = pair2[DYN_IDX(c * (a.T * a.F) + t * a.F + a.F - 1, a.C * a.T * a.F)].w;
 }
 
 // true when every pair row has a load threshold (vlim is NaN for a row whose TBT decreases somewhere)
@@ -68,7 +69,7 @@ __global__ void mixed_inva_kernel(const MixedArgs a) {
     const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
     if (i >= int64_t(a.C) * a.K) return;
     const int c = int(i / a.K);
-    const uint32_t tup = a.tuples[i - int64_t(c) * a.K].x;
+    const uint32_t tup = a.tuples[DYN_IDX(i - int64_t(c) * a.K, a.K)].x;
     double A = 0.0;
     for (int t = 0; t < a.T; ++t) A += double((tup >> (8 * t)) & 255u) * double(a.caph[c * a.T + t]);
     a.inva[i] = float(1.0 / A);                              // +inf when no degree of the tuple has capacity: infeasible
@@ -83,8 +84,8 @@ __global__ void __launch_bounds__(kThreads) mixed_select_kernel(const MixedArgs 
     const int64_t nwarps = int64_t(gridDim.x) * kWarps;
     for (int64_t i = int64_t(blockIdx.x) * kWarps + (threadIdx.x >> 5); i < a.tiles; i += nwarps) {
         const int c = int(i % a.C);
-        const float L = fmaxf(a.load[i], 0.f);              // negative / NaN -> 0
-        const float slo = a.slo[c];
+        const float L = fmaxf(a.load[DYN_IDX(i, a.tiles)], 0.f);              // negative / NaN -> 0
+        const float slo = a.slo[DYN_IDX(c, a.C)];
         float caph[T];
 #pragma unroll
         for (int t = 0; t < T; ++t) caph[t] = a.caph[c * T + t];
@@ -92,7 +93,7 @@ __global__ void __launch_bounds__(kThreads) mixed_select_kernel(const MixedArgs 
         uint32_t bnum = 0xffffffffu, btup = 0;               // number and counts of the lane's best tuple
         uint32_t bq = 0;                                     // its frequencies, 8 bits per TP index
         for (int64_t k = lane; k < a.K; k += 32) {
-            const uint2 tk = __ldg(a.tuples + k);
+            const uint2 tk = __ldg(a.tuples + DYN_IDX(k, a.K));
             const uint32_t tup = tk.x;
             float A = 0.f;
 #pragma unroll
@@ -105,8 +106,8 @@ __global__ void __launch_bounds__(kThreads) mixed_select_kernel(const MixedArgs 
                 const uint32_t n = (tup >> (8 * t)) & 255u;
                 if (n == 0) continue;
                 const float l = frac * caph[t], nf = float(n);
-                const float4 *rows_t = a.rows + (size_t(c) * P + t * a.F) * RS;
-                const float2 *pc_t = a.pairc + c * P + t * a.F;
+                const float4 *rows_t = a.rows + size_t(DYN_IDX(c * P + t * a.F, a.C * P - a.F + 1)) * RS;
+                const float2 *pc_t = a.pairc + DYN_IDX(c * P + t * a.F, a.C * P - a.F + 1);
                 float eg = CUDART_INF_F;
                 uint32_t qg = 0;
                 for (int q = 0; q < a.F; ++q) {
@@ -134,11 +135,11 @@ __global__ void __launch_bounds__(kThreads) mixed_select_kernel(const MixedArgs 
         const uint32_t kmin = __reduce_min_sync(kFull, best == Emin ? bnum : 0xffffffffu);
         if (Emin == CUDART_INF_F) {
             if (lane < T) {
-                a.counts[i * T + lane] = -1;
-                a.freq[i * T + lane] = -1;
+                a.counts[DYN_IDX(i * T + lane, a.tiles * T)] = -1;
+                a.freq[DYN_IDX(i * T + lane, a.tiles * T)] = -1;
             }
             if (lane == 0) {
-                a.tuple[i] = -1;
+                a.tuple[DYN_IDX(i, a.tiles)] = -1;
                 a.best_E[i] = CUDART_INF_F;
             }
             continue;
@@ -147,10 +148,10 @@ __global__ void __launch_bounds__(kThreads) mixed_select_kernel(const MixedArgs 
 #pragma unroll
             for (int t = 0; t < T; ++t) {
                 const uint32_t n = (btup >> (8 * t)) & 255u;
-                a.counts[i * T + t] = int32_t(n);
+                a.counts[DYN_IDX(i * T + t, a.tiles * T)] = int32_t(n);
                 a.freq[i * T + t] = n ? int32_t((bq >> (8 * t)) & 255u) : -1;
             }
-            a.tuple[i] = int32_t(kmin);
+            a.tuple[DYN_IDX(i, a.tiles)] = int32_t(kmin);
             a.best_E[i] = Emin;
         }
     }
@@ -167,6 +168,8 @@ __global__ void __launch_bounds__(kThreads, 3) mixed_fast_kernel(const MixedArgs
         const int n16 = (a.off_end - a.off_pair2) / 16;
         for (int i = threadIdx.x; i < n16; i += blockDim.x) smem[i] = src[i];
         __syncthreads();
+        DYN_SET_RANGES(uint32_t(__cvta_generic_to_shared(smem)), uint32_t(__cvta_generic_to_shared(smem)) + uint32_t(n16) * 16u,
+                       uint32_t(a.off_end));
     }
     uint32_t origin = table_origin<true>();
     asm volatile("" : "+r"(origin) : : "memory");        // table loads stay behind the staging barrier
@@ -197,7 +200,7 @@ __global__ void __launch_bounds__(kThreads, 3) mixed_fast_kernel(const MixedArgs
                 tup[j] = tk.x;
                 num[j] = tk.y;
                 // every instance runs at this fraction of its top-frequency capacity
-                frac[j] = k < a.K ? L * __ldg(a.inva + int64_t(c) * a.K + k) : 0.f;
+                frac[j] = k < a.K ? L * __ldg(a.inva + DYN_IDX(int64_t(c) * a.K + k, int64_t(a.C) * a.K)) : 0.f;
                 E[j] = tk.x ? 0.f : CUDART_INF_F;            // a slot past the end of the list never wins
             }
 #pragma unroll
@@ -220,7 +223,7 @@ __global__ void __launch_bounds__(kThreads, 3) mixed_fast_kernel(const MixedArgs
 #pragma unroll 4
                 for (int q = 0; q < F; ++q) {
                     uint64_t icm2, lim2;
-                    asm("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(icm2), "=l"(lim2) : "r"(cpair + uint32_t(q) * 16u));
+                    asm("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(icm2), "=l"(lim2) : "r"(DYN_SMEM_ADDR(cpair + uint32_t(q) * 16u, 16u)));
                     const float lim = __uint_as_float(uint32_t(lim2));
                     fast_two(lnA, icm2, off2, two23_2, eight2, lim, lim, e1[0], e1[1]);
                     fast_two(lnB, icm2, off2, two23_2, eight2, lim, lim, e1[2], e1[3]);
@@ -244,11 +247,11 @@ __global__ void __launch_bounds__(kThreads, 3) mixed_fast_kernel(const MixedArgs
         const uint32_t kmin = __reduce_min_sync(kFull, best == Emin ? bnum : 0xffffffffu);
         if (Emin == CUDART_INF_F) {
             if (lane < T) {
-                a.counts[i * T + lane] = -1;
-                a.freq[i * T + lane] = -1;
+                a.counts[DYN_IDX(i * T + lane, a.tiles * T)] = -1;
+                a.freq[DYN_IDX(i * T + lane, a.tiles * T)] = -1;
             }
             if (lane == 0) {
-                a.tuple[i] = -1;
+                a.tuple[DYN_IDX(i, a.tiles)] = -1;
                 a.best_E[i] = CUDART_INF_F;
             }
             continue;
@@ -291,10 +294,10 @@ __global__ void __launch_bounds__(kThreads, 3) mixed_fast_kernel(const MixedArgs
 #pragma unroll
             for (int t = 0; t < T; ++t) {
                 const uint32_t n = (wt >> (8 * t)) & 255u;
-                a.counts[i * T + t] = int32_t(n);
+                a.counts[DYN_IDX(i * T + t, a.tiles * T)] = int32_t(n);
                 a.freq[i * T + t] = n ? gq[t] : -1;
             }
-            a.tuple[i] = int32_t(kmin);
+            a.tuple[DYN_IDX(i, a.tiles)] = int32_t(kmin);
             a.best_E[i] = Emin;
         }
     }

@@ -1,5 +1,6 @@
 // Whole path from host buffers: copy in, bin, evaluate + select, totals, copy out.  Device memory is
 // carved from the caller's arena; nothing is allocated here.
+#define DYN_TU_ID 6
 #include "dyn_internal.cuh"
 
 namespace {

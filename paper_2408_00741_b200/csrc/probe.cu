@@ -15,6 +15,7 @@
 //                             sweep's time.
 //
 // The caller times the launches (events on the stream, or dyn_set_timing_events).
+#define DYN_TU_ID 12
 #include "dyn_internal.cuh"
 #include "eval_dev.cuh"
 
@@ -62,6 +63,8 @@ sweep_inner_probe_kernel(const int iters, const float scale, const float feasibl
     for (int i = threadIdx.x; i < kProbeP * RS; i += blockDim.x)
         rows2[i] = make_float2(1.0f + float(i % RS), 0.5f + 0.001f * float(i / RS));
     __syncthreads();
+    DYN_SET_RANGES(uint32_t(__cvta_generic_to_shared(smem)),
+                   uint32_t(__cvta_generic_to_shared(smem)) + uint32_t(kProbeP) * 16u + uint32_t(kProbeP * RS) * 8u, 0u);
     uint32_t origin = table_origin<true>();
     asm volatile("" : "+r"(origin) : : "memory");
     const uint32_t cpair = origin;
@@ -121,6 +124,15 @@ __global__ void self_check_kernel(const float m_plus_two23, const uint32_t bytes
     g_self_check = (__float_as_uint(z) == want) ? 1 : 2;
 }
 
+#ifdef DYN_CHECK
+// a planted violation: index 5 into an array of 3, which the check records and replaces by 0
+__global__ void check_selftest_kernel(int *out) {
+    int a[3] = {7, 8, 9};
+    const int i = DYN_IDX(5 + int(threadIdx.x), 3);
+    *out = a[i];
+}
+#endif
+
 }  // namespace
 
 }  // namespace dyn
@@ -128,6 +140,19 @@ __global__ void self_check_kernel(const float m_plus_two23, const uint32_t bytes
 using namespace dyn;
 
 extern "C" {
+
+int dyn_debug_selftest(int32_t *d_out, void *stream) {
+#ifdef DYN_CHECK
+    if (!d_out) return DYN_EINVAL;
+    check_selftest_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(d_out);
+    DYN_CUDA_TRY(cudaGetLastError());
+    return DYN_OK;
+#else
+    (void)d_out;
+    (void)stream;
+    return DYN_EUNSUPPORTED;
+#endif
+}
 
 int dyn_self_check(void *stream) {
     cudaStream_t st = static_cast<cudaStream_t>(stream);

@@ -13,6 +13,7 @@
 //                       to their minimum, which is accumulated in fp64, so that fp32 holds only differences.
 //   reconf_back_kernel  the walk back, one warp per (scenario, class): it finds each predecessor again with the
 //                       same addition (lowest source on ties) and writes the chosen candidates.
+#define DYN_TU_ID 10
 #include "dyn_internal.cuh"
 
 #include <cuda_pipeline.h>
@@ -54,14 +55,14 @@ __global__ void __launch_bounds__(kThreads) reconf_cost_kernel(const ReconfArgs 
         const int c = int(sc % a.C);
         const int64_t s = sc / a.C;
         const int n = g / a.T + 1, t = g - (n - 1) * a.T;
-        const float L = fmaxf(a.load[(s * a.W + w) * a.C + c], 0.f);
+        const float L = fmaxf(a.load[DYN_IDX((s * a.W + w) * a.C + c, a.S * a.W * a.C)], 0.f);
         const float nf = float(n), ln = L * (1.0f / nf);
         const float slo = a.slo[c];
         float best = CUDART_INF_F;
         int bq = 0;
         if (a.budget <= 0 || int64_t(n) * a.tp[t] <= int64_t(a.budget)) {
-            const float4 *rows_t = a.rows + (size_t(c) * P + t * a.F) * RS;
-            const float2 *pc_t = a.pairc + c * P + t * a.F;
+            const float4 *rows_t = a.rows + size_t(DYN_IDX(c * P + t * a.F, a.C * P - a.F + 1)) * RS;
+            const float2 *pc_t = a.pairc + DYN_IDX(c * P + t * a.F, a.C * P - a.F + 1);
             for (int q = 0; q < a.F; ++q) {
                 bool ok;
                 const float E = eval_pair(rows_t + size_t(q) * RS, __ldg(pc_t + q).x, Mf, ln, nf, slo, ok);
@@ -71,8 +72,8 @@ __global__ void __launch_bounds__(kThreads) reconf_cost_kernel(const ReconfArgs 
                 }
             }
         }
-        a.cost[e] = best;
-        a.qbest[e] = uint8_t(bq);
+        a.cost[DYN_IDX(e, total)] = best;
+        a.qbest[DYN_IDX(e, total)] = uint8_t(bq);
     }
 }
 
@@ -133,7 +134,8 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
     // t0..t3 and plane 1 the same for t2, t3, so that the lanes of a warp read neighbouring 16-byte pieces
     for (int i = tid; i < rows_s * RSd; i += kPathThreads) {
         const int h = i / RSd, g = i - h * RSd, j = g & 3;
-        Rs[size_t(h >> 1) * (2 * RSd) + (j >> 1) * RSd + (g & ~3) + (j & 1) * 2 + (h & 1)] = g < NS ? a.R[size_t(h) * NS + g] : 0.f;
+        Rs[DYN_IDX(size_t(h >> 1) * (2 * RSd) + (j >> 1) * RSd + (g & ~3) + (j & 1) * 2 + (h & 1), size_t(rows_s) * RSd)] =
+            g < NS ? a.R[DYN_IDX(size_t(h) * NS + g, size_t(NS) * NS)] : 0.f;
     }
     // rows of R that do not fit in shared memory: the first G * kRegRows of them stay in registers, each source
     // group holding kRegRows rows (its four columns of them); any further rows are read through L1 / L2
@@ -148,7 +150,7 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
             const bool have = worker && h < NS;              // no such row: +inf never wins
             const float *row = a.R + size_t(h) * NS + 4 * tg;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) v[i][j] = have ? (4 * tg + j < NS ? __ldg(row + j) : 0.f) : CUDART_INF_F;
+            for (int j = 0; j < 4; ++j) v[i][j] = have ? (4 * tg + j < NS ? __ldg(DYN_PTR(row + j, a.R, int64_t(NS) * NS)) : 0.f) : CUDART_INF_F;
         }
         rp0[k] = make_float4(v[0][0], v[1][0], v[0][1], v[1][1]);
         rp1[k] = make_float4(v[0][2], v[1][2], v[0][3], v[1][3]);
@@ -200,14 +202,14 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
         const float shift = (mprev < CUDART_INF_F) ? mprev : 0.f;
         base += double(shift);
         if (tid == 0) s_min[w & 1] = 0xffffffffu;            // this window's slot; last read before the previous barrier
-        for (int g = tid; g < NS; g += kPathThreads) hist[(w - 1) * NS + g] = Dp[g] - shift;
+        for (int g = tid; g < NS; g += kPathThreads) hist[DYN_IDX((w - 1) * NS + g, W * NS)] = Dp[DYN_IDX(g, NS4)] - shift;
         if (worker) {
             float b0 = CUDART_INF_F, b1 = CUDART_INF_F, b2 = CUDART_INF_F, b3 = CUDART_INF_F;
             const float2 nshift = make_float2(-shift, -shift);                  // d + (-shift) is d - shift bit for bit
 #pragma unroll 1
             for (int q = q_lo; q < q_hi; ++q) {
-                const float4 d4 = reinterpret_cast<const float4 *>(Dp)[q];
-                const float *rq = Rs + size_t(2 * q) * (2 * RSd) + 4 * tg;
+                const float4 d4 = reinterpret_cast<const float4 *>(Dp)[DYN_IDX(q, TG)];
+                const float *rq = Rs + DYN_IDX(size_t(2 * q) * (2 * RSd) + 4 * tg, size_t(rows_s) * RSd - 3 * RSd - 3);
                 relax_pair(b0, b1, b2, b3, __fadd2_rn(make_float2(d4.x, d4.y), nshift), *reinterpret_cast<const float4 *>(rq),
                            *reinterpret_cast<const float4 *>(rq + RSd));
                 relax_pair(b0, b1, b2, b3, __fadd2_rn(make_float2(d4.z, d4.w), nshift), *reinterpret_cast<const float4 *>(rq + 2 * RSd),
@@ -229,7 +231,7 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
                 if (4 * tg + 2 < NS) b2 = fminf(b2, d + __ldg(row + 2));
                 if (4 * tg + 3 < NS) b3 = fminf(b3, d + __ldg(row + 3));
             }
-            reinterpret_cast<float4 *>(part + size_t(hg) * NS4)[tg] = make_float4(b0, b1, b2, b3);
+            reinterpret_cast<float4 *>(part + size_t(DYN_IDX(hg, G)) * NS4)[DYN_IDX(tg, TG)] = make_float4(b0, b1, b2, b3);
         }
         __syncthreads();                                     // every reader of Dp is done; the partial minima are in
         float lmin = CUDART_INF_F;
@@ -239,17 +241,18 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
         for (int o = 0; o < kOwn; ++o) {
             const int g = tid + o * kPathThreads;
             if (g < NS) {
-                float best = part[g];
-                for (int k = 1; k < G; ++k) best = fminf(best, part[k * NS4 + g]);
-                const float d = cslot[g] + best;
-                Dp[g] = d;
+                float best = part[DYN_IDX(g, NS4)];
+                for (int k = 1; k < G; ++k) best = fminf(best, part[DYN_IDX(k * NS4 + g, G * NS4)]);
+                const float d = cslot[DYN_IDX(g, NS4)] + best;
+                Dp[DYN_IDX(g, NS4)] = d;
                 lmin = fminf(lmin, d);
             }
         }
         publish_min(lmin, int(w & 1));
         // the slot is free (its values went into the minimum just published): ask for the costs kRing windows on
         if (w + kRing < W)
-            for (int g = tid; g < NS; g += kPathThreads) __pipeline_memcpy_async(cslot + g, cost + (w + kRing) * NS + g, 4);
+            for (int g = tid; g < NS; g += kPathThreads)
+                __pipeline_memcpy_async(cslot + g, cost + DYN_IDX((w + kRing) * NS + g, W * NS), 4);
         __pipeline_commit();
         __syncthreads();                                     // publishes Dp and the minimum
     }
@@ -259,7 +262,7 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
         return;
     }
     // the last window's vector goes to the row of `hist` that the recursion leaves free; the walk back starts there
-    for (int g = tid; g < NS; g += kPathThreads) hist[(W - 1) * NS + g] = Dp[g];
+    for (int g = tid; g < NS; g += kPathThreads) hist[DYN_IDX((W - 1) * NS + g, W * NS)] = Dp[g];
     if (tid == 0) a.path_total[sc] = (m < CUDART_INF_F) ? base + double(m) : double(CUDART_INF_F);
 }
 
@@ -273,7 +276,7 @@ __global__ void reconf_transpose_kernel(const ReconfArgs a) {
     const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
     if (i >= int64_t(a.NS) * a.NS) return;
     const int g = int(i / a.NS), h = int(i - int64_t(g) * a.NS);
-    a.Rt[i] = a.R[size_t(h) * a.NS + g];
+    a.Rt[i] = a.R[DYN_IDX(size_t(h) * a.NS + g, size_t(a.NS) * a.NS)];
 }
 
 constexpr int kBackWarps = 1;
@@ -331,10 +334,10 @@ __global__ void __launch_bounds__(kBackThreads) reconf_back_kernel(const ReconfA
     const bool ahead = NS <= 256;
     float *ring = Rts + size_t(rows_b) * NS;                 // [kBackRing][256]
     auto ask = [&](int64_t row, int slot) {                  // entries of vector `row` (clamped; rows < 0 are never used)
-        const float *src = hist + (row > 0 ? row : 0) * NS;
+        const float *src = hist + DYN_IDX(row > 0 ? row : 0, W) * NS;
 #pragma unroll
         for (int j = 0; j < 8; ++j)
-            if (lane + 32 * j < NS) __pipeline_memcpy_async(ring + slot * 256 + lane + 32 * j, src + lane + 32 * j, 4);
+            if (lane + 32 * j < NS) __pipeline_memcpy_async(ring + DYN_IDX(slot, kBackRing) * 256 + lane + 32 * j, src + lane + 32 * j, 4);
         __pipeline_commit();
     };
     if (ahead)
@@ -350,14 +353,14 @@ __global__ void __launch_bounds__(kBackThreads) reconf_back_kernel(const ReconfA
         for (int k = 0; k < 8; ++k) {
             const int64_t w = wb - k;
             if (w >= 0) {
-                if (lane == 0) path[seg_hi - 1 - w] = cur;
+                if (lane == 0) path[DYN_IDX(seg_hi - 1 - w, kBackChunk)] = cur;
                 if (ahead) __pipeline_wait_prior(kBackRing - 1);        // this window's vector has arrived
                 if (cur >= 0 && w > 0) {
                     float mm;
                     uint32_t arg = 0xffffffffu;
                     if (ahead) {
                         if (rcol_of != cur) {                // warp-uniform
-                            const float *col = cur < rows_b ? Rts + size_t(cur) * NS : Rt + size_t(cur) * NS;
+                            const float *col = cur < rows_b ? Rts + size_t(cur) * NS : Rt + size_t(DYN_IDX(cur, NS)) * NS;
 #pragma unroll
                             for (int j = 0; j < 8; ++j) rcol[j] = lane + 32 * j < NS ? col[lane + 32 * j] : CUDART_INF_F;
                             rcol_of = cur;
@@ -395,11 +398,11 @@ __global__ void __launch_bounds__(kBackThreads) reconf_back_kernel(const ReconfA
         if (seg_hi - lo >= kBackChunk || lo == 0) {
             __syncwarp();
             for (int64_t w = lo + lane; w < seg_hi; w += 32) {
-                const int g = path[seg_hi - 1 - w];
-                const int64_t i = (s * W + w) * a.C + c;
+                const int g = path[DYN_IDX(seg_hi - 1 - w, kBackChunk)];
+                const int64_t i = DYN_IDX((s * W + w) * a.C + c, a.S * W * a.C);
                 if (g >= 0) {
-                    a.best_idx[i] = g * a.F + int(a.qbest[sc * W * NS + w * NS + g]);
-                    a.best_E[i] = cost[w * NS + g];
+                    a.best_idx[i] = g * a.F + int(a.qbest[DYN_IDX(sc * W * NS + w * NS + g, a.S * a.C * W * NS)]);
+                    a.best_E[i] = cost[DYN_IDX(w * NS + g, W * NS)];
                 } else {
                     a.best_idx[i] = -1;
                     a.best_E[i] = CUDART_INF_F;

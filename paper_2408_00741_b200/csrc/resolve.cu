@@ -7,6 +7,7 @@
 // value and slope of TBT and of the per-instance window energy, plus the scale from per-instance load
 // to table position.  Interpolating in f here and in u inside the sweep equals the bilinear
 // interpolation of the definition.
+#define DYN_TU_ID 3
 #include "dyn_internal.cuh"
 
 namespace dyn {
@@ -68,6 +69,7 @@ __global__ void resolve_kernel(const ResolveParams rp, float4 *__restrict__ rows
         const int r = rp.row[q];
         const double w = double(rp.weight[q]);
         const size_t ct = (size_t(c) * rp.T + t) * rp.R;
+        (void)DYN_IDX(ct + r + 1, size_t(rp.C) * rp.T * rp.R);        // rows r and r + 1 of the profile tables exist
         const float *tb0 = rp.d_tbt + (ct + r) * M, *tb1 = tb0 + M;
         const float *pw0 = rp.d_pow + (ct + r) * M, *pw1 = pw0 + M;
         const double ttft = lerp64(rp.d_ttft[ct + r], rp.d_ttft[ct + r + 1], w);
@@ -88,7 +90,7 @@ __global__ void resolve_kernel(const ResolveParams rp, float4 *__restrict__ rows
             v = make_float4(kInf, 0.f, float(pw_m), 0.f);
         }
         if (!pair_ok) v.x = kInf;
-        rows[(size_t(c) * P + p) * RS + m] = v;
+        rows[DYN_IDX((size_t(c) * P + p) * RS + m, size_t(total))] = v;
         // threshold path: the same energy as a line in the per-instance load l, e(l) = a + l*b (x = l*(M-1)/cap);
         // the lines of neighbouring segments meet at the knots, so a position that rounding puts on
         // either side of a knot gets the same value
@@ -97,7 +99,7 @@ __global__ void resolve_kernel(const ResolveParams rp, float4 *__restrict__ rows
             const double d = lerp64(pw0[m + 1], pw1[m + 1], w) * scale - pw_m;
             line = make_float2(float(pw_m - double(m) * d), float(d * double(M - 1) / cap));
         }
-        rows2[(size_t(c) * P + p) * RS + m] = line;
+        rows2[DYN_IDX((size_t(c) * P + p) * RS + m, size_t(total))] = line;
         if (m == 0) {
             // Load threshold of the pair.  TBT is piecewise linear along the row, so {x : TBT(x) <= slo} is a
             // union of intervals; when it is empty or one interval that starts at x = 0, "TBT <= slo and
@@ -130,13 +132,13 @@ __global__ void resolve_kernel(const ResolveParams rp, float4 *__restrict__ rows
             if (!single) xlim = -1.0;            // the threshold path skips this row; the general path serves it
             if (pair_ok && xlim >= 0.0) vlim = xlim / double(M);
             // x = u*(M-1) is formed as sat(L/n * ic) * M, so that saturation at 1 means x = M
-            pairc[size_t(c) * P + p] = make_float2(pair_ok ? float(double(M - 1) / (double(M) * cap)) : 0.f,
+            pairc[DYN_IDX(size_t(c) * P + p, size_t(rp.C) * P)] = make_float2(pair_ok ? float(double(M - 1) / (double(M) * cap)) : 0.f,
                                                    single ? float(vlim) : __int_as_float(0x7fc00000));
             // threshold path: table position per unit of per-instance load (twice: the sweep uses it as a
             // packed pair) and the largest per-instance load within the SLO and the capacity
             const float icm = pair_ok ? float(double(M - 1) / cap) : 0.f;
             const float llim = (pair_ok && xlim >= 0.0) ? float(xlim / double(M - 1) * cap) : -1.f;
-            pair2[size_t(c) * P + p] = make_float4(icm, icm, llim, float(cap));   // cap as interpolated, feasible or not
+            pair2[DYN_IDX(size_t(c) * P + p, size_t(rp.C) * P)] = make_float4(icm, icm, llim, float(cap));   // cap as interpolated, feasible or not
             if (p == 0) slo[c] = rp.slo_tbt[c];
             if (c == 0 && p < rp.T) tp[p] = rp.tp[p];
         }

@@ -9,6 +9,7 @@
 // lane keeps its first minimum, then two warp-wide integer min-reductions pick (energy, index).
 // totals: fp64 sums in a fixed order (thread: the classes of its window in order; block: a fixed tree
 // over 256 windows; scenario: chunks in order), so results repeat bit for bit.
+#define DYN_TU_ID 5
 #include "dyn_internal.cuh"
 
 #include <math_constants.h>
@@ -34,7 +35,7 @@ select_kernel(const float *__restrict__ E, int64_t tiles, int J, int32_t *__rest
     const int lane = threadIdx.x & 31;
     const int64_t nwarps = int64_t(gridDim.x) * kWarps;
     for (int64_t i = int64_t(blockIdx.x) * kWarps + (threadIdx.x >> 5); i < tiles; i += nwarps) {
-        const float *row = E + size_t(i) * size_t(J);
+        const float *row = E + size_t(DYN_IDX(i, tiles)) * size_t(J);
         float best = CUDART_INF_F;
         int bj = 0x7fffffff;
         if (VEC4) {
@@ -42,7 +43,7 @@ select_kernel(const float *__restrict__ E, int64_t tiles, int J, int32_t *__rest
             const int J4 = J >> 2;
 #pragma unroll 4
             for (int q = lane; q < J4; q += 32) {
-                const float4 v = __ldcs(row4 + q);
+                const float4 v = __ldcs(row4 + DYN_IDX(q, J4));
                 const int j = q << 2;
                 if (v.x < best) { best = v.x; bj = j; }
                 if (v.y < best) { best = v.y; bj = j + 1; }
@@ -52,7 +53,7 @@ select_kernel(const float *__restrict__ E, int64_t tiles, int J, int32_t *__rest
         } else {
 #pragma unroll 4
             for (int j = lane; j < J; j += 32) {
-                const float v = __ldcs(row + j);
+                const float v = __ldcs(row + DYN_IDX(j, J));
                 if (v < best) { best = v; bj = j; }
             }
         }
@@ -97,20 +98,20 @@ __global__ void __launch_bounds__(kThreads) totals_partial_kernel(const TotalsAr
     for (int c = 0; c < a.C; ++c) {                 // every lane takes every trip: the match below is warp-wide
         int32_t j = -1;
         if (have) {
-            j = a.o.best_idx[base + c];
+            j = a.o.best_idx[DYN_IDX(base + c, size_t(a.S) * a.W * a.C)];
             if (j < 0) ++bad;
-            else ew += double(a.o.best_E[base + c]);
+            else ew += double(a.o.best_E[DYN_IDX(base + c, size_t(a.S) * a.W * a.C)]);
         }
         if (a.o.hist) {
             // neighbouring windows of a class often choose the same candidate: one atomic per distinct
             // candidate in the warp, by the lowest lane that holds it
             const unsigned peers = __match_any_sync(kFull, j);
             if (j >= 0 && lane == __ffs(peers) - 1)
-                atomicAdd(&a.o.hist[size_t(s) * size_t(a.J) + size_t(j)], uint32_t(__popc(peers)));
+                atomicAdd(&a.o.hist[size_t(s) * size_t(a.J) + size_t(DYN_IDX(j, a.J))], uint32_t(__popc(peers)));
         }
         if (a.o.gpus && j >= 0) {
-            if (a.nj) g += uint32_t(a.nj[j] * a.tj[j]);
-            else g += uint32_t((j / TF + 1) * a.tp[(j / a.F) % a.T]);
+            if (a.nj) g += uint32_t(a.nj[DYN_IDX(j, a.J)] * a.tj[DYN_IDX(j, a.J)]);
+            else g += uint32_t((j / TF + 1) * a.tp[DYN_IDX((j / a.F) % a.T, a.T)]);
         }
     }
     if (have) {
@@ -139,8 +140,8 @@ __global__ void totals_final_kernel(const TotalsArgs a) {
     double sum = 0.0;
     uint32_t bad = 0;
     for (int64_t ch = 0; ch < a.chunks; ++ch) {
-        sum += a.partial[s * a.chunks + ch];
-        bad += a.partial_bad[s * a.chunks + ch];
+        sum += a.partial[DYN_IDX(s * a.chunks + ch, a.S * a.chunks)];
+        bad += a.partial_bad[DYN_IDX(s * a.chunks + ch, a.S * a.chunks)];
     }
     a.o.E_total[s] = sum;
     a.o.n_infeasible[s] = bad;

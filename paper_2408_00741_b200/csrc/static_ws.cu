@@ -1,5 +1,6 @@
 // dyn_eval_select_static: the fused evaluate+select call for callers that cannot allocate device
 // memory.  Its scratch is a fixed array in the library image instead of a caller workspace.
+#define DYN_TU_ID 7
 #include "dyn_internal.cuh"
 
 #include <mutex>

@@ -34,6 +34,7 @@
 //     re-evaluating that instance count for 32 pairs at a time with bit-identical arithmetic.
 // The resolved tables of all classes are staged in shared memory once per CTA when they fit; larger
 // tables are read through L1 or staged per class.
+#define DYN_TU_ID 4
 #include "dyn_internal.cuh"
 #include "eval_dev.cuh"
 
@@ -91,8 +92,11 @@ __device__ __forceinline__ void stage(const SweepArgs &a, int from, int to) {
     extern __shared__ float4 smem[];
     const float4 *src = reinterpret_cast<const float4 *>(a.ws + from);
     const int n16 = (to - from) / 16;
-    for (int i = threadIdx.x; i < n16; i += blockDim.x) smem[i] = src[i];
+    for (int i = threadIdx.x; i < n16; i += blockDim.x) smem[DYN_IDX(i, a.smem_bytes / 16)] = src[i];
     __syncthreads();
+    // (checking build) the range the arithmetically formed table addresses must stay in
+    DYN_SET_RANGES(uint32_t(__cvta_generic_to_shared(smem)), uint32_t(__cvta_generic_to_shared(smem)) + uint32_t(to - from),
+                   uint32_t(a.off_end));
 }
 
 // number of pair rows among [first, first + n) without a load threshold (the resolve step stores NaN as
@@ -267,7 +271,7 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
             float ln[NCH];
 #pragma unroll
             for (int t = 0; t < TT; ++t) {
-                const float L = t < nt ? fmaxf(lp[t * C], 0.f) : 0.f;   // negative / NaN -> 0
+                const float L = t < nt ? fmaxf(*DYN_PTR(lp + t * C, a.load, a.tiles), 0.f) : 0.f;   // negative / NaN -> 0
 #pragma unroll
                 for (int k = 0; k < NPL; ++k) {
                     ln[t * NPL + k] = L * rn[k];
@@ -283,7 +287,7 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
 #pragma unroll kPairUnroll
             for (int p = 0; p < P; ++p) {
                 uint64_t icm2, lim2;
-                asm("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(icm2), "=l"(lim2) : "r"(cpair + uint32_t(p) * 16u));
+                asm("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(icm2), "=l"(lim2) : "r"(DYN_SMEM_ADDR(cpair + uint32_t(p) * 16u, 16u)));
                 const float lim = __uint_as_float(uint32_t(lim2));
 #pragma unroll
                 for (int q = 0; q < NCH; q += 2)
@@ -425,8 +429,8 @@ __device__ __forceinline__ void sweep_body(const SweepArgs &a, const Tables tb, 
             }
         }
         if (nl < nt) {
-            best_idx[oi + nl * C] = my_idx;
-            best_E[oi + nl * C] = my_E;
+            best_idx[DYN_IDX(oi + nl * C, a.tiles)] = my_idx;
+            best_E[DYN_IDX(oi + nl * C, a.tiles)] = my_E;
         }
     }
 }
@@ -439,6 +443,7 @@ eval_select_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, float *__r
     Tables tb;
     tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.pair2 = a.off_pair2; tb.rows2 = a.off_rows2;
     const int bad = rows_without_threshold(a, 0, a.C * a.P);     // uniform over the grid: every CTA reads the same flags
+    if (!SMEM) DYN_SET_RANGES(0u, 0u, uint32_t(a.off_end));
     if (bad * 4 <= a.C * a.P) {
         if (SMEM) {
             stage(a, a.off_pair2, a.off_end);        // pair2 | rows2
@@ -475,10 +480,13 @@ eval_select_class_kernel(const SweepArgs a, int32_t *__restrict__ best_idx, floa
         for (int i = threadIdx.x; i < np16; i += blockDim.x) smem[i] = src_p[i];
         for (int i = threadIdx.x; i < nr16; i += blockDim.x) smem[np16 + i] = src_r[i];
         __syncthreads();
+        DYN_SET_RANGES(uint32_t(__cvta_generic_to_shared(smem)), uint32_t(__cvta_generic_to_shared(smem)) + uint32_t((np16 + nr16) * 16),
+                       uint32_t(a.off_end));
         tb.pair2 = 0; tb.rows2 = uint32_t(pair_bytes);
         if (bad == 0) sweep_body<NPL, TT, BUDGET, true, true, true, true>(a, tb, best_idx, best_E);
         else sweep_body<NPL, TT, BUDGET, true, true, true, true, true>(a, tb, best_idx, best_E);
     } else {
+        DYN_SET_RANGES(0u, 0u, uint32_t(a.off_end));
         const int c = blockIdx.y;
         tb.rows = a.off_rows + uint32_t(c) * uint32_t(a.P * (a.M + 1)) * 16u;
         tb.pairc = a.off_pairc + uint32_t(c) * uint32_t(a.P) * 8u;
@@ -515,7 +523,7 @@ __device__ __forceinline__ void configs_body(const SweepArgs &a, const Tables tb
         const int c = int(i % a.C);
         const bool active = p < P;
         const int pp = active ? p : 0;
-        const float L = fmaxf(a.load[i], 0.f);
+        const float L = fmaxf(a.load[DYN_IDX(i, a.tiles)], 0.f);
         const float slo_c = __ldg(reinterpret_cast<const float *>(ws + a.off_slo) + c);
         const uint32_t row = origin + (FAST ? tb.rows2 : tb.rows) + uint32_t((c * P + pp) * RS) * ESZ;
         float ic, lim;                                // threshold path: {icm, llim}; general: {ic, slo}
@@ -540,7 +548,7 @@ __device__ __forceinline__ void configs_body(const SweepArgs &a, const Tables tb
             const int64_t q = int64_t(a.budget) / a.tp[pp / a.F];
             nlim = q < Nmax ? int(q) : Nmax;
         }
-        float *out = E_out + size_t(i) * size_t(a.J) + p;     // candidates of this pair are P floats apart
+        float *out = E_out + size_t(DYN_IDX(i, a.tiles)) * size_t(a.J) + (active ? p : 0);     // candidates of this pair are P floats apart
         if (FAST && SMEM) {
             // two instance counts per trip with the packed form of the fused kernel (same arithmetic)
             const uint64_t L2 = pack2(L, L), icm2 = pack2(ic, ic);
@@ -551,7 +559,7 @@ __device__ __forceinline__ void configs_body(const SweepArgs &a, const Tables tb
 #pragma unroll 4
             for (int h = 0; h < pairs; ++h, out += 2 * P) {
                 uint64_t rn2, nf2;                            // {1/n, 1/(n+1)}, {n, n+1}
-                asm("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(rn2), "=l"(nf2) : "r"(sn_addr + uint32_t(h) * 16u));
+                asm("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(rn2), "=l"(nf2) : "r"(sn_addr + uint32_t(DYN_IDX(h, 129)) * 16u));
                 const float limA = (!BUDGET || 2 * h + 1 <= nlim) ? lim : -1.f;
                 const float limB = (!BUDGET || 2 * h + 2 <= nlim) ? lim : -1.f;
                 float EA, EB;
@@ -622,6 +630,7 @@ eval_configs_kernel(const SweepArgs a, const int64_t units_total, float *__restr
     Tables tb;
     tb.rows = a.off_rows; tb.pairc = a.off_pairc; tb.slo = a.off_slo; tb.pair2 = a.off_pair2; tb.rows2 = a.off_rows2;
     const int bad = rows_without_threshold(a, 0, a.C * a.P);     // (also a barrier for s_n)
+    if (!SMEM) DYN_SET_RANGES(0u, 0u, uint32_t(a.off_end));
     if (bad * 4 <= a.C * a.P) {                      // load-threshold path: 8-byte lookups
         if (SMEM) {
             stage(a, a.off_pair2, a.off_end);

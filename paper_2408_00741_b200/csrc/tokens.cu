@@ -13,6 +13,7 @@
 //
 // carbon: window energies times the grid's carbon intensity, summed over the windows in a fixed order
 // [Sec. 6.4]; fp64, one warp per scenario, bit-identical from run to run.
+#define DYN_TU_ID 11
 #include "dyn_internal.cuh"
 
 namespace dyn {
@@ -65,10 +66,10 @@ __device__ __forceinline__ void add_request(const BinParams &bp, const TokenBins
     const uint32_t c = token_class<NI, NO>(bp, a, b);
     const uint32_t rel = w - tb.w_lo;                        // wraps for w < w_lo: then rel >= nwin
     if (rel < tb.nwin) {
-        add_shared(s_lane + ((rel * tb.C + c) << tb.copies_log2), tb.stride, a, b);
+        add_shared(s_lane + DYN_IDX((rel * tb.C + c) << tb.copies_log2, tb.stride), tb.stride, a, b);
     } else {
-        atomicAdd(&tok_in[size_t(w) * tb.C + c], (unsigned long long)a);
-        atomicAdd(&tok_out[size_t(w) * tb.C + c], (unsigned long long)b);
+        atomicAdd(&tok_in[DYN_IDX(size_t(w) * tb.C + c, size_t(tb.W) * tb.C)], (unsigned long long)a);
+        atomicAdd(&tok_out[DYN_IDX(size_t(w) * tb.C + c, size_t(tb.W) * tb.C)], (unsigned long long)b);
     }
 }
 
@@ -85,10 +86,10 @@ __device__ __forceinline__ void add_four(const BinParams &bp, const TokenBins &t
             r1 = fastdiv(vt.y, bp.win) - tb.w_lo;
             r2 = fastdiv(vt.z, bp.win) - tb.w_lo;
         }
-        add_shared(s_lane + ((r0 * tb.C + token_class<NI, NO>(bp, va.x, vb.x)) << tb.copies_log2), tb.stride, va.x, vb.x);
-        add_shared(s_lane + ((r1 * tb.C + token_class<NI, NO>(bp, va.y, vb.y)) << tb.copies_log2), tb.stride, va.y, vb.y);
-        add_shared(s_lane + ((r2 * tb.C + token_class<NI, NO>(bp, va.z, vb.z)) << tb.copies_log2), tb.stride, va.z, vb.z);
-        add_shared(s_lane + ((r3 * tb.C + token_class<NI, NO>(bp, va.w, vb.w)) << tb.copies_log2), tb.stride, va.w, vb.w);
+        add_shared(s_lane + DYN_IDX(((r0 * tb.C + token_class<NI, NO>(bp, va.x, vb.x)) << tb.copies_log2), tb.stride), tb.stride, va.x, vb.x);
+        add_shared(s_lane + DYN_IDX(((r1 * tb.C + token_class<NI, NO>(bp, va.y, vb.y)) << tb.copies_log2), tb.stride), tb.stride, va.y, vb.y);
+        add_shared(s_lane + DYN_IDX(((r2 * tb.C + token_class<NI, NO>(bp, va.z, vb.z)) << tb.copies_log2), tb.stride), tb.stride, va.z, vb.z);
+        add_shared(s_lane + DYN_IDX(((r3 * tb.C + token_class<NI, NO>(bp, va.w, vb.w)) << tb.copies_log2), tb.stride), tb.stride, va.w, vb.w);
     } else {
         add_request<NI, NO>(bp, tb, s_lane, vt.x, va.x, vb.x, tok_in, tok_out);
         add_request<NI, NO>(bp, tb, s_lane, vt.y, va.y, vb.y, tok_in, tok_out);
@@ -124,7 +125,7 @@ bin_tokens_kernel(const BinParams bp, const uint32_t *__restrict__ t_ms, const u
     const uint32_t nbins = tb.nwin * tb.C;
     tb.copies_log2 = 0;
     while (tb.copies_log2 < 5 && (nbins << (tb.copies_log2 + 1)) <= uint32_t(kWords)) ++tb.copies_log2;
-    tb.stride = nbins << tb.copies_log2;
+    tb.stride = DYN_IDX(nbins << tb.copies_log2, uint32_t(kWords) + 1u);      // four word arrays of this length fit in s_sum
     for (uint32_t i = threadIdx.x; i < tb.stride; i += kThreads)
         s_sum[i] = s_sum[i + tb.stride] = s_sum[i + 2 * tb.stride] = s_sum[i + 3 * tb.stride] = 0u;
     __syncthreads();
@@ -138,8 +139,9 @@ bin_tokens_kernel(const BinParams bp, const uint32_t *__restrict__ t_ms, const u
                     *b4 = reinterpret_cast<const uint4 *>(out_tok);
         uint32_t i = threadIdx.x;
         for (; i + kThreads < n4; i += 2 * kThreads) {
-            const uint4 t0 = __ldcs(t4 + i), a0 = __ldcs(a4 + i), b0 = __ldcs(b4 + i);
-            const uint4 t1 = __ldcs(t4 + i + kThreads), a1 = __ldcs(a4 + i + kThreads), b1 = __ldcs(b4 + i + kThreads);
+            const uint32_t j0 = DYN_IDX(i, n4), j1 = DYN_IDX(i + kThreads, n4);
+            const uint4 t0 = __ldcs(t4 + j0), a0 = __ldcs(a4 + j0), b0 = __ldcs(b4 + j0);
+            const uint4 t1 = __ldcs(t4 + j1), a1 = __ldcs(a4 + j1), b1 = __ldcs(b4 + j1);
             add_four<NI, NO>(bp, tb, s_lane, t0, a0, b0, tok_in, tok_out);
             add_four<NI, NO>(bp, tb, s_lane, t1, a1, b1, tok_in, tok_out);
         }
@@ -163,15 +165,15 @@ bin_tokens_kernel(const BinParams bp, const uint32_t *__restrict__ t_ms, const u
         const uint32_t *q = s_sum + (i << tb.copies_log2);
         const unsigned long long si = (unsigned long long)q[0] + ((unsigned long long)q[tb.stride] << 16);
         const unsigned long long so = (unsigned long long)q[2 * tb.stride] + ((unsigned long long)q[3 * tb.stride] << 16);
-        if (si) atomicAdd(&tok_in[size_t(tb.w_lo) * tb.C + i], si);
-        if (so) atomicAdd(&tok_out[size_t(tb.w_lo) * tb.C + i], so);
+        if (si) atomicAdd(&tok_in[DYN_IDX(size_t(tb.w_lo) * tb.C + i, size_t(tb.W) * tb.C)], si);
+        if (so) atomicAdd(&tok_out[DYN_IDX(size_t(tb.w_lo) * tb.C + i, size_t(tb.W) * tb.C)], so);
     }
 }
 
 __global__ void tokens_to_tps_kernel(const unsigned long long *__restrict__ tok_in, const unsigned long long *__restrict__ tok_out,
                                      float *__restrict__ tps, uint64_t n, float window_s) {
     for (uint64_t i = uint64_t(blockIdx.x) * blockDim.x + threadIdx.x; i < n; i += uint64_t(gridDim.x) * blockDim.x)
-        tps[i] = __fdiv_rn(float(tok_in[i] + tok_out[i]), window_s);
+        tps[DYN_IDX(i, n)] = __fdiv_rn(float(tok_in[DYN_IDX(i, n)] + tok_out[DYN_IDX(i, n)]), window_s);
 }
 
 // one warp per scenario; lane l sums windows l, l+32, ... in order, then the lanes are added in a fixed tree
@@ -181,7 +183,7 @@ __global__ void __launch_bounds__(kThreads) carbon_kernel(const double *__restri
     const int64_t s = int64_t(blockIdx.x) * (kThreads / 32) + (threadIdx.x >> 5);
     if (s >= S) return;
     double acc = 0.0;
-    for (int64_t w = lane; w < W; w += 32) acc += E_window[s * W + w] * double(intensity[w]) / 1000.0;
+    for (int64_t w = lane; w < W; w += 32) acc += E_window[DYN_IDX(s * W + w, S * W)] * double(intensity[DYN_IDX(w, W)]) / 1000.0;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, off);
     if (lane == 0) carbon[s] = acc;
