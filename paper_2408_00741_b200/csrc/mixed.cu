@@ -11,12 +11,12 @@
 // Work per tile is (tuples) x (TP degrees in use) x F single-type evaluations; the loads and results are
 // 4 + 12 + 8T bytes per tile.  The energy of a group is n x (energy of one instance at its per-instance load l),
 // and l = (L/A) x capH_t, so for one TP degree the 32 x 4 tuples a warp holds are 128 per-instance loads run
-// against that degree's F table rows: the inner loop of the single-type sweep.  When every TBT row is
-// monotone in load (the resolve step's flags) and the threshold tables fit in shared memory, the kernel uses
+// against that degree's F table rows: the inner loop of the single-type sweep.  When the threshold tables fit
+// in shared memory, the kernel uses
 // that loop (compare on l, segment address from a subnormal FMA, one FMA per candidate, predicated min) and
-// recovers the frequencies of the winning tuple afterwards with the same arithmetic; otherwise a plain
-// variant evaluates from the general-path tables through L1.  Both are launched; each looks at the flags
-// and only the one they select does the work.
+// recovers the frequencies of the winning tuple afterwards with the same arithmetic.  A class with a table row
+// that has no load threshold is evaluated tile by tile from the general-path tables through L1 (the same
+// kernel, a warp-uniform choice per tile), as is everything when the tables do not fit.
 #define DYN_TU_ID 9
 #include "dyn_internal.cuh"
 #include "eval_dev.cuh"
@@ -27,6 +27,9 @@ namespace dyn {
 
 namespace {
 
+#ifndef DYN_MIXED_SHORT
+#define DYN_MIXED_SHORT 0
+#endif
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 
@@ -57,13 +60,6 @@ __global__ void mixed_caph_kernel(const MixedArgs a) {
     a.caph[i] = pair2[DYN_IDX(c * (a.T * a.F) + t * a.F + a.F - 1, a.C * a.T * a.F)].w;
 }
 
-// true when every pair row has a load threshold (vlim is NaN for a row whose TBT decreases somewhere)
-__device__ __forceinline__ bool rows_monotone(const MixedArgs &a) {
-    int bad = 0;
-    for (int i = threadIdx.x; i < a.C * a.T * a.F; i += blockDim.x) bad |= isnan(__ldg(a.pairc + i).y) ? 1 : 0;
-    return __syncthreads_or(bad) == 0;
-}
-
 // 1 / A of every (class, tuple): A = sum_t n_t * capH_t, the pool's capacity at the highest candidate frequency
 __global__ void mixed_inva_kernel(const MixedArgs a) {
     const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -75,14 +71,12 @@ __global__ void mixed_inva_kernel(const MixedArgs a) {
     a.inva[i] = float(1.0 / A);                              // +inf when no degree of the tuple has capacity: infeasible
 }
 
+// one tile on the general-path tables (through L1): lane l takes tuples l, l + 32, ... of the list
 template <int T>
-__global__ void __launch_bounds__(kThreads) mixed_select_kernel(const MixedArgs a) {
-    if (a.use_fast && rows_monotone(a)) return;              // the threshold variant does this call
-    const int lane = threadIdx.x & 31;
+__device__ __noinline__ void mixed_tile_plain(const MixedArgs &a, const int64_t i, const int lane) {
     const int P = T * a.F, RS = a.M + 1;
     const float Mf = float(a.M);
-    const int64_t nwarps = int64_t(gridDim.x) * kWarps;
-    for (int64_t i = int64_t(blockIdx.x) * kWarps + (threadIdx.x >> 5); i < a.tiles; i += nwarps) {
+    {
         const int c = int(i % a.C);
         const float L = fmaxf(a.load[DYN_IDX(i, a.tiles)], 0.f);              // negative / NaN -> 0
         const float slo = a.slo[DYN_IDX(c, a.C)];
@@ -142,7 +136,7 @@ __global__ void __launch_bounds__(kThreads) mixed_select_kernel(const MixedArgs 
                 a.tuple[DYN_IDX(i, a.tiles)] = -1;
                 a.best_E[i] = CUDART_INF_F;
             }
-            continue;
+            return;
         }
         if (best == Emin && bnum == kmin) {                  // exactly one lane: tuple numbers are distinct
 #pragma unroll
@@ -157,11 +151,27 @@ __global__ void __launch_bounds__(kThreads) mixed_select_kernel(const MixedArgs 
     }
 }
 
-
-// threshold variant: tables of all classes in shared memory, four tuples per lane and pass
 template <int T>
+__global__ void __launch_bounds__(kThreads) mixed_select_kernel(const MixedArgs a) {
+    DYN_SET_RANGES(0u, 0u, uint32_t(a.off_end));
+    const int lane = threadIdx.x & 31;
+    const int64_t nwarps = int64_t(gridDim.x) * kWarps;
+    for (int64_t i = int64_t(blockIdx.x) * kWarps + (threadIdx.x >> 5); i < a.tiles; i += nwarps) mixed_tile_plain<T>(a, i, lane);
+}
+
+
+// threshold variant: tables of all classes in shared memory, SL tuples per lane and pass (32 * SL tuples side by side;
+// the list is sorted by the set of degrees in use, and a pass skips the degrees none of its tuples uses: short
+// passes skip more, long ones share a pair's constants among more candidates)
+template <int T, int SL>
 __global__ void __launch_bounds__(kThreads, 3) mixed_fast_kernel(const MixedArgs a) {
-    if (!rows_monotone(a)) return;                           // the plain variant does this call
+    // classes with a table row that has no load threshold (the resolve step's flags) take the general path
+    __shared__ unsigned char s_general[256];
+    for (int c = threadIdx.x; c < a.C; c += blockDim.x) {
+        bool bad = false;
+        for (int p = 0; p < a.T * a.F; ++p) bad |= isnan(__ldg(a.pairc + c * a.T * a.F + p).y);
+        s_general[c] = bad ? 1 : 0;
+    }
     extern __shared__ float4 smem[];
     {
         const float4 *src = reinterpret_cast<const float4 *>(a.ws + a.off_pair2);
@@ -184,17 +194,21 @@ __global__ void __launch_bounds__(kThreads, 3) mixed_fast_kernel(const MixedArgs
     const int64_t nwarps = int64_t(gridDim.x) * kWarps;
     for (int64_t i = int64_t(blockIdx.x) * kWarps + (threadIdx.x >> 5); i < a.tiles; i += nwarps) {
         const int c = int(i % a.C);
-        const float L = fmaxf(a.load[i], 0.f);              // negative / NaN -> 0
+        if (s_general[c]) {                                  // warp-uniform
+            mixed_tile_plain<T>(a, i, lane);
+            continue;
+        }
+        const float L = fmaxf(a.load[DYN_IDX(i, a.tiles)], 0.f);              // negative / NaN -> 0
         float caph[T];
 #pragma unroll
         for (int t = 0; t < T; ++t) caph[t] = a.caph[c * T + t];
         float best = CUDART_INF_F, bfrac = 0.f;
         uint32_t bnum = 0xffffffffu, btup = 0;
-        for (int64_t base = 0; base < a.K; base += 128) {
-            uint32_t tup[4], num[4];
-            float frac[4], E[4];
+        for (int64_t base = 0; base < a.K; base += 32 * SL) {
+            uint32_t tup[SL], num[SL];
+            float frac[SL], E[SL];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
+            for (int j = 0; j < SL; ++j) {
                 const int64_t k = base + j * 32 + lane;
                 const uint2 tk = k < a.K ? __ldg(a.tuples + k) : make_uint2(0u, 0xffffffffu);
                 tup[j] = tk.x;
@@ -205,18 +219,20 @@ __global__ void __launch_bounds__(kThreads, 3) mixed_fast_kernel(const MixedArgs
             }
 #pragma unroll
             for (int t = 0; t < T; ++t) {
-                uint32_t n[4];
-                float ln[4], e1[4];
+                uint32_t n[SL];
+                float ln[SL], e1[SL];
                 uint32_t any = 0;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                for (int j = 0; j < SL; ++j) {
                     n[j] = (tup[j] >> (8 * t)) & 255u;
                     any |= n[j];
                     ln[j] = n[j] ? frac[j] * caph[t] : CUDART_INF_F;      // no instance of this degree: nothing to serve
                     e1[j] = CUDART_INF_F;
                 }
                 if (!__any_sync(kFull, any != 0)) continue;              // no tuple of the pass uses this degree
-                const uint64_t lnA = pack2(ln[0], ln[1]), lnB = pack2(ln[2], ln[3]);
+                uint64_t ln2[SL / 2];
+#pragma unroll
+                for (int j = 0; j < SL; j += 2) ln2[j / 2] = pack2(ln[j], ln[j + 1]);
                 const uint32_t cpair = origin + uint32_t(c * P + t * F) * 16u;
                 const float off0 = row_offset_units(rows2 + uint32_t((c * P + t * F) * RS) * 8u);
                 uint64_t off2 = pack2(off0, off0);
@@ -225,16 +241,16 @@ __global__ void __launch_bounds__(kThreads, 3) mixed_fast_kernel(const MixedArgs
                     uint64_t icm2, lim2;
                     asm("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(icm2), "=l"(lim2) : "r"(DYN_SMEM_ADDR(cpair + uint32_t(q) * 16u, 16u)));
                     const float lim = __uint_as_float(uint32_t(lim2));
-                    fast_two(lnA, icm2, off2, two23_2, eight2, lim, lim, e1[0], e1[1]);
-                    fast_two(lnB, icm2, off2, two23_2, eight2, lim, lim, e1[2], e1[3]);
+#pragma unroll
+                    for (int j = 0; j < SL; j += 2) fast_two(ln2[j / 2], icm2, off2, two23_2, eight2, lim, lim, e1[j], e1[j + 1]);
                     off2 = add2(off2, off2_step);
                 }
 #pragma unroll
-                for (int j = 0; j < 4; ++j)
+                for (int j = 0; j < SL; ++j)
                     if (n[j]) E[j] += float(n[j]) * e1[j];   // ascending TP index; +inf if the group has no frequency
             }
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
+            for (int j = 0; j < SL; ++j)
                 if (E[j] < best || (E[j] == best && num[j] < bnum)) {     // lowest tuple number on ties
                     best = E[j];
                     bnum = num[j];
@@ -334,18 +350,28 @@ cudaError_t launch_mixed(const ResolvedLayout &lay, void *d_ws, size_t off_tuple
     a.off_pair2 = int32_t(lay.off_pair2); a.off_rows2 = int32_t(lay.off_rows2); a.off_end = int32_t(lay.off_tp);
     const size_t fast_bytes = lay.off_tp - lay.off_pair2;
     a.use_fast = fast_bytes <= 96 * 1024 ? 1 : 0;
+    // (passes of 64 tuples skip more degrees than passes of 128 but share a pair's constants among fewer candidates:
+    // measured slower at 200 tuples, so the long passes serve every list)
+    const bool short_passes = K <= DYN_MIXED_SHORT;
     e = record_start(st);
     if (e != cudaSuccess) return e;
 #define DYN_MIXED_LAUNCH(TT)                                                                                      \
     do {                                                                                                          \
         if (a.use_fast) {                                                                                         \
-            e = cudaFuncSetAttribute(mixed_fast_kernel<TT>, cudaFuncAttributeMaxDynamicSharedMemorySize,          \
-                                     int(fast_bytes));                                                            \
-            if (e != cudaSuccess) return e;                                                                       \
-            mixed_fast_kernel<TT><<<int(grid), kThreads, fast_bytes, st>>>(a);                                    \
-            if ((e = cudaGetLastError()) != cudaSuccess) return e;                                                \
+            if (short_passes) {                                                                                   \
+                e = cudaFuncSetAttribute(mixed_fast_kernel<TT, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,   \
+                                         int(fast_bytes));                                                        \
+                if (e != cudaSuccess) return e;                                                                   \
+                mixed_fast_kernel<TT, 2><<<int(grid), kThreads, fast_bytes, st>>>(a);                             \
+            } else {                                                                                              \
+                e = cudaFuncSetAttribute(mixed_fast_kernel<TT, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,   \
+                                         int(fast_bytes));                                                        \
+                if (e != cudaSuccess) return e;                                                                   \
+                mixed_fast_kernel<TT, 4><<<int(grid), kThreads, fast_bytes, st>>>(a);                             \
+            }                                                                                                     \
+        } else {                                                                                                  \
+            mixed_select_kernel<TT><<<int(grid), kThreads, 0, st>>>(a);                                           \
         }                                                                                                         \
-        mixed_select_kernel<TT><<<int(grid), kThreads, 0, st>>>(a);                                               \
     } while (0)
     switch (lay.T) {
         case 1: DYN_MIXED_LAUNCH(1); break;

@@ -47,6 +47,12 @@ __device__ __forceinline__ uint32_t token_class(const BinParams &bp, uint32_t in
     }
 }
 
+// the same for a request whose token counts are known to be below 65536: the high halves add nothing
+__device__ __forceinline__ void add_shared_low(uint32_t *p, uint32_t stride, uint32_t a, uint32_t b) {
+    atomicAdd(p, a);
+    atomicAdd(p + 2 * stride, b);
+}
+
 // adds one request's tokens to the sums of shared-memory bin `p` (the lane's copy)
 __device__ __forceinline__ void add_shared(uint32_t *p, uint32_t stride, uint32_t a, uint32_t b) {
     atomicAdd(p, a & 0xffffu);
@@ -86,10 +92,21 @@ __device__ __forceinline__ void add_four(const BinParams &bp, const TokenBins &t
             r1 = fastdiv(vt.y, bp.win) - tb.w_lo;
             r2 = fastdiv(vt.z, bp.win) - tb.w_lo;
         }
-        add_shared(s_lane + DYN_IDX(((r0 * tb.C + token_class<NI, NO>(bp, va.x, vb.x)) << tb.copies_log2), tb.stride), tb.stride, va.x, vb.x);
-        add_shared(s_lane + DYN_IDX(((r1 * tb.C + token_class<NI, NO>(bp, va.y, vb.y)) << tb.copies_log2), tb.stride), tb.stride, va.y, vb.y);
-        add_shared(s_lane + DYN_IDX(((r2 * tb.C + token_class<NI, NO>(bp, va.z, vb.z)) << tb.copies_log2), tb.stride), tb.stride, va.z, vb.z);
-        add_shared(s_lane + DYN_IDX(((r3 * tb.C + token_class<NI, NO>(bp, va.w, vb.w)) << tb.copies_log2), tb.stride), tb.stride, va.w, vb.w);
+        uint32_t *p0 = s_lane + DYN_IDX(((r0 * tb.C + token_class<NI, NO>(bp, va.x, vb.x)) << tb.copies_log2), tb.stride);
+        uint32_t *p1 = s_lane + DYN_IDX(((r1 * tb.C + token_class<NI, NO>(bp, va.y, vb.y)) << tb.copies_log2), tb.stride);
+        uint32_t *p2 = s_lane + DYN_IDX(((r2 * tb.C + token_class<NI, NO>(bp, va.z, vb.z)) << tb.copies_log2), tb.stride);
+        uint32_t *p3 = s_lane + DYN_IDX(((r3 * tb.C + token_class<NI, NO>(bp, va.w, vb.w)) << tb.copies_log2), tb.stride);
+        if (((va.x | va.y | va.z | va.w | vb.x | vb.y | vb.z | vb.w) >> 16) == 0u) {      // one test for all eight counts
+            add_shared_low(p0, tb.stride, va.x, vb.x);
+            add_shared_low(p1, tb.stride, va.y, vb.y);
+            add_shared_low(p2, tb.stride, va.z, vb.z);
+            add_shared_low(p3, tb.stride, va.w, vb.w);
+        } else {
+            add_shared(p0, tb.stride, va.x, vb.x);
+            add_shared(p1, tb.stride, va.y, vb.y);
+            add_shared(p2, tb.stride, va.z, vb.z);
+            add_shared(p3, tb.stride, va.w, vb.w);
+        }
     } else {
         add_request<NI, NO>(bp, tb, s_lane, vt.x, va.x, vb.x, tok_in, tok_out);
         add_request<NI, NO>(bp, tb, s_lane, vt.y, va.y, vb.y, tok_in, tok_out);

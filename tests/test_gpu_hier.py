@@ -116,3 +116,13 @@ def test_hier_free_form_tables(dyn, monotone, large):
     prof, sp = random_tables(29, monotone, large)
     load = gen.random_loads((2, 24, 9), seed=36, mean=5.0)
     _check(dyn, prof, sp, 12, 4, load, max_exempt=0.03)
+
+
+def test_hier_classes_with_and_without_load_thresholds(dyn):
+    """A few table rows (classes 0, 4 and 8) cross the SLO twice: the warps of those classes evaluate from the
+    general-path tables, the other six classes keep the threshold path, in the same launches."""
+    from parity import tables_with_few_rows_without_threshold
+    prof, sp, bad = tables_with_few_rows_without_threshold(31)
+    assert {c for c, _, _ in bad} == {0, 4, 8}
+    load = gen.random_loads((2, 24, 9), seed=37, mean=5.0)
+    _check(dyn, prof, sp, 12, 4, load, max_exempt=0.03)

@@ -144,3 +144,14 @@ def test_free_form_tables(dyn, monotone, large):
     sp = gen.make_space(sp0.f_cand_mhz[::5] if large else sp0.f_cand_mhz, 6, 60.0, slo_ttft=0.8, slo_tbt=0.1, gpu_budget=14)
     load = gen.random_loads((2, 9, 9), seed=35, mean=6.0)
     _check(dyn, prof, sp, load, max_exempt=0.03)
+
+
+def test_classes_with_and_without_load_thresholds_side_by_side(dyn):
+    """A few table rows (classes 0, 4 and 8) cross the SLO twice: tiles of those classes take the general path, the
+    other six classes keep the threshold path, in the same launch."""
+    from parity import tables_with_few_rows_without_threshold
+    prof, sp0, bad = tables_with_few_rows_without_threshold(29)
+    assert {c for c, _, _ in bad} == {0, 4, 8}
+    sp = gen.make_space(sp0.f_cand_mhz, 6, 60.0, slo_ttft=0.8, slo_tbt=0.1, gpu_budget=14)
+    load = gen.random_loads((2, 11, 9), seed=36, mean=6.0)
+    _check(dyn, prof, sp, load, max_exempt=0.03)
