@@ -107,7 +107,7 @@ constexpr int kOwn = 4;                         // entries of the state vector a
 // One CTA per (scenario, class).  Dynamic shared memory: Dp[NS4] | part[G][NS4] | cring[kRing][NS4] | Rs[rows_s / 2][2][NS4 + 4].
 // Forward: D_w(g) = cost_w(g) + min_h (D_{w-1}(h) + R[h][g]).  Only the minimum is formed here (half a packed add and half a three-input min per
 // step): a thread takes four neighbouring targets and a share of the sources, four sources per trip (one 16-byte
-// read of the state vector, four of R).  The values D_{w-1}, relative to their minimum, are written to `hist`,
+// read of the state vector, four of R).  The values D_{w-1}, as held (relative to the running base), are written to `hist`,
 // and the walk back finds each predecessor again as the lowest h that attains the minimum, with the same addition.
 __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfArgs a, const int rows_s) {
     extern __shared__ float4 smem4[];
@@ -197,22 +197,22 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
     }
     __syncthreads();                                         // publishes Dp, the minimum and Rs
     for (int64_t w = 1; w < W; ++w) {
-        // keep differences only: the previous minimum goes to the fp64 base (all +inf stays +inf)
+        // keep differences only: the minimum of the previous vector goes to the fp64 base (all +inf stays +inf) and
+        // is taken off the vector computed in this window
         const float mprev = val_of(s_min[(w - 1) & 1]);
         const float shift = (mprev < CUDART_INF_F) ? mprev : 0.f;
         base += double(shift);
         if (tid == 0) s_min[w & 1] = 0xffffffffu;            // this window's slot; last read before the previous barrier
-        for (int g = tid; g < NS; g += kPathThreads) hist[DYN_IDX((w - 1) * NS + g, W * NS)] = Dp[DYN_IDX(g, NS4)] - shift;
+        for (int g = tid; g < NS; g += kPathThreads) hist[DYN_IDX((w - 1) * NS + g, W * NS)] = Dp[DYN_IDX(g, NS4)];
         if (worker) {
             float b0 = CUDART_INF_F, b1 = CUDART_INF_F, b2 = CUDART_INF_F, b3 = CUDART_INF_F;
-            const float2 nshift = make_float2(-shift, -shift);                  // d + (-shift) is d - shift bit for bit
 #pragma unroll 1
             for (int q = q_lo; q < q_hi; ++q) {
                 const float4 d4 = reinterpret_cast<const float4 *>(Dp)[DYN_IDX(q, TG)];
                 const float *rq = Rs + DYN_IDX(size_t(2 * q) * (2 * RSd) + 4 * tg, size_t(rows_s) * RSd - 3 * RSd - 3);
-                relax_pair(b0, b1, b2, b3, __fadd2_rn(make_float2(d4.x, d4.y), nshift), *reinterpret_cast<const float4 *>(rq),
+                relax_pair(b0, b1, b2, b3, make_float2(d4.x, d4.y), *reinterpret_cast<const float4 *>(rq),
                            *reinterpret_cast<const float4 *>(rq + RSd));
-                relax_pair(b0, b1, b2, b3, __fadd2_rn(make_float2(d4.z, d4.w), nshift), *reinterpret_cast<const float4 *>(rq + 2 * RSd),
+                relax_pair(b0, b1, b2, b3, make_float2(d4.z, d4.w), *reinterpret_cast<const float4 *>(rq + 2 * RSd),
                            *reinterpret_cast<const float4 *>(rq + 3 * RSd));
             }
 #pragma unroll
@@ -220,11 +220,11 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
                 // past the last quad of the vector the rows hold +inf, so any entries of the vector will do
                 const int hq = h_reg / 4 + j4 < TG ? h_reg / 4 + j4 : TG - 1;
                 const float4 d4 = reinterpret_cast<const float4 *>(Dp)[hq];
-                relax_pair(b0, b1, b2, b3, __fadd2_rn(make_float2(d4.x, d4.y), nshift), rp0[2 * j4], rp1[2 * j4]);
-                relax_pair(b0, b1, b2, b3, __fadd2_rn(make_float2(d4.z, d4.w), nshift), rp0[2 * j4 + 1], rp1[2 * j4 + 1]);
+                relax_pair(b0, b1, b2, b3, make_float2(d4.x, d4.y), rp0[2 * j4], rp1[2 * j4]);
+                relax_pair(b0, b1, b2, b3, make_float2(d4.z, d4.w), rp0[2 * j4 + 1], rp1[2 * j4 + 1]);
             }
             for (int h = g_lo; h < g_hi; ++h) {
-                const float d = Dp[h] - shift;
+                const float d = Dp[h];
                 const float *row = a.R + size_t(h) * NS + 4 * tg;
                 b0 = fminf(b0, d + __ldg(row));
                 if (4 * tg + 1 < NS) b1 = fminf(b1, d + __ldg(row + 1));
@@ -243,7 +243,9 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
             if (g < NS) {
                 float best = part[DYN_IDX(g, NS4)];
                 for (int k = 1; k < G; ++k) best = fminf(best, part[DYN_IDX(k * NS4 + g, G * NS4)]);
-                const float d = cslot[DYN_IDX(g, NS4)] + best;
+                // the minimum of the PREVIOUS vector comes off here, one window late: one subtraction per entry
+                // instead of one per source in the scan; the values stay within two windows' growth of zero
+                const float d = (cslot[DYN_IDX(g, NS4)] + best) - shift;
                 Dp[DYN_IDX(g, NS4)] = d;
                 lmin = fminf(lmin, d);
             }
@@ -256,7 +258,7 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
         __pipeline_commit();
         __syncthreads();                                     // publishes Dp and the minimum
     }
-    const float m = W > 0 ? val_of(s_min[(W - 1) & 1]) : 0.f;
+    const float m = W > 0 ? val_of(s_min[(W - 1) & 1]) : 0.f;      // minimum of the last vector (relative to `base`)
     if (W == 0) {
         if (tid == 0) a.path_total[sc] = 0.0;
         return;
