@@ -307,25 +307,39 @@ def feasible_share(dyn, P, SP, d_load_sample):
     return float(torch.isfinite(E).sum().item()) / float(E.numel())
 
 
-def executed_work(dyn, peaks, sampler, wl_name, kernel_rate, share):
-    """Hardware-side figures of the sweep: its instruction rate against the measured issue ceiling (instruction
-    count from recorded profiler counters, null once the kernel's sources have changed), and its rate against
-    the library's probe of the sweep's inner loop at the workload's share of feasible candidates."""
+def pipe_fractions(peaks, kernel, key, kernel_rate):
+    """Hardware-side figures of a kernel from its recorded profiler counters (per 32 evaluations: warp instructions
+    executed, shared-memory wavefronts) and the rate of this run: the share of the issue ceiling and of the
+    shared-memory data path it uses.  The ceilings come from the multiply-add probe of this run (one warp
+    instruction per scheduler and clock = its rate / 64; one wavefront per SM and clock = a quarter of that).
+    None without counters; the figures are None once the kernel's sources have changed since they were taken."""
     from paper_2408_00741_b200 import counters
-    out = {"issue": None, "inner_loop_probe": None}
-    rec = counters.lookup("eval_select_kernel", wl_name)
-    if rec is not None and rec.get("warp_inst_per_32_evals") is not None:
-        if rec["stale"]:
-            out["issue"] = {"warp_inst_per_32_evals": None, "frac": None, "counters": "stale: the kernel's sources "
-                            "changed after the counters were taken"}
-        else:
-            ipe = rec["warp_inst_per_32_evals"]
-            rate = ipe * kernel_rate / 32.0
-            out["issue"] = {"warp_inst_per_32_evals": ipe, "achieved_warp_inst_per_s": rate,
-                            "peak_warp_inst_per_s": peaks["issue_warp_inst_per_s"],
-                            "frac": rate / peaks["issue_warp_inst_per_s"],
-                            "counters": "smsp__inst_executed.sum of one launch, recorded for the current sources; "
-                                        "ceiling = measured multiply-add rate / 64"}
+    rec = counters.lookup(kernel, key)
+    if rec is None:
+        return None
+    if rec["stale"]:
+        return {"counters": "stale: the kernel's sources changed after the counters were taken", "issue_frac": None,
+                "shared_memory_frac": None, "frac": None}
+    out = {"counters": "one launch under the profiler, recorded for the current sources", "issue_frac": None,
+           "shared_memory_frac": None}
+    issue_peak = peaks["issue_warp_inst_per_s"]
+    if rec.get("warp_inst_per_32_evals") is not None:
+        out["warp_inst_per_32_evals"] = rec["warp_inst_per_32_evals"]
+        out["issue_frac"] = rec["warp_inst_per_32_evals"] * kernel_rate / 32.0 / issue_peak
+    if rec.get("shared_wavefronts_per_32_evals") is not None:
+        out["shared_wavefronts_per_32_evals"] = rec["shared_wavefronts_per_32_evals"]
+        out["shared_memory_frac"] = rec["shared_wavefronts_per_32_evals"] * kernel_rate / 32.0 / (issue_peak / 4.0)
+    fr = [x for x in (out["issue_frac"], out["shared_memory_frac"]) if x is not None]
+    out["frac"] = max(fr) if fr else None                 # the pipe that binds
+    out["dram_bytes_per_unit"] = rec.get("dram_bytes_per_unit")
+    return out
+
+
+def executed_work(dyn, peaks, sampler, wl_name, kernel_rate, share):
+    """Hardware-side figures of the sweep: its instruction and shared-memory rates against the measured ceilings
+    (counts from recorded profiler counters), and its rate against the library's probe of the sweep's inner loop
+    at the workload's share of feasible candidates."""
+    out = {"pipes": pipe_fractions(peaks, "eval_select_kernel", wl_name, kernel_rate), "inner_loop_probe": None}
     if share is not None:
         work = []
         ms, _, _, t0, t1 = timed_kernel(dyn, lambda: work.append(dyn.dyn_probe_sweep_inner(400, share, peaks["sink"])),
@@ -360,7 +374,7 @@ def rows_without_threshold(prof, sp, which):
     return tbt, n
 
 
-def measure_config(dyn, gen, dev, sampler, peaks, flush, name, S=1, general=None, trace=None, with_bin=True):
+def measure_config(dyn, gen, dev, sampler, peaks, flush, name, S=1, general=None, trace=None, with_bin=True, key=None):
     """One benchmark configuration: the histogram kernel on its trace and the fused sweep on its loads (S > 1:
     Poisson-resampled scenarios of the binned trace; general = "one" / "all": one row / every row that is feasible
     at all crosses the SLO twice and takes the path that interpolates TBT per candidate)."""
@@ -412,6 +426,12 @@ def measure_config(dyn, gen, dev, sampler, peaks, flush, name, S=1, general=None
                   "l2": "flushed" if small(d_load.numel() * 4) is not None else "inputs_larger_than_L2",
                   "clocks": sampler.window(t0, t1) if sampler else None,
                   "E_total_scenario0_Wh": float(out.E_total[0].item())})
+    if key is not None:
+        entry["executed"] = pipe_fractions(peaks, "eval_select_kernel", key, evals / (ms * 1e-3))
+        if with_bin and "bin" in entry:
+            bx = pipe_fractions(peaks, "bin_trace_kernel", key, n_req / (entry["bin"]["kernel_ms"] * 1e-3))
+            entry["bin"]["executed"] = bx
+            entry["bin"]["traffic"] = (bx["dram_bytes_per_unit"] * n_req if bx and bx.get("dram_bytes_per_unit") else None)
     return entry
 
 
@@ -604,7 +624,7 @@ def run_ours(args, rank, world, local_rank):
                                                            trace=trace if wl.name in ("cfg2", "cfg4") else None)),
                         ("cfg2_x256_general", dict(name="cfg2", S=256, general="all", with_bin=False,
                                                    trace=trace if wl.name in ("cfg2", "cfg4") else None))):
-            pc[key] = guarded(measure_config, dyn, gen, dev, sampler, peaks, flush, **kw)
+            pc[key] = guarded(measure_config, dyn, gen, dev, sampler, peaks, flush, key=key, **kw)
         roofline["per_config"] = pc
         if isinstance(pc.get("cfg3"), dict) and "bin" in pc["cfg3"]:
             result["trace_requests_per_s"] = pc["cfg3"]["bin"]["requests_per_s"]
@@ -858,7 +878,7 @@ def run_only(args, local_rank):
     res = {"peaks": {k: v for k, v in peaks.items() if k != "sink"}}
     for key in args.only.split(","):
         if key in per_config:
-            res[key] = measure_config(dyn, gen, dev, sampler, peaks, flush, **per_config[key])
+            res[key] = measure_config(dyn, gen, dev, sampler, peaks, flush, key=key, **per_config[key])
         elif key == "bin_trace":
             res[key] = measure_bin(dyn, gen, dev, peaks=peaks)
         elif key == "materialised":
