@@ -188,6 +188,11 @@ int64_t enumerate_tuples(const dyn_profile *p, const dyn_space *sp, int64_t limi
 
 constexpr int64_t kMaxTuples = int64_t(1) << 20;
 
+// entries the list of (tuple, TP index) pairs can take: one per tuple and index plus the padding of every index
+size_t mixed_pairs_capacity(int64_t K, int T) {
+    return K <= kMixedPairsMaxTuples ? size_t(K) * size_t(T) + size_t(T) * size_t(kMixedPairsChunk) : 0;
+}
+
 int check_mixed(const dyn_profile *p, const dyn_space *sp, int64_t S, int64_t W, ResolveParams *rp) {
     const int rc = check_problem(p, sp, S, W, rp);
     if (rc != DYN_OK) return rc;
@@ -402,7 +407,7 @@ size_t dyn_mixed_workspace_bytes(const dyn_profile *profile, const dyn_space *sp
     const int64_t K = dyn_mixed_tuple_count(profile, space);
     if (!base || K <= 0) return 0;
     return base + align256(size_t(K) * sizeof(uint2)) + align256(size_t(profile->C) * profile->T * sizeof(float)) +
-           align256(size_t(profile->C) * size_t(K) * sizeof(float));
+           align256(size_t(profile->C) * size_t(K) * sizeof(float)) + align256(mixed_pairs_capacity(K, profile->T) * sizeof(uint32_t));
 }
 
 int dyn_mixed_select(const dyn_profile *profile, const dyn_space *space, const float *d_load, int64_t S, int64_t W,
@@ -429,16 +434,33 @@ int dyn_mixed_select(const dyn_profile *profile, const dyn_space *space, const f
     const ResolvedLayout lay = resolved_layout(profile->C, profile->T, space->F, profile->M, space->Nmax, S, W);
     const size_t off_tuples = lay.total, off_caph = off_tuples + align256(size_t(K) * sizeof(uint2));
     const size_t off_inva = off_caph + align256(size_t(profile->C) * profile->T * sizeof(float));
-    const size_t need = off_inva + align256(size_t(profile->C) * size_t(K) * sizeof(float));
+    const size_t off_pairs = off_inva + align256(size_t(profile->C) * size_t(K) * sizeof(float));
+    const size_t need = off_pairs + align256(mixed_pairs_capacity(K, profile->T) * sizeof(uint32_t));
     rc = check_ws(d_ws, ws_bytes, need);
     if (rc != DYN_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     char *ws = static_cast<char *>(d_ws);
     // pageable host memory: the copy is staged before the call returns
     DYN_CUDA_TRY(cudaMemcpyAsync(ws + off_tuples, tuples.data(), size_t(K) * sizeof(uint2), cudaMemcpyHostToDevice, st));
+    // short lists: the (tuple, TP index) pairs that hold instances, by TP index and padded per index to whole
+    // chunks of a warp, so that the search spends no evaluation on a parallelism a tuple does not use
+    int64_t n_pairs = 0;
+    if (K <= kMixedPairsMaxTuples) {
+        static thread_local std::vector<uint32_t> pairs;
+        pairs.clear();
+        for (int t = 0; t < profile->T; ++t) {
+            for (int64_t k = 0; k < K; ++k) {
+                const uint32_t n = (tuples[size_t(k)].x >> (8 * t)) & 255u;
+                if (n) pairs.push_back(uint32_t(k) | (n << 16) | (uint32_t(t) << 24));
+            }
+            while (pairs.size() % size_t(kMixedPairsChunk)) pairs.push_back(uint32_t(t) << 24);     // no instance: never evaluated
+        }
+        n_pairs = int64_t(pairs.size());
+        DYN_CUDA_TRY(cudaMemcpyAsync(ws + off_pairs, pairs.data(), pairs.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, st));
+    }
     DYN_CUDA_TRY(launch_resolve(rp, lay, d_ws, st));
-    DYN_CUDA_TRY(launch_mixed(lay, d_ws, off_tuples, off_caph, off_inva, K, d_load, tiles, out->d_counts, out->d_freq,
-                              out->d_tuple, out->d_best_E, st));
+    DYN_CUDA_TRY(launch_mixed(lay, d_ws, off_tuples, off_caph, off_inva, off_pairs, n_pairs, K, d_load, tiles, out->d_counts,
+                              out->d_freq, out->d_tuple, out->d_best_E, st));
     SelectOut so{};
     so.best_idx = out->d_tuple; so.best_E = out->d_best_E; so.E_total = out->d_E_total; so.n_infeasible = out->d_n_infeasible;
     const int64_t chunks = totals_chunks(W);

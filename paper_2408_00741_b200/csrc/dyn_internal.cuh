@@ -110,9 +110,13 @@ cudaError_t launch_hier(const ResolveParams &rp, const ResolvedLayout &lay, void
                         int32_t *d_shard, int32_t *best_idx, float *best_E, cudaStream_t st);
 
 // pools that mix tensor parallelisms: `tuples` holds K count tuples, 8 bits per TP index
-cudaError_t launch_mixed(const ResolvedLayout &lay, void *d_ws, size_t off_tuples, size_t off_caph, size_t off_inva, int64_t K,
-                         const float *d_load, int64_t tiles, int32_t *d_counts, int32_t *d_freq, int32_t *d_tuple,
-                         float *d_best_E, cudaStream_t st);
+// `pairs` (n_pairs entries, 0: none): tuple index | count << 16 | TP index << 24, by TP index, every index padded to
+// whole chunks of kMixedPairsChunk entries; built for lists of at most kMixedPairsMaxTuples tuples
+constexpr int64_t kMixedPairsMaxTuples = 512;
+constexpr int kMixedPairsChunk = 64;
+cudaError_t launch_mixed(const ResolvedLayout &lay, void *d_ws, size_t off_tuples, size_t off_caph, size_t off_inva, size_t off_pairs,
+                         int64_t n_pairs, int64_t K, const float *d_load, int64_t tiles, int32_t *d_counts, int32_t *d_freq,
+                         int32_t *d_tuple, float *d_best_E, cudaStream_t st);
 
 // selection with re-configuration costs (shortest path over the windows)
 cudaError_t launch_reconf(const ResolvedLayout &lay, void *d_ws, size_t off_cost, size_t off_q, size_t off_from, size_t off_rt,

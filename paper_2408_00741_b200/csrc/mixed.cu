@@ -43,6 +43,8 @@ struct MixedArgs {
     float *caph;              // [C][T] capacity at the highest candidate frequency
     float *inva;              // [C][K] 1 / (sum_t n_t * capH_t) of every tuple (threshold variant)
     const uint2 *tuples;      // [K] {counts, 8 bits per TP index; tuple number}, sorted by the set of TP indices in use
+    const uint32_t *pairs;    // [n_pairs] tuple index | count << 16 | TP index << 24, by TP index, padded per index to whole chunks
+    int64_t n_pairs;
     const float *load;        // [tiles]
     int64_t tiles, K;
     int32_t C, T, F, M;
@@ -160,6 +162,73 @@ __global__ void __launch_bounds__(kThreads) mixed_select_kernel(const MixedArgs 
 }
 
 
+// End of a tile in the threshold variants: the warp's best tuple (least energy, lowest tuple number among equals)
+// from the lanes' candidates, its frequencies recovered with the arithmetic of the search, the results written.
+template <int T>
+__device__ __forceinline__ void finish_tile(const MixedArgs &a, const int64_t i, const int c, const int lane, float best,
+                                            const uint32_t bnum, const uint32_t btup, const float bfrac, const float (&caph)[T],
+                                            const uint32_t origin, const uint32_t rows2) {
+    const int F = a.F, P = T * F, RS = a.M + 1;
+    best += 0.f;                                         // -0 -> +0
+    const float Emin = warp_min(best);
+    const uint32_t kmin = __reduce_min_sync(kFull, best == Emin ? bnum : 0xffffffffu);
+    if (Emin == CUDART_INF_F) {
+        if (lane < T) {
+            a.counts[DYN_IDX(i * T + lane, a.tiles * T)] = -1;
+            a.freq[DYN_IDX(i * T + lane, a.tiles * T)] = -1;
+        }
+        if (lane == 0) {
+            a.tuple[DYN_IDX(i, a.tiles)] = -1;
+            a.best_E[i] = CUDART_INF_F;
+        }
+        return;
+    }
+    // the winning tuple and its load fraction, from the lane that holds it (tuple numbers are distinct)
+    const int wl = __ffs(__ballot_sync(kFull, best == Emin && bnum == kmin)) - 1;
+    const uint32_t wt = __shfl_sync(kFull, btup, wl);
+    const float wf = __shfl_sync(kFull, bfrac, wl);
+    // its frequencies: lane p re-evaluates pair (t, q) = (p / F, p % F) with the same arithmetic; per degree
+    // the least energy, lowest q among equals
+    float gmin[T];
+    int gq[T];
+#pragma unroll
+    for (int t = 0; t < T; ++t) { gmin[t] = CUDART_INF_F; gq[t] = -1; }
+    for (int p0 = 0; p0 < P; p0 += 32) {
+        const int p = p0 + lane;
+        const int tp = p < P ? p / F : 0;
+        float val = CUDART_INF_F;
+        if (p < P && ((wt >> (8 * tp)) & 255u)) {
+            float ctp = caph[0];
+#pragma unroll
+            for (int t = 1; t < T; ++t) ctp = (t == tp) ? caph[t] : ctp;
+            const float4 pc = load16<true>(a.ws, origin + uint32_t(c * P + p) * 16u);
+            float e;
+            bool ok;
+            fast_one<true>(a.ws, rows2 + uint32_t((c * P + p) * RS) * 8u, wf * ctp, pc.x, pc.z, e, ok);
+            if (ok) val = e;
+        }
+#pragma unroll
+        for (int t = 0; t < T; ++t) {
+            const bool mine = p < P && tp == t;
+            const float m = warp_min(mine ? val : CUDART_INF_F);
+            if (m < gmin[t]) {                           // strictly better than the earlier rounds (lower q)
+                gmin[t] = m;
+                gq[t] = p0 + __ffs(__ballot_sync(kFull, mine && val == m)) - 1 - t * F;
+            }
+        }
+    }
+    if (lane == 0) {
+#pragma unroll
+        for (int t = 0; t < T; ++t) {
+            const uint32_t n = (wt >> (8 * t)) & 255u;
+            a.counts[DYN_IDX(i * T + t, a.tiles * T)] = int32_t(n);
+            a.freq[i * T + t] = n ? gq[t] : -1;
+        }
+        a.tuple[DYN_IDX(i, a.tiles)] = int32_t(kmin);
+        a.best_E[i] = Emin;
+    }
+}
+
 // threshold variant: tables of all classes in shared memory, SL tuples per lane and pass (32 * SL tuples side by side;
 // the list is sorted by the set of degrees in use, and a pass skips the degrees none of its tuples uses: short
 // passes skip more, long ones share a pair's constants among more candidates)
@@ -258,72 +327,108 @@ __global__ void __launch_bounds__(kThreads, 3) mixed_fast_kernel(const MixedArgs
                     bfrac = frac[j];
                 }
         }
-        best += 0.f;                                         // -0 -> +0
-        const float Emin = warp_min(best);
-        const uint32_t kmin = __reduce_min_sync(kFull, best == Emin ? bnum : 0xffffffffu);
-        if (Emin == CUDART_INF_F) {
-            if (lane < T) {
-                a.counts[DYN_IDX(i * T + lane, a.tiles * T)] = -1;
-                a.freq[DYN_IDX(i * T + lane, a.tiles * T)] = -1;
-            }
-            if (lane == 0) {
-                a.tuple[DYN_IDX(i, a.tiles)] = -1;
-                a.best_E[i] = CUDART_INF_F;
-            }
+        finish_tile<T>(a, i, c, lane, best, bnum, btup, bfrac, caph, origin, rows2);
+    }
+}
+
+// threshold variant for short lists: the (tuple, TP index) pairs that hold instances are listed by TP index (the host
+// pads every index to whole chunks of 64 pairs), a warp takes a chunk at a time, two pairs per lane, against the F
+// table rows of the chunk's index, and adds n x (energy of one instance) to the tuple's sum in a per-warp array in
+// shared memory.  Chunks come in ascending TP index, so a tuple's sum forms in the same order as in the other
+// variants; no evaluation is spent on a parallelism that a tuple does not use.  Then the lanes scan the sums.
+template <int T>
+__global__ void __launch_bounds__(kThreads, 3) mixed_pairs_kernel(const MixedArgs a, const int table_bytes) {
+    __shared__ unsigned char s_general[256];
+    for (int c = threadIdx.x; c < a.C; c += blockDim.x) {
+        bool bad = false;
+        for (int p = 0; p < a.T * a.F; ++p) bad |= isnan(__ldg(a.pairc + c * a.T * a.F + p).y);
+        s_general[c] = bad ? 1 : 0;
+    }
+    extern __shared__ float4 smem[];
+    {
+        const float4 *src = reinterpret_cast<const float4 *>(a.ws + a.off_pair2);
+        const int n16 = (a.off_end - a.off_pair2) / 16;
+        for (int i = threadIdx.x; i < n16; i += blockDim.x) smem[i] = src[i];
+        __syncthreads();
+        DYN_SET_RANGES(uint32_t(__cvta_generic_to_shared(smem)), uint32_t(__cvta_generic_to_shared(smem)) + uint32_t(n16) * 16u,
+                       uint32_t(a.off_end));
+    }
+    uint32_t origin = table_origin<true>();
+    asm volatile("" : "+r"(origin) : : "memory");        // table loads stay behind the staging barrier
+    const int lane = threadIdx.x & 31;
+    const int K = int(a.K), Kpad = (K + 31) & ~31;
+    float *Es = reinterpret_cast<float *>(reinterpret_cast<char *>(smem) + table_bytes) + (threadIdx.x >> 5) * Kpad;   // this warp's sums
+    const int F = a.F, P = T * F, RS = a.M + 1;
+    const uint32_t pstep = uint32_t(RS) * 8u;
+    const uint32_t rows2 = origin + uint32_t(a.off_rows2 - a.off_pair2);
+    const uint64_t two23_2 = pack2(kTwo23, kTwo23);
+    const uint64_t eight2 = pack2(units(8u), units(8u));
+    const float offs = float(int(pstep)) * units(1u);
+    const uint64_t off2_step = pack2(offs, offs);
+    const int64_t nwarps = int64_t(gridDim.x) * kWarps;
+    for (int64_t i = int64_t(blockIdx.x) * kWarps + (threadIdx.x >> 5); i < a.tiles; i += nwarps) {
+        const int c = int(i % a.C);
+        if (s_general[c]) {                                  // warp-uniform
+            mixed_tile_plain<T>(a, i, lane);
             continue;
         }
-        // the winning tuple and its load fraction, from the lane that holds it (tuple numbers are distinct)
-        const int wl = __ffs(__ballot_sync(kFull, best == Emin && bnum == kmin)) - 1;
-        const uint32_t wt = __shfl_sync(kFull, btup, wl);
-        const float wf = __shfl_sync(kFull, bfrac, wl);
-        // its frequencies: lane p re-evaluates pair (t, q) = (p / F, p % F) with the same arithmetic; per degree
-        // the least energy, lowest q among equals
-        float gmin[T];
-        int gq[T];
+        const float L = fmaxf(a.load[DYN_IDX(i, a.tiles)], 0.f);              // negative / NaN -> 0
+        float caph[T];
 #pragma unroll
-        for (int t = 0; t < T; ++t) { gmin[t] = CUDART_INF_F; gq[t] = -1; }
-        for (int p0 = 0; p0 < P; p0 += 32) {
-            const int p = p0 + lane;
-            const int tp = p < P ? p / F : 0;
-            float val = CUDART_INF_F;
-            if (p < P && ((wt >> (8 * tp)) & 255u)) {
-                float ctp = caph[0];
+        for (int t = 0; t < T; ++t) caph[t] = a.caph[c * T + t];
+        const float *inva_c = a.inva + int64_t(c) * a.K;
+        for (int k = lane; k < Kpad; k += 32) Es[DYN_IDX(k, Kpad)] = 0.f;
+        __syncwarp();
+        for (int64_t e0 = 0; e0 < a.n_pairs; e0 += kMixedPairsChunk) {
+            const uint32_t entA = __ldg(a.pairs + DYN_IDX(e0 + lane, a.n_pairs)), entB = __ldg(a.pairs + DYN_IDX(e0 + 32 + lane, a.n_pairs));
+            const int t = int(__shfl_sync(kFull, entA, 0) >> 24);             // the chunk's TP index (the same in every entry)
+            const uint32_t kA = entA & 0xffffu, kB = entB & 0xffffu, nA = (entA >> 16) & 255u, nB = (entB >> 16) & 255u;
+            float ct = caph[0];
 #pragma unroll
-                for (int t = 1; t < T; ++t) ctp = (t == tp) ? caph[t] : ctp;
-                const float4 pc = load16<true>(a.ws, origin + uint32_t(c * P + p) * 16u);
-                float e;
-                bool ok;
-                fast_one<true>(a.ws, rows2 + uint32_t((c * P + p) * RS) * 8u, wf * ctp, pc.x, pc.z, e, ok);
-                if (ok) val = e;
+            for (int u = 1; u < T; ++u) ct = (u == t) ? caph[u] : ct;
+            // every instance of a tuple runs at the fraction L / A of its top-frequency capacity
+            const float lA = nA ? (L * __ldg(inva_c + DYN_IDX(kA, a.K))) * ct : CUDART_INF_F;
+            const float lB = nB ? (L * __ldg(inva_c + DYN_IDX(kB, a.K))) * ct : CUDART_INF_F;
+            const uint64_t ln2 = pack2(lA, lB);
+            float eA = CUDART_INF_F, eB = CUDART_INF_F;
+            const uint32_t cpair = origin + uint32_t(c * P + t * F) * 16u;
+            const float off0 = row_offset_units(rows2 + uint32_t((c * P + t * F) * RS) * 8u);
+            uint64_t off2 = pack2(off0, off0);
+#pragma unroll 4
+            for (int q = 0; q < F; ++q) {
+                uint64_t icm2, lim2;
+                asm("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(icm2), "=l"(lim2) : "r"(DYN_SMEM_ADDR(cpair + uint32_t(q) * 16u, 16u)));
+                const float lim = __uint_as_float(uint32_t(lim2));
+                fast_two(ln2, icm2, off2, two23_2, eight2, lim, lim, eA, eB);
+                off2 = add2(off2, off2_step);
             }
-#pragma unroll
-            for (int t = 0; t < T; ++t) {
-                const bool mine = p < P && tp == t;
-                const float m = warp_min(mine ? val : CUDART_INF_F);
-                if (m < gmin[t]) {                           // strictly better than the earlier rounds (lower q)
-                    gmin[t] = m;
-                    gq[t] = p0 + __ffs(__ballot_sync(kFull, mine && val == m)) - 1 - t * F;
-                }
+            // the pairs of a chunk belong to different tuples (one TP index): no two lanes meet on a sum
+            if (nA) Es[DYN_IDX(kA, Kpad)] += float(nA) * eA;                  // +inf if the group has no frequency
+            if (nB) Es[DYN_IDX(kB, Kpad)] += float(nB) * eB;
+            __syncwarp();
+        }
+        float best = CUDART_INF_F, bfrac = 0.f;
+        uint32_t bnum = 0xffffffffu, btup = 0;
+        for (int k = lane; k < K; k += 32) {
+            const float E = Es[DYN_IDX(k, Kpad)];
+            const uint2 tk = __ldg(a.tuples + k);
+            if (E < best || (E == best && tk.y < bnum)) {    // lowest tuple number on ties
+                best = E;
+                bnum = tk.y;
+                btup = tk.x;
+                bfrac = L * __ldg(inva_c + k);
             }
         }
-        if (lane == 0) {
-#pragma unroll
-            for (int t = 0; t < T; ++t) {
-                const uint32_t n = (wt >> (8 * t)) & 255u;
-                a.counts[DYN_IDX(i * T + t, a.tiles * T)] = int32_t(n);
-                a.freq[i * T + t] = n ? gq[t] : -1;
-            }
-            a.tuple[DYN_IDX(i, a.tiles)] = int32_t(kmin);
-            a.best_E[i] = Emin;
-        }
+        __syncwarp();                                        // the sums are read before the next tile clears them
+        finish_tile<T>(a, i, c, lane, best, bnum, btup, bfrac, caph, origin, rows2);
     }
 }
 
 }  // namespace
 
-cudaError_t launch_mixed(const ResolvedLayout &lay, void *d_ws, size_t off_tuples, size_t off_caph, size_t off_inva, int64_t K,
-                         const float *d_load, int64_t tiles, int32_t *d_counts, int32_t *d_freq, int32_t *d_tuple,
-                         float *d_best_E, cudaStream_t st) {
+cudaError_t launch_mixed(const ResolvedLayout &lay, void *d_ws, size_t off_tuples, size_t off_caph, size_t off_inva, size_t off_pairs,
+                         int64_t n_pairs, int64_t K, const float *d_load, int64_t tiles, int32_t *d_counts, int32_t *d_freq,
+                         int32_t *d_tuple, float *d_best_E, cudaStream_t st) {
     char *ws = static_cast<char *>(d_ws);
     MixedArgs a{};
     a.rows = reinterpret_cast<const float4 *>(ws + lay.off_rows);
@@ -332,6 +437,8 @@ cudaError_t launch_mixed(const ResolvedLayout &lay, void *d_ws, size_t off_tuple
     a.caph = reinterpret_cast<float *>(ws + off_caph);
     a.inva = reinterpret_cast<float *>(ws + off_inva);
     a.tuples = reinterpret_cast<const uint2 *>(ws + off_tuples);
+    a.pairs = reinterpret_cast<const uint32_t *>(ws + off_pairs);
+    a.n_pairs = n_pairs;
     a.load = d_load;
     a.tiles = tiles; a.K = K;
     a.C = lay.C; a.T = lay.T; a.F = lay.F; a.M = lay.M;
@@ -355,9 +462,17 @@ cudaError_t launch_mixed(const ResolvedLayout &lay, void *d_ws, size_t off_tuple
     const bool short_passes = K <= DYN_MIXED_SHORT;
     e = record_start(st);
     if (e != cudaSuccess) return e;
+    // short lists: the compact list of (tuple, TP index) pairs; per-warp sums behind the tables in shared memory
+    const size_t pairs_bytes = fast_bytes + size_t(kWarps) * size_t((K + 31) & ~int64_t(31)) * sizeof(float);
+    const bool use_pairs = a.use_fast && n_pairs > 0 && K <= kMixedPairsMaxTuples && K <= 0xffff;
 #define DYN_MIXED_LAUNCH(TT)                                                                                      \
     do {                                                                                                          \
-        if (a.use_fast) {                                                                                         \
+        if (use_pairs) {                                                                                          \
+            e = cudaFuncSetAttribute(mixed_pairs_kernel<TT>, cudaFuncAttributeMaxDynamicSharedMemorySize,         \
+                                     int(pairs_bytes));                                                           \
+            if (e != cudaSuccess) return e;                                                                       \
+            mixed_pairs_kernel<TT><<<int(grid), kThreads, pairs_bytes, st>>>(a, int(fast_bytes));                 \
+        } else if (a.use_fast) {                                                                                  \
             if (short_passes) {                                                                                   \
                 e = cudaFuncSetAttribute(mixed_fast_kernel<TT, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,   \
                                          int(fast_bytes));                                                        \
