@@ -206,6 +206,43 @@ __global__ void __launch_bounds__(256, FAST ? 4 : 1) hier_shard_kernel(const Hie
         e_floor *= 0.99999f;
         if (!(e_floor > 0.f)) e_floor = 0.f;          // no positive floor: no pruning
     }
+    // A sharper bound per degree: a line under the row's energy, e_t(l) >= alpha_t + beta_t * l on [0, limit] (beta_t the
+    // row's secant slope, alpha_t the least knot value of e - beta_t * l; the rows are piecewise linear, so the knots
+    // decide).  A pool of n instances at the epoch's peak PL then costs at least n * alpha_t + PL * beta_t at degree t
+    // (n * e_t(PL / n)), whatever segment PL / n falls in: a candidate whose bound reaches the best energy found is
+    // skipped, and once that holds for every degree and every alpha_t is non-negative (the bounds grow with n) the
+    // walk stops.  For a power model that is linear in the load the bound is the energy itself, so the walk ends
+    // right after the first feasible count.  (Both coefficients are taken a little low against rounding.)
+    float alpha[4], beta[4];
+    bool grows = true;                                // every bound is non-decreasing in n
+#pragma unroll
+    for (int t = 0; t < 4; ++t) { alpha[t] = 0.f; beta[t] = 0.f; }
+    if (packed) {
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            if (t >= a.T || !(llim[t] >= 0.f)) continue;
+            // knot m sits at l_m = m / icm; its energy is the segment's line there (the last knot closes segment M-2)
+            const float2 e0 = load8<true>(a.ws, row[t]);
+            const float2 eL = load8<true>(a.ws, row[t] + uint32_t(a.M - 2) * 8u);
+            const float lL = float(a.M - 1) / icm[t];
+            const float first = e0.x, last = fmaf(lL, eL.y, eL.x);
+            float b = lL > 0.f ? (last - first) / lL : 0.f;
+            if (!(b > 0.f) || !(b < CUDART_INF_F)) b = 0.f;
+            b *= 0.9999f;
+            float al = CUDART_INF_F;
+            for (int m = 0; m < a.M; ++m) {
+                const int seg = m < a.M - 1 ? m : a.M - 2;
+                const float2 en = load8<true>(a.ws, row[t] + uint32_t(seg) * 8u);
+                const float lm = float(m) / icm[t];
+                al = fminf(al, fmaf(lm, en.y, en.x) - b * lm);
+            }
+            al = al > 0.f ? al * 0.9999f : al * 1.0001f;
+            if (!(al > -CUDART_INF_F) || !(al < CUDART_INF_F)) { al = 0.f; b = 0.f; }
+            alpha[t] = al;
+            beta[t] = b;
+            grows = grows && al >= 0.f;
+        }
+    }
     const uint64_t two23_2 = pack2(kTwo23, kTwo23), eight2 = pack2(units(8u), units(8u));
     for (int64_t s = blockIdx.y; s < a.S; s += gridDim.y) {
         const float *ld = a.load + size_t(s) * size_t(a.W) * a.C + c;
@@ -219,39 +256,35 @@ __global__ void __launch_bounds__(256, FAST ? 4 : 1) hier_shard_kernel(const Hie
         float best = CUDART_INF_F;
         int bnt = -1;
         if (packed) {
-            int nlim[4];
-            float xmin = CUDART_INF_F;                // least n (as a real number) that carries PL at some degree
+            // Degree by degree: counts below the least one that carries PL at the degree are infeasible there and are
+            // not visited; from there on the counts are walked two at a time with the sweep's packed evaluation until
+            // the degree's bound (see above) or the energy floor reaches the best energy found.  Ties go to the lowest
+            // index (n - 1) * T + t, as in a walk in index order.
+            int bidx = 0x7fffffff;
 #pragma unroll
             for (int t = 0; t < 4; ++t) {
-                nlim[t] = t < a.T ? budget / a.tp[t < a.T ? t : 0] : 0;     // TP ascending: the limits descend
-                xmin = fminf(xmin, PL * inv_llim[t]);
-            }
-            // every n below xmin - 1 is infeasible at every degree by a margin of 1/n, far above rounding
-            int n = xmin < 300.f ? max(1, int(xmin) - 1) : nmax + 1;
-            int bn = 0;
-            for (; n <= nmax; n += 2) {
-                if (float(n) * e_floor >= best) break;       // n and every larger count cost at least `best`
-                const float lnA = PL * s_rn[DYN_IDX(n, 257)], lnB = n + 1 <= nmax ? PL * s_rn[DYN_IDX(n + 1, 257)] : CUDART_INF_F;
-                const uint64_t ln2 = pack2(lnA, lnB);
-                float eA = CUDART_INF_F, eB = CUDART_INF_F;
-#pragma unroll
-                for (int t = 0; t < 4; ++t)
-                    fast_two(ln2, icm2[t], off2[t], two23_2, eight2, n <= nlim[t] ? llim[t] : -1.f,
-                             n + 1 <= nlim[t] ? llim[t] : -1.f, eA, eB);
-                const float EA = float(n) * eA, EB = float(n + 1) * eB;
-                if (EA < best) { best = EA; bn = n; }         // ascending n: strict compare keeps the lowest
-                if (EB < best) { best = EB; bn = n + 1; }
-            }
-            if (bn > 0) {
-                const float nf = float(bn), ln = PL * s_rn[bn];
-#pragma unroll
-                for (int t = 3; t >= 0; --t) {               // descending, so the lowest matching degree stays
-                    float e;
-                    bool ok;
-                    fast_one<true>(a.ws, row[t], ln, icm[t], bn <= nlim[t] ? llim[t] : -1.f, e, ok);
-                    if (ok && nf * e == best) bnt = (bn - 1) * a.T + t;
+                if (t >= a.T || !(llim[t] >= 0.f)) continue;
+                int nl = budget / a.tp[t];
+                if (nl > a.Nmax) nl = a.Nmax;
+                const float plb = PL * beta[t];
+                float xf = PL * inv_llim[t] * 0.9999f;       // a little below the least count that carries PL here
+                if (!(xf < 1e9f)) xf = 1e9f;
+                int n = xf < 1.f ? 1 : (xf < 300.f ? int(xf) : nl + 1);
+                for (; n <= nl; n += 2) {
+                    const float nf = float(n);
+                    if (nf * e_floor >= best) break;         // n and every larger count cost more than `best`
+                    if (alpha[t] >= 0.f && fmaf(fmaxf(nf, xf), alpha[t], plb) >= best) break;   // so does every count from n on at this degree
+                    const bool two = n + 1 <= nl;
+                    const uint64_t ln2 = pack2(PL * s_rn[DYN_IDX(n, 257)], two ? PL * s_rn[DYN_IDX(n + 1, 257)] : CUDART_INF_F);
+                    float eA = CUDART_INF_F, eB = CUDART_INF_F;
+                    fast_two(ln2, icm2[t], off2[t], two23_2, eight2, llim[t], two ? llim[t] : -1.f, eA, eB);
+                    const float EA = nf * eA, EB = (nf + 1.0f) * eB;
+                    const int iA = (n - 1) * a.T + t, iB = n * a.T + t;
+                    if (EA < best || (EA == best && EA < CUDART_INF_F && iA < bidx)) { best = EA; bidx = iA; }
+                    if (EB < best || (EB == best && EB < CUDART_INF_F && iB < bidx)) { best = EB; bidx = iB; }
                 }
             }
+            if (best < CUDART_INF_F) bnt = bidx;
         } else
         for (int n = 1; n <= nmax; ++n) {
             const float nf = float(n), ln = PL * s_rn[n];
