@@ -7,6 +7,10 @@
 // a move sigma' -> sigma between consecutive windows costs R[sigma'][sigma] (the caller's table, Wh).
 //   reconf_cost_kernel  cost[s][c][w][sigma] and the frequency that attains it: one thread per entry, a warp
 //                       covers 32 shardings of one tile (one load, the table rows of T degrees), F evaluations each
+//   reconf_cost_fast_kernel  the same on the threshold tables in shared memory, the form the sweep uses: a warp takes a
+//                       tile, lanes hold instance counts, the (TP, f) pairs are the inner loop (packed evaluation of
+//                       two counts), the frequency is noted whenever the running minimum falls; classes with a row
+//                       that has no load threshold are evaluated as in reconf_cost_kernel
 //   reconf_path_kernel  one CTA per (scenario, class): forward recursion over the windows (min-plus product of the
 //                       state vector with R: add + min per step; R in shared memory as far as it fits, the state
 //                       vector too), the vectors written to global memory.  The running values are kept relative
@@ -15,6 +19,7 @@
 //                       same addition (lowest source on ties) and writes the chosen candidates.
 #define DYN_TU_ID 10
 #include "dyn_internal.cuh"
+#include "eval_dev.cuh"
 
 #include <cuda_pipeline.h>
 #include <math_constants.h>
@@ -41,6 +46,8 @@ struct ReconfArgs {
     int32_t *best_idx;
     float *best_E;
     double *path_total;       // [S][C]
+    const char *ws;           // scratch block (threshold tables at off_pair2 .. off_end)
+    int32_t off_pair2, off_rows2, off_end;
 };
 
 __global__ void __launch_bounds__(kThreads) reconf_cost_kernel(const ReconfArgs a) {
@@ -74,6 +81,121 @@ __global__ void __launch_bounds__(kThreads) reconf_cost_kernel(const ReconfArgs 
         }
         a.cost[DYN_IDX(e, total)] = best;
         a.qbest[DYN_IDX(e, total)] = uint8_t(bq);
+    }
+}
+
+// one entry of the cost tensor from the general-path tables (any class)
+__device__ __forceinline__ void cost_entry_general(const ReconfArgs &a, int c, float L, int g, float &best, int &bq) {
+    const int P = a.T * a.F, RS = a.M + 1;
+    const int n = g / a.T + 1, t = g - (n - 1) * a.T;
+    const float nf = float(n), ln = L * (1.0f / nf);
+    const float slo = a.slo[c];
+    best = CUDART_INF_F;
+    bq = 0;
+    if (a.budget <= 0 || int64_t(n) * a.tp[t] <= int64_t(a.budget)) {
+        const float4 *rows_t = a.rows + size_t(DYN_IDX(c * P + t * a.F, a.C * P - a.F + 1)) * RS;
+        const float2 *pc_t = a.pairc + DYN_IDX(c * P + t * a.F, a.C * P - a.F + 1);
+        for (int q = 0; q < a.F; ++q) {
+            bool ok;
+            const float E = eval_pair(rows_t + size_t(q) * RS, __ldg(pc_t + q).x, float(a.M), ln, nf, slo, ok);
+            if (ok && E < best) {                            // ascending q: strict compare keeps the lowest
+                best = E;
+                bq = q;
+            }
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads) reconf_cost_fast_kernel(const ReconfArgs a, const int table_bytes) {
+    __shared__ unsigned char s_general[256];
+    for (int c = threadIdx.x; c < a.C; c += blockDim.x) {
+        bool bad = false;
+        for (int p = 0; p < a.T * a.F; ++p) bad |= isnan(__ldg(a.pairc + c * a.T * a.F + p).y);
+        s_general[c] = bad ? 1 : 0;
+    }
+    extern __shared__ float4 smem[];
+    {
+        const float4 *src = reinterpret_cast<const float4 *>(a.ws + a.off_pair2);
+        const int n16 = (a.off_end - a.off_pair2) / 16;
+        for (int i = threadIdx.x; i < n16; i += blockDim.x) smem[i] = src[i];
+        __syncthreads();
+        DYN_SET_RANGES(uint32_t(__cvta_generic_to_shared(smem)), uint32_t(__cvta_generic_to_shared(smem)) + uint32_t(n16) * 16u,
+                       uint32_t(a.off_end));
+    }
+    uint32_t origin = table_origin<true>();
+    asm volatile("" : "+r"(origin) : : "memory");        // table loads stay behind the staging barrier
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, warps = kThreads / 32;
+    const int NS = a.NS, NS4 = (NS + 3) & ~3;
+    // this warp's results of a tile: NS costs, then NS frequencies
+    float *oc = reinterpret_cast<float *>(reinterpret_cast<char *>(smem) + table_bytes) + size_t(warp) * NS4;
+    unsigned char *oq = reinterpret_cast<unsigned char *>(reinterpret_cast<float *>(reinterpret_cast<char *>(smem) + table_bytes) +
+                                                          size_t(warps) * NS4) + size_t(warp) * NS4;
+    const int F = a.F, T = a.T, P = T * F, RS = a.M + 1;
+    const uint32_t pstep = uint32_t(RS) * 8u;
+    const uint32_t rows2 = origin + uint32_t(a.off_rows2 - a.off_pair2);
+    const uint64_t two23_2 = pack2(kTwo23, kTwo23);
+    const uint64_t eight2 = pack2(units(8u), units(8u));
+    const float offs = float(int(pstep)) * units(1u);
+    const uint64_t off2_step = pack2(offs, offs);
+    const int64_t tiles = a.S * a.C * a.W;
+    for (int64_t i = int64_t(blockIdx.x) * warps + warp; i < tiles; i += int64_t(gridDim.x) * warps) {
+        const int64_t w = i % a.W, sc = i / a.W;
+        const int c = int(sc % a.C);
+        const int64_t s = sc / a.C;
+        const float L = fmaxf(a.load[DYN_IDX((s * a.W + w) * a.C + c, a.S * a.W * a.C)], 0.f);
+        float *cost_i = a.cost + i * NS;
+        uint8_t *q_i = a.qbest + i * NS;
+        if (s_general[c]) {                                  // warp-uniform
+            for (int g = lane; g < NS; g += 32) {
+                float best;
+                int bq;
+                cost_entry_general(a, c, L, g, best, bq);
+                cost_i[DYN_IDX(g, NS)] = best;
+                q_i[DYN_IDX(g, NS)] = uint8_t(bq);
+            }
+            continue;
+        }
+        for (int k0 = 0; k0 < a.Nmax; k0 += 64) {
+            const int nA = k0 + lane + 1, nB = nA + 32;
+            const bool inA = nA <= a.Nmax, inB = nB <= a.Nmax;
+            const float nfA = float(nA), nfB = float(nB);
+            const uint64_t ln2 = pack2(inA ? L * (1.0f / nfA) : CUDART_INF_F, inB ? L * (1.0f / nfB) : CUDART_INF_F);
+            for (int t = 0; t < T; ++t) {
+                const int tpt = __ldg(a.tp + t);
+                const bool okA = inA && (a.budget <= 0 || int64_t(nA) * tpt <= int64_t(a.budget));
+                const bool okB = inB && (a.budget <= 0 || int64_t(nB) * tpt <= int64_t(a.budget));
+                float eA = CUDART_INF_F, eB = CUDART_INF_F;
+                int qA = 0, qB = 0;
+                const uint32_t cpair = origin + uint32_t(c * P + t * F) * 16u;
+                const float off0 = row_offset_units(rows2 + uint32_t((c * P + t * F) * RS) * 8u);
+                uint64_t off2 = pack2(off0, off0);
+#pragma unroll 4
+                for (int q = 0; q < F; ++q) {
+                    uint64_t icm2, lim2;
+                    asm("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(icm2), "=l"(lim2) : "r"(DYN_SMEM_ADDR(cpair + uint32_t(q) * 16u, 16u)));
+                    const float lim = __uint_as_float(uint32_t(lim2));
+                    const float pA = eA, pB = eB;
+                    fast_two(ln2, icm2, off2, two23_2, eight2, okA ? lim : -1.f, okB ? lim : -1.f, eA, eB);
+                    qA = eA < pA ? q : qA;                   // ascending q: the lowest frequency that attains the minimum
+                    qB = eB < pB ? q : qB;
+                    off2 = add2(off2, off2_step);
+                }
+                if (inA) {
+                    oc[DYN_IDX((nA - 1) * T + t, NS4)] = nfA * eA;           // +inf where no frequency is feasible
+                    oq[DYN_IDX((nA - 1) * T + t, NS4)] = (unsigned char)qA;
+                }
+                if (inB) {
+                    oc[DYN_IDX((nB - 1) * T + t, NS4)] = nfB * eB;
+                    oq[DYN_IDX((nB - 1) * T + t, NS4)] = (unsigned char)qB;
+                }
+            }
+        }
+        __syncwarp();
+        for (int g = lane; g < NS; g += 32) {
+            cost_i[DYN_IDX(g, NS)] = oc[g];
+            q_i[DYN_IDX(g, NS)] = oq[g];
+        }
+        __syncwarp();                                        // the tile is out before the next one overwrites it
     }
 }
 
@@ -459,8 +581,24 @@ cudaError_t launch_reconf(const ResolvedLayout &lay, void *d_ws, size_t off_cost
         int64_t grid = (total + kThreads - 1) / kThreads;
         const int64_t cap = int64_t(sm_count()) * 16;
         if (grid > cap) grid = cap;
-        reconf_cost_kernel<<<unsigned(grid), kThreads, 0, st>>>(a);
-        cudaError_t e = cudaGetLastError();
+        // threshold tables and a tile's results per warp in shared memory when they fit
+        const size_t table_bytes = lay.off_tp - lay.off_pair2;
+        const int NS4c = (a.NS + 3) & ~3;
+        const size_t fast_smem = table_bytes + size_t(kThreads / 32) * NS4c * (sizeof(float) + 1);
+        cudaError_t e;
+        if (fast_smem <= 96 * 1024 && lay.F <= 256) {
+            a.ws = ws;
+            a.off_pair2 = int32_t(lay.off_pair2); a.off_rows2 = int32_t(lay.off_rows2); a.off_end = int32_t(lay.off_tp);
+            if ((e = cudaFuncSetAttribute(reconf_cost_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(fast_smem))) != cudaSuccess)
+                return e;
+            int64_t g2 = (S * lay.C * W + kThreads / 32 - 1) / (kThreads / 32);
+            const int64_t cap2 = int64_t(sm_count()) * 4;
+            if (g2 > cap2) g2 = cap2;
+            reconf_cost_fast_kernel<<<unsigned(g2), kThreads, fast_smem, st>>>(a, int(table_bytes));
+        } else {
+            reconf_cost_kernel<<<unsigned(grid), kThreads, 0, st>>>(a);
+        }
+        e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
     int dev = 0, lim = 48 * 1024;
