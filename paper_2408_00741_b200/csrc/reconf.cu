@@ -281,11 +281,12 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
     // the rest, split evenly over the source groups
     const int n_rest = NS > rows_sr ? NS - rows_sr : 0;
     const int g_lo = rows_sr + int(int64_t(hg) * n_rest / G), g_hi = worker ? rows_sr + int(int64_t(hg + 1) * n_rest / G) : g_lo;
-    // Two barriers per window.  Dp holds the vector of the previous window as computed (not yet relative to its
-    // minimum); the minimum is gathered with one shared atomic per warp on an order-preserving integer key, in
-    // one of two slots that alternate between windows.  A thread owns entries tid, tid + kPathThreads, ... (kOwn of
-    // them) of the vector outside the scan.  Padding entries past NS are sources that never win: +inf.
-    __shared__ unsigned int s_min[2];
+    // Two barriers per window.  Dp holds the vector of the previous window as computed; every fourth window (and the
+    // last) its minimum is gathered with one shared atomic per warp on an order-preserving integer key (two slots
+    // that alternate, a third for the last window) and comes off the vector of the window after.  A thread owns
+    // entries tid, tid + kPathThreads, ... (kOwn of them) of the vector outside the scan and writes them to `hist`
+    // as it forms them.  Padding entries past NS are sources that never win: +inf.
+    __shared__ unsigned int s_min[3];                        // two alternating slots for every fourth window, one for the last
     auto key_of = [](float v) {
         const unsigned int b = __float_as_uint(v);
         return b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
@@ -296,7 +297,7 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
         asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(wm) : "f"(lmin));
         if ((tid & 31) == 0) atomicMin(&s_min[slot], key_of(wm));
     };
-    if (tid == 0) s_min[0] = s_min[1] = 0xffffffffu;
+    if (tid == 0) s_min[0] = s_min[1] = s_min[2] = 0xffffffffu;
     __syncthreads();
     double base = 0.0;
     {
@@ -304,9 +305,10 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
         for (int g = tid; g < NS4; g += kPathThreads) {
             const float v = g < NS ? (W > 0 ? cost[g] : 0.f) : CUDART_INF_F;
             Dp[g] = v;
+            if (g < NS && W > 0) hist[g] = v;                // row 0: the first window's vector as held
             lmin = fminf(lmin, v);
         }
-        publish_min(lmin, 0);
+        publish_min(lmin, W == 1 ? 2 : 0);
     }
     // The window costs come from DRAM; a thread asks for its own entries of the next kRing windows ahead of time
     // (asynchronous copies into a ring in shared memory, one group per window), so the recursion never waits
@@ -321,11 +323,15 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
     for (int64_t w = 1; w < W; ++w) {
         // keep differences only: the minimum of the previous vector goes to the fp64 base (all +inf stays +inf) and
         // is taken off the vector computed in this window
-        const float mprev = val_of(s_min[(w - 1) & 1]);
+        // (the minimum is gathered for every fourth window only: between two of them the values grow by a few
+        // windows' costs, which fp32 resolves just as well)
+        const bool had_min = ((w - 1) & 3) == 0;             // the previous window published its minimum
+        const float mprev = had_min ? val_of(s_min[((w - 1) >> 2) & 1]) : 0.f;
         const float shift = (mprev < CUDART_INF_F) ? mprev : 0.f;
         base += double(shift);
-        if (tid == 0) s_min[w & 1] = 0xffffffffu;            // this window's slot; last read before the previous barrier
-        for (int g = tid; g < NS; g += kPathThreads) hist[DYN_IDX((w - 1) * NS + g, W * NS)] = Dp[DYN_IDX(g, NS4)];
+        const bool pub = (w & 3) == 0 || w == W - 1;         // this window publishes; the last window has a slot of its own
+        const int pub_slot = w == W - 1 ? 2 : int((w >> 2) & 1);
+        if (tid == 0 && pub && w != W - 1) s_min[pub_slot] = 0xffffffffu;   // last read eight windows ago
         if (worker) {
             float b0 = CUDART_INF_F, b1 = CUDART_INF_F, b2 = CUDART_INF_F, b3 = CUDART_INF_F;
 #pragma unroll 1
@@ -369,10 +375,11 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
                 // instead of one per source in the scan; the values stay within two windows' growth of zero
                 const float d = (cslot[DYN_IDX(g, NS4)] + best) - shift;
                 Dp[DYN_IDX(g, NS4)] = d;
+                hist[DYN_IDX(w * NS + g, W * NS)] = d;       // the vector as held: the walk back reads it
                 lmin = fminf(lmin, d);
             }
         }
-        publish_min(lmin, int(w & 1));
+        if (pub) publish_min(lmin, pub_slot);
         // the slot is free (its values went into the minimum just published): ask for the costs kRing windows on
         if (w + kRing < W)
             for (int g = tid; g < NS; g += kPathThreads)
@@ -380,13 +387,12 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
         __pipeline_commit();
         __syncthreads();                                     // publishes Dp and the minimum
     }
-    const float m = W > 0 ? val_of(s_min[(W - 1) & 1]) : 0.f;      // minimum of the last vector (relative to `base`)
+    const float m = W > 0 ? val_of(s_min[2]) : 0.f;          // minimum of the last vector (relative to `base`)
     if (W == 0) {
         if (tid == 0) a.path_total[sc] = 0.0;
         return;
     }
-    // the last window's vector goes to the row of `hist` that the recursion leaves free; the walk back starts there
-    for (int g = tid; g < NS; g += kPathThreads) hist[DYN_IDX((W - 1) * NS + g, W * NS)] = Dp[g];
+    // (every window's vector, the last one included, went to `hist` as it was formed; the walk back starts at the last)
     if (tid == 0) a.path_total[sc] = (m < CUDART_INF_F) ? base + double(m) : double(CUDART_INF_F);
 }
 
