@@ -226,7 +226,15 @@ constexpr int kOwn = 4;                         // entries of the state vector a
 
 // R[h][g]: rows_s rows sit in shared memory, NS4 + 4 floats per row (NS4 = NS rounded up to a multiple of 4; the
 // pieces stay 16-byte aligned), pairs of rows interleaved as described at the copy loop
-// One CTA per (scenario, class).  Dynamic shared memory: Dp[NS4] | part[G][NS4] | cring[kRing][NS4] | Rs[rows_s / 2][2][NS4 + 4].
+// One CTA per (scenario, class).  Dynamic shared memory: Dp[NS4] | part[G][NS4] | cring[kRing][NS4] | rlo[NS4] | Rs[rows_s / 2][2][NS4 + 4].
+// Sources that cannot attain any minimum are skipped, four at a time: with a reference state h0 every target g has
+// min_h (D(h) + R[h][g]) <= D(h0) + R[h0][g] <= D(h0) + max_g R[h0][g] =: bound, while source h offers at least
+// D(h) + min_g R[h][g] =: D(h) + rlo(h); a quad of sources whose four values D(h) + rlo(h) all exceed the bound is not
+// scanned (rounding is monotone, so the comparison of the rounded sums decides the same way as the exact one would for
+// the rounded candidates: the minima formed are bit for bit those of the full scan).  h0 is the state that attained
+// the last gathered minimum; any state gives a valid bound.  Where transitions cost little next to the spread of the
+// window costs over the shardings -- the regime of the paper's overhead table -- most quads are skipped; with a
+// prohibitive table none is, and the test costs a few instructions per quad.
 // Forward: D_w(g) = cost_w(g) + min_h (D_{w-1}(h) + R[h][g]).  Only the minimum is formed here (half a packed add and half a three-input min per
 // step): a thread takes four neighbouring targets and a share of the sources, four sources per trip (one 16-byte
 // read of the state vector, four of R).  The values D_{w-1}, as held (relative to the running base), are written to `hist`,
@@ -240,7 +248,9 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
     float *Dp = reinterpret_cast<float *>(smem4);
     float *part = Dp + NS4;
     float *cring = part + size_t(G) * NS4;                   // [kRing][NS4]: costs of the next windows
-    float *Rs = cring + size_t(kRing) * NS4;
+    float *rlo = cring + size_t(kRing) * NS4;               // [NS4] least entry of every row of R (+inf past NS)
+    float *Rs = rlo + NS4;
+    __shared__ float s_rhi[1024];                            // largest entry of every row of R (NS <= 1024)
     const int64_t sc = blockIdx.x;                           // s * C + c
     const int64_t W = a.W;
     const float *cost = a.cost + sc * W * NS;
@@ -258,6 +268,23 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
         const int h = i / RSd, g = i - h * RSd, j = g & 3;
         Rs[DYN_IDX(size_t(h >> 1) * (2 * RSd) + (j >> 1) * RSd + (g & ~3) + (j & 1) * 2 + (h & 1), size_t(rows_s) * RSd)] =
             g < NS ? a.R[DYN_IDX(size_t(h) * NS + g, size_t(NS) * NS)] : 0.f;
+    }
+    // least and largest entry of every row: a warp per row, lanes across it
+    for (int h = tid >> 5; h < NS4; h += kPathThreads / 32) {
+        float lo = CUDART_INF_F, hi = -CUDART_INF_F;
+        if (h < NS)
+            for (int g = tid & 31; g < NS; g += 32) {
+                const float v = __ldg(a.R + DYN_IDX(size_t(h) * NS + g, size_t(NS) * NS));
+                lo = fminf(lo, v);
+                hi = fmaxf(hi, v);
+            }
+        float wlo, whi;
+        asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(wlo) : "f"(lo));
+        asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(whi) : "f"(hi));
+        if ((tid & 31) == 0) {
+            rlo[h] = wlo;                                    // +inf past NS: such a source is never scanned
+            if (h < 1024) s_rhi[h] = whi;
+        }
     }
     // rows of R that do not fit in shared memory: the first G * kRegRows of them stay in registers, each source
     // group holding kRegRows rows (its four columns of them); any further rows are read through L1 / L2
@@ -281,34 +308,54 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
     // the rest, split evenly over the source groups
     const int n_rest = NS > rows_sr ? NS - rows_sr : 0;
     const int g_lo = rows_sr + int(int64_t(hg) * n_rest / G), g_hi = worker ? rows_sr + int(int64_t(hg + 1) * n_rest / G) : g_lo;
-    // Two barriers per window.  Dp holds the vector of the previous window as computed; every fourth window (and the
-    // last) its minimum is gathered with one shared atomic per warp on an order-preserving integer key (two slots
-    // that alternate, a third for the last window) and comes off the vector of the window after.  A thread owns
-    // entries tid, tid + kPathThreads, ... (kOwn of them) of the vector outside the scan and writes them to `hist`
-    // as it forms them.  Padding entries past NS are sources that never win: +inf.
-    __shared__ unsigned int s_min[3];                        // two alternating slots for every fourth window, one for the last
-    auto key_of = [](float v) {
-        const unsigned int b = __float_as_uint(v);
-        return b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
-    };
-    auto val_of = [](unsigned int k) { return __uint_as_float(k ^ ((k >> 31) ? 0x80000000u : 0xffffffffu)); };
-    auto publish_min = [&](float lmin, int slot) {
+    // Two barriers per window.  Dp holds the vector of the previous window as computed.  Its minimum and a state that
+    // attains it are gathered without atomics: every warp leaves the minimum of its threads' entries and where it
+    // sits in a slot of its own, and at the start of the next window every thread takes the least of the
+    // kPathThreads / 32 slots.  The minimum comes off the vector of the window after (one window late); the state is
+    // the reference of the bound that lets the scan skip sources.  A thread owns entries tid, tid + kPathThreads, ...
+    // (kOwn of them) of the vector outside the scan and writes them to `hist` as it forms them.  Padding entries past
+    // NS are sources that never win: +inf.
+    constexpr int kPW = kPathThreads / 32;
+    __shared__ __align__(16) float s_wmin[kPW];
+    __shared__ __align__(16) int s_warg[kPW];
+    auto publish_min = [&](float lmin, int larg) {           // larg: an entry of this thread that holds lmin (any valid state if none)
         float wm;
         asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(wm) : "f"(lmin));
-        if ((tid & 31) == 0) atomicMin(&s_min[slot], key_of(wm));
+        const int src = __ffs(__ballot_sync(0xffffffffu, lmin == wm)) - 1;       // some lane holds it (no NaNs here)
+        const int arg = __shfl_sync(0xffffffffu, larg, src);
+        if ((tid & 31) == 0) {
+            s_wmin[tid >> 5] = wm;
+            s_warg[tid >> 5] = arg;
+        }
     };
-    if (tid == 0) s_min[0] = s_min[1] = s_min[2] = 0xffffffffu;
+    auto gathered_min = [&](int &arg) {                      // least slot (the lowest warp among equals) and its state
+        float m = s_wmin[0];
+        arg = s_warg[0];
+#pragma unroll
+        for (int k = 1; k < kPW; ++k) {
+            const float v = s_wmin[k];
+            if (v < m) {
+                m = v;
+                arg = s_warg[k];
+            }
+        }
+        return m;
+    };
     __syncthreads();
     double base = 0.0;
     {
         float lmin = CUDART_INF_F;
+        int larg = 0;
         for (int g = tid; g < NS4; g += kPathThreads) {
             const float v = g < NS ? (W > 0 ? cost[g] : 0.f) : CUDART_INF_F;
             Dp[g] = v;
             if (g < NS && W > 0) hist[g] = v;                // row 0: the first window's vector as held
-            lmin = fminf(lmin, v);
+            if (v < lmin) {
+                lmin = v;
+                larg = g;
+            }
         }
-        publish_min(lmin, W == 1 ? 2 : 0);
+        publish_min(lmin, larg);
     }
     // The window costs come from DRAM; a thread asks for its own entries of the next kRing windows ahead of time
     // (asynchronous copies into a ring in shared memory, one group per window), so the recursion never waits
@@ -323,19 +370,32 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
     for (int64_t w = 1; w < W; ++w) {
         // keep differences only: the minimum of the previous vector goes to the fp64 base (all +inf stays +inf) and
         // is taken off the vector computed in this window
-        // (the minimum is gathered for every fourth window only: between two of them the values grow by a few
-        // windows' costs, which fp32 resolves just as well)
-        const bool had_min = ((w - 1) & 3) == 0;             // the previous window published its minimum
-        const float mprev = had_min ? val_of(s_min[((w - 1) >> 2) & 1]) : 0.f;
+        int h0;
+        const float mprev = gathered_min(h0);
         const float shift = (mprev < CUDART_INF_F) ? mprev : 0.f;
         base += double(shift);
-        const bool pub = (w & 3) == 0 || w == W - 1;         // this window publishes; the last window has a slot of its own
-        const int pub_slot = w == W - 1 ? 2 : int((w >> 2) & 1);
-        if (tid == 0 && pub && w != W - 1) s_min[pub_slot] = 0xffffffffu;   // last read eight windows ago
+        const float bound = mprev + s_rhi[DYN_IDX(h0, 1024)];               // D(h0) = mprev
+        auto quad_live = [&](int qd) {                       // some source of quad qd can still attain a minimum
+            const float4 d4 = reinterpret_cast<const float4 *>(Dp)[DYN_IDX(qd, TG)];
+            const float4 m4 = reinterpret_cast<const float4 *>(rlo)[DYN_IDX(qd, TG)];
+            return fminf(fminf(d4.x + m4.x, d4.y + m4.y), fminf(d4.z + m4.z, d4.w + m4.w)) <= bound;
+        };
+        // which quads of this warp's source group are live: one lane per quad, gathered by a vote (bit b of live_s:
+        // shared-memory quad q_lo + b, the first 32 of them; bit j of live_r: register quad j)
+        uint32_t live_s = 0xffffffffu, live_r = 0xffffffffu;
+        if (hg < G) {                                        // the same in every thread of a warp
+            const int lane = tid & 31;
+            const int nsm = int(int64_t(hg + 1) * SQ / G) - q_lo;
+            live_s = __ballot_sync(0xffffffffu, lane < nsm && quad_live(q_lo + lane));
+            const int hq = h_reg / 4 + lane;
+            live_r = __ballot_sync(0xffffffffu, lane < kRegRows / 4 && hq < TG && quad_live(hq));
+        }
         if (worker) {
             float b0 = CUDART_INF_F, b1 = CUDART_INF_F, b2 = CUDART_INF_F, b3 = CUDART_INF_F;
-#pragma unroll 1
-            for (int q = q_lo; q < q_hi; ++q) {
+            // only the live quads are visited: the set bits of the votes, then any shared-memory quads beyond the 32
+            // a vote covers (those are scanned in full)
+            for (uint32_t m = live_s; m; m &= m - 1u) {
+                const int q = q_lo + __ffs(int(m)) - 1;
                 const float4 d4 = reinterpret_cast<const float4 *>(Dp)[DYN_IDX(q, TG)];
                 const float *rq = Rs + DYN_IDX(size_t(2 * q) * (2 * RSd) + 4 * tg, size_t(rows_s) * RSd - 3 * RSd - 3);
                 relax_pair(b0, b1, b2, b3, make_float2(d4.x, d4.y), *reinterpret_cast<const float4 *>(rq),
@@ -343,16 +403,36 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
                 relax_pair(b0, b1, b2, b3, make_float2(d4.z, d4.w), *reinterpret_cast<const float4 *>(rq + 2 * RSd),
                            *reinterpret_cast<const float4 *>(rq + 3 * RSd));
             }
-#pragma unroll
-            for (int j4 = 0; j4 < kRegRows / 4; ++j4) {
-                // past the last quad of the vector the rows hold +inf, so any entries of the vector will do
-                const int hq = h_reg / 4 + j4 < TG ? h_reg / 4 + j4 : TG - 1;
-                const float4 d4 = reinterpret_cast<const float4 *>(Dp)[hq];
-                relax_pair(b0, b1, b2, b3, make_float2(d4.x, d4.y), rp0[2 * j4], rp1[2 * j4]);
-                relax_pair(b0, b1, b2, b3, make_float2(d4.z, d4.w), rp0[2 * j4 + 1], rp1[2 * j4 + 1]);
+#pragma unroll 1
+            for (int q = q_lo + 32; q < q_hi; ++q) {
+                const float4 d4 = reinterpret_cast<const float4 *>(Dp)[DYN_IDX(q, TG)];
+                const float *rq = Rs + DYN_IDX(size_t(2 * q) * (2 * RSd) + 4 * tg, size_t(rows_s) * RSd - 3 * RSd - 3);
+                relax_pair(b0, b1, b2, b3, make_float2(d4.x, d4.y), *reinterpret_cast<const float4 *>(rq),
+                           *reinterpret_cast<const float4 *>(rq + RSd));
+                relax_pair(b0, b1, b2, b3, make_float2(d4.z, d4.w), *reinterpret_cast<const float4 *>(rq + 2 * RSd),
+                           *reinterpret_cast<const float4 *>(rq + 3 * RSd));
+            }
+            // register quads: a jump per live quad into the code that names its registers
+            static_assert(kRegRows == 40, "ten register quads are spelled out below");
+            for (uint32_t m = live_r; m; m &= m - 1u) {
+                const int j4 = __ffs(int(m)) - 1;
+                const float4 d4 = reinterpret_cast<const float4 *>(Dp)[DYN_IDX(h_reg / 4 + j4, TG)];
+                const float2 dA = make_float2(d4.x, d4.y), dB = make_float2(d4.z, d4.w);
+                switch (j4) {
+#define DYN_REG_QUAD(J)                                              \
+    case J:                                                          \
+        relax_pair(b0, b1, b2, b3, dA, rp0[2 * J], rp1[2 * J]);         \
+        relax_pair(b0, b1, b2, b3, dB, rp0[2 * J + 1], rp1[2 * J + 1]); \
+        break;
+                    DYN_REG_QUAD(0) DYN_REG_QUAD(1) DYN_REG_QUAD(2) DYN_REG_QUAD(3) DYN_REG_QUAD(4)
+                    DYN_REG_QUAD(5) DYN_REG_QUAD(6) DYN_REG_QUAD(7) DYN_REG_QUAD(8) DYN_REG_QUAD(9)
+#undef DYN_REG_QUAD
+                    default: break;
+                }
             }
             for (int h = g_lo; h < g_hi; ++h) {
                 const float d = Dp[h];
+                if (!(d + rlo[h] <= bound)) continue;
                 const float *row = a.R + size_t(h) * NS + 4 * tg;
                 b0 = fminf(b0, d + __ldg(row));
                 if (4 * tg + 1 < NS) b1 = fminf(b1, d + __ldg(row + 1));
@@ -363,6 +443,7 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
         }
         __syncthreads();                                     // every reader of Dp is done; the partial minima are in
         float lmin = CUDART_INF_F;
+        int larg = 0;
         __pipeline_wait_prior(kRing - 1);                    // this window's costs have arrived (the thread's own entries)
         float *cslot = cring + size_t(w % kRing) * NS4;
 #pragma unroll
@@ -376,10 +457,13 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
                 const float d = (cslot[DYN_IDX(g, NS4)] + best) - shift;
                 Dp[DYN_IDX(g, NS4)] = d;
                 hist[DYN_IDX(w * NS + g, W * NS)] = d;       // the vector as held: the walk back reads it
-                lmin = fminf(lmin, d);
+                if (d < lmin) {
+                    lmin = d;
+                    larg = g;
+                }
             }
         }
-        if (pub) publish_min(lmin, pub_slot);
+        publish_min(lmin, larg);
         // the slot is free (its values went into the minimum just published): ask for the costs kRing windows on
         if (w + kRing < W)
             for (int g = tid; g < NS; g += kPathThreads)
@@ -387,7 +471,8 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
         __pipeline_commit();
         __syncthreads();                                     // publishes Dp and the minimum
     }
-    const float m = W > 0 ? val_of(s_min[2]) : 0.f;          // minimum of the last vector (relative to `base`)
+    int h_last;
+    const float m = W > 0 ? gathered_min(h_last) : 0.f;      // minimum of the last vector (relative to `base`)
     if (W == 0) {
         if (tid == 0) a.path_total[sc] = 0.0;
         return;
@@ -549,11 +634,11 @@ __global__ void __launch_bounds__(kBackThreads) reconf_back_kernel(const ReconfA
 // rows of R kept in shared memory for NS states, given the device's limit
 static size_t reconf_fixed_floats(int32_t NS) {
     const int NS4 = (NS + 3) & ~3, TG = NS4 / 4, lanes_t = (TG + 31) / 32 * 32, G = kPathThreads / lanes_t;
-    return size_t(1 + G + kRing) * NS4;
+    return size_t(1 + G + kRing + 1) * NS4;
 }
 static int reconf_rows_in_smem(int32_t NS, size_t limit) {
     const int NS4 = (NS + 3) & ~3;
-    const size_t fixed = reconf_fixed_floats(NS) * sizeof(float) + 1024;
+    const size_t fixed = reconf_fixed_floats(NS) * sizeof(float) + 6144;      // the kernel's static shared memory on top
     if (limit <= fixed) return 0;
     int64_t rows = int64_t((limit - fixed) / (size_t(NS4 + 4) * sizeof(float)));
     // the registers come first (no shared-memory traffic): shared memory holds what they leave
