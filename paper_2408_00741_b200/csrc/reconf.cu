@@ -221,12 +221,11 @@ __device__ __forceinline__ void relax_pair(float &b0, float &b1, float &b2, floa
 
 constexpr int kPathThreads = 256;
 constexpr int kRegRows = 40;                    // rows of R a thread keeps in registers (its four columns of them); whole quads
-constexpr int kRing = 4;                        // windows whose costs are on their way into shared memory
 constexpr int kOwn = 4;                         // entries of the state vector a thread owns outside the scan (NS <= 1024)
 
 // R[h][g]: rows_s rows sit in shared memory, NS4 + 4 floats per row (NS4 = NS rounded up to a multiple of 4; the
 // pieces stay 16-byte aligned), pairs of rows interleaved as described at the copy loop
-// One CTA per (scenario, class).  Dynamic shared memory: Dp[NS4] | part[G][NS4] | cring[kRing][NS4] | rlo[NS4] | Rs[rows_s / 2][2][NS4 + 4].
+// One CTA per (scenario, class).  Dynamic shared memory: Dp[NS4] | part[G][NS4] | rlo[NS4] | Rs[rows_s / 2][2][NS4 + 4].
 // Sources that cannot attain any minimum are skipped, four at a time: with a reference state h0 every target g has
 // min_h (D(h) + R[h][g]) <= D(h0) + R[h0][g] <= D(h0) + max_g R[h0][g] =: bound, while source h offers at least
 // D(h) + min_g R[h][g] =: D(h) + rlo(h); a quad of sources whose four values D(h) + rlo(h) all exceed the bound is not
@@ -247,8 +246,7 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
     const int G = kPathThreads / lanes_t;                    // thread groups that split the sources
     float *Dp = reinterpret_cast<float *>(smem4);
     float *part = Dp + NS4;
-    float *cring = part + size_t(G) * NS4;                   // [kRing][NS4]: costs of the next windows
-    float *rlo = cring + size_t(kRing) * NS4;               // [NS4] least entry of every row of R (+inf past NS)
+    float *rlo = part + size_t(G) * NS4;                   // [NS4] least entry of every row of R (+inf past NS)
     float *Rs = rlo + NS4;
     __shared__ float s_rhi[1024];                            // largest entry of every row of R (NS <= 1024)
     const int64_t sc = blockIdx.x;                           // s * C + c
@@ -321,11 +319,9 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
     auto publish_min = [&](float lmin, int larg) {           // larg: an entry of this thread that holds lmin (any valid state if none)
         float wm;
         asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(wm) : "f"(lmin));
-        const int src = __ffs(__ballot_sync(0xffffffffu, lmin == wm)) - 1;       // some lane holds it (no NaNs here)
-        const int arg = __shfl_sync(0xffffffffu, larg, src);
-        if ((tid & 31) == 0) {
+        if (lmin == wm) {                                    // some lane holds it (no NaNs here); any of them will do
             s_wmin[tid >> 5] = wm;
-            s_warg[tid >> 5] = arg;
+            s_warg[tid >> 5] = larg;
         }
     };
     auto gathered_min = [&](int &arg) {                      // least slot (the lowest warp among equals) and its state
@@ -357,14 +353,14 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
         }
         publish_min(lmin, larg);
     }
-    // The window costs come from DRAM; a thread asks for its own entries of the next kRing windows ahead of time
-    // (asynchronous copies into a ring in shared memory, one group per window), so the recursion never waits
-    // for memory.  A thread reads only what it copied itself: no barrier is needed for the ring.
+    // The window costs come from DRAM: a thread loads its own entries of the NEXT window at the start of a window and
+    // uses them a whole window later, so the recursion does not wait for memory.
+    float cnow[kOwn], cnext[kOwn];
 #pragma unroll
-    for (int r = 1; r <= kRing; ++r) {
-        if (r < W)
-            for (int g = tid; g < NS; g += kPathThreads) __pipeline_memcpy_async(cring + size_t(r % kRing) * NS4 + g, cost + r * NS + g, 4);
-        __pipeline_commit();
+    for (int o = 0; o < kOwn; ++o) {
+        const int g = tid + o * kPathThreads;
+        cnow[o] = (g < NS && W > 1) ? __ldg(cost + NS + g) : 0.f;
+        cnext[o] = 0.f;
     }
     __syncthreads();                                         // publishes Dp, the minimum and Rs
     for (int64_t w = 1; w < W; ++w) {
@@ -375,6 +371,13 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
         const float shift = (mprev < CUDART_INF_F) ? mprev : 0.f;
         base += double(shift);
         const float bound = mprev + s_rhi[DYN_IDX(h0, 1024)];               // D(h0) = mprev
+        if (w + 1 < W) {
+#pragma unroll
+            for (int o = 0; o < kOwn; ++o) {
+                const int g = tid + o * kPathThreads;
+                if (g < NS) cnext[o] = __ldg(cost + DYN_IDX((w + 1) * NS + g, W * NS));
+            }
+        }
         auto quad_live = [&](int qd) {                       // some source of quad qd can still attain a minimum
             const float4 d4 = reinterpret_cast<const float4 *>(Dp)[DYN_IDX(qd, TG)];
             const float4 m4 = reinterpret_cast<const float4 *>(rlo)[DYN_IDX(qd, TG)];
@@ -386,9 +389,19 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
         if (hg < G) {                                        // the same in every thread of a warp
             const int lane = tid & 31;
             const int nsm = int(int64_t(hg + 1) * SQ / G) - q_lo;
-            live_s = __ballot_sync(0xffffffffu, lane < nsm && quad_live(q_lo + lane));
-            const int hq = h_reg / 4 + lane;
-            live_r = __ballot_sync(0xffffffffu, lane < kRegRows / 4 && hq < TG && quad_live(hq));
+            if (nsm + kRegRows / 4 <= 32) {
+                // one vote serves both kinds: lanes 0 .. nsm-1 the shared-memory quads, the next ten the register quads
+                const int jr = lane - nsm;
+                const int qd = lane < nsm ? q_lo + lane : h_reg / 4 + jr;
+                const bool have = lane < nsm || (jr < kRegRows / 4 && qd < TG);
+                const uint32_t bal = __ballot_sync(0xffffffffu, quad_live(have ? qd : 0) && have);
+                live_s = bal & ((1u << nsm) - 1u);
+                live_r = (bal >> nsm) & ((1u << (kRegRows / 4)) - 1u);
+            } else {
+                live_s = __ballot_sync(0xffffffffu, lane < nsm && quad_live(q_lo + lane));
+                const int hq = h_reg / 4 + lane;
+                live_r = __ballot_sync(0xffffffffu, lane < kRegRows / 4 && hq < TG && quad_live(hq));
+            }
         }
         if (worker) {
             float b0 = CUDART_INF_F, b1 = CUDART_INF_F, b2 = CUDART_INF_F, b3 = CUDART_INF_F;
@@ -444,17 +457,19 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
         __syncthreads();                                     // every reader of Dp is done; the partial minima are in
         float lmin = CUDART_INF_F;
         int larg = 0;
-        __pipeline_wait_prior(kRing - 1);                    // this window's costs have arrived (the thread's own entries)
-        float *cslot = cring + size_t(w % kRing) * NS4;
 #pragma unroll
         for (int o = 0; o < kOwn; ++o) {
             const int g = tid + o * kPathThreads;
             if (g < NS) {
-                float best = part[DYN_IDX(g, NS4)];
-                for (int k = 1; k < G; ++k) best = fminf(best, part[DYN_IDX(k * NS4 + g, G * NS4)]);
+                float best = part[DYN_IDX(g, NS4)];               // G is 1, 2, 4 or 8: independent loads
+                if (G >= 2) best = fminf(best, part[DYN_IDX(NS4 + g, G * NS4)]);
+                if (G >= 4) best = min3f(best, part[DYN_IDX(2 * NS4 + g, G * NS4)], part[DYN_IDX(3 * NS4 + g, G * NS4)]);
+                if (G >= 8)
+                    best = fminf(min3f(best, part[DYN_IDX(4 * NS4 + g, G * NS4)], part[DYN_IDX(5 * NS4 + g, G * NS4)]),
+                                 fminf(part[DYN_IDX(6 * NS4 + g, G * NS4)], part[DYN_IDX(7 * NS4 + g, G * NS4)]));
                 // the minimum of the PREVIOUS vector comes off here, one window late: one subtraction per entry
                 // instead of one per source in the scan; the values stay within two windows' growth of zero
-                const float d = (cslot[DYN_IDX(g, NS4)] + best) - shift;
+                const float d = (cnow[o] + best) - shift;
                 Dp[DYN_IDX(g, NS4)] = d;
                 hist[DYN_IDX(w * NS + g, W * NS)] = d;       // the vector as held: the walk back reads it
                 if (d < lmin) {
@@ -464,11 +479,8 @@ __global__ void __launch_bounds__(kPathThreads) reconf_path_kernel(const ReconfA
             }
         }
         publish_min(lmin, larg);
-        // the slot is free (its values went into the minimum just published): ask for the costs kRing windows on
-        if (w + kRing < W)
-            for (int g = tid; g < NS; g += kPathThreads)
-                __pipeline_memcpy_async(cslot + g, cost + DYN_IDX((w + kRing) * NS + g, W * NS), 4);
-        __pipeline_commit();
+#pragma unroll
+        for (int o = 0; o < kOwn; ++o) cnow[o] = cnext[o];
         __syncthreads();                                     // publishes Dp and the minimum
     }
     int h_last;
@@ -634,7 +646,7 @@ __global__ void __launch_bounds__(kBackThreads) reconf_back_kernel(const ReconfA
 // rows of R kept in shared memory for NS states, given the device's limit
 static size_t reconf_fixed_floats(int32_t NS) {
     const int NS4 = (NS + 3) & ~3, TG = NS4 / 4, lanes_t = (TG + 31) / 32 * 32, G = kPathThreads / lanes_t;
-    return size_t(1 + G + kRing + 1) * NS4;
+    return size_t(1 + G + 1) * NS4;
 }
 static int reconf_rows_in_smem(int32_t NS, size_t limit) {
     const int NS4 = (NS + 3) & ~3;
