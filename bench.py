@@ -779,7 +779,7 @@ def measure_hier(dyn, gen, dev, S=2048, peaks=None):
     return {"workload": f"cfg2 shape x {S} scenarios, epochs {e1}/{e2}/1 windows", "tiles": int(tiles), "call_ms": ms,
             "tiles_per_s": tiles / (ms * 1e-3), "candidates_upper_bound": int(cands),
             "roofline": {"bound": "alu", "achieved": tfl, "peak": fp32_peak, "unit": "TFLOP/s", "frac": tfl / fp32_peak,
-                         "traffic": None, "peak_source": peak_src + "; candidates are an upper bound (node budget prunes)"},
+                         "traffic": None, "peak_source": peak_src + "; candidates of the definition (every count and degree within the node budget, every frequency): the sharding level decides most of them by a lower bound without evaluating them, so this fraction says how fast the definition's work is done, not how busy the pipes are"},
             "energy_over_joint_optimum": hier_total / joint_total}
 
 
@@ -855,7 +855,7 @@ def measure_reconf(dyn, gen, dev, S=16, peaks=None):
             "path_kernel_ms": ms, "call_ms": c0.elapsed_time(c1) / K, "minplus_steps": int(steps),
             "steps_per_s": steps / (ms * 1e-3),
             "roofline": {"bound": "alu", "achieved": tfl, "peak": fp32_peak, "unit": "TFLOP/s", "frac": tfl / fp32_peak,
-                         "traffic": None, "peak_source": peak_src + "; 2 flop (add, compare) per step"},
+                         "traffic": None, "peak_source": peak_src + "; 2 flop (add, compare) per step of the definition (W x NS^2 per problem); sources that cannot attain any minimum are skipped, so the executed steps are fewer on tables whose entries are small next to the spread of the window costs"},
             "window_energy_over_free_optimum": float(out.E_total.sum().item() / jout.E_total.sum().item()),
             "schedules": int(torch.isfinite(total).sum().item())}
 
