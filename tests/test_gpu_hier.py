@@ -126,3 +126,27 @@ def test_hier_classes_with_and_without_load_thresholds(dyn):
     assert {c for c, _, _ in bad} == {0, 4, 8}
     load = gen.random_loads((2, 24, 9), seed=37, mean=5.0)
     _check(dyn, prof, sp, 12, 4, load, max_exempt=0.03)
+
+
+@pytest.mark.parametrize("shape", ["convex", "concave", "falling"])
+def test_hier_energy_rows_that_are_not_lines(dyn, shape):
+    """The sharding level stops its walk over the counts on a line under the degree's energy row.  Rows that bend
+    upwards (the line's intercept is negative: no early stop at that degree), bend downwards, or fall with the load
+    must give the choices of the full walk, which the oracle does."""
+    import dataclasses
+    wl = gen.workload("cfg2")
+    prof, sp = wl.profile(), wl.space()
+    u = np.linspace(0.0, 1.0, prof.M, dtype=np.float64)
+    tp = prof.tp.astype(np.float64)[None, :, None, None]
+    s3 = (prof.f_grid_mhz.astype(np.float64) / 1980.0)[None, None, :, None] ** 3
+    if shape == "convex":
+        pw = 5.0 * tp + 900.0 * tp * s3 * u ** 3
+    elif shape == "concave":
+        pw = 120.0 * tp + 500.0 * tp * s3 * np.sqrt(u)
+    else:
+        pw = 700.0 * tp - 450.0 * tp * s3 * u
+    pw = np.broadcast_to(pw, prof.pow.shape).astype(np.float32).copy()
+    prof = dataclasses.replace(prof, pow=pw)
+    load = gen.random_loads((2, 48, 9), seed=41, mean=4.0)
+    load[1, :, 2] *= 6.0                                     # a class that needs many instances
+    _check(dyn, prof, sp, 12, 4, load, max_exempt=0.03)

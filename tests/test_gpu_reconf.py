@@ -146,3 +146,27 @@ def test_free_form_tables(dyn, monotone):
     sp = gen.make_space(sp0.f_cand_mhz, 12, 60.0, slo_ttft=0.8, slo_tbt=0.1)
     load = gen.random_loads((1, 14, 9), seed=57, mean=6.0, zero_frac=0.0)
     _check(dyn, prof, sp, _table(sp.n_max * prof.T, 6, 4.0), load)
+
+
+@pytest.mark.parametrize("kind", ["cheap-next-to-the-cost-spread", "few-cheap-moves", "staying-costs-too"])
+def test_tables_that_let_the_forward_pass_skip_sources(dyn, kind):
+    """The forward pass skips sources that cannot attain any minimum (a bound from the state of the last minimum and
+    the row extremes of the table).  Tables with small entries (nearly every source is skipped), with a few cheap
+    moves among prohibitive ones (the row minima are far below the row maxima) and with a non-zero diagonal must give
+    the optimum of the full scan, which the oracle does."""
+    wl = gen.workload("cfg2")
+    prof, sp = wl.profile(), gen.make_space(wl.f_cand_mhz, 24, wl.window_s)
+    NS = sp.n_max * prof.T
+    rng = np.random.default_rng(61)
+    if kind == "cheap-next-to-the-cost-spread":
+        R = rng.uniform(0.0, 0.5, (NS, NS)).astype(np.float32)
+        np.fill_diagonal(R, 0.0)
+    elif kind == "few-cheap-moves":
+        R = np.full((NS, NS), 5e3, np.float32)
+        cheap = rng.random((NS, NS)) < 0.05
+        R[cheap] = rng.uniform(0.0, 3.0, int(cheap.sum())).astype(np.float32)
+        np.fill_diagonal(R, 0.0)
+    else:
+        R = rng.uniform(1.0, 4.0, (NS, NS)).astype(np.float32)              # the diagonal too: no move is free
+    load = gen.random_loads((2, 40, 9), seed=62, mean=3.0)
+    _check(dyn, prof, sp, R, load)
