@@ -188,9 +188,10 @@ int64_t enumerate_tuples(const dyn_profile *p, const dyn_space *sp, int64_t limi
 
 constexpr int64_t kMaxTuples = int64_t(1) << 20;
 
-// entries the list of (tuple, TP index) pairs can take: one per tuple and index plus the padding of every index
+// entries the list of (tuple, TP index) pairs can take: one per tuple and index, plus at most one padded-out chunk per
+// index and at the end
 size_t mixed_pairs_capacity(int64_t K, int T) {
-    return K <= kMixedPairsMaxTuples ? size_t(K) * size_t(T) + size_t(T) * size_t(kMixedPairsChunk) : 0;
+    return K <= kMixedPairsMaxTuples ? size_t(K) * size_t(T) + size_t(T + 1) * size_t(kMixedPairsChunk) : 0;
 }
 
 int check_mixed(const dyn_profile *p, const dyn_space *sp, int64_t S, int64_t W, ResolveParams *rp) {
@@ -448,15 +449,40 @@ int dyn_mixed_select(const dyn_profile *profile, const dyn_space *space, const f
     if (K <= kMixedPairsMaxTuples) {
         static thread_local std::vector<uint32_t> pairs;
         pairs.clear();
+        // A lane takes two neighbouring entries, which must share their TP index (every index is padded to an even
+        // count); a chunk of kMixedPairsChunk entries may run over from one index into the next as long as no tuple
+        // appears in it twice (the sums of a chunk are added without looking at each other): where one would, the
+        // chunk is padded out.  Padding entries hold no instance and are never evaluated.
+        static thread_local std::vector<uint8_t> in_chunk;
+        in_chunk.assign(size_t(K), 0);
+        size_t chunk_begin = 0;
+        auto new_chunk_if_full = [&]() {
+            if (pairs.size() - chunk_begin == size_t(kMixedPairsChunk)) {
+                for (size_t e = chunk_begin; e < pairs.size(); ++e) in_chunk[pairs[e] & 0xffffu] = 0;
+                chunk_begin = pairs.size();
+            }
+        };
         for (int t = 0; t < profile->T; ++t) {
             for (int64_t k = 0; k < K; ++k) {
                 const uint32_t n = (tuples[size_t(k)].x >> (8 * t)) & 255u;
-                if (n) pairs.push_back(uint32_t(k) | (n << 16) | (uint32_t(t) << 24));
+                if (!n) continue;
+                if (in_chunk[size_t(k)]) {                   // the tuple is in this chunk already (at a lower index): pad it out
+                    while (pairs.size() - chunk_begin < size_t(kMixedPairsChunk)) pairs.push_back(uint32_t(t) << 24);
+                    new_chunk_if_full();
+                }
+                pairs.push_back(uint32_t(k) | (n << 16) | (uint32_t(t) << 24));
+                in_chunk[size_t(k)] = 1;
+                new_chunk_if_full();
             }
-            while (pairs.size() % size_t(kMixedPairsChunk)) pairs.push_back(uint32_t(t) << 24);     // no instance: never evaluated
+            if (pairs.size() & 1u) {                         // an even count per index; the padding entry names tuple 0 with no instance
+                pairs.push_back(uint32_t(t) << 24);
+                new_chunk_if_full();
+            }
         }
-        n_pairs = int64_t(pairs.size());
-        DYN_CUDA_TRY(cudaMemcpyAsync(ws + off_pairs, pairs.data(), pairs.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, st));
+        while (pairs.size() % size_t(kMixedPairsChunk)) pairs.push_back(uint32_t(profile->T - 1) << 24);
+        n_pairs = pairs.size() <= mixed_pairs_capacity(K, profile->T) ? int64_t(pairs.size()) : 0;     // (0: the kernel for long lists)
+        if (n_pairs > 0)
+            DYN_CUDA_TRY(cudaMemcpyAsync(ws + off_pairs, pairs.data(), pairs.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, st));
     }
     DYN_CUDA_TRY(launch_resolve(rp, lay, d_ws, st));
     DYN_CUDA_TRY(launch_mixed(lay, d_ws, off_tuples, off_caph, off_inva, off_pairs, n_pairs, K, d_load, tiles, out->d_counts,

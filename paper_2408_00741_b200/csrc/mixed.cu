@@ -331,10 +331,10 @@ __global__ void __launch_bounds__(kThreads, 3) mixed_fast_kernel(const MixedArgs
     }
 }
 
-// threshold variant for short lists: the (tuple, TP index) pairs that hold instances are listed by TP index (the host
-// pads every index to whole chunks of 64 pairs), a warp takes a chunk at a time, two pairs per lane, against the F
-// table rows of the chunk's index, and adds n x (energy of one instance) to the tuple's sum in a per-warp array in
-// shared memory.  Chunks come in ascending TP index, so a tuple's sum forms in the same order as in the other
+// threshold variant for short lists: the (tuple, TP index) pairs that hold instances are listed by TP index, a warp
+// takes a chunk of 64 at a time, two neighbouring pairs per lane, against the F table rows of the lane's index, and
+// adds n x (energy of one instance) to the tuple's sum in a per-warp array in shared memory.  A chunk may run over
+// from one index into the next, but holds no tuple twice (the host sees to that).  Chunks come in ascending TP index, so a tuple's sum forms in the same order as in the other
 // variants; no evaluation is spent on a parallelism that a tuple does not use.  Then the lanes scan the sums.
 template <int T>
 __global__ void __launch_bounds__(kThreads, 3) mixed_pairs_kernel(const MixedArgs a, const int table_bytes) {
@@ -380,9 +380,10 @@ __global__ void __launch_bounds__(kThreads, 3) mixed_pairs_kernel(const MixedArg
         for (int k = lane; k < Kpad; k += 32) Es[DYN_IDX(k, Kpad)] = 0.f;
         __syncwarp();
         for (int64_t e0 = 0; e0 < a.n_pairs; e0 += kMixedPairsChunk) {
-            const uint32_t entA = __ldg(a.pairs + DYN_IDX(e0 + lane, a.n_pairs)), entB = __ldg(a.pairs + DYN_IDX(e0 + 32 + lane, a.n_pairs));
-            const int t = int(__shfl_sync(kFull, entA, 0) >> 24);             // the chunk's TP index (the same in every entry)
-            const uint32_t kA = entA & 0xffffu, kB = entB & 0xffffu, nA = (entA >> 16) & 255u, nB = (entB >> 16) & 255u;
+            // a lane's two neighbouring entries share their TP index; the chunk may run over from one index into the next
+            const uint2 ent = __ldg(reinterpret_cast<const uint2 *>(a.pairs + DYN_IDX(e0 + 2 * lane, a.n_pairs - 1)));
+            const int t = int(ent.x >> 24);
+            const uint32_t kA = ent.x & 0xffffu, kB = ent.y & 0xffffu, nA = (ent.x >> 16) & 255u, nB = (ent.y >> 16) & 255u;
             float ct = caph[0];
 #pragma unroll
             for (int u = 1; u < T; ++u) ct = (u == t) ? caph[u] : ct;
@@ -391,18 +392,18 @@ __global__ void __launch_bounds__(kThreads, 3) mixed_pairs_kernel(const MixedArg
             const float lB = nB ? (L * __ldg(inva_c + DYN_IDX(kB, a.K))) * ct : CUDART_INF_F;
             const uint64_t ln2 = pack2(lA, lB);
             float eA = CUDART_INF_F, eB = CUDART_INF_F;
-            const uint32_t cpair = origin + uint32_t(c * P + t * F) * 16u;
+            uint32_t cpair = origin + uint32_t(c * P + t * F) * 16u;
             const float off0 = row_offset_units(rows2 + uint32_t((c * P + t * F) * RS) * 8u);
             uint64_t off2 = pack2(off0, off0);
 #pragma unroll 4
-            for (int q = 0; q < F; ++q) {
+            for (int q = 0; q < F; ++q, cpair += 16u) {
                 uint64_t icm2, lim2;
-                asm("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(icm2), "=l"(lim2) : "r"(DYN_SMEM_ADDR(cpair + uint32_t(q) * 16u, 16u)));
+                asm("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(icm2), "=l"(lim2) : "r"(DYN_SMEM_ADDR(cpair, 16u)));
                 const float lim = __uint_as_float(uint32_t(lim2));
                 fast_two(ln2, icm2, off2, two23_2, eight2, lim, lim, eA, eB);
                 off2 = add2(off2, off2_step);
             }
-            // the pairs of a chunk belong to different tuples (one TP index): no two lanes meet on a sum
+            // no tuple appears twice in a chunk (the host pads a chunk out where one would): no two lanes meet on a sum
             if (nA) Es[DYN_IDX(kA, Kpad)] += float(nA) * eA;                  // +inf if the group has no frequency
             if (nB) Es[DYN_IDX(kB, Kpad)] += float(nB) * eB;
             __syncwarp();
