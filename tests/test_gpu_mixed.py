@@ -155,3 +155,17 @@ def test_classes_with_and_without_load_thresholds_side_by_side(dyn):
     sp = gen.make_space(sp0.f_cand_mhz, 6, 60.0, slo_ttft=0.8, slo_tbt=0.1, gpu_budget=14)
     load = gen.random_loads((2, 11, 9), seed=36, mean=6.0)
     _check(dyn, prof, sp, load, max_exempt=0.03)
+
+
+@pytest.mark.parametrize("tps,n_max,budget", [((1, 2, 4, 8), 3, 5), ((1, 2, 4, 8), 9, 9), ((1, 2, 4, 8), 16, 16),
+                                              ((1, 2, 4, 8), 20, 21), ((2, 8), 12, 24), ((1, 4, 8), 24, 24),
+                                              ((1, 2, 4, 8), 24, 26)])
+def test_list_lengths_around_the_chunk_and_kernel_limits(dyn, tps, n_max, budget):
+    """Short tuple lists are evaluated as (tuple, TP index) pairs in chunks of 64 that may run over from one TP index
+    into the next; lists beyond 512 tuples take the kernel that holds tuples in lanes.  Lists of 14 to about 900 tuples,
+    with two to four parallelisms, cover chunks that are padded out, chunks that run over, and both kernels."""
+    wl = gen.workload("cfg2")
+    prof = gen.make_profile(tps, wl.f_grid_mhz, wl.M, gen.class_coefficients(7))
+    sp = gen.make_space(wl.f_cand_mhz, n_max, wl.window_s, gpu_budget=budget)
+    load = gen.random_loads((2, 24, 9), seed=71, mean=2.0)
+    _check(dyn, prof, sp, load)
